@@ -1,0 +1,253 @@
+/*
+ * pd.h - C ABI of the B200 (sm_100a) prefill/decode benchmarking library.
+ *
+ * The library measures one dense decoder layer in the two modes the allocation
+ * method needs as inputs (paper, Method: "Acquire prefill throughput under TTFT
+ * constraints" wants the maximum prefill throughput of a saturated instance;
+ * "Acquire decode throughput under TPOT constraints" wants the TPOT-versus-batch
+ * curve), and evaluates the allocation model itself (Eq. 1-13).
+ *
+ * Conventions
+ *   - Every function returns a pd_status; nothing throws or aborts.
+ *   - "device" pointers are CUDA global memory of the current device; "host"
+ *     pointers are ordinary process memory.  The library never takes ownership of
+ *     a caller's pointer; the only library-owned objects are pd_layer handles.
+ *   - bf16 tensors are raw 16-bit patterns, row-major, innermost index contiguous.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).  Layer calls
+ *     only enqueue work: they neither allocate nor synchronise.
+ *   - Structs start with `struct_size = sizeof(struct)` so that fields can be appended.
+ */
+#ifndef PD_H_
+#define PD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  PD_OK = 0,
+  PD_ERR_INVALID_ARG = -1,
+  PD_ERR_UNSUPPORTED_SHAPE = -2,
+  PD_ERR_WORKSPACE_TOO_SMALL = -3,
+  PD_ERR_CUDA = -4,
+  PD_ERR_DEVICE_TIMEOUT = -5,
+  PD_ERR_INFEASIBLE_TTFT = -6,
+  PD_ERR_INFEASIBLE_TPOT = -7,
+  PD_ERR_ARCH = -8
+} pd_status;
+
+/* Static string for a status code. */
+const char* pd_status_str(pd_status s);
+/* cudaError_t (as int) recorded by the calling thread's last PD_ERR_CUDA. */
+int pd_last_cuda_error(void);
+/* Library version, for the binding's sanity check. */
+int pd_version(void);
+
+/* ------------------------------------------------------------------ layer */
+
+/* Shape of one decoder layer.  Supported: head_dim 64 or 128, n_q_heads a multiple
+ * of n_kv_heads with group size <= 16, d_model and d_ff multiples of 64,
+ * max_pos = largest token position + 1 ever used (RoPE table length). */
+typedef struct {
+  uint32_t struct_size;
+  int32_t d_model, n_q_heads, n_kv_heads, head_dim, d_ff;
+  float rms_eps, rope_theta;
+  int32_t max_pos;
+} pd_layer_cfg;
+
+/* Caller's weights: device pointers, bf16, row-major [out_features, in_features]. */
+typedef struct {
+  uint32_t struct_size;
+  const void* w_qkv;  /* [(Hq+2Hkv)*hd, d]: q heads, then k heads, then v heads */
+  const void* w_o;    /* [d, Hq*hd] */
+  const void* w_gate; /* [F, d] */
+  const void* w_up;   /* [F, d] */
+  const void* w_down; /* [d, F] */
+  const void* g_attn; /* [d] RMSNorm gain before attention */
+  const void* g_mlp;  /* [d] RMSNorm gain before the MLP */
+} pd_layer_weights;
+
+typedef struct pd_layer pd_layer; /* opaque; owns repacked weight copies, tensor maps, RoPE table */
+
+/* Copies and repacks the weights on `stream` (cudaMalloc inside).  The caller may free
+ * its own weight buffers once `stream` has been synchronised.  PD_ERR_ARCH if the
+ * current device is not compute capability 10.x. */
+pd_status pd_layer_create(const pd_layer_cfg* cfg, const pd_layer_weights* w, void* stream, pd_layer** out);
+pd_status pd_layer_destroy(pd_layer* layer);
+
+/* Bytes of scratch the layer calls need for at most `max_tokens` prefill tokens per
+ * call, `max_batch` decode sequences and KV length `max_kv_len`. */
+pd_status pd_workspace_bytes(const pd_layer_cfg* cfg, int32_t max_tokens, int32_t max_batch,
+                             int32_t max_kv_len, size_t* out_bytes);
+
+/* Caller-owned KV cache: K and V device bf16 [batch_cap, Hkv, len_cap, hd], one
+ * contiguous run per (sequence, kv head). */
+typedef struct {
+  uint32_t struct_size;
+  void* k;
+  void* v;
+  int32_t batch_cap, len_cap;
+} pd_kv_cache;
+
+/* Prefill mode (paper: the compute-bound phase whose saturated throughput is the
+ * "maximum prefill throughput").  One layer over a packed ragged batch:
+ *   x, out        device bf16 [T, d]; out may alias x
+ *   cu_seqlens    n_req+1 int32, cu[0] = 0, cu[n_req] = T; request r owns rows cu[r]..cu[r+1]-1
+ *                 at positions 0..len_r-1 and attends causally within itself.  Given twice:
+ *                 `_dev` (device copy read by the kernels) and `_host` (validated, sizes grids).
+ *   slots_dev     device int32[n_req] (NULL: slot r = r): K/V of request r are written to
+ *                 cache sequence slots[r], positions 0..len_r-1.  A slot outside the cache is
+ *                 skipped by the kernels and reported by pd_layer_check.
+ * Errors: INVALID_ARG (NULL, non-monotone cu, length beyond the cache or the RoPE table; T = 0
+ * is accepted and does nothing), WORKSPACE_TOO_SMALL, CUDA (launch failure). */
+pd_status pd_prefill_layer(pd_layer* layer, const void* x, void* out, const int32_t* cu_seqlens_dev,
+                           const int32_t* cu_seqlens_host, int32_t n_req, const int32_t* slots_dev,
+                           const pd_kv_cache* cache, void* workspace, size_t workspace_bytes, void* stream);
+
+/* Decode mode (paper: the memory-bandwidth-bound phase measured as TPOT versus batch).
+ *   x, out        device bf16 [B, d]; out may alias x
+ *   kv_len_dev    device int32[B]: tokens already cached for sequence b (= position of the new
+ *                 token).  The new K/V are appended at index kv_len[b]; attention covers
+ *                 kv_len[b]+1 entries.  kv_len itself is not modified.
+ *   max_kv_len    host upper bound of kv_len[b]+1 (sizes the split of the KV range); must be
+ *                 <= cache->len_cap.  Sequence b uses cache slot b.
+ * B = 0 is accepted and does nothing. */
+pd_status pd_decode_layer(pd_layer* layer, const void* x, void* out, const int32_t* kv_len_dev, int32_t B,
+                          int32_t max_kv_len, const pd_kv_cache* cache, void* workspace,
+                          size_t workspace_bytes, void* stream);
+
+/* The same two modes over a stack of n_layers layers run back to back (layer i+1 reads layer
+ * i's output), layer i using caches[i % n_caches].  With io_on_host = 0, x/out/cu_seqlens_dev/
+ * kv_len are device pointers and the call only enqueues work.  With io_on_host = 1 they are
+ * host pointers (pinned memory advised): the call copies the inputs to the device on `stream`,
+ * runs the stack, copies `out` back and synchronises `stream` before returning; for prefill
+ * `cu_seqlens_dev` is then ignored (the host copy is uploaded).  The workspace must come from
+ * pd_workspace_bytes (it includes room for the staged activations). */
+pd_status pd_prefill_stack(pd_layer* const* layers, const pd_kv_cache* caches, int32_t n_layers, int32_t n_caches,
+                           const void* x, void* out, int32_t io_on_host, const int32_t* cu_seqlens_dev,
+                           const int32_t* cu_seqlens_host, int32_t n_req, void* workspace,
+                           size_t workspace_bytes, void* stream);
+pd_status pd_decode_stack(pd_layer* const* layers, const pd_kv_cache* caches, int32_t n_layers, int32_t n_caches,
+                          const void* x, void* out, int32_t io_on_host, const int32_t* kv_len, int32_t B,
+                          int32_t max_kv_len, void* workspace, size_t workspace_bytes, void* stream);
+
+/* Reads and clears the device-side error word of the layer (set when a bounded wait inside
+ * a kernel gave up).  Synchronises `stream`.  PD_OK or PD_ERR_DEVICE_TIMEOUT. */
+pd_status pd_layer_check(pd_layer* layer, void* stream);
+
+/* Plain C[M,N] = A[M,K] * B[N,K]^T in bf16 with fp32 accumulation on the tensor cores
+ * (the contraction every projection of the layer uses), exposed for unit tests and
+ * roofline measurement.  A, B, C device bf16 row-major; K a multiple of 64, N of 16.
+ * `err_word` device int32 (may be NULL), set non-zero if a bounded wait gave up. */
+pd_status pd_gemm_bf16(const void* a, const void* b, void* c, int32_t m, int32_t n, int32_t k,
+                       int32_t* err_word, void* stream);
+
+/* Kernels launched so far by the calling thread through this library. */
+int64_t pd_launch_count(void);
+
+/* Optional per-kernel-class timing for roofline reports.  Between pd_trace_begin and
+ * pd_trace_end every kernel the calling thread launches through the layer calls is bracketed
+ * by a pair of CUDA events on its stream; pd_trace_end waits for them and sums the elapsed
+ * time and the launch count per class.  Tracing adds two event records per kernel, so a
+ * traced pass is for attribution, not for the headline time. */
+#define PD_TRACE_CLASSES 16
+enum {
+  PD_K_GEMM_QKV = 0, PD_K_GEMM_O = 1, PD_K_GEMM_GATE_UP = 2, PD_K_GEMM_DOWN = 3, PD_K_ATTN_PREFILL = 4,
+  PD_K_ATTN_DECODE = 5, PD_K_RMSNORM = 6, PD_K_ROPE_KV = 7, PD_K_SWIGLU = 8
+};
+typedef struct {
+  uint32_t struct_size;
+  double time_s[PD_TRACE_CLASSES];
+  int64_t launches[PD_TRACE_CLASSES];
+} pd_trace_report;
+pd_status pd_trace_begin(void);
+pd_status pd_trace_end(pd_trace_report* out);
+
+/* ---------------------------------------------------------------- measure */
+
+/* One measurement job on the current device with synthetic seeded data.
+ * Prefill (paper, "Acquire prefill throughput ..."): one batch of n_req requests with host
+ * lengths l_in[] is pushed through n_layers_run distinct layers back to back, `reps` times;
+ * the maximum prefill throughput is tokens / median time, scaled to n_layers_model layers.
+ * Decode (paper, "Acquire decode throughput ..."): for every batch size, steps t = 0,
+ * step_stride, ... < n_steps (and the last step) run the stack at kv_len = kv_len_start + t;
+ * TPOT(B) is the mean step time scaled to n_layers_model layers.
+ * Either part is skipped when its count (n_req / n_batch_sizes) is 0. */
+typedef struct {
+  uint32_t struct_size;
+  int32_t n_layers_run, n_layers_model;
+  int32_t warmup, reps;
+  uint64_t seed;
+  const int32_t* l_in; /* host int32[n_req] */
+  int32_t n_req;
+  const int32_t* batch_sizes; /* host int32[n_batch_sizes], at most 32 */
+  int32_t n_batch_sizes;
+  int32_t kv_len_start, n_steps, step_stride;
+  const int32_t* kv_len_mix; /* optional host int32[max batch]: per-sequence start lengths (ragged); NULL = kv_len_start */
+} pd_measure_cfg;
+
+typedef struct {
+  uint32_t struct_size;
+  double prefill_time_s;   /* median, n_layers_model layers */
+  double prefill_tok_s;    /* maximum prefill throughput */
+  double prefill_flops;    /* algorithmic flops of that pass (causal half of attention) */
+  double prefill_frac_bf16_peak;
+  int32_t n_points;
+  int32_t batch[32];
+  double tpot_s[32];                /* TPOT(B), n_layers_model layers */
+  double decode_bytes[32];          /* algorithmic bytes per step */
+  double decode_frac_hbm_peak[32];
+  double attn_time_s[32];           /* decode-attention kernel alone, per layer, mean over the steps */
+  double attn_frac_hbm_peak[32];
+  int32_t gpu_launches;             /* kernels launched inside the timed regions */
+} pd_measurement;
+
+pd_status pd_measure(const pd_layer_cfg* cfg, const pd_measure_cfg* mcfg, double peak_bf16_flops,
+                     double peak_hbm_bytes_s, pd_measurement* out);
+
+/* --------------------------------------------------------------- allocate */
+
+/* Inputs of the allocation model.  Throughputs in tokens/s, times in seconds; l_in and
+ * l_out are the mean input and output lengths (Eq. 1); the curve (batch[i], tpot_s[i]) is
+ * the measured TPOT per decode batch size. */
+typedef struct {
+  uint32_t struct_size;
+  double tp_total_tok_s, l_in, l_out, ttft_slo_s, tpot_slo_s, t_overhead_s;
+  double prefill_max_tok_s;
+  int32_t n_points;
+  const int32_t* batch;
+  const double* tpot_s;
+} pd_alloc_in;
+
+typedef struct {
+  uint32_t struct_size;
+  double tp_prefill_eff; /* Eq. 13 */
+  double tp_decode_eff;  /* B* / TPOT(B*) */
+  double mu, lambda, rho; /* Eq. 9-11 */
+  int32_t feasible_batch; /* B*: largest sweep point whose whole prefix meets the TPOT SLO */
+  int32_t sweep_capped;   /* 1 if B* is the largest measured batch */
+  double n_prefill_frac, n_decode_frac; /* Eq. 5, 6 */
+  double ratio_pd;                       /* Eq. 7 */
+  int32_t n_prefill, n_decode;           /* nearest integer (half up), at least 1 */
+  int32_t n_prefill_ceil, n_decode_ceil; /* ceiling, at least 1 */
+  double achieved_total_tok_s;           /* Eq. 1 with T_total = max(Eq. 2, Eq. 3) at the integer counts */
+} pd_alloc_out;
+
+/* Pure host code, usable without a GPU.  PD_ERR_INFEASIBLE_TTFT when TTFT - T_overhead <= 0
+ * or Eq. 13 is not positive; PD_ERR_INFEASIBLE_TPOT when no sweep point meets the TPOT SLO.
+ * Fields that can still be computed are filled; the others are NaN / 0. */
+pd_status pd_allocate(const pd_alloc_in* in, pd_alloc_out* out);
+
+/* FIFO single-server replay of n requests (host): request i arrives gaps[i] after request
+ * i-1 and needs service[i] seconds.  Outputs the mean sojourn time (what Eq. 12 predicts as
+ * 1/(mu - lambda)) and the mean waiting time. */
+pd_status pd_queue_replay(const double* gaps, const double* service, int64_t n, double* mean_sojourn_s,
+                          double* mean_wait_s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PD_H_ */

@@ -1,0 +1,145 @@
+// Shared host-side helpers of the CUDA translation units: status plumbing, the
+// layer object, tensor-map creation and kernel launcher declarations.
+#pragma once
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "pd.h"
+
+namespace pd {
+
+typedef __nv_bfloat16 bf16;
+
+pd_status cuda_fail(cudaError_t e);  // records e for pd_last_cuda_error(), returns PD_ERR_CUDA
+
+#define PD_CUDA_TRY(expr)                              \
+  do {                                                 \
+    cudaError_t pd_e_ = (expr);                        \
+    if (pd_e_ != cudaSuccess) return ::pd::cuda_fail(pd_e_); \
+  } while (0)
+
+#define PD_TRY(expr)                    \
+  do {                                  \
+    pd_status pd_s_ = (expr);           \
+    if (pd_s_ != PD_OK) return pd_s_;   \
+  } while (0)
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// Counts kernel launches made by this thread (reported by pd_measure).
+extern thread_local long long g_launch_count;
+inline void count_launch(int n = 1) { g_launch_count += n; }
+
+// Brackets the kernels launched in its scope with CUDA events while a trace is active
+// (pd_trace_begin .. pd_trace_end); free otherwise.
+class TraceScope {
+ public:
+  TraceScope(int cls, cudaStream_t s);
+  ~TraceScope();
+  TraceScope(const TraceScope&) = delete;
+  TraceScope& operator=(const TraceScope&) = delete;
+
+ private:
+  cudaStream_t stream_;
+  int idx_;
+};
+
+// ------------------------------------------------------------ tensor maps
+// 2-D bf16 row-major tensor [rows, cols] with row pitch `ld` elements, tiled in boxes of
+// box_rows x 64 columns with the 128-byte shared-memory swizzle.
+pd_status make_tmap_bf16(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint64_t ld,
+                         uint32_t box_rows);
+
+// ------------------------------------------------------------------ GEMM
+enum GemmEpilogue : int {
+  EPI_STORE = 0,     // C = acc
+  EPI_RESIDUAL = 1,  // C = R + acc
+};
+
+struct GemmArgs {
+  const bf16* a;  // [M, K], row pitch lda
+  const bf16* b;  // [N, K], row pitch ldb
+  bf16* c;        // [M, N], row pitch ldc
+  const bf16* r;  // residual [M, N], row pitch ldr (EPI_RESIDUAL); may alias c
+  int m, n, k;
+  int lda, ldb, ldc, ldr;
+  int epilogue;
+  int* err_word;              // device int32, set non-zero on a device-side timeout; may be NULL
+};
+
+// Tensor-core GEMM (tcgen05 + TMEM accumulators, operands staged by TMA).
+pd_status gemm_tc(const GemmArgs& g, cudaStream_t stream);
+// Plain CUDA-core GEMM with the same contract: debugging reference, selected with PD_GEMM=simt.
+pd_status gemm_simt(const GemmArgs& g, cudaStream_t stream);
+// Dispatches on the PD_GEMM environment variable (read once).
+pd_status gemm(const GemmArgs& g, cudaStream_t stream);
+// Box height (rows of B per tile) the tensor-core GEMM will use for this problem.
+int gemm_tc_block_n(int m, int n, int k);
+
+// ------------------------------------------------------------ elementwise
+pd_status launch_rmsnorm(const bf16* x, const bf16* gain, bf16* y, int rows, int d, float eps, cudaStream_t s);
+
+struct RopeArgs {
+  bf16* qkv;              // [T, n_qkv] in/out: q part is rotated in place
+  bf16* k_cache;          // [batch_cap, Hkv, len_cap, hd]
+  bf16* v_cache;
+  const float2* rope_tab; // [max_pos, hd/2] (cos, sin)
+  const int32_t* cu_seqlens;  // prefill: device [n_req+1]; decode: NULL
+  const int32_t* slots;       // prefill: device [n_req] cache slot per request, or NULL (slot = request)
+  const int32_t* kv_len;      // decode: device [B] position of the new token; prefill: NULL
+  int n_req;
+  int n_tokens, n_q_heads, n_kv_heads, head_dim, len_cap;
+  int max_pos;                // rows of rope_tab
+  int batch_cap;              // sequences in the cache
+  int* err_word;              // set to 2 when a position or slot falls outside the cache or the table
+};
+pd_status launch_rope_scatter(const RopeArgs& a, cudaStream_t s);
+
+// a[T, F] = silu(gu[T, 0:F]) * gu[T, F:2F]
+pd_status launch_swiglu(const bf16* gu, bf16* a, int rows, int f, cudaStream_t s);
+
+// -------------------------------------------------------------- attention
+struct PrefillAttnArgs {
+  const bf16* q;       // [T, ldq] (head h at column h*hd)
+  int ldq;
+  const bf16* k_cache; // [batch_cap, Hkv, len_cap, hd]
+  const bf16* v_cache;
+  bf16* o;             // [T, Hq*hd]
+  const int32_t* cu_seqlens;  // device [n_req+1]
+  const int32_t* slots;       // device [n_req] or NULL
+  int n_req, n_tokens, max_len;
+  int n_q_heads, n_kv_heads, head_dim, len_cap, batch_cap;
+};
+pd_status launch_prefill_attention(const PrefillAttnArgs& a, cudaStream_t s);
+
+struct DecodeAttnArgs {
+  const bf16* q;       // [B, ldq]
+  int ldq;
+  const bf16* k_cache;
+  const bf16* v_cache;
+  bf16* o;             // [B, Hq*hd]
+  const int32_t* kv_len;  // device [B]; attention covers kv_len[b] + 1 entries
+  float* partial;         // workspace [B, Hkv, n_splits, G, hd + 2] fp32 (when n_splits > 1)
+  int batch, max_kv_len, n_splits;
+  int n_q_heads, n_kv_heads, head_dim, len_cap;
+};
+int decode_attention_splits(int batch, int n_kv_heads, int max_kv_len);
+pd_status launch_decode_attention(const DecodeAttnArgs& a, cudaStream_t s);
+
+// Seeded N(mean, std) fill in bf16 (counter-based; value i depends only on seed, stream, i).
+pd_status launch_fill_normal(bf16* dst, size_t n, uint64_t seed, uint64_t stream_id, float mean, float std,
+                             cudaStream_t s);
+
+}  // namespace pd
+
+// The opaque layer object.
+struct pd_layer {
+  pd_layer_cfg cfg;
+  int n_qkv;
+  pd::bf16 *w_qkv, *w_o, *w_gu, *w_down;  // owned copies; w_gu = [2F, d]: gate rows then up rows
+  pd::bf16 *g_attn, *g_mlp;
+  float2* rope_tab;                        // [max_pos, hd/2]
+  int* err_word;                           // device int32
+};

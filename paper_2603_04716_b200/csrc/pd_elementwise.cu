@@ -1,0 +1,223 @@
+// Memory-bound glue kernels of the layer: RMSNorm, RoPE with the KV-cache write, SwiGLU,
+// and the seeded synthetic fill used by the measurement harness.  All use 128-bit accesses.
+#include "pd_common.cuh"
+#include "pd_ptx.cuh"
+
+namespace pd {
+namespace {
+
+__device__ __forceinline__ void unpack8(const uint4& v, float (&f)[8]) {
+  f[0] = ptx::bf16_lo(v.x); f[1] = ptx::bf16_hi(v.x);
+  f[2] = ptx::bf16_lo(v.y); f[3] = ptx::bf16_hi(v.y);
+  f[4] = ptx::bf16_lo(v.z); f[5] = ptx::bf16_hi(v.z);
+  f[6] = ptx::bf16_lo(v.w); f[7] = ptx::bf16_hi(v.w);
+}
+__device__ __forceinline__ uint4 pack8(const float (&f)[8]) {
+  uint4 o;
+  o.x = ptx::pack_bf16(f[0], f[1]);
+  o.y = ptx::pack_bf16(f[2], f[3]);
+  o.z = ptx::pack_bf16(f[4], f[5]);
+  o.w = ptx::pack_bf16(f[6], f[7]);
+  return o;
+}
+
+// ------------------------------------------------------------------- RMSNorm
+// y = x * rsqrt(mean(x^2) + eps) * g; one block per row, row kept in registers.
+constexpr int RMS_THREADS = 256;
+constexpr int RMS_MAX_CHUNKS = 8;  // 8 chunks * 8 elements * 256 threads = d up to 16384
+
+__global__ void __launch_bounds__(RMS_THREADS) rmsnorm_kernel(const bf16* __restrict__ x,
+                                                               const bf16* __restrict__ gain, bf16* __restrict__ y,
+                                                               int d, float eps) {
+  const int row = blockIdx.x;
+  const uint4* xr = reinterpret_cast<const uint4*>(x + static_cast<size_t>(row) * d);
+  const uint4* gr = reinterpret_cast<const uint4*>(gain);
+  uint4* yr = reinterpret_cast<uint4*>(y + static_cast<size_t>(row) * d);
+  const int chunks = d / 8;
+  uint4 v[RMS_MAX_CHUNKS];
+  float ss = 0.f;
+#pragma unroll
+  for (int i = 0; i < RMS_MAX_CHUNKS; ++i) {
+    const int c = threadIdx.x + i * RMS_THREADS;
+    if (c < chunks) {
+      v[i] = xr[c];
+      float f[8];
+      unpack8(v[i], f);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) ss = fmaf(f[e], f[e], ss);
+    }
+  }
+  __shared__ float red[RMS_THREADS / 32];
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+  __syncthreads();
+  float tot = 0.f;
+#pragma unroll
+  for (int w = 0; w < RMS_THREADS / 32; ++w) tot += red[w];
+  const float scale = rsqrtf(tot / static_cast<float>(d) + eps);
+#pragma unroll
+  for (int i = 0; i < RMS_MAX_CHUNKS; ++i) {
+    const int c = threadIdx.x + i * RMS_THREADS;
+    if (c < chunks) {
+      float f[8], g[8];
+      unpack8(v[i], f);
+      unpack8(gr[c], g);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) f[e] = f[e] * scale * g[e];
+      yr[c] = pack8(f);
+    }
+  }
+}
+
+// ------------------------------------------------------- RoPE + KV-cache write
+// One block per token.  Each thread owns 8 rotation pairs (i, i + hd/2) of one head: it
+// loads 16 bytes from each half, rotates by the table entry of the token's position and
+// stores q back in place or k into the cache; v heads are copied to the cache unchanged.
+__global__ void __launch_bounds__(128) rope_scatter_kernel(RopeArgs a) {
+  const int t = blockIdx.x;
+  __shared__ int s_pos, s_slot;
+  if (threadIdx.x == 0) {
+    if (a.cu_seqlens) {
+      int lo = 0, hi = a.n_req;  // find r with cu[r] <= t < cu[r+1]
+      while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (a.cu_seqlens[mid] <= t) lo = mid; else hi = mid;
+      }
+      s_pos = t - a.cu_seqlens[lo];
+      s_slot = a.slots ? a.slots[lo] : lo;
+    } else {
+      s_pos = a.kv_len[t];
+      s_slot = t;
+    }
+  }
+  __syncthreads();
+  const int pos = s_pos, slot = s_slot;
+  if (pos < 0 || pos >= a.len_cap || pos >= a.max_pos || slot < 0 || slot >= a.batch_cap) {
+    // would write outside the cache: record and skip
+    if (threadIdx.x == 0 && a.err_word) atomicExch(a.err_word, 2);
+    return;
+  }
+  const int hd = a.head_dim, half = hd / 2;
+  const int per_head = half / 8;  // threads per head
+  const int n_heads = a.n_q_heads + 2 * a.n_kv_heads;
+  const int n_qkv = n_heads * hd;
+  bf16* row = a.qkv + static_cast<size_t>(t) * n_qkv;
+  const float2* tab = a.rope_tab + static_cast<size_t>(pos) * half;
+  for (int w = threadIdx.x; w < n_heads * per_head; w += blockDim.x) {
+    const int h = w / per_head;
+    const int i0 = (w - h * per_head) * 8;
+    bf16* src = row + h * hd;
+    const uint4 lo4 = *reinterpret_cast<const uint4*>(src + i0);
+    const uint4 hi4 = *reinterpret_cast<const uint4*>(src + half + i0);
+    if (h < a.n_q_heads + a.n_kv_heads) {
+      float lo[8], hi[8], olo[8], ohi[8];
+      unpack8(lo4, lo);
+      unpack8(hi4, hi);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        const float2 cs = tab[i0 + e];
+        olo[e] = lo[e] * cs.x - hi[e] * cs.y;
+        ohi[e] = hi[e] * cs.x + lo[e] * cs.y;
+      }
+      bf16* dst;
+      if (h < a.n_q_heads) {
+        dst = src;
+      } else {
+        const int j = h - a.n_q_heads;
+        dst = a.k_cache + ((static_cast<size_t>(slot) * a.n_kv_heads + j) * a.len_cap + pos) * hd;
+      }
+      *reinterpret_cast<uint4*>(dst + i0) = pack8(olo);
+      *reinterpret_cast<uint4*>(dst + half + i0) = pack8(ohi);
+    } else {
+      const int j = h - a.n_q_heads - a.n_kv_heads;
+      bf16* dst = a.v_cache + ((static_cast<size_t>(slot) * a.n_kv_heads + j) * a.len_cap + pos) * hd;
+      *reinterpret_cast<uint4*>(dst + i0) = lo4;
+      *reinterpret_cast<uint4*>(dst + half + i0) = hi4;
+    }
+  }
+}
+
+// -------------------------------------------------------------------- SwiGLU
+__global__ void __launch_bounds__(256) swiglu_kernel(const bf16* __restrict__ gu, bf16* __restrict__ out,
+                                                      size_t rows, int f) {
+  const int chunks_per_row = f / 8;
+  const size_t total = rows * chunks_per_row;
+  for (size_t idx = blockIdx.x * static_cast<size_t>(blockDim.x) + threadIdx.x; idx < total;
+       idx += static_cast<size_t>(gridDim.x) * blockDim.x) {
+    const size_t r = idx / chunks_per_row;
+    const int c = static_cast<int>(idx - r * chunks_per_row);
+    const bf16* base = gu + r * (2 * static_cast<size_t>(f));
+    float g[8], u[8], o[8];
+    unpack8(*reinterpret_cast<const uint4*>(base + c * 8), g);
+    unpack8(*reinterpret_cast<const uint4*>(base + f + c * 8), u);
+#pragma unroll
+    for (int e = 0; e < 8; ++e) o[e] = g[e] / (1.f + __expf(-g[e])) * u[e];
+    *reinterpret_cast<uint4*>(out + r * f + c * 8) = pack8(o);
+  }
+}
+
+// ------------------------------------------------------------- seeded fill
+__device__ __forceinline__ uint64_t splitmix64(uint64_t z) {
+  z += 0x9E3779B97F4A7C15ull;
+  z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+  z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+  return z ^ (z >> 31);
+}
+
+__global__ void __launch_bounds__(256) fill_normal_kernel(bf16* dst, size_t n, uint64_t key, float mean, float std) {
+  // One hash per pair of outputs, Box-Muller on its two 32-bit halves.
+  const size_t pairs = (n + 1) / 2;
+  for (size_t i = blockIdx.x * static_cast<size_t>(blockDim.x) + threadIdx.x; i < pairs;
+       i += static_cast<size_t>(gridDim.x) * blockDim.x) {
+    const uint64_t h = splitmix64(key ^ splitmix64(i));
+    const float u1 = (static_cast<float>(static_cast<uint32_t>(h >> 32) >> 8) + 0.5f) * (1.0f / 16777216.0f);
+    const float u2 = (static_cast<float>(static_cast<uint32_t>(h) >> 8) + 0.5f) * (1.0f / 16777216.0f);
+    const float rad = sqrtf(-2.0f * __logf(u1));
+    float s, c;
+    __sincosf(6.283185307179586f * u2, &s, &c);
+    dst[2 * i] = __float2bfloat16(mean + std * rad * c);
+    if (2 * i + 1 < n) dst[2 * i + 1] = __float2bfloat16(mean + std * rad * s);
+  }
+}
+
+}  // namespace
+
+pd_status launch_rmsnorm(const bf16* x, const bf16* gain, bf16* y, int rows, int d, float eps, cudaStream_t s) {
+  if (rows == 0) return PD_OK;
+  if (d % 8 != 0 || d > RMS_THREADS * RMS_MAX_CHUNKS * 8) return PD_ERR_UNSUPPORTED_SHAPE;
+  rmsnorm_kernel<<<rows, RMS_THREADS, 0, s>>>(x, gain, y, d, eps);
+  count_launch();
+  PD_CUDA_TRY(cudaGetLastError());
+  return PD_OK;
+}
+
+pd_status launch_rope_scatter(const RopeArgs& a, cudaStream_t s) {
+  if (a.n_tokens == 0) return PD_OK;
+  rope_scatter_kernel<<<a.n_tokens, 128, 0, s>>>(a);
+  count_launch();
+  PD_CUDA_TRY(cudaGetLastError());
+  return PD_OK;
+}
+
+pd_status launch_swiglu(const bf16* gu, bf16* out, int rows, int f, cudaStream_t s) {
+  if (rows == 0) return PD_OK;
+  const size_t total = static_cast<size_t>(rows) * (f / 8);
+  size_t blocks = (total + 255) / 256;
+  if (blocks > 148 * 16) blocks = 148 * 16;
+  swiglu_kernel<<<static_cast<unsigned>(blocks), 256, 0, s>>>(gu, out, static_cast<size_t>(rows), f);
+  count_launch();
+  PD_CUDA_TRY(cudaGetLastError());
+  return PD_OK;
+}
+
+pd_status launch_fill_normal(bf16* dst, size_t n, uint64_t seed, uint64_t stream_id, float mean, float std,
+                             cudaStream_t s) {
+  if (n == 0) return PD_OK;
+  const uint64_t key = seed * 0xD1342543DE82EF95ull + stream_id * 0x2545F4914F6CDD1Dull + 0x632BE59BD9B4E019ull;
+  fill_normal_kernel<<<148 * 8, 256, 0, s>>>(dst, n, key, mean, std);
+  PD_CUDA_TRY(cudaGetLastError());
+  return PD_OK;
+}
+
+}  // namespace pd

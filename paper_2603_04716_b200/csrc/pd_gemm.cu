@@ -1,0 +1,431 @@
+// C[M,N] = A[M,K] * B[N,K]^T (+ residual), bf16 operands, fp32 accumulation.
+//
+// Tensor-core path: a persistent, warp-specialised kernel.  One thread issues TMA tile
+// loads of A (128 x 64) and B (BN x 64) into a ring of shared-memory stages; one thread
+// issues tcgen05.mma (128 x BN x 16 per instruction) accumulating in tensor memory; four
+// warps drain the accumulator (tcgen05.ld) and run the epilogue.  Two accumulator buffers
+// in tensor memory let the epilogue of tile i overlap the main loop of tile i+1.
+// Every barrier wait is wall-clock bounded; on a timeout the block raises a shared abort
+// flag, records an error word in global memory and leaves through the normal teardown.
+#include <cstdlib>
+#include <cstring>
+#include <mutex>
+
+#include "pd_common.cuh"
+#include "pd_ptx.cuh"
+
+namespace pd {
+
+// ------------------------------------------------------------------ tensor maps
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn get_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  });
+  return fn;
+}
+
+pd_status make_tmap_bf16(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint64_t ld,
+                         uint32_t box_rows) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return PD_ERR_CUDA;
+  if ((reinterpret_cast<uintptr_t>(base) & 15u) || (ld * 2) % 16 != 0 || box_rows == 0 || box_rows > 256)
+    return PD_ERR_INVALID_ARG;
+  cuuint64_t dims[2] = {cols, rows};
+  cuuint64_t strides[1] = {ld * 2};
+  cuuint32_t box[2] = {64, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? PD_OK : PD_ERR_INVALID_ARG;
+}
+
+// ---------------------------------------------------------------- tcgen05 GEMM
+namespace {
+
+constexpr int BM = 128;
+constexpr int BK = 64;
+constexpr int GEMM_THREADS = 192;  // warp 0: TMA, warp 1: MMA, warps 2-5: epilogue
+constexpr int TMEM_COLS = 512;
+
+template <int BN>
+struct GemmCfg {
+  static constexpr int A_BYTES = BM * BK * 2;
+  static constexpr int B_BYTES = BN * BK * 2;
+  static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+  static constexpr int STAGES = (BN >= 256) ? 4 : (BN >= 128 ? 6 : 8);
+  static constexpr int ACC_COLS = BN;  // columns per accumulator buffer
+  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+};
+
+struct GemmDev {
+  bf16* c;
+  const bf16* r;
+  int m, n, k;
+  int ldc, ldr;
+  int tiles_m, tiles_n;
+  int* err_word;
+};
+
+__device__ __forceinline__ void tile_coords(int tile, int tiles_m, int tiles_n, int& tm, int& tn) {
+  // Groups of up to 8 row-tiles share the same column-tiles while they are resident, so
+  // concurrently running blocks hit the same A and B tiles in L2.
+  constexpr int GROUP = 8;
+  const int per_group = GROUP * tiles_n;
+  const int g = tile / per_group;
+  const int first_m = g * GROUP;
+  const int rows_in_group = min(GROUP, tiles_m - first_m);
+  const int t = tile - g * per_group;
+  tm = first_m + t % rows_in_group;
+  tn = t / rows_in_group;
+}
+
+template <int BN, int EPI>
+__global__ void __launch_bounds__(GEMM_THREADS, 1)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b, GemmDev p) {
+  using Cfg = GemmCfg<BN>;
+  constexpr int STAGES = Cfg::STAGES;
+  extern __shared__ uint8_t smem_raw[];
+  // tiles need 1024-byte alignment for the 128-byte swizzle pattern
+  const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem_al = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem_al + STAGES * Cfg::STAGE_BYTES);
+  // bars[0..S): full, [S..2S): empty, [2S..2S+2): acc full, [2S+2..2S+4): acc empty
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const uint32_t bar0 = ptx::smem_u32(bars);
+  auto full_bar = [&](int s) { return bar0 + 8u * s; };
+  auto empty_bar = [&](int s) { return bar0 + 8u * (STAGES + s); };
+  auto accf_bar = [&](int a) { return bar0 + 8u * (2 * STAGES + a); };
+  auto acce_bar = [&](int a) { return bar0 + 8u * (2 * STAGES + 2 + a); };
+
+  if (threadIdx.x == 0) {
+    *abort_flag = 0;
+    for (int s = 0; s < STAGES; ++s) {
+      ptx::mbar_init(full_bar(s), 1);
+      ptx::mbar_init(empty_bar(s), 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      ptx::mbar_init(accf_bar(a), 1);
+      ptx::mbar_init(acce_bar(a), 4);
+    }
+    ptx::fence_barrier_init();
+    ptx::prefetch_tensormap(&tmap_a);
+    ptx::prefetch_tensormap(&tmap_b);
+  }
+  if (warp == 1) {
+    ptx::tmem_alloc(ptx::smem_u32(tmem_slot), TMEM_COLS);
+    ptx::tmem_relinquish();
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  const int n_tiles = p.tiles_m * p.tiles_n;
+  const int k_blocks = p.k / BK;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+        int tm, tn;
+        tile_coords(tile, p.tiles_m, p.tiles_n, tm, tn);
+        for (int kb = 0; kb < k_blocks; ++kb) {
+          if (!ptx::mbar_wait_bounded(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
+          const uint32_t sa = smem_base + stage * Cfg::STAGE_BYTES;
+          const uint32_t sb = sa + Cfg::A_BYTES;
+          ptx::mbar_arrive_expect_tx(full_bar(stage), Cfg::STAGE_BYTES);
+          ptx::tma_load_2d(sa, &tmap_a, kb * BK, tm * BM, full_bar(stage));
+          ptx::tma_load_2d(sb, &tmap_b, kb * BK, tn * BN, full_bar(stage));
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+      }
+      if (!ok) {
+        // give loads already in flight time to land before the block's shared memory is released
+        for (int i = 0; i < 2000; ++i) __nanosleep(1000);
+      }
+    }
+  } else if (warp == 1) {
+    // -------------------------------------------------------------- MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc = ptx::umma_idesc_bf16(BM, BN);
+      int stage = 0;
+      uint32_t phase = 0;
+      int acc = 0;
+      uint32_t acc_phase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+        if (!ptx::mbar_wait_bounded(acce_bar(acc), acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+        ptx::tc_fence_after();
+        const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * Cfg::ACC_COLS);
+        for (int kb = 0; kb < k_blocks; ++kb) {
+          if (!ptx::mbar_wait_bounded(full_bar(stage), phase, abort_flag)) { ok = false; break; }
+          ptx::tc_fence_after();
+          const uint32_t sa = smem_base + stage * Cfg::STAGE_BYTES;
+          const uint32_t sb = sa + Cfg::A_BYTES;
+          const uint64_t da = ptx::umma_desc_sw128(sa);
+          const uint64_t db = ptx::umma_desc_sw128(sb);
+#pragma unroll
+          for (int kk = 0; kk < BK / 16; ++kk) {
+            // 16 bf16 = 32 bytes along K inside the 128-byte swizzled row: +2 in 16-byte units
+            ptx::umma_bf16(d_tmem, da + 2u * kk, db + 2u * kk, idesc, (kb > 0 || kk > 0) ? 1u : 0u);
+          }
+          ptx::umma_commit(empty_bar(stage));  // stage is free once these MMAs have read it
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        ptx::umma_commit(accf_bar(acc));  // accumulator complete
+        if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+      }
+    }
+  } else {
+    // ---------------------------------------------------------------- epilogue
+    const int lane_group = warp & 3;  // tensor-memory lanes 32*lane_group .. +31 belong to this warp
+    int acc = 0;
+    uint32_t acc_phase = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+      int tm, tn;
+      tile_coords(tile, p.tiles_m, p.tiles_n, tm, tn);
+      // warp-uniform outcome: tcgen05.ld below needs the whole warp
+      ok = __all_sync(0xffffffffu, ptx::mbar_wait_bounded(accf_bar(acc), acc_phase, abort_flag));
+      if (!ok) break;
+      ptx::tc_fence_after();
+      const int row = tm * BM + lane_group * 32 + lane;
+      const uint32_t t_row = tmem_base + (static_cast<uint32_t>(lane_group * 32) << 16) +
+                             static_cast<uint32_t>(acc * Cfg::ACC_COLS);
+      constexpr int CHUNK = 32;
+#pragma unroll 1
+      for (int c0 = 0; c0 < BN; c0 += 32) {
+        uint32_t v[32];
+        ptx::tmem_ld_32x32(t_row + c0, v);
+        ptx::tmem_ld_wait();
+        const int col = tn * BN + c0;
+        if (row < p.m) {
+          bf16* crow = p.c + static_cast<size_t>(row) * p.ldc + col;
+          const bf16* rrow = (EPI == EPI_RESIDUAL) ? p.r + static_cast<size_t>(row) * p.ldr + col : nullptr;
+#pragma unroll
+          for (int j = 0; j < CHUNK; j += 8) {
+            if (col + j < p.n) {
+              float f[8];
+#pragma unroll
+              for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(v[j + e]);
+              if (EPI == EPI_RESIDUAL) {
+                const uint4 rr = *reinterpret_cast<const uint4*>(rrow + j);
+                f[0] += ptx::bf16_lo(rr.x); f[1] += ptx::bf16_hi(rr.x);
+                f[2] += ptx::bf16_lo(rr.y); f[3] += ptx::bf16_hi(rr.y);
+                f[4] += ptx::bf16_lo(rr.z); f[5] += ptx::bf16_hi(rr.z);
+                f[6] += ptx::bf16_lo(rr.w); f[7] += ptx::bf16_hi(rr.w);
+              }
+              uint4 o;
+              o.x = ptx::pack_bf16(f[0], f[1]);
+              o.y = ptx::pack_bf16(f[2], f[3]);
+              o.z = ptx::pack_bf16(f[4], f[5]);
+              o.w = ptx::pack_bf16(f[6], f[7]);
+              *reinterpret_cast<uint4*>(crow + j) = o;
+            }
+          }
+        }
+      }
+      // all of this warp's reads of the accumulator are complete: hand the buffer back
+      ptx::tc_fence_before();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(acce_bar(acc));
+      if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+    }
+  }
+
+  ptx::tc_fence_before();
+  __syncthreads();
+  if (*abort_flag && threadIdx.x == 0 && p.err_word) atomicExch(p.err_word, 1);
+  if (warp == 1) {
+    __syncwarp();
+    ptx::tc_fence_after();
+    ptx::tmem_dealloc(tmem_base, TMEM_COLS);
+  }
+}
+
+int g_sm_count = 0;
+int sm_count() {
+  if (g_sm_count == 0) {
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess &&
+        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0)
+      g_sm_count = n;
+    else
+      g_sm_count = 148;
+  }
+  return g_sm_count;
+}
+
+template <int BN, int EPI>
+pd_status launch_tc(const GemmArgs& g, cudaStream_t stream) {
+  using Cfg = GemmCfg<BN>;
+  static bool attr_set = false;
+  auto kern = gemm_tc_kernel<BN, EPI>;
+  if (!attr_set) {
+    PD_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES));
+    attr_set = true;
+  }
+  CUtensorMap ta, tb;
+  PD_TRY(make_tmap_bf16(&ta, g.a, g.m, g.k, g.lda, BM));
+  PD_TRY(make_tmap_bf16(&tb, g.b, g.n, g.k, g.ldb, BN));
+  GemmDev p;
+  p.c = g.c; p.r = g.r; p.m = g.m; p.n = g.n; p.k = g.k; p.ldc = g.ldc; p.ldr = g.ldr;
+  p.tiles_m = (g.m + BM - 1) / BM;
+  p.tiles_n = (g.n + BN - 1) / BN;
+  p.err_word = g.err_word;
+  const int tiles = p.tiles_m * p.tiles_n;
+  const int grid = tiles < sm_count() ? tiles : sm_count();
+  kern<<<grid, GEMM_THREADS, Cfg::SMEM_BYTES, stream>>>(ta, tb, p);
+  count_launch();
+  PD_CUDA_TRY(cudaGetLastError());
+  return PD_OK;
+}
+
+template <int BN>
+pd_status launch_tc_epi(const GemmArgs& g, cudaStream_t stream) {
+  return g.epilogue == EPI_RESIDUAL ? launch_tc<BN, EPI_RESIDUAL>(g, stream) : launch_tc<BN, EPI_STORE>(g, stream);
+}
+
+}  // namespace
+
+int gemm_tc_block_n(int m, int n, int k) {
+  (void)k;
+  // Pick the widest tile whose tile count still fills the machine reasonably: cost model =
+  // waves * per-tile time, per-tile time ~ BN (+ a fixed part for the A operand traffic).
+  const int sms = sm_count();
+  const int tiles_m = (m + BM - 1) / BM;
+  int best = 256;
+  double best_cost = 1e300;
+  const int cands[3] = {256, 128, 64};
+  for (int bn : cands) {
+    if (bn > n && bn != 64) continue;
+    const long long tiles = 1ll * tiles_m * ((n + bn - 1) / bn);
+    const long long waves = (tiles + sms - 1) / sms;
+    const double cost = static_cast<double>(waves) * (bn + 32.0);
+    if (cost < best_cost) { best_cost = cost; best = bn; }
+  }
+  return best;
+}
+
+static pd_status check_gemm_args(const GemmArgs& g) {
+  if (!g.a || !g.b || !g.c || g.m < 0 || g.n <= 0 || g.k <= 0) return PD_ERR_INVALID_ARG;
+  if (g.epilogue == EPI_RESIDUAL && !g.r) return PD_ERR_INVALID_ARG;
+  if (g.k % BK != 0 || g.n % 16 != 0) return PD_ERR_UNSUPPORTED_SHAPE;
+  if (g.lda % 8 || g.ldb % 8 || g.ldc % 8 || (g.epilogue == EPI_RESIDUAL && g.ldr % 8)) return PD_ERR_UNSUPPORTED_SHAPE;
+  return PD_OK;
+}
+
+pd_status gemm_tc(const GemmArgs& g, cudaStream_t stream) {
+  PD_TRY(check_gemm_args(g));
+  if (g.m == 0) return PD_OK;
+  switch (gemm_tc_block_n(g.m, g.n, g.k)) {
+    case 256: return launch_tc_epi<256>(g, stream);
+    case 128: return launch_tc_epi<128>(g, stream);
+    default: return launch_tc_epi<64>(g, stream);
+  }
+}
+
+// ------------------------------------------------------------- CUDA-core GEMM
+namespace {
+template <int EPI>
+__global__ void __launch_bounds__(256) gemm_simt_kernel(const bf16* __restrict__ a, const bf16* __restrict__ b,
+                                                         bf16* c, const bf16* r, int m, int n, int k, int lda,
+                                                         int ldb, int ldc, int ldr) {
+  // 64 x 64 tile, 16-wide K slices, 4 x 4 outputs per thread.
+  __shared__ float sa[16][64 + 1];
+  __shared__ float sb[16][64 + 1];
+  const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+  const int row0 = blockIdx.y * 64, col0 = blockIdx.x * 64;
+  float acc[4][4] = {};
+  for (int k0 = 0; k0 < k; k0 += 16) {
+    for (int i = threadIdx.x; i < 64 * 16; i += 256) {
+      const int rr = i >> 4, kk = i & 15;
+      const int gr = row0 + rr, gc = col0 + rr;
+      sa[kk][rr] = (gr < m) ? __bfloat162float(a[static_cast<size_t>(gr) * lda + k0 + kk]) : 0.f;
+      sb[kk][rr] = (gc < n) ? __bfloat162float(b[static_cast<size_t>(gc) * ldb + k0 + kk]) : 0.f;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int kk = 0; kk < 16; ++kk) {
+      float av[4], bv[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) { av[i] = sa[kk][ty * 4 + i]; bv[i] = sb[kk][tx * 4 + i]; }
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
+    }
+    __syncthreads();
+  }
+  for (int i = 0; i < 4; ++i) {
+    const int gr = row0 + ty * 4 + i;
+    if (gr >= m) continue;
+    for (int j = 0; j < 4; ++j) {
+      const int gc = col0 + tx * 4 + j;
+      if (gc >= n) continue;
+      float v = acc[i][j];
+      if (EPI == EPI_RESIDUAL) v += __bfloat162float(r[static_cast<size_t>(gr) * ldr + gc]);
+      c[static_cast<size_t>(gr) * ldc + gc] = __float2bfloat16(v);
+    }
+  }
+}
+}  // namespace
+
+pd_status gemm_simt(const GemmArgs& g, cudaStream_t stream) {
+  PD_TRY(check_gemm_args(g));
+  if (g.m == 0) return PD_OK;
+  dim3 grid((g.n + 63) / 64, (g.m + 63) / 64);
+  if (g.epilogue == EPI_RESIDUAL)
+    gemm_simt_kernel<EPI_RESIDUAL><<<grid, 256, 0, stream>>>(g.a, g.b, g.c, g.r, g.m, g.n, g.k, g.lda, g.ldb,
+                                                            g.ldc, g.ldr);
+  else
+    gemm_simt_kernel<EPI_STORE><<<grid, 256, 0, stream>>>(g.a, g.b, g.c, g.r, g.m, g.n, g.k, g.lda, g.ldb, g.ldc,
+                                                         g.ldr);
+  count_launch();
+  PD_CUDA_TRY(cudaGetLastError());
+  return PD_OK;
+}
+
+pd_status gemm(const GemmArgs& g, cudaStream_t stream) {
+  static int use_simt = -1;
+  if (use_simt < 0) {
+    const char* e = std::getenv("PD_GEMM");
+    use_simt = (e && std::strcmp(e, "simt") == 0) ? 1 : 0;
+  }
+  return use_simt ? gemm_simt(g, stream) : gemm_tc(g, stream);
+}
+
+}  // namespace pd
+
+extern "C" pd_status pd_gemm_bf16(const void* a, const void* b, void* c, int32_t m, int32_t n, int32_t k,
+                                  int32_t* err_word, void* stream) {
+  pd::GemmArgs g{};
+  g.a = static_cast<const pd::bf16*>(a);
+  g.b = static_cast<const pd::bf16*>(b);
+  g.c = static_cast<pd::bf16*>(c);
+  g.r = nullptr;
+  g.m = m; g.n = n; g.k = k;
+  g.lda = k; g.ldb = k; g.ldc = n; g.ldr = 0;
+  g.epilogue = pd::EPI_STORE;
+  g.err_word = err_word;
+  return pd::gemm(g, static_cast<cudaStream_t>(stream));
+}

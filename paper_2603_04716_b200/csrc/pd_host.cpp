@@ -1,0 +1,130 @@
+// Host-side scalar part of the library: the allocation model (Eq. 1-13) and the
+// FIFO queue replay used to check the M/M/1 prediction of Eq. 12.
+// Compiled with floating-point contraction off so that the integer results do not
+// depend on whether the compiler fuses a multiply with an add.
+#include <cmath>
+#include <cstring>
+#include <limits>
+#include <vector>
+#include <algorithm>
+
+#include "pd.h"
+
+namespace {
+
+int32_t nearest_count(double n) {
+  double r = std::floor(n + 0.5);
+  if (!(r >= 1.0)) return 1;
+  if (r > 2147483647.0) return 2147483647;
+  return static_cast<int32_t>(r);
+}
+
+int32_t ceil_count(double n) {
+  double r = std::ceil(n);
+  if (!(r >= 1.0)) return 1;
+  if (r > 2147483647.0) return 2147483647;
+  return static_cast<int32_t>(r);
+}
+
+}  // namespace
+
+extern "C" const char* pd_status_str(pd_status s) {
+  switch (s) {
+    case PD_OK: return "ok";
+    case PD_ERR_INVALID_ARG: return "invalid argument";
+    case PD_ERR_UNSUPPORTED_SHAPE: return "unsupported shape";
+    case PD_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+    case PD_ERR_CUDA: return "CUDA error";
+    case PD_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
+    case PD_ERR_INFEASIBLE_TTFT: return "TTFT SLO infeasible";
+    case PD_ERR_INFEASIBLE_TPOT: return "TPOT SLO infeasible";
+    case PD_ERR_ARCH: return "device is not sm_100";
+  }
+  return "unknown status";
+}
+
+extern "C" int pd_version(void) { return 1; }
+
+extern "C" pd_status pd_allocate(const pd_alloc_in* in, pd_alloc_out* out) {
+  if (!in || !out || in->struct_size != sizeof(pd_alloc_in)) return PD_ERR_INVALID_ARG;
+  const double nan = std::numeric_limits<double>::quiet_NaN();
+  std::memset(out, 0, sizeof(*out));
+  out->struct_size = sizeof(pd_alloc_out);
+  out->tp_prefill_eff = out->tp_decode_eff = out->mu = out->lambda = out->rho = nan;
+  out->n_prefill_frac = out->n_decode_frac = out->ratio_pd = out->achieved_total_tok_s = nan;
+
+  const double L_in = in->l_in, L_out = in->l_out;
+  if (!(in->tp_total_tok_s > 0.0) || !(L_in > 0.0) || !(L_out > 0.0) || !(in->prefill_max_tok_s > 0.0) ||
+      !(in->tpot_slo_s > 0.0) || !(in->t_overhead_s >= 0.0) || in->n_points < 0 ||
+      (in->n_points > 0 && (!in->batch || !in->tpot_s)))
+    return PD_ERR_INVALID_ARG;
+  for (int i = 0; i < in->n_points; ++i)
+    if (in->batch[i] <= 0 || !(in->tpot_s[i] > 0.0)) return PD_ERR_INVALID_ARG;
+
+  pd_status status = PD_OK;
+
+  // Prefill side: service rate (Eq. 9), TTFT budget (Eq. 8, 12), effective throughput (Eq. 13).
+  out->mu = in->prefill_max_tok_s / L_in;
+  const double budget = in->ttft_slo_s - in->t_overhead_s;
+  bool prefill_ok = false;
+  if (budget > 0.0) {
+    out->tp_prefill_eff = in->prefill_max_tok_s - L_in / budget;
+    prefill_ok = out->tp_prefill_eff > 0.0;
+  }
+  if (prefill_ok) {
+    out->lambda = out->tp_prefill_eff / L_in;  // Eq. 11 solved for lambda with Eq. 10
+    out->rho = out->lambda / out->mu;           // Eq. 10
+  } else {
+    status = PD_ERR_INFEASIBLE_TTFT;
+  }
+
+  // Decode side: walk the curve in order of batch size; stop at the first point over the SLO.
+  std::vector<int> order(in->n_points);
+  for (int i = 0; i < in->n_points; ++i) order[i] = i;
+  std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return in->batch[a] < in->batch[b]; });
+  int best = -1;
+  for (int idx : order) {
+    if (in->tpot_s[idx] <= in->tpot_slo_s) best = idx; else break;
+  }
+  if (best < 0) {
+    if (status == PD_OK) status = PD_ERR_INFEASIBLE_TPOT;
+  } else {
+    out->feasible_batch = in->batch[best];
+    out->sweep_capped = (best == order.back()) ? 1 : 0;
+    out->tp_decode_eff = static_cast<double>(in->batch[best]) / in->tpot_s[best];
+  }
+  if (status != PD_OK) return status;
+
+  const double TP_total = in->tp_total_tok_s, TP_p = out->tp_prefill_eff, TP_d = out->tp_decode_eff;
+  out->n_prefill_frac = (TP_total * L_in) / ((L_in + L_out) * TP_p);   // Eq. 5
+  out->n_decode_frac = (TP_total * L_out) / ((L_in + L_out) * TP_d);   // Eq. 6
+  out->ratio_pd = (L_in * TP_d) / (L_out * TP_p);                      // Eq. 7
+  out->n_prefill = nearest_count(out->n_prefill_frac);
+  out->n_decode = nearest_count(out->n_decode_frac);
+  out->n_prefill_ceil = ceil_count(out->n_prefill_frac);
+  out->n_decode_ceil = ceil_count(out->n_decode_frac);
+  // Pipelined phases: the slower one sets the pace (Eq. 2-4), total tokens per request L_in + L_out (Eq. 1).
+  const double side_p = out->n_prefill * TP_p * (L_in + L_out) / L_in;
+  const double side_d = out->n_decode * TP_d * (L_in + L_out) / L_out;
+  out->achieved_total_tok_s = side_p < side_d ? side_p : side_d;
+  return PD_OK;
+}
+
+extern "C" pd_status pd_queue_replay(const double* gaps, const double* service, int64_t n, double* mean_sojourn_s,
+                                     double* mean_wait_s) {
+  if (!gaps || !service || n <= 0 || !mean_sojourn_s || !mean_wait_s) return PD_ERR_INVALID_ARG;
+  // Lindley recursion: W(i) = max(0, W(i-1) + S(i-1) - gap(i)).
+  double wait = 0.0, sum_wait = 0.0, sum_soj = 0.0;
+  for (int64_t i = 0; i < n; ++i) {
+    if (!(service[i] >= 0.0) || !(gaps[i] >= 0.0)) return PD_ERR_INVALID_ARG;
+    if (i > 0) {
+      double w = wait + service[i - 1] - gaps[i];
+      wait = w > 0.0 ? w : 0.0;
+    }
+    sum_wait += wait;
+    sum_soj += wait + service[i];
+  }
+  *mean_sojourn_s = sum_soj / static_cast<double>(n);
+  *mean_wait_s = sum_wait / static_cast<double>(n);
+  return PD_OK;
+}

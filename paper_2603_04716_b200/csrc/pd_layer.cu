@@ -1,0 +1,377 @@
+// The layer object and the two layer passes (prefill, decode): argument validation on
+// the host, workspace carving, and the kernel sequence.  Nothing here allocates or
+// synchronises except pd_layer_create / pd_layer_destroy / pd_layer_check and the
+// host-I/O variants of the stack calls.
+#include <cmath>
+#include <new>
+#include <vector>
+
+#include "pd_common.cuh"
+
+using pd::bf16;
+
+namespace {
+
+struct Workspace {
+  // byte offsets into the caller's workspace
+  size_t norm, qkv, attn_o, resid, gate_up, act, partial, stage_a, stage_b, meta, total;
+};
+
+Workspace carve(const pd_layer_cfg& c, size_t tokens, size_t max_batch, int max_kv_len) {
+  const size_t d = c.d_model, nqkv = static_cast<size_t>(c.n_q_heads + 2 * c.n_kv_heads) * c.head_dim;
+  const size_t hq = static_cast<size_t>(c.n_q_heads) * c.head_dim, f = c.d_ff;
+  Workspace w{};
+  size_t off = 0;
+  auto take = [&](size_t bytes) {
+    const size_t o = off;
+    off += pd::align_up(bytes, 256);
+    return o;
+  };
+  w.norm = take(tokens * d * 2);
+  w.qkv = take(tokens * nqkv * 2);
+  w.attn_o = take(tokens * hq * 2);
+  w.resid = take(tokens * d * 2);
+  w.gate_up = take(tokens * 2 * f * 2);
+  w.act = take(tokens * f * 2);
+  const int splits = max_batch ? pd::decode_attention_splits(1, c.n_kv_heads, max_kv_len) : 1;  // worst case: B = 1
+  w.partial = take(max_batch * c.n_kv_heads * static_cast<size_t>(splits) * (c.n_q_heads / c.n_kv_heads) *
+                   (c.head_dim + 2) * 4);
+  w.stage_a = take(tokens * d * 2);  // activations between layers of a stack / staged host input
+  w.stage_b = take(tokens * d * 2);
+  w.meta = take(4096 * 4);           // staged cu_seqlens / kv_len of the host-I/O stack calls
+  w.total = off;
+  return w;
+}
+
+pd_status check_cfg(const pd_layer_cfg* c) {
+  if (!c || c->struct_size != sizeof(pd_layer_cfg)) return PD_ERR_INVALID_ARG;
+  if (c->d_model <= 0 || c->n_q_heads <= 0 || c->n_kv_heads <= 0 || c->d_ff <= 0 || c->max_pos <= 0 ||
+      !(c->rms_eps > 0.f) || !(c->rope_theta > 0.f))
+    return PD_ERR_INVALID_ARG;
+  if (c->head_dim != 64 && c->head_dim != 128) return PD_ERR_UNSUPPORTED_SHAPE;
+  if (c->n_q_heads % c->n_kv_heads != 0 || c->n_q_heads / c->n_kv_heads > 16) return PD_ERR_UNSUPPORTED_SHAPE;
+  if (c->d_model % 64 != 0 || c->d_ff % 64 != 0 || c->d_model > 16384) return PD_ERR_UNSUPPORTED_SHAPE;
+  return PD_OK;
+}
+
+pd_status check_cache(const pd_layer* L, const pd_kv_cache* c) {
+  (void)L;
+  if (!c || c->struct_size != sizeof(pd_kv_cache) || !c->k || !c->v || c->batch_cap <= 0 || c->len_cap <= 0)
+    return PD_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(c->k) & 15u) || (reinterpret_cast<uintptr_t>(c->v) & 15u)) return PD_ERR_INVALID_ARG;
+  return PD_OK;
+}
+
+// MLP half shared by both modes: h (residual stream after attention) -> out.
+pd_status mlp_half(pd_layer* L, const bf16* h, bf16* out, int tokens, uint8_t* ws, const Workspace& w,
+                   cudaStream_t st) {
+  const pd_layer_cfg& c = L->cfg;
+  bf16* norm = reinterpret_cast<bf16*>(ws + w.norm);
+  bf16* gu = reinterpret_cast<bf16*>(ws + w.gate_up);
+  bf16* act = reinterpret_cast<bf16*>(ws + w.act);
+  { pd::TraceScope ts(PD_K_RMSNORM, st); PD_TRY(pd::launch_rmsnorm(h, L->g_mlp, norm, tokens, c.d_model, c.rms_eps, st)); }
+  pd::GemmArgs g{};
+  g.a = norm; g.b = L->w_gu; g.c = gu; g.m = tokens; g.n = 2 * c.d_ff; g.k = c.d_model;
+  g.lda = c.d_model; g.ldb = c.d_model; g.ldc = 2 * c.d_ff; g.epilogue = pd::EPI_STORE; g.err_word = L->err_word;
+  { pd::TraceScope ts(PD_K_GEMM_GATE_UP, st); PD_TRY(pd::gemm(g, st)); }
+  { pd::TraceScope ts(PD_K_SWIGLU, st); PD_TRY(pd::launch_swiglu(gu, act, tokens, c.d_ff, st)); }
+  pd::GemmArgs g2{};
+  g2.a = act; g2.b = L->w_down; g2.c = out; g2.r = h; g2.m = tokens; g2.n = c.d_model; g2.k = c.d_ff;
+  g2.lda = c.d_ff; g2.ldb = c.d_ff; g2.ldc = c.d_model; g2.ldr = c.d_model; g2.epilogue = pd::EPI_RESIDUAL;
+  g2.err_word = L->err_word;
+  { pd::TraceScope ts(PD_K_GEMM_DOWN, st); PD_TRY(pd::gemm(g2, st)); }
+  return PD_OK;
+}
+
+// Attention-input half shared by both modes: x -> qkv (q rotated in place, k/v written to the cache).
+pd_status qkv_half(pd_layer* L, const bf16* x, int tokens, const pd::RopeArgs& rope_in, uint8_t* ws,
+                   const Workspace& w, cudaStream_t st) {
+  const pd_layer_cfg& c = L->cfg;
+  bf16* norm = reinterpret_cast<bf16*>(ws + w.norm);
+  bf16* qkv = reinterpret_cast<bf16*>(ws + w.qkv);
+  { pd::TraceScope ts(PD_K_RMSNORM, st); PD_TRY(pd::launch_rmsnorm(x, L->g_attn, norm, tokens, c.d_model, c.rms_eps, st)); }
+  pd::GemmArgs g{};
+  g.a = norm; g.b = L->w_qkv; g.c = qkv; g.m = tokens; g.n = L->n_qkv; g.k = c.d_model;
+  g.lda = c.d_model; g.ldb = c.d_model; g.ldc = L->n_qkv; g.epilogue = pd::EPI_STORE; g.err_word = L->err_word;
+  { pd::TraceScope ts(PD_K_GEMM_QKV, st); PD_TRY(pd::gemm(g, st)); }
+  pd::RopeArgs r = rope_in;
+  r.qkv = qkv;
+  { pd::TraceScope ts(PD_K_ROPE_KV, st); PD_TRY(pd::launch_rope_scatter(r, st)); }
+  return PD_OK;
+}
+
+pd_status oproj(pd_layer* L, const bf16* x, int tokens, uint8_t* ws, const Workspace& w, cudaStream_t st) {
+  const pd_layer_cfg& c = L->cfg;
+  const int hq = c.n_q_heads * c.head_dim;
+  pd::GemmArgs g{};
+  g.a = reinterpret_cast<bf16*>(ws + w.attn_o); g.b = L->w_o; g.c = reinterpret_cast<bf16*>(ws + w.resid); g.r = x;
+  g.m = tokens; g.n = c.d_model; g.k = hq; g.lda = hq; g.ldb = hq; g.ldc = c.d_model; g.ldr = c.d_model;
+  g.epilogue = pd::EPI_RESIDUAL; g.err_word = L->err_word;
+  pd::TraceScope ts(PD_K_GEMM_O, st);
+  return pd::gemm(g, st);
+}
+
+pd_status validate_prefill(const pd_layer* L, const int32_t* cu_host, int n_req, const pd_kv_cache* cache,
+                           bool default_slots, int* tokens, int* max_len) {
+  if (!L || !cu_host || n_req < 0 || n_req > 4095) return PD_ERR_INVALID_ARG;
+  PD_TRY(check_cache(L, cache));
+  if (cu_host[0] != 0) return PD_ERR_INVALID_ARG;
+  int mx = 0;
+  for (int r = 0; r < n_req; ++r) {
+    const int len = cu_host[r + 1] - cu_host[r];
+    if (len < 0) return PD_ERR_INVALID_ARG;
+    if (len > cache->len_cap || len > L->cfg.max_pos) return PD_ERR_INVALID_ARG;
+    if (len > mx) mx = len;
+  }
+  if (default_slots && n_req > cache->batch_cap) return PD_ERR_INVALID_ARG;
+  *tokens = cu_host[n_req];
+  *max_len = mx;
+  return PD_OK;
+}
+
+pd_status prefill_impl(pd_layer* L, const bf16* x, bf16* out, const int32_t* cu_dev, int n_req, int tokens,
+                       int max_len, const int32_t* slots_dev, const pd_kv_cache* cache, uint8_t* ws,
+                       const Workspace& w, cudaStream_t st) {
+  const pd_layer_cfg& c = L->cfg;
+  pd::RopeArgs r{};
+  r.k_cache = static_cast<bf16*>(cache->k); r.v_cache = static_cast<bf16*>(cache->v); r.rope_tab = L->rope_tab;
+  r.cu_seqlens = cu_dev; r.slots = slots_dev; r.kv_len = nullptr; r.n_req = n_req; r.n_tokens = tokens;
+  r.n_q_heads = c.n_q_heads; r.n_kv_heads = c.n_kv_heads; r.head_dim = c.head_dim; r.len_cap = cache->len_cap;
+  r.max_pos = c.max_pos; r.batch_cap = cache->batch_cap; r.err_word = L->err_word;
+  PD_TRY(qkv_half(L, x, tokens, r, ws, w, st));
+  pd::PrefillAttnArgs a{};
+  a.q = reinterpret_cast<bf16*>(ws + w.qkv); a.ldq = L->n_qkv;
+  a.k_cache = static_cast<bf16*>(cache->k); a.v_cache = static_cast<bf16*>(cache->v);
+  a.o = reinterpret_cast<bf16*>(ws + w.attn_o); a.cu_seqlens = cu_dev; a.slots = slots_dev;
+  a.n_req = n_req; a.n_tokens = tokens; a.max_len = max_len;
+  a.n_q_heads = c.n_q_heads; a.n_kv_heads = c.n_kv_heads; a.head_dim = c.head_dim; a.len_cap = cache->len_cap;
+  a.batch_cap = cache->batch_cap;
+  { pd::TraceScope ts(PD_K_ATTN_PREFILL, st); PD_TRY(pd::launch_prefill_attention(a, st)); }
+  PD_TRY(oproj(L, x, tokens, ws, w, st));
+  PD_TRY(mlp_half(L, reinterpret_cast<bf16*>(ws + w.resid), out, tokens, ws, w, st));
+  return PD_OK;
+}
+
+pd_status decode_impl(pd_layer* L, const bf16* x, bf16* out, const int32_t* kv_len_dev, int B, int max_kv_len,
+                      const pd_kv_cache* cache, uint8_t* ws, const Workspace& w, cudaStream_t st) {
+  const pd_layer_cfg& c = L->cfg;
+  pd::RopeArgs r{};
+  r.k_cache = static_cast<bf16*>(cache->k); r.v_cache = static_cast<bf16*>(cache->v); r.rope_tab = L->rope_tab;
+  r.cu_seqlens = nullptr; r.slots = nullptr; r.kv_len = kv_len_dev; r.n_req = B; r.n_tokens = B;
+  r.n_q_heads = c.n_q_heads; r.n_kv_heads = c.n_kv_heads; r.head_dim = c.head_dim; r.len_cap = cache->len_cap;
+  r.max_pos = c.max_pos; r.batch_cap = cache->batch_cap; r.err_word = L->err_word;
+  PD_TRY(qkv_half(L, x, B, r, ws, w, st));
+  pd::DecodeAttnArgs a{};
+  a.q = reinterpret_cast<bf16*>(ws + w.qkv); a.ldq = L->n_qkv;
+  a.k_cache = static_cast<bf16*>(cache->k); a.v_cache = static_cast<bf16*>(cache->v);
+  a.o = reinterpret_cast<bf16*>(ws + w.attn_o); a.kv_len = kv_len_dev;
+  a.partial = reinterpret_cast<float*>(ws + w.partial);
+  a.batch = B; a.max_kv_len = max_kv_len; a.n_splits = pd::decode_attention_splits(B, c.n_kv_heads, max_kv_len);
+  a.n_q_heads = c.n_q_heads; a.n_kv_heads = c.n_kv_heads; a.head_dim = c.head_dim; a.len_cap = cache->len_cap;
+  { pd::TraceScope ts(PD_K_ATTN_DECODE, st); PD_TRY(pd::launch_decode_attention(a, st)); }
+  PD_TRY(oproj(L, x, B, ws, w, st));
+  PD_TRY(mlp_half(L, reinterpret_cast<bf16*>(ws + w.resid), out, B, ws, w, st));
+  return PD_OK;
+}
+
+}  // namespace
+
+extern "C" pd_status pd_workspace_bytes(const pd_layer_cfg* cfg, int32_t max_tokens, int32_t max_batch,
+                                        int32_t max_kv_len, size_t* out_bytes) {
+  PD_TRY(check_cfg(cfg));
+  if (!out_bytes || max_tokens < 0 || max_batch < 0 || max_kv_len < 0) return PD_ERR_INVALID_ARG;
+  const size_t tokens = static_cast<size_t>(max_tokens > max_batch ? max_tokens : max_batch);
+  *out_bytes = carve(*cfg, tokens, static_cast<size_t>(max_batch), max_kv_len).total;
+  return PD_OK;
+}
+
+extern "C" pd_status pd_layer_create(const pd_layer_cfg* cfg, const pd_layer_weights* w, void* stream,
+                                     pd_layer** out) {
+  PD_TRY(check_cfg(cfg));
+  if (!w || w->struct_size != sizeof(pd_layer_weights) || !out) return PD_ERR_INVALID_ARG;
+  if (!w->w_qkv || !w->w_o || !w->w_gate || !w->w_up || !w->w_down || !w->g_attn || !w->g_mlp)
+    return PD_ERR_INVALID_ARG;
+  int dev = 0, major = 0;
+  PD_CUDA_TRY(cudaGetDevice(&dev));
+  PD_CUDA_TRY(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev));
+  if (major != 10) return PD_ERR_ARCH;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+
+  pd_layer* L = new (std::nothrow) pd_layer();
+  if (!L) return PD_ERR_INVALID_ARG;
+  L->cfg = *cfg;
+  L->n_qkv = (cfg->n_q_heads + 2 * cfg->n_kv_heads) * cfg->head_dim;
+  const size_t d = cfg->d_model, f = cfg->d_ff, hq = static_cast<size_t>(cfg->n_q_heads) * cfg->head_dim;
+  const size_t half = cfg->head_dim / 2;
+  auto fail = [&](cudaError_t e) {
+    pd_layer_destroy(L);
+    return pd::cuda_fail(e);
+  };
+  cudaError_t e;
+  if ((e = cudaMalloc(&L->w_qkv, L->n_qkv * d * 2)) != cudaSuccess) return fail(e);
+  if ((e = cudaMalloc(&L->w_o, d * hq * 2)) != cudaSuccess) return fail(e);
+  if ((e = cudaMalloc(&L->w_gu, 2 * f * d * 2)) != cudaSuccess) return fail(e);
+  if ((e = cudaMalloc(&L->w_down, d * f * 2)) != cudaSuccess) return fail(e);
+  if ((e = cudaMalloc(&L->g_attn, d * 2)) != cudaSuccess) return fail(e);
+  if ((e = cudaMalloc(&L->g_mlp, d * 2)) != cudaSuccess) return fail(e);
+  if ((e = cudaMalloc(&L->rope_tab, static_cast<size_t>(cfg->max_pos) * half * sizeof(float2))) != cudaSuccess)
+    return fail(e);
+  if ((e = cudaMalloc(&L->err_word, sizeof(int))) != cudaSuccess) return fail(e);
+  const cudaMemcpyKind d2d = cudaMemcpyDeviceToDevice;
+  if ((e = cudaMemcpyAsync(L->w_qkv, w->w_qkv, L->n_qkv * d * 2, d2d, st)) != cudaSuccess) return fail(e);
+  if ((e = cudaMemcpyAsync(L->w_o, w->w_o, d * hq * 2, d2d, st)) != cudaSuccess) return fail(e);
+  // gate rows first, then up rows, so one GEMM produces both halves of the SwiGLU input
+  if ((e = cudaMemcpyAsync(L->w_gu, w->w_gate, f * d * 2, d2d, st)) != cudaSuccess) return fail(e);
+  if ((e = cudaMemcpyAsync(L->w_gu + f * d, w->w_up, f * d * 2, d2d, st)) != cudaSuccess) return fail(e);
+  if ((e = cudaMemcpyAsync(L->w_down, w->w_down, d * f * 2, d2d, st)) != cudaSuccess) return fail(e);
+  if ((e = cudaMemcpyAsync(L->g_attn, w->g_attn, d * 2, d2d, st)) != cudaSuccess) return fail(e);
+  if ((e = cudaMemcpyAsync(L->g_mlp, w->g_mlp, d * 2, d2d, st)) != cudaSuccess) return fail(e);
+  if ((e = cudaMemsetAsync(L->err_word, 0, sizeof(int), st)) != cudaSuccess) return fail(e);
+
+  // RoPE table in double on the host: (cos, sin)(pos * theta^(-2i/hd))
+  std::vector<float2> tab(static_cast<size_t>(cfg->max_pos) * half);
+  std::vector<double> inv_freq(half);
+  for (size_t i = 0; i < half; ++i)
+    inv_freq[i] = std::pow(static_cast<double>(cfg->rope_theta), -2.0 * static_cast<double>(i) / cfg->head_dim);
+  for (int p = 0; p < cfg->max_pos; ++p)
+    for (size_t i = 0; i < half; ++i) {
+      const double ang = static_cast<double>(p) * inv_freq[i];
+      tab[static_cast<size_t>(p) * half + i] = make_float2(static_cast<float>(std::cos(ang)), static_cast<float>(std::sin(ang)));
+    }
+  // the table is a stack temporary: copy synchronously with respect to the host
+  if ((e = cudaMemcpy(L->rope_tab, tab.data(), tab.size() * sizeof(float2), cudaMemcpyHostToDevice)) != cudaSuccess)
+    return fail(e);
+  *out = L;
+  return PD_OK;
+}
+
+extern "C" pd_status pd_layer_destroy(pd_layer* L) {
+  if (!L) return PD_OK;
+  cudaFree(L->w_qkv); cudaFree(L->w_o); cudaFree(L->w_gu); cudaFree(L->w_down);
+  cudaFree(L->g_attn); cudaFree(L->g_mlp); cudaFree(L->rope_tab); cudaFree(L->err_word);
+  delete L;
+  return PD_OK;
+}
+
+extern "C" pd_status pd_layer_check(pd_layer* L, void* stream) {
+  if (!L) return PD_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int word = 0;
+  PD_CUDA_TRY(cudaMemcpyAsync(&word, L->err_word, sizeof(int), cudaMemcpyDeviceToHost, st));
+  PD_CUDA_TRY(cudaStreamSynchronize(st));
+  if (word != 0) {
+    PD_CUDA_TRY(cudaMemsetAsync(L->err_word, 0, sizeof(int), st));
+    return word == 2 ? PD_ERR_INVALID_ARG : PD_ERR_DEVICE_TIMEOUT;
+  }
+  return PD_OK;
+}
+
+extern "C" pd_status pd_prefill_layer(pd_layer* L, const void* x, void* out, const int32_t* cu_dev,
+                                      const int32_t* cu_host, int32_t n_req, const int32_t* slots_dev,
+                                      const pd_kv_cache* cache, void* workspace, size_t workspace_bytes,
+                                      void* stream) {
+  int tokens = 0, max_len = 0;
+  PD_TRY(validate_prefill(L, cu_host, n_req, cache, slots_dev == nullptr, &tokens, &max_len));
+  if (tokens == 0) return PD_OK;
+  if (!x || !out || !cu_dev || !workspace) return PD_ERR_INVALID_ARG;
+  const Workspace w = carve(L->cfg, tokens, 0, 0);
+  if (workspace_bytes < w.total) return PD_ERR_WORKSPACE_TOO_SMALL;
+  if (reinterpret_cast<uintptr_t>(workspace) & 255u) return PD_ERR_INVALID_ARG;
+  return prefill_impl(L, static_cast<const bf16*>(x), static_cast<bf16*>(out), cu_dev, n_req, tokens, max_len,
+                      slots_dev, cache, static_cast<uint8_t*>(workspace), w, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" pd_status pd_decode_layer(pd_layer* L, const void* x, void* out, const int32_t* kv_len_dev, int32_t B,
+                                     int32_t max_kv_len, const pd_kv_cache* cache, void* workspace,
+                                     size_t workspace_bytes, void* stream) {
+  if (!L || B < 0) return PD_ERR_INVALID_ARG;
+  if (B == 0) return PD_OK;
+  PD_TRY(check_cache(L, cache));
+  if (!x || !out || !kv_len_dev || !workspace) return PD_ERR_INVALID_ARG;
+  if (B > cache->batch_cap || max_kv_len <= 0 || max_kv_len > cache->len_cap || max_kv_len > L->cfg.max_pos)
+    return PD_ERR_INVALID_ARG;
+  const Workspace w = carve(L->cfg, B, B, max_kv_len);
+  if (workspace_bytes < w.total) return PD_ERR_WORKSPACE_TOO_SMALL;
+  if (reinterpret_cast<uintptr_t>(workspace) & 255u) return PD_ERR_INVALID_ARG;
+  return decode_impl(L, static_cast<const bf16*>(x), static_cast<bf16*>(out), kv_len_dev, B, max_kv_len, cache,
+                     static_cast<uint8_t*>(workspace), w, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" pd_status pd_prefill_stack(pd_layer* const* layers, const pd_kv_cache* caches, int32_t n_layers,
+                                      int32_t n_caches, const void* x, void* out, int32_t io_on_host,
+                                      const int32_t* cu_dev, const int32_t* cu_host, int32_t n_req, void* workspace,
+                                      size_t workspace_bytes, void* stream) {
+  if (!layers || !caches || n_layers <= 0 || n_caches <= 0 || !layers[0]) return PD_ERR_INVALID_ARG;
+  int tokens = 0, max_len = 0;
+  for (int i = 0; i < n_layers; ++i) {
+    if (!layers[i]) return PD_ERR_INVALID_ARG;
+    PD_TRY(validate_prefill(layers[i], cu_host, n_req, &caches[i % n_caches], true, &tokens, &max_len));
+  }
+  if (tokens == 0) return PD_OK;
+  if (!x || !out || !workspace || (!io_on_host && !cu_dev)) return PD_ERR_INVALID_ARG;
+  const Workspace w = carve(layers[0]->cfg, tokens, 0, 0);
+  if (workspace_bytes < w.total) return PD_ERR_WORKSPACE_TOO_SMALL;
+  if (reinterpret_cast<uintptr_t>(workspace) & 255u) return PD_ERR_INVALID_ARG;
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const size_t act_bytes = static_cast<size_t>(tokens) * layers[0]->cfg.d_model * 2;
+  bf16* buf[2] = {reinterpret_cast<bf16*>(ws + w.stage_a), reinterpret_cast<bf16*>(ws + w.stage_b)};
+  const bf16* cur = static_cast<const bf16*>(x);
+  if (io_on_host) {
+    PD_CUDA_TRY(cudaMemcpyAsync(buf[0], x, act_bytes, cudaMemcpyHostToDevice, st));
+    PD_CUDA_TRY(cudaMemcpyAsync(ws + w.meta, cu_host, (n_req + 1) * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+    cu_dev = reinterpret_cast<const int32_t*>(ws + w.meta);
+    cur = buf[0];
+  }
+  for (int i = 0; i < n_layers; ++i) {
+    bf16* dst = (i == n_layers - 1 && !io_on_host) ? static_cast<bf16*>(out) : buf[(i + 1) & 1];
+    PD_TRY(prefill_impl(layers[i], cur, dst, cu_dev, n_req, tokens, max_len, nullptr, &caches[i % n_caches], ws, w, st));
+    cur = dst;
+  }
+  if (io_on_host) {
+    PD_CUDA_TRY(cudaMemcpyAsync(out, cur, act_bytes, cudaMemcpyDeviceToHost, st));
+    PD_CUDA_TRY(cudaStreamSynchronize(st));
+  }
+  return PD_OK;
+}
+
+extern "C" pd_status pd_decode_stack(pd_layer* const* layers, const pd_kv_cache* caches, int32_t n_layers,
+                                     int32_t n_caches, const void* x, void* out, int32_t io_on_host,
+                                     const int32_t* kv_len, int32_t B, int32_t max_kv_len, void* workspace,
+                                     size_t workspace_bytes, void* stream) {
+  if (!layers || !caches || n_layers <= 0 || n_caches <= 0 || B < 0 || B > 4096) return PD_ERR_INVALID_ARG;
+  if (B == 0) return PD_OK;
+  for (int i = 0; i < n_layers; ++i) {
+    if (!layers[i]) return PD_ERR_INVALID_ARG;
+    const pd_kv_cache* c = &caches[i % n_caches];
+    PD_TRY(check_cache(layers[i], c));
+    if (B > c->batch_cap || max_kv_len <= 0 || max_kv_len > c->len_cap || max_kv_len > layers[i]->cfg.max_pos)
+      return PD_ERR_INVALID_ARG;
+  }
+  if (!x || !out || !kv_len || !workspace) return PD_ERR_INVALID_ARG;
+  const Workspace w = carve(layers[0]->cfg, B, B, max_kv_len);
+  if (workspace_bytes < w.total) return PD_ERR_WORKSPACE_TOO_SMALL;
+  if (reinterpret_cast<uintptr_t>(workspace) & 255u) return PD_ERR_INVALID_ARG;
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const size_t act_bytes = static_cast<size_t>(B) * layers[0]->cfg.d_model * 2;
+  bf16* buf[2] = {reinterpret_cast<bf16*>(ws + w.stage_a), reinterpret_cast<bf16*>(ws + w.stage_b)};
+  const bf16* cur = static_cast<const bf16*>(x);
+  const int32_t* kv_dev = kv_len;
+  if (io_on_host) {
+    PD_CUDA_TRY(cudaMemcpyAsync(buf[0], x, act_bytes, cudaMemcpyHostToDevice, st));
+    PD_CUDA_TRY(cudaMemcpyAsync(ws + w.meta, kv_len, B * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+    kv_dev = reinterpret_cast<const int32_t*>(ws + w.meta);
+    cur = buf[0];
+  }
+  for (int i = 0; i < n_layers; ++i) {
+    bf16* dst = (i == n_layers - 1 && !io_on_host) ? static_cast<bf16*>(out) : buf[(i + 1) & 1];
+    PD_TRY(decode_impl(layers[i], cur, dst, kv_dev, B, max_kv_len, &caches[i % n_caches], ws, w, st));
+    cur = dst;
+  }
+  if (io_on_host) {
+    PD_CUDA_TRY(cudaMemcpyAsync(out, cur, act_bytes, cudaMemcpyDeviceToHost, st));
+    PD_CUDA_TRY(cudaStreamSynchronize(st));
+  }
+  return PD_OK;
+}

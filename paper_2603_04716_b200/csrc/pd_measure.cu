@@ -1,0 +1,302 @@
+// Measurement harness: the empirical benchmarking the allocation method feeds on.
+// Builds a stack of distinct synthetic layers on the current device, times the prefill
+// pass (maximum prefill throughput) and decode steps over a batch sweep (TPOT versus
+// batch) with CUDA events, and reports algorithmic work against the given peaks.
+#include <algorithm>
+#include <cstring>
+#include <vector>
+
+#include "pd_common.cuh"
+
+using pd::bf16;
+
+namespace {
+
+struct DevBuf {
+  void* p = nullptr;
+  ~DevBuf() { if (p) cudaFree(p); }
+  cudaError_t alloc(size_t bytes) { return cudaMalloc(&p, bytes ? bytes : 16); }
+};
+
+struct Stack {
+  std::vector<pd_layer*> layers;
+  ~Stack() { for (pd_layer* l : layers) pd_layer_destroy(l); }
+};
+
+struct Events {
+  cudaEvent_t a = nullptr, b = nullptr;
+  ~Events() { if (a) cudaEventDestroy(a); if (b) cudaEventDestroy(b); }
+};
+
+double median(std::vector<double> v) {
+  std::sort(v.begin(), v.end());
+  const size_t n = v.size();
+  return n % 2 ? v[n / 2] : 0.5 * (v[n / 2 - 1] + v[n / 2]);
+}
+
+size_t layer_param_count(const pd_layer_cfg& c) {
+  const size_t d = c.d_model, nqkv = static_cast<size_t>(c.n_q_heads + 2 * c.n_kv_heads) * c.head_dim;
+  return d * nqkv + static_cast<size_t>(c.n_q_heads) * c.head_dim * d + 3 * d * static_cast<size_t>(c.d_ff);
+}
+
+pd_status build_stack(const pd_layer_cfg& cfg, int n_layers, uint64_t seed, cudaStream_t st, Stack* out) {
+  const size_t d = cfg.d_model, f = cfg.d_ff, hq = static_cast<size_t>(cfg.n_q_heads) * cfg.head_dim;
+  const size_t nqkv = static_cast<size_t>(cfg.n_q_heads + 2 * cfg.n_kv_heads) * cfg.head_dim;
+  DevBuf wqkv, wo, wg, wu, wd, ga, gm;
+  PD_CUDA_TRY(wqkv.alloc(nqkv * d * 2));
+  PD_CUDA_TRY(wo.alloc(d * hq * 2));
+  PD_CUDA_TRY(wg.alloc(f * d * 2));
+  PD_CUDA_TRY(wu.alloc(f * d * 2));
+  PD_CUDA_TRY(wd.alloc(d * f * 2));
+  PD_CUDA_TRY(ga.alloc(d * 2));
+  PD_CUDA_TRY(gm.alloc(d * 2));
+  for (int l = 0; l < n_layers; ++l) {
+    const uint64_t s0 = static_cast<uint64_t>(l) * 16;
+    PD_TRY(pd::launch_fill_normal(static_cast<bf16*>(wqkv.p), nqkv * d, seed, s0 + 0, 0.f, 0.02f, st));
+    PD_TRY(pd::launch_fill_normal(static_cast<bf16*>(wo.p), d * hq, seed, s0 + 1, 0.f, 0.02f, st));
+    PD_TRY(pd::launch_fill_normal(static_cast<bf16*>(wg.p), f * d, seed, s0 + 2, 0.f, 0.02f, st));
+    PD_TRY(pd::launch_fill_normal(static_cast<bf16*>(wu.p), f * d, seed, s0 + 3, 0.f, 0.02f, st));
+    PD_TRY(pd::launch_fill_normal(static_cast<bf16*>(wd.p), d * f, seed, s0 + 4, 0.f, 0.02f, st));
+    PD_TRY(pd::launch_fill_normal(static_cast<bf16*>(ga.p), d, seed, s0 + 5, 1.f, 0.02f, st));
+    PD_TRY(pd::launch_fill_normal(static_cast<bf16*>(gm.p), d, seed, s0 + 6, 1.f, 0.02f, st));
+    pd_layer_weights w{};
+    w.struct_size = sizeof(w);
+    w.w_qkv = wqkv.p; w.w_o = wo.p; w.w_gate = wg.p; w.w_up = wu.p; w.w_down = wd.p; w.g_attn = ga.p; w.g_mlp = gm.p;
+    pd_layer* L = nullptr;
+    PD_TRY(pd_layer_create(&cfg, &w, st, &L));
+    out->layers.push_back(L);
+    PD_CUDA_TRY(cudaStreamSynchronize(st));  // the temporaries are refilled for the next layer
+  }
+  return PD_OK;
+}
+
+// Number of KV buffers to cycle through: one per layer if memory allows, otherwise as many as
+// fit in 70 % of the free memory (still far larger than L2 in total).
+int cache_ring(size_t bytes_per_cache, int n_layers) {
+  size_t free_b = 0, total_b = 0;
+  if (cudaMemGetInfo(&free_b, &total_b) != cudaSuccess) return 1;
+  const size_t budget = static_cast<size_t>(0.7 * static_cast<double>(free_b));
+  size_t fit = bytes_per_cache ? budget / bytes_per_cache : static_cast<size_t>(n_layers);
+  if (fit < 1) fit = 1;
+  return static_cast<int>(std::min<size_t>(fit, static_cast<size_t>(n_layers)));
+}
+
+}  // namespace
+
+extern "C" pd_status pd_measure(const pd_layer_cfg* cfg_in, const pd_measure_cfg* m, double peak_bf16_flops,
+                                double peak_hbm_bytes_s, pd_measurement* out) {
+  if (!cfg_in || !m || !out || m->struct_size != sizeof(pd_measure_cfg) || cfg_in->struct_size != sizeof(pd_layer_cfg))
+    return PD_ERR_INVALID_ARG;
+  if (m->n_layers_run <= 0 || m->n_layers_model <= 0 || m->warmup < 0 || m->reps <= 0) return PD_ERR_INVALID_ARG;
+  if (m->n_req < 0 || m->n_batch_sizes < 0 || m->n_batch_sizes > 32) return PD_ERR_INVALID_ARG;
+  if ((m->n_req > 0 && !m->l_in) || (m->n_batch_sizes > 0 && (!m->batch_sizes || m->n_steps <= 0 || m->kv_len_start < 0)))
+    return PD_ERR_INVALID_ARG;
+  std::memset(out, 0, sizeof(*out));
+  out->struct_size = sizeof(pd_measurement);
+  pd_layer_cfg cfg = *cfg_in;
+  const double scale_layers = static_cast<double>(m->n_layers_model) / m->n_layers_run;
+  const int nl = m->n_layers_run;
+  const size_t d = cfg.d_model;
+  const size_t kv_row = static_cast<size_t>(cfg.n_kv_heads) * cfg.head_dim * 2;  // bytes of K (or V) per token
+
+  cudaStream_t st = nullptr;
+  PD_CUDA_TRY(cudaStreamCreateWithFlags(&st, cudaStreamNonBlocking));
+  struct StreamGuard { cudaStream_t s; ~StreamGuard() { cudaStreamDestroy(s); } } sg{st};
+  Events ev;
+  PD_CUDA_TRY(cudaEventCreate(&ev.a));
+  PD_CUDA_TRY(cudaEventCreate(&ev.b));
+
+  Stack stack;
+  PD_TRY(build_stack(cfg, nl, m->seed, st, &stack));
+  const long long launches_before = pd::g_launch_count;
+  long long timed_launches = 0;
+
+  // ------------------------------------------------------------------ prefill
+  if (m->n_req > 0) {
+    std::vector<int32_t> cu(m->n_req + 1, 0);
+    int max_len = 0;
+    double attn_flops = 0.0;
+    for (int r = 0; r < m->n_req; ++r) {
+      if (m->l_in[r] < 0 || m->l_in[r] > cfg.max_pos) return PD_ERR_INVALID_ARG;
+      cu[r + 1] = cu[r] + m->l_in[r];
+      max_len = std::max(max_len, m->l_in[r]);
+      const double l = m->l_in[r];
+      attn_flops += 4.0 * cfg.n_q_heads * cfg.head_dim * (l * (l + 1.0) / 2.0);
+    }
+    const int tokens = cu[m->n_req];
+    if (tokens > 0) {
+      const double gemm_flops = 2.0 * tokens * static_cast<double>(layer_param_count(cfg));
+      out->prefill_flops = (gemm_flops + attn_flops) * m->n_layers_model;
+
+      const size_t cache_bytes = static_cast<size_t>(m->n_req) * max_len * kv_row;
+      const int ring = cache_ring(2 * cache_bytes, nl);
+      std::vector<DevBuf> kbuf(ring), vbuf(ring);
+      std::vector<pd_kv_cache> caches(ring);
+      for (int i = 0; i < ring; ++i) {
+        PD_CUDA_TRY(kbuf[i].alloc(cache_bytes));
+        PD_CUDA_TRY(vbuf[i].alloc(cache_bytes));
+        caches[i].struct_size = sizeof(pd_kv_cache);
+        caches[i].k = kbuf[i].p; caches[i].v = vbuf[i].p;
+        caches[i].batch_cap = m->n_req; caches[i].len_cap = max_len;
+      }
+      size_t ws_bytes = 0;
+      PD_TRY(pd_workspace_bytes(&cfg, tokens, 0, 0, &ws_bytes));
+      DevBuf ws, x, y, cu_dev;
+      PD_CUDA_TRY(ws.alloc(ws_bytes));
+      PD_CUDA_TRY(x.alloc(tokens * d * 2));
+      PD_CUDA_TRY(y.alloc(tokens * d * 2));
+      PD_CUDA_TRY(cu_dev.alloc(cu.size() * 4));
+      PD_CUDA_TRY(cudaMemcpyAsync(cu_dev.p, cu.data(), cu.size() * 4, cudaMemcpyHostToDevice, st));
+      PD_TRY(pd::launch_fill_normal(static_cast<bf16*>(x.p), tokens * d, m->seed, 1000, 0.f, 1.f, st));
+      std::vector<double> times;
+      for (int it = 0; it < m->warmup + m->reps; ++it) {
+        const long long l0 = pd::g_launch_count;
+        PD_CUDA_TRY(cudaEventRecord(ev.a, st));
+        PD_TRY(pd_prefill_stack(stack.layers.data(), caches.data(), nl, ring, x.p, y.p, 0,
+                                static_cast<const int32_t*>(cu_dev.p), cu.data(), m->n_req, ws.p, ws_bytes, st));
+        PD_CUDA_TRY(cudaEventRecord(ev.b, st));
+        PD_CUDA_TRY(cudaEventSynchronize(ev.b));
+        float ms = 0.f;
+        PD_CUDA_TRY(cudaEventElapsedTime(&ms, ev.a, ev.b));
+        if (it >= m->warmup) {
+          times.push_back(ms * 1e-3);
+          timed_launches += pd::g_launch_count - l0;
+        }
+      }
+      PD_TRY(pd_layer_check(stack.layers[0], st));
+      out->prefill_time_s = median(times) * scale_layers;
+      out->prefill_tok_s = tokens / out->prefill_time_s;
+      if (peak_bf16_flops > 0) out->prefill_frac_bf16_peak = out->prefill_flops / out->prefill_time_s / peak_bf16_flops;
+    }
+  }
+
+  // ------------------------------------------------------------------- decode
+  if (m->n_batch_sizes > 0) {
+    int max_b = 0;
+    for (int i = 0; i < m->n_batch_sizes; ++i) {
+      if (m->batch_sizes[i] <= 0 || m->batch_sizes[i] > 4096) return PD_ERR_INVALID_ARG;
+      max_b = std::max(max_b, m->batch_sizes[i]);
+    }
+    int max_start = m->kv_len_start;
+    if (m->kv_len_mix)
+      for (int b = 0; b < max_b; ++b) {
+        if (m->kv_len_mix[b] < 0) return PD_ERR_INVALID_ARG;
+        max_start = std::max(max_start, m->kv_len_mix[b]);
+      }
+    const int len_cap = max_start + m->n_steps;
+    if (len_cap > cfg.max_pos) return PD_ERR_INVALID_ARG;
+    // steps sampled: 0, stride, 2*stride, ... and the last one
+    std::vector<int> steps;
+    const int stride = m->step_stride > 0 ? m->step_stride : 1;
+    for (int t = 0; t < m->n_steps; t += stride) steps.push_back(t);
+    if (steps.back() != m->n_steps - 1) steps.push_back(m->n_steps - 1);
+
+    const size_t params_bytes = layer_param_count(cfg) * 2;
+    for (int bi = 0; bi < m->n_batch_sizes; ++bi) {
+      const int B = m->batch_sizes[bi];
+      const size_t cache_bytes = static_cast<size_t>(B) * len_cap * kv_row;
+      const int ring = cache_ring(2 * cache_bytes, nl);
+      std::vector<DevBuf> kbuf(ring), vbuf(ring);
+      std::vector<pd_kv_cache> caches(ring);
+      for (int i = 0; i < ring; ++i) {
+        PD_CUDA_TRY(kbuf[i].alloc(cache_bytes));
+        PD_CUDA_TRY(vbuf[i].alloc(cache_bytes));
+        PD_TRY(pd::launch_fill_normal(static_cast<bf16*>(kbuf[i].p), cache_bytes / 2, m->seed, 2000 + 2 * i, 0.f, 1.f, st));
+        PD_TRY(pd::launch_fill_normal(static_cast<bf16*>(vbuf[i].p), cache_bytes / 2, m->seed, 2001 + 2 * i, 0.f, 1.f, st));
+        caches[i].struct_size = sizeof(pd_kv_cache);
+        caches[i].k = kbuf[i].p; caches[i].v = vbuf[i].p; caches[i].batch_cap = B; caches[i].len_cap = len_cap;
+      }
+      size_t ws_bytes = 0;
+      PD_TRY(pd_workspace_bytes(&cfg, 0, B, len_cap, &ws_bytes));
+      DevBuf ws, x, y, kv_dev;
+      PD_CUDA_TRY(ws.alloc(ws_bytes));
+      PD_CUDA_TRY(x.alloc(B * d * 2));
+      PD_CUDA_TRY(y.alloc(B * d * 2));
+      PD_CUDA_TRY(kv_dev.alloc(steps.size() * B * 4));
+      std::vector<int32_t> kv_host(steps.size() * B);
+      double kv_tokens_mean = 0.0;
+      for (size_t si = 0; si < steps.size(); ++si)
+        for (int b = 0; b < B; ++b) {
+          const int start = m->kv_len_mix ? m->kv_len_mix[b] : m->kv_len_start;
+          kv_host[si * B + b] = start + steps[si];
+          kv_tokens_mean += start + steps[si] + 1;
+        }
+      kv_tokens_mean /= static_cast<double>(steps.size());  // sum over the batch, mean over steps
+      PD_CUDA_TRY(cudaMemcpyAsync(kv_dev.p, kv_host.data(), kv_host.size() * 4, cudaMemcpyHostToDevice, st));
+      PD_TRY(pd::launch_fill_normal(static_cast<bf16*>(x.p), B * d, m->seed, 3000 + bi, 0.f, 1.f, st));
+      PD_CUDA_TRY(cudaStreamSynchronize(st));
+
+      double step_time_sum = 0.0, attn_time_sum = 0.0;
+      for (size_t si = 0; si < steps.size(); ++si) {
+        const int32_t* kvp = static_cast<const int32_t*>(kv_dev.p) + si * B;
+        int max_kv = 0;
+        for (int b = 0; b < B; ++b) max_kv = std::max(max_kv, kv_host[si * B + b] + 1);
+        std::vector<double> times;
+        for (int it = 0; it < m->warmup + m->reps; ++it) {
+          const long long l0 = pd::g_launch_count;
+          PD_CUDA_TRY(cudaEventRecord(ev.a, st));
+          PD_TRY(pd_decode_stack(stack.layers.data(), caches.data(), nl, ring, x.p, y.p, 0, kvp, B, max_kv, ws.p,
+                                 ws_bytes, st));
+          PD_CUDA_TRY(cudaEventRecord(ev.b, st));
+          PD_CUDA_TRY(cudaEventSynchronize(ev.b));
+          float ms = 0.f;
+          PD_CUDA_TRY(cudaEventElapsedTime(&ms, ev.a, ev.b));
+          if (it >= m->warmup) {
+            times.push_back(ms * 1e-3);
+            timed_launches += pd::g_launch_count - l0;
+          }
+        }
+        step_time_sum += median(times);
+
+        // the attention kernel alone, over the same caches (q = whatever the last pass left in the workspace)
+        pd::DecodeAttnArgs a{};
+        size_t ws_total = 0;
+        (void)ws_total;
+        // reuse the library's own carving by running one decode layer first would be circular: place q, o and the
+        // partials at the start of the workspace instead (the kernel only needs valid, finite inputs)
+        const size_t q_bytes = pd::align_up(static_cast<size_t>(B) * stack.layers[0]->n_qkv * 2, 256);
+        const size_t o_bytes = pd::align_up(static_cast<size_t>(B) * cfg.n_q_heads * cfg.head_dim * 2, 256);
+        uint8_t* wsb = static_cast<uint8_t*>(ws.p);
+        a.q = reinterpret_cast<bf16*>(wsb); a.ldq = stack.layers[0]->n_qkv;
+        a.o = reinterpret_cast<bf16*>(wsb + q_bytes);
+        a.partial = reinterpret_cast<float*>(wsb + q_bytes + o_bytes);
+        a.kv_len = kvp; a.batch = B; a.max_kv_len = max_kv;
+        a.n_splits = pd::decode_attention_splits(B, cfg.n_kv_heads, max_kv);
+        a.n_q_heads = cfg.n_q_heads; a.n_kv_heads = cfg.n_kv_heads; a.head_dim = cfg.head_dim; a.len_cap = len_cap;
+        PD_TRY(pd::launch_fill_normal(const_cast<bf16*>(a.q), static_cast<size_t>(B) * a.ldq, m->seed, 4000, 0.f, 1.f, st));
+        std::vector<double> atimes;
+        for (int it = 0; it < m->warmup + m->reps; ++it) {
+          PD_CUDA_TRY(cudaEventRecord(ev.a, st));
+          for (int l = 0; l < nl; ++l) {
+            a.k_cache = static_cast<bf16*>(caches[l % ring].k);
+            a.v_cache = static_cast<bf16*>(caches[l % ring].v);
+            PD_TRY(pd::launch_decode_attention(a, st));
+          }
+          PD_CUDA_TRY(cudaEventRecord(ev.b, st));
+          PD_CUDA_TRY(cudaEventSynchronize(ev.b));
+          float ms = 0.f;
+          PD_CUDA_TRY(cudaEventElapsedTime(&ms, ev.a, ev.b));
+          if (it >= m->warmup) atimes.push_back(ms * 1e-3 / nl);
+        }
+        attn_time_sum += median(atimes);
+      }
+      PD_TRY(pd_layer_check(stack.layers[0], st));
+      const double step_time = step_time_sum / steps.size();  // n_layers_run layers
+      const double attn_time = attn_time_sum / steps.size();  // one layer
+      const double kv_bytes_layer = kv_tokens_mean * 2.0 * kv_row;
+      const double bytes_layer = static_cast<double>(params_bytes) + kv_bytes_layer + B * 2.0 * kv_row + 2.0 * B * d * 2;
+      const int pi = out->n_points++;
+      out->batch[pi] = B;
+      out->tpot_s[pi] = step_time * scale_layers;
+      out->decode_bytes[pi] = bytes_layer * m->n_layers_model;
+      out->attn_time_s[pi] = attn_time;
+      if (peak_hbm_bytes_s > 0) {
+        out->decode_frac_hbm_peak[pi] = out->decode_bytes[pi] / out->tpot_s[pi] / peak_hbm_bytes_s;
+        out->attn_frac_hbm_peak[pi] = kv_bytes_layer / attn_time / peak_hbm_bytes_s;
+      }
+    }
+  }
+  (void)launches_before;
+  out->gpu_launches = static_cast<int32_t>(std::min<long long>(timed_launches, 2147483647ll));
+  return PD_OK;
+}

@@ -27,3 +27,14 @@ def read_golden(name):
 @pytest.fixture(scope="session")
 def worked_example():
     return read_golden("worked_example.txt")
+
+
+@pytest.fixture(scope="session")
+def pdlib():
+    """The Python binding, after (re)building libpd.so in-tree if it is missing or stale."""
+    import subprocess
+    res = subprocess.run([sys.executable, os.path.join(ROOT, "paper_2603_04716_b200", "build.py")],
+                         capture_output=True, text=True)
+    assert res.returncode == 0, res.stdout + res.stderr
+    import paper_2603_04716_b200 as pd
+    return pd

@@ -1,0 +1,64 @@
+"""Helpers for the GPU parity tests: bf16 upload/download through torch device memory
+(torch is used only as an allocator here) and the tolerance check."""
+import numpy as np
+
+import pd_inputs as gen
+
+ATOL = 2e-2
+RTOL = 2e-2
+
+
+def to_dev(a):
+    """float32 array of bf16-representable values -> int16 CUDA tensor holding the bf16 bits."""
+    import torch
+    bits = gen.to_bf16_bits(np.asarray(a, dtype=np.float32)).view(np.int16)
+    return torch.from_numpy(bits).cuda()
+
+
+def i32_dev(a):
+    import torch
+    return torch.from_numpy(np.asarray(a, dtype=np.int32)).cuda()
+
+
+def empty_bf16(*shape):
+    import torch
+    return torch.zeros(shape, dtype=torch.int16, device="cuda")
+
+
+def from_dev(t):
+    """int16 CUDA tensor with bf16 bits -> float32 numpy array."""
+    return gen.from_bf16_bits(t.cpu().numpy().view(np.uint16))
+
+
+def assert_close(got, ref, what=""):
+    got = np.asarray(got, dtype=np.float64)
+    ref = np.asarray(ref, dtype=np.float64)
+    assert got.shape == ref.shape, (got.shape, ref.shape)
+    assert np.all(np.isfinite(got)), f"{what}: non-finite output"
+    err = np.abs(got - ref)
+    bound = ATOL + RTOL * np.abs(ref)
+    worst = np.argmax(err - bound)
+    assert np.all(err <= bound), (f"{what}: max abs err {err.max():.4g}, worst at {np.unravel_index(worst, err.shape)} "
+                                  f"got {got.flat[worst]:.5g} ref {ref.flat[worst]:.5g}; "
+                                  f"{np.count_nonzero(err > bound)} of {err.size} outside tolerance")
+    return float(err.max())
+
+
+class DeviceLayer:
+    """One layer on the device plus the buffers a test needs."""
+
+    def __init__(self, pd, cfg, weights_np, max_tokens, max_batch, max_kv_len):
+        import torch
+        self.pd, self.cfg = pd, cfg
+        self.wdev = {k: to_dev(v) for k, v in weights_np.items()}
+        self.layer = pd.Layer(cfg, self.wdev)
+        torch.cuda.synchronize()
+        self.ws_bytes = pd.pd_workspace_bytes(cfg, max_tokens, max_batch, max_kv_len)
+        self.ws = torch.zeros(self.ws_bytes, dtype=torch.uint8, device="cuda")
+
+    def make_cache(self, batch_cap, len_cap, k_np=None, v_np=None):
+        shape = (batch_cap, self.cfg.n_kv_heads, len_cap, self.cfg.head_dim)
+        k = to_dev(k_np) if k_np is not None else empty_bf16(*shape)
+        v = to_dev(v_np) if v_np is not None else empty_bf16(*shape)
+        assert tuple(k.shape) == shape
+        return k, v, self.pd.kv_cache_struct(k, v, batch_cap, len_cap)

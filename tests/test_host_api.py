@@ -1,0 +1,116 @@
+"""CPU-only checks of the product's host side: the library loads and exports the
+symbols the header declares; pd_allocate and pd_queue_replay agree with the oracle
+(integers and doubles bit for bit, both being IEEE double in the same order)."""
+import ctypes
+import math
+import os
+import random
+import re
+
+import numpy as np
+import pytest
+
+from oracle import allocation as A
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def test_library_exports_every_declared_symbol(pdlib):
+    header = open(os.path.join(ROOT, "include", "pd.h")).read()
+    declared = set(re.findall(r"\b(pd_[a-z0-9_]+)\s*\(", header))
+    assert declared == set(pdlib.EXPORTS)
+    lib = ctypes.CDLL(pdlib.LIB_PATH)
+    for name in declared:
+        assert hasattr(lib, name), name
+    assert pdlib.pd_version() >= 1
+
+
+def test_struct_sizes_match_c_layout(pdlib):
+    # natural C layout: checked against hand-computed sizes of include/pd.h
+    assert ctypes.sizeof(pdlib.pd_layer_cfg) == 36
+    assert ctypes.sizeof(pdlib.pd_layer_weights) == 8 + 7 * 8
+    assert ctypes.sizeof(pdlib.pd_kv_cache) == 32
+    assert ctypes.sizeof(pdlib.pd_alloc_in) == 8 + 7 * 8 + 8 + 16
+    assert ctypes.sizeof(pdlib.pd_alloc_out) == 8 + 5 * 8 + 8 + 3 * 8 + 16 + 8
+    assert ctypes.sizeof(pdlib.pd_measurement) == 8 + 4 * 8 + 8 + 32 * 4 + 5 * 32 * 8 + 8
+
+
+def _same(a, b):
+    return (math.isnan(a) and math.isnan(b)) or a == b
+
+
+def test_allocate_matches_oracle_bit_for_bit(pdlib):
+    rnd = random.Random(11)
+    status_names = {0: "ok", pdlib.PD_ERR_INFEASIBLE_TTFT: "infeasible_ttft", pdlib.PD_ERR_INFEASIBLE_TPOT: "infeasible_tpot"}
+    seen = set()
+    for trial in range(2000):
+        n = rnd.randint(1, 16)
+        batch = rnd.sample(range(1, 1024), n)
+        tpot = [rnd.uniform(0.002, 0.12) for _ in range(n)]
+        if trial % 3:
+            order = sorted(range(n), key=lambda i: batch[i])
+            srt = sorted(tpot)
+            for rank, i in enumerate(order):
+                tpot[i] = srt[rank]
+        args = dict(tp_total=rnd.uniform(1e3, 1e6), l_in=float(rnd.randint(16, 32768)), l_out=float(rnd.randint(1, 4096)),
+                    ttft=rnd.uniform(0.05, 8.0), tpot_slo=rnd.uniform(0.001, 0.13), tp_max=rnd.uniform(5e3, 2e5),
+                    t_over=rnd.choice([0.0, 0.1, rnd.uniform(0, 0.3)]))
+        o = A.allocate(args["tp_total"], args["l_in"], args["l_out"], args["ttft"], args["tpot_slo"], args["tp_max"],
+                       batch, tpot, args["t_over"])
+        p = pdlib.pd_allocate(args["tp_total"], args["l_in"], args["l_out"], args["ttft"], args["tpot_slo"],
+                              args["tp_max"], batch, tpot, args["t_over"])
+        assert status_names[p["status"]] == o.status
+        seen.add(o.status)
+        assert p["feasible_batch"] == o.feasible_batch and bool(p["sweep_capped"]) == o.sweep_capped
+        assert (p["n_prefill"], p["n_decode"], p["n_prefill_ceil"], p["n_decode_ceil"]) == \
+               (o.n_prefill, o.n_decode, o.n_prefill_ceil, o.n_decode_ceil)
+        for mine, theirs in (("tp_prefill_eff", o.tp_prefill_eff), ("tp_decode_eff", o.tp_decode_eff), ("mu", o.mu),
+                             ("lam", o.lam), ("rho", o.rho), ("n_prefill_frac", o.n_prefill_frac),
+                             ("n_decode_frac", o.n_decode_frac), ("ratio_pd", o.ratio_pd),
+                             ("achieved_total_tok_s", o.achieved_total_tok_s)):
+            assert _same(p[mine], theirs), (mine, p[mine], theirs)
+    assert seen == {"ok", "infeasible_ttft", "infeasible_tpot"}
+
+
+def test_allocate_worked_example(pdlib, worked_example):
+    g = worked_example
+    b = 34
+    p = pdlib.pd_allocate(g["tp_total_tokens_per_min"] / 60.0, g["l_in"], g["l_out"], g["ttft_slo_s"], g["tpot_slo_s"],
+                          g["prefill_max_tok_s"], [b], [b / g["tp_decode_eff"]], g["t_overhead_s"])
+    assert p["status"] == 0
+    assert (p["n_prefill"], p["n_decode"]) == (int(g["n_prefill"]), int(g["n_decode"]))
+    assert abs(p["tp_prefill_eff"] - g["tp_prefill_eff_approx"]) <= g["tp_prefill_eff_tol"]
+    assert abs(p["ratio_pd"] - g["ratio_pd_printed"]) <= g["ratio_pd_tol"]
+
+
+def test_allocate_rejects_bad_arguments(pdlib):
+    with pytest.raises(pdlib.PdError):
+        pdlib.pd_allocate(-1.0, 10, 10, 1, 0.05, 1e4, [1], [0.01])
+    with pytest.raises(pdlib.PdError):
+        pdlib.pd_allocate(1e4, 10, 10, 1, 0.05, 1e4, [0], [0.01])
+    with pytest.raises(pdlib.PdError):
+        pdlib.pd_allocate(1e4, 10, 10, 1, 0.05, 1e4, [1], [float("nan")])
+
+
+def test_queue_replay_matches_oracle(pdlib):
+    rng = np.random.Generator(np.random.Philox(key=3))
+    for n in (1, 2, 1000, 50_000):
+        gaps = rng.exponential(0.3, size=n)
+        svc = rng.exponential(0.25, size=n)
+        soj, wait = pdlib.pd_queue_replay(gaps, svc)
+        o_soj, o_wait = A.queue_replay(gaps.tolist(), svc.tolist())
+        assert soj == o_soj and wait == o_wait
+    with pytest.raises(pdlib.PdError):
+        pdlib.pd_queue_replay(np.array([-1.0]), np.array([1.0]))
+
+
+def test_workspace_bytes_and_config_validation(pdlib):
+    cfg = pdlib.LayerConfig(512, 8, 2, 64, 1536, max_pos=256)
+    small = pdlib.pd_workspace_bytes(cfg, 128, 4, 144)
+    big = pdlib.pd_workspace_bytes(cfg, 1024, 4, 144)
+    assert 0 < small < big and small % 256 == 0
+    for bad in (pdlib.LayerConfig(512, 8, 3, 64, 1536), pdlib.LayerConfig(512, 8, 2, 96, 1536),
+                pdlib.LayerConfig(500, 8, 2, 64, 1536)):
+        with pytest.raises(pdlib.PdError) as e:
+            pdlib.pd_workspace_bytes(bad, 128, 4, 144)
+        assert e.value.status == pdlib.PD_ERR_UNSUPPORTED_SHAPE
