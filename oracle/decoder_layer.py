@@ -23,6 +23,16 @@ Layouts (all row-major numpy arrays):
     g_attn   [d_model]            g_mlp [d_model]
     KV cache [batch, Hkv, len_cap, hd]  (K and V separate)
 
+Storage rounding.  The definition above is exact arithmetic on the given inputs.
+The data layout the GPU library is measured with keeps every tensor that crosses
+HBM between two operations in bf16 (normalised activations, q, the K/V cache, the
+attention output, the residual stream, the SwiGLU output, the layer output).  Passing
+``store=<rounding function>`` applies that function at exactly those hand-over
+points and nowhere else (no rounding inside a contraction, the softmax or SwiGLU);
+``store=None`` (default) is the unrounded definition.  With it the tests can separate
+"the kernels compute the right function" (tight, against the rounded variant) from
+"bf16 storage costs this much accuracy" (against the exact variant).
+
 Parity pins (see tests/test_oracle_layer.py): softmax rows sum to one, decode
 step t equals prefill row t, zero-weight and single-token special cases,
 rotation invariants of RoPE, permutation invariance over packed requests, a
@@ -124,16 +134,20 @@ def _attend(q: np.ndarray, k: np.ndarray, v: np.ndarray, q_pos: np.ndarray,
     return o.reshape(tq, cfg.n_q_heads * cfg.head_dim)
 
 
+def _identity(a: np.ndarray) -> np.ndarray:
+    return a
+
+
 def _mlp_and_residuals(x_rows: np.ndarray, o_rows: np.ndarray, w: LayerWeights,
-                       cfg: LayerConfig, dt) -> np.ndarray:
-    h = x_rows + o_rows @ w.w_o.astype(dt).T
-    n2 = rmsnorm(h, w.g_mlp.astype(dt), cfg.rms_eps)
-    a = silu(n2 @ w.w_gate.astype(dt).T) * (n2 @ w.w_up.astype(dt).T)
-    return h + a @ w.w_down.astype(dt).T
+                       cfg: LayerConfig, dt, st) -> np.ndarray:
+    h = st(x_rows + o_rows @ w.w_o.astype(dt).T)
+    n2 = st(rmsnorm(h, w.g_mlp.astype(dt), cfg.rms_eps))
+    a = st(silu(n2 @ w.w_gate.astype(dt).T) * (n2 @ w.w_up.astype(dt).T))
+    return st(h + a @ w.w_down.astype(dt).T)
 
 
 def prefill_layer(cfg: LayerConfig, w: LayerWeights, x: np.ndarray, cu_seqlens,
-                  rows=None, dtype=np.float64, probs_out: list | None = None):
+                  rows=None, dtype=np.float64, probs_out: list | None = None, store=None):
     """One layer over a packed ragged batch of requests.
 
     ``cu_seqlens`` has n_req + 1 entries; request r owns rows cu[r]..cu[r+1]-1 at
@@ -144,6 +158,7 @@ def prefill_layer(cfg: LayerConfig, w: LayerWeights, x: np.ndarray, cu_seqlens,
     Returns (out, k, v): out[len(rows) or T, d]; k, v[T, Hkv, hd] (k after RoPE).
     """
     dt = dtype
+    st = store or _identity
     x = np.asarray(x, dtype=dt)
     cu = np.asarray(cu_seqlens, dtype=np.int64)
     t_total = x.shape[0]
@@ -152,14 +167,14 @@ def prefill_layer(cfg: LayerConfig, w: LayerWeights, x: np.ndarray, cu_seqlens,
     req = np.repeat(np.arange(len(cu) - 1), np.diff(cu))
     pos = np.arange(t_total) - cu[req]
 
-    n1 = rmsnorm(x, w.g_attn.astype(dt), cfg.rms_eps)
+    n1 = st(rmsnorm(x, w.g_attn.astype(dt), cfg.rms_eps))
     w_qkv = w.w_qkv.astype(dt)
     w_q, w_k, w_v = w_qkv[:hq * hd], w_qkv[hq * hd:(hq + hkv) * hd], w_qkv[(hq + hkv) * hd:]
-    k = rope((n1 @ w_k.T).reshape(t_total, hkv, hd), pos, cfg.rope_theta)
-    v = (n1 @ w_v.T).reshape(t_total, hkv, hd)
+    k = st(rope((n1 @ w_k.T).reshape(t_total, hkv, hd), pos, cfg.rope_theta))
+    v = st((n1 @ w_v.T).reshape(t_total, hkv, hd))
 
     sel = np.arange(t_total) if rows is None else np.asarray(rows, dtype=np.int64)
-    q = rope((n1[sel] @ w_q.T).reshape(len(sel), hq, hd), pos[sel], cfg.rope_theta)
+    q = st(rope((n1[sel] @ w_q.T).reshape(len(sel), hq, hd), pos[sel], cfg.rope_theta))
 
     o = np.empty((len(sel), hq * hd), dtype=dt)
     for r in range(len(cu) - 1):
@@ -168,13 +183,13 @@ def prefill_layer(cfg: LayerConfig, w: LayerWeights, x: np.ndarray, cu_seqlens,
             continue
         lo, hi = cu[r], cu[r + 1]
         o[mine] = _attend(q[mine], k[lo:hi], v[lo:hi], pos[sel][mine], pos[lo:hi], cfg, probs_out)
-    out = _mlp_and_residuals(x[sel], o, w, cfg, dt)
+    out = _mlp_and_residuals(x[sel], st(o), w, cfg, dt, st)
     return out, k, v
 
 
 def decode_layer(cfg: LayerConfig, w: LayerWeights, x: np.ndarray, kv_len,
                  k_cache: np.ndarray, v_cache: np.ndarray, dtype=np.float64,
-                 probs_out: list | None = None) -> np.ndarray:
+                 probs_out: list | None = None, store=None) -> np.ndarray:
     """One decode step for a batch of B sequences, one new token each.
 
     kv_len[b] tokens are already cached for sequence b; the new token has
@@ -183,17 +198,18 @@ def decode_layer(cfg: LayerConfig, w: LayerWeights, x: np.ndarray, kv_len,
     Returns out[B, d].
     """
     dt = dtype
+    st = store or _identity
     x = np.asarray(x, dtype=dt)
     kv_len = np.asarray(kv_len, dtype=np.int64)
     b_sz = x.shape[0]
     hq, hkv, hd = cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim
     assert np.all(kv_len < k_cache.shape[2])
 
-    n1 = rmsnorm(x, w.g_attn.astype(dt), cfg.rms_eps)
+    n1 = st(rmsnorm(x, w.g_attn.astype(dt), cfg.rms_eps))
     qkv = n1 @ w.w_qkv.astype(dt).T
-    q = rope(qkv[:, :hq * hd].reshape(b_sz, hq, hd), kv_len, cfg.rope_theta)
-    k = rope(qkv[:, hq * hd:(hq + hkv) * hd].reshape(b_sz, hkv, hd), kv_len, cfg.rope_theta)
-    v = qkv[:, (hq + hkv) * hd:].reshape(b_sz, hkv, hd)
+    q = st(rope(qkv[:, :hq * hd].reshape(b_sz, hq, hd), kv_len, cfg.rope_theta))
+    k = st(rope(qkv[:, hq * hd:(hq + hkv) * hd].reshape(b_sz, hkv, hd), kv_len, cfg.rope_theta))
+    v = st(qkv[:, (hq + hkv) * hd:].reshape(b_sz, hkv, hd))
 
     o = np.empty((b_sz, hq * hd), dtype=dt)
     for b in range(b_sz):
@@ -203,7 +219,7 @@ def decode_layer(cfg: LayerConfig, w: LayerWeights, x: np.ndarray, kv_len,
         keys = np.ascontiguousarray(k_cache[b, :, :n + 1, :].transpose(1, 0, 2)).astype(dt)
         vals = np.ascontiguousarray(v_cache[b, :, :n + 1, :].transpose(1, 0, 2)).astype(dt)
         o[b:b + 1] = _attend(q[b:b + 1], keys, vals, kv_len[b:b + 1], np.arange(n + 1), cfg, probs_out)
-    return _mlp_and_residuals(x, o, w, cfg, dt)
+    return _mlp_and_residuals(x, st(o), w, cfg, dt, st)
 
 
 def layer_flops_prefill(cfg: LayerConfig, lens) -> float:

@@ -256,3 +256,34 @@ def test_flop_count_matches_hand_numbers():
     # GEMM flops per token: 2 * (4096*6144 + 4096*4096 + 3*4096*14336) = 436.2 M
     assert L.layer_flops_prefill(cfg, [1]) - 4 * 32 * 128 == pytest.approx(436.2e6, rel=1e-3)
     assert L.layer_flops_prefill(cfg, [4096]) == pytest.approx(1.924e12, rel=2e-3)
+
+
+def test_storage_rounding_variant():
+    """store=None is the exact definition; an identity store changes nothing; a bf16 store
+    returns bf16-representable outputs and cache entries and stays within the error model
+    (S rounding points of relative size 2^-9, amplified about twice by the gated MLP)."""
+    cfg = TINY
+    w = make_weights(cfg)
+    x = gen.activations(0, 64, cfg.d_model)
+    exact, k, v = L.prefill_layer(cfg, w, x, [0, 64])
+    same, _, _ = L.prefill_layer(cfg, w, x, [0, 64], store=lambda a: a)
+    np.testing.assert_array_equal(exact, same)
+    calls = []
+
+    def r(a):
+        calls.append(a.shape)
+        return gen.bf16_round(np.asarray(a, dtype=np.float32)).astype(np.float64)
+    rounded, kr, vr = L.prefill_layer(cfg, w, x, [0, 64], store=r)
+    assert len(calls) == 9          # n1, k, v, q, o, h, n2, a, out
+    for t in (rounded, kr, vr):
+        np.testing.assert_array_equal(t, gen.bf16_round(t.astype(np.float32)).astype(np.float64))
+    rel = np.linalg.norm(rounded - exact) / np.linalg.norm(exact)
+    assert 1e-4 < rel < 2.0 * 2.0 ** -9 * np.sqrt(9 / 3) * 2
+    # decode: same hand-over points, cache receives rounded entries
+    kc = np.zeros((1, cfg.n_kv_heads, 65, cfg.head_dim)); vc = np.zeros_like(kc)
+    kc[0, :, :64] = kr.transpose(1, 0, 2); vc[0, :, :64] = vr.transpose(1, 0, 2)
+    calls.clear()
+    d = L.decode_layer(cfg, w, x[:1], [64], kc, vc, store=r)
+    assert len(calls) == 9
+    np.testing.assert_array_equal(kc[0, :, 64], gen.bf16_round(kc[0, :, 64].astype(np.float32)))
+    np.testing.assert_array_equal(d, gen.bf16_round(d.astype(np.float32)))
