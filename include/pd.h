@@ -119,6 +119,20 @@ pd_status pd_decode_layer(pd_layer* layer, const void* x, void* out, const int32
                           int32_t max_kv_len, const pd_kv_cache* cache, void* workspace,
                           size_t workspace_bytes, void* stream);
 
+/* The decode-attention kernel on its own (the HBM-bound part of decode mode; paper: decode is
+ * memory-bandwidth-bound), for roofline measurement and unit tests.
+ *   q, out        device bf16 [B, Hq*hd]; q has row pitch ldq elements (a multiple of 8)
+ *   kv_len_dev    device int32[B]; sequence b attends over entries 0..kv_len[b] of cache slot b
+ *                 (kv_len[b]+1 entries, all of which must already be in the cache)
+ *   workspace     scratch for the partial results of the KV-range splits, at least
+ *                 pd_decode_attention_workspace_bytes(cfg, B, max_kv_len) bytes, 256-byte aligned
+ * Only n_q_heads, n_kv_heads and head_dim of cfg are used. */
+pd_status pd_decode_attention_workspace_bytes(const pd_layer_cfg* cfg, int32_t B, int32_t max_kv_len,
+                                              size_t* out_bytes);
+pd_status pd_decode_attention(const pd_layer_cfg* cfg, const void* q, int32_t ldq, void* out,
+                              const int32_t* kv_len_dev, int32_t B, int32_t max_kv_len, const pd_kv_cache* cache,
+                              void* workspace, size_t workspace_bytes, void* stream);
+
 /* The same two modes over a stack of n_layers layers run back to back (layer i+1 reads layer
  * i's output), layer i using caches[i % n_caches].  With io_on_host = 0, x/out/cu_seqlens_dev/
  * kv_len are device pointers and the call only enqueues work.  With io_on_host = 1 they are
@@ -156,7 +170,7 @@ int64_t pd_launch_count(void);
 #define PD_TRACE_CLASSES 16
 enum {
   PD_K_GEMM_QKV = 0, PD_K_GEMM_O = 1, PD_K_GEMM_GATE_UP = 2, PD_K_GEMM_DOWN = 3, PD_K_ATTN_PREFILL = 4,
-  PD_K_ATTN_DECODE = 5, PD_K_RMSNORM = 6, PD_K_ROPE_KV = 7, PD_K_SWIGLU = 8
+  PD_K_ATTN_DECODE = 5, PD_K_RMSNORM = 6
 };
 typedef struct {
   uint32_t struct_size;

@@ -34,11 +34,10 @@ EXPORTS = [
     "pd_status_str", "pd_last_cuda_error", "pd_version", "pd_layer_create", "pd_layer_destroy",
     "pd_workspace_bytes", "pd_prefill_layer", "pd_decode_layer", "pd_prefill_stack", "pd_decode_stack",
     "pd_layer_check", "pd_gemm_bf16", "pd_measure", "pd_allocate", "pd_queue_replay",
-    "pd_launch_count", "pd_trace_begin", "pd_trace_end",
+    "pd_launch_count", "pd_trace_begin", "pd_trace_end", "pd_decode_attention", "pd_decode_attention_workspace_bytes",
 ]
 
-TRACE_CLASSES = ["gemm_qkv", "gemm_o", "gemm_gate_up", "gemm_down", "attn_prefill", "attn_decode", "rmsnorm",
-                 "rope_kv", "swiglu"]
+TRACE_CLASSES = ["gemm_qkv", "gemm_o", "gemm_gate_up", "gemm_down", "attn_prefill", "attn_decode", "rmsnorm"]
 
 
 class PdError(RuntimeError):
@@ -126,6 +125,10 @@ _lib.pd_measure.argtypes = [C.POINTER(pd_layer_cfg), C.POINTER(pd_measure_cfg), 
 _lib.pd_allocate.argtypes = [C.POINTER(pd_alloc_in), C.POINTER(pd_alloc_out)]
 _lib.pd_queue_replay.argtypes = [C.POINTER(C.c_double), C.POINTER(C.c_double), C.c_int64, C.POINTER(C.c_double),
                                  C.POINTER(C.c_double)]
+_lib.pd_decode_attention_workspace_bytes.argtypes = [C.POINTER(pd_layer_cfg), C.c_int32, C.c_int32,
+                                                     C.POINTER(C.c_size_t)]
+_lib.pd_decode_attention.argtypes = [C.POINTER(pd_layer_cfg), _P, C.c_int32, _P, _P, C.c_int32, C.c_int32,
+                                     C.POINTER(pd_kv_cache), _P, C.c_size_t, _P]
 _lib.pd_launch_count.restype = C.c_int64
 _lib.pd_trace_end.argtypes = [C.POINTER(pd_trace_report)]
 for _n in EXPORTS:
@@ -253,6 +256,20 @@ def pd_decode_layer(layer: Layer, x, out, kv_len_dev, batch: int, max_kv_len: in
     _check(_lib.pd_decode_layer(layer.handle, _ptr(x), _ptr(out), _ptr(kv_len_dev), batch, max_kv_len,
                                 C.byref(cache), _ptr(workspace), workspace_bytes, _stream_ptr(stream)),
            "pd_decode_layer")
+
+
+def pd_decode_attention_workspace_bytes(cfg: LayerConfig, batch: int, max_kv_len: int) -> int:
+    out = C.c_size_t(0)
+    _check(_lib.pd_decode_attention_workspace_bytes(C.byref(cfg.c_struct()), batch, max_kv_len, C.byref(out)),
+           "pd_decode_attention_workspace_bytes")
+    return out.value
+
+
+def pd_decode_attention(cfg: LayerConfig, q, ldq: int, out, kv_len_dev, batch: int, max_kv_len: int,
+                        cache: pd_kv_cache, workspace, workspace_bytes: int, stream=None):
+    _check(_lib.pd_decode_attention(C.byref(cfg.c_struct()), _ptr(q), ldq, _ptr(out), _ptr(kv_len_dev), batch,
+                                    max_kv_len, C.byref(cache), _ptr(workspace), workspace_bytes,
+                                    _stream_ptr(stream)), "pd_decode_attention")
 
 
 def _layer_array(layers):

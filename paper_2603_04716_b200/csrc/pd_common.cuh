@@ -56,49 +56,42 @@ pd_status make_tmap_bf16(CUtensorMap* out, const void* base, uint64_t rows, uint
 enum GemmEpilogue : int {
   EPI_STORE = 0,     // C = acc
   EPI_RESIDUAL = 1,  // C = R + acc
+  EPI_SWIGLU = 2,    // C[M, N/2] = silu(gate) * up, B rows interleaved gate/up in blocks of 64
+  EPI_ROPE_KV = 3,   // rotate-half RoPE on q and k heads; q -> C, k and v -> the KV cache
+};
+
+// What the RoPE / KV-write epilogue needs besides the accumulator.  Row t of the product is token t:
+// prefill finds its request by binary search in cu_seqlens (position = offset in the request, cache
+// sequence = slots[request] or the request index); decode uses position kv_len[t], sequence t.
+struct RopeEpilogue {
+  const float2* rope_tab;     // [max_pos, hd/2] (cos, sin)
+  const int32_t* cu_seqlens;  // prefill: device [n_req + 1]; decode: NULL
+  const int32_t* slots;       // prefill: device [n_req] or NULL
+  const int32_t* kv_len;      // decode: device [B]
+  bf16* k_cache;              // [batch_cap, Hkv, len_cap, hd]
+  bf16* v_cache;
+  int n_req, n_q_heads, n_kv_heads, head_dim, len_cap, batch_cap, max_pos;
 };
 
 struct GemmArgs {
   const bf16* a;  // [M, K], row pitch lda
   const bf16* b;  // [N, K], row pitch ldb
-  bf16* c;        // [M, N], row pitch ldc
+  bf16* c;        // [M, N] (EPI_SWIGLU: [M, N/2]; EPI_ROPE_KV: q heads only), row pitch ldc
   const bf16* r;  // residual [M, N], row pitch ldr (EPI_RESIDUAL); may alias c
   int m, n, k;
   int lda, ldb, ldc, ldr;
   int epilogue;
-  int* err_word;              // device int32, set non-zero on a device-side timeout; may be NULL
+  const RopeEpilogue* rope;   // EPI_ROPE_KV
+  int* err_word;              // device int32: 1 = a bounded wait gave up, 2 = a position or slot was out of range
 };
 
 // Tensor-core GEMM (tcgen05 + TMEM accumulators, operands staged by TMA).
-pd_status gemm_tc(const GemmArgs& g, cudaStream_t stream);
-// Plain CUDA-core GEMM with the same contract: debugging reference, selected with PD_GEMM=simt.
-pd_status gemm_simt(const GemmArgs& g, cudaStream_t stream);
-// Dispatches on the PD_GEMM environment variable (read once).
 pd_status gemm(const GemmArgs& g, cudaStream_t stream);
-// Box height (rows of B per tile) the tensor-core GEMM will use for this problem.
-int gemm_tc_block_n(int m, int n, int k);
+// Tile width (rows of B per tile) the GEMM will use for this problem.
+int gemm_block_n(int m, int n, int epilogue);
 
 // ------------------------------------------------------------ elementwise
 pd_status launch_rmsnorm(const bf16* x, const bf16* gain, bf16* y, int rows, int d, float eps, cudaStream_t s);
-
-struct RopeArgs {
-  bf16* qkv;              // [T, n_qkv] in/out: q part is rotated in place
-  bf16* k_cache;          // [batch_cap, Hkv, len_cap, hd]
-  bf16* v_cache;
-  const float2* rope_tab; // [max_pos, hd/2] (cos, sin)
-  const int32_t* cu_seqlens;  // prefill: device [n_req+1]; decode: NULL
-  const int32_t* slots;       // prefill: device [n_req] cache slot per request, or NULL (slot = request)
-  const int32_t* kv_len;      // decode: device [B] position of the new token; prefill: NULL
-  int n_req;
-  int n_tokens, n_q_heads, n_kv_heads, head_dim, len_cap;
-  int max_pos;                // rows of rope_tab
-  int batch_cap;              // sequences in the cache
-  int* err_word;              // set to 2 when a position or slot falls outside the cache or the table
-};
-pd_status launch_rope_scatter(const RopeArgs& a, cudaStream_t s);
-
-// a[T, F] = silu(gu[T, 0:F]) * gu[T, F:2F]
-pd_status launch_swiglu(const bf16* gu, bf16* a, int rows, int f, cudaStream_t s);
 
 // -------------------------------------------------------------- attention
 struct PrefillAttnArgs {
@@ -138,7 +131,7 @@ pd_status launch_fill_normal(bf16* dst, size_t n, uint64_t seed, uint64_t stream
 struct pd_layer {
   pd_layer_cfg cfg;
   int n_qkv;
-  pd::bf16 *w_qkv, *w_o, *w_gu, *w_down;  // owned copies; w_gu = [2F, d]: gate rows then up rows
+  pd::bf16 *w_qkv, *w_o, *w_gu, *w_down;  // owned copies; w_gu = [2F, d]: 64 gate rows, 64 up rows, alternating
   pd::bf16 *g_attn, *g_mlp;
   float2* rope_tab;                        // [max_pos, hd/2]
   int* err_word;                           // device int32

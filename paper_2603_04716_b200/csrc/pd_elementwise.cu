@@ -1,5 +1,5 @@
-// Memory-bound glue kernels of the layer: RMSNorm, RoPE with the KV-cache write, SwiGLU,
-// and the seeded synthetic fill used by the measurement harness.  All use 128-bit accesses.
+// Memory-bound glue kernels: RMSNorm (RoPE, the KV-cache write and SwiGLU live in the GEMM
+// epilogues) and the seeded synthetic fill used by the measurement harness.
 #include "pd_common.cuh"
 #include "pd_ptx.cuh"
 
@@ -70,93 +70,6 @@ __global__ void __launch_bounds__(RMS_THREADS) rmsnorm_kernel(const bf16* __rest
   }
 }
 
-// ------------------------------------------------------- RoPE + KV-cache write
-// One block per token.  Each thread owns 8 rotation pairs (i, i + hd/2) of one head: it
-// loads 16 bytes from each half, rotates by the table entry of the token's position and
-// stores q back in place or k into the cache; v heads are copied to the cache unchanged.
-__global__ void __launch_bounds__(128) rope_scatter_kernel(RopeArgs a) {
-  const int t = blockIdx.x;
-  __shared__ int s_pos, s_slot;
-  if (threadIdx.x == 0) {
-    if (a.cu_seqlens) {
-      int lo = 0, hi = a.n_req;  // find r with cu[r] <= t < cu[r+1]
-      while (hi - lo > 1) {
-        const int mid = (lo + hi) >> 1;
-        if (a.cu_seqlens[mid] <= t) lo = mid; else hi = mid;
-      }
-      s_pos = t - a.cu_seqlens[lo];
-      s_slot = a.slots ? a.slots[lo] : lo;
-    } else {
-      s_pos = a.kv_len[t];
-      s_slot = t;
-    }
-  }
-  __syncthreads();
-  const int pos = s_pos, slot = s_slot;
-  if (pos < 0 || pos >= a.len_cap || pos >= a.max_pos || slot < 0 || slot >= a.batch_cap) {
-    // would write outside the cache: record and skip
-    if (threadIdx.x == 0 && a.err_word) atomicExch(a.err_word, 2);
-    return;
-  }
-  const int hd = a.head_dim, half = hd / 2;
-  const int per_head = half / 8;  // threads per head
-  const int n_heads = a.n_q_heads + 2 * a.n_kv_heads;
-  const int n_qkv = n_heads * hd;
-  bf16* row = a.qkv + static_cast<size_t>(t) * n_qkv;
-  const float2* tab = a.rope_tab + static_cast<size_t>(pos) * half;
-  for (int w = threadIdx.x; w < n_heads * per_head; w += blockDim.x) {
-    const int h = w / per_head;
-    const int i0 = (w - h * per_head) * 8;
-    bf16* src = row + h * hd;
-    const uint4 lo4 = *reinterpret_cast<const uint4*>(src + i0);
-    const uint4 hi4 = *reinterpret_cast<const uint4*>(src + half + i0);
-    if (h < a.n_q_heads + a.n_kv_heads) {
-      float lo[8], hi[8], olo[8], ohi[8];
-      unpack8(lo4, lo);
-      unpack8(hi4, hi);
-#pragma unroll
-      for (int e = 0; e < 8; ++e) {
-        const float2 cs = tab[i0 + e];
-        olo[e] = lo[e] * cs.x - hi[e] * cs.y;
-        ohi[e] = hi[e] * cs.x + lo[e] * cs.y;
-      }
-      bf16* dst;
-      if (h < a.n_q_heads) {
-        dst = src;
-      } else {
-        const int j = h - a.n_q_heads;
-        dst = a.k_cache + ((static_cast<size_t>(slot) * a.n_kv_heads + j) * a.len_cap + pos) * hd;
-      }
-      *reinterpret_cast<uint4*>(dst + i0) = pack8(olo);
-      *reinterpret_cast<uint4*>(dst + half + i0) = pack8(ohi);
-    } else {
-      const int j = h - a.n_q_heads - a.n_kv_heads;
-      bf16* dst = a.v_cache + ((static_cast<size_t>(slot) * a.n_kv_heads + j) * a.len_cap + pos) * hd;
-      *reinterpret_cast<uint4*>(dst + i0) = lo4;
-      *reinterpret_cast<uint4*>(dst + half + i0) = hi4;
-    }
-  }
-}
-
-// -------------------------------------------------------------------- SwiGLU
-__global__ void __launch_bounds__(256) swiglu_kernel(const bf16* __restrict__ gu, bf16* __restrict__ out,
-                                                      size_t rows, int f) {
-  const int chunks_per_row = f / 8;
-  const size_t total = rows * chunks_per_row;
-  for (size_t idx = blockIdx.x * static_cast<size_t>(blockDim.x) + threadIdx.x; idx < total;
-       idx += static_cast<size_t>(gridDim.x) * blockDim.x) {
-    const size_t r = idx / chunks_per_row;
-    const int c = static_cast<int>(idx - r * chunks_per_row);
-    const bf16* base = gu + r * (2 * static_cast<size_t>(f));
-    float g[8], u[8], o[8];
-    unpack8(*reinterpret_cast<const uint4*>(base + c * 8), g);
-    unpack8(*reinterpret_cast<const uint4*>(base + f + c * 8), u);
-#pragma unroll
-    for (int e = 0; e < 8; ++e) o[e] = g[e] / (1.f + __expf(-g[e])) * u[e];
-    *reinterpret_cast<uint4*>(out + r * f + c * 8) = pack8(o);
-  }
-}
-
 // ------------------------------------------------------------- seeded fill
 __device__ __forceinline__ uint64_t splitmix64(uint64_t z) {
   z += 0x9E3779B97F4A7C15ull;
@@ -187,25 +100,6 @@ pd_status launch_rmsnorm(const bf16* x, const bf16* gain, bf16* y, int rows, int
   if (rows == 0) return PD_OK;
   if (d % 8 != 0 || d > RMS_THREADS * RMS_MAX_CHUNKS * 8) return PD_ERR_UNSUPPORTED_SHAPE;
   rmsnorm_kernel<<<rows, RMS_THREADS, 0, s>>>(x, gain, y, d, eps);
-  count_launch();
-  PD_CUDA_TRY(cudaGetLastError());
-  return PD_OK;
-}
-
-pd_status launch_rope_scatter(const RopeArgs& a, cudaStream_t s) {
-  if (a.n_tokens == 0) return PD_OK;
-  rope_scatter_kernel<<<a.n_tokens, 128, 0, s>>>(a);
-  count_launch();
-  PD_CUDA_TRY(cudaGetLastError());
-  return PD_OK;
-}
-
-pd_status launch_swiglu(const bf16* gu, bf16* out, int rows, int f, cudaStream_t s) {
-  if (rows == 0) return PD_OK;
-  const size_t total = static_cast<size_t>(rows) * (f / 8);
-  size_t blocks = (total + 255) / 256;
-  if (blocks > 148 * 16) blocks = 148 * 16;
-  swiglu_kernel<<<static_cast<unsigned>(blocks), 256, 0, s>>>(gu, out, static_cast<size_t>(rows), f);
   count_launch();
   PD_CUDA_TRY(cudaGetLastError());
   return PD_OK;

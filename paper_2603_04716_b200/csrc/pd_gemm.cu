@@ -1,14 +1,15 @@
 // C[M,N] = A[M,K] * B[N,K]^T (+ residual), bf16 operands, fp32 accumulation.
 //
-// Tensor-core path: a persistent, warp-specialised kernel.  One thread issues TMA tile
+// A persistent, warp-specialised kernel.  One thread issues TMA tile
 // loads of A (128 x 64) and B (BN x 64) into a ring of shared-memory stages; one thread
 // issues tcgen05.mma (128 x BN x 16 per instruction) accumulating in tensor memory; four
 // warps drain the accumulator (tcgen05.ld) and run the epilogue.  Two accumulator buffers
 // in tensor memory let the epilogue of tile i overlap the main loop of tile i+1.
+// Epilogues: plain store, residual add, SwiGLU (gate and up columns interleaved in blocks
+// of 64 so one tile holds both halves), and RoPE with the scatter of q, k, v to the q buffer
+// and the KV cache (a tile holds whole heads).
 // Every barrier wait is wall-clock bounded; on a timeout the block raises a shared abort
 // flag, records an error word in global memory and leaves through the normal teardown.
-#include <cstdlib>
-#include <cstring>
 #include <mutex>
 
 #include "pd_common.cuh"
@@ -75,7 +76,17 @@ struct GemmDev {
   int ldc, ldr;
   int tiles_m, tiles_n;
   int* err_word;
+  RopeEpilogue rope;  // EPI_ROPE_KV only
 };
+
+__device__ __forceinline__ uint4 pack8(const float (&f)[8]) {
+  uint4 o;
+  o.x = ptx::pack_bf16(f[0], f[1]);
+  o.y = ptx::pack_bf16(f[2], f[3]);
+  o.z = ptx::pack_bf16(f[4], f[5]);
+  o.w = ptx::pack_bf16(f[6], f[7]);
+  return o;
+}
 
 __device__ __forceinline__ void tile_coords(int tile, int tiles_m, int tiles_n, int& tm, int& tn) {
   // Groups of up to 8 row-tiles share the same column-tiles while they are resident, so
@@ -211,35 +222,123 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       const int row = tm * BM + lane_group * 32 + lane;
       const uint32_t t_row = tmem_base + (static_cast<uint32_t>(lane_group * 32) << 16) +
                              static_cast<uint32_t>(acc * Cfg::ACC_COLS);
-      constexpr int CHUNK = 32;
+      if constexpr (EPI == EPI_STORE || EPI == EPI_RESIDUAL) {
 #pragma unroll 1
-      for (int c0 = 0; c0 < BN; c0 += 32) {
-        uint32_t v[32];
-        ptx::tmem_ld_32x32(t_row + c0, v);
-        ptx::tmem_ld_wait();
-        const int col = tn * BN + c0;
-        if (row < p.m) {
-          bf16* crow = p.c + static_cast<size_t>(row) * p.ldc + col;
-          const bf16* rrow = (EPI == EPI_RESIDUAL) ? p.r + static_cast<size_t>(row) * p.ldr + col : nullptr;
+        for (int c0 = 0; c0 < BN; c0 += 32) {
+          uint32_t v[32];
+          ptx::tmem_ld_32x32(t_row + c0, v);
+          ptx::tmem_ld_wait();
+          const int col = tn * BN + c0;
+          if (row < p.m) {
+            bf16* crow = p.c + static_cast<size_t>(row) * p.ldc + col;
+            const bf16* rrow = (EPI == EPI_RESIDUAL) ? p.r + static_cast<size_t>(row) * p.ldr + col : nullptr;
 #pragma unroll
-          for (int j = 0; j < CHUNK; j += 8) {
-            if (col + j < p.n) {
+            for (int j = 0; j < 32; j += 8) {
+              if (col + j < p.n) {
+                float f[8];
+#pragma unroll
+                for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(v[j + e]);
+                if (EPI == EPI_RESIDUAL) {
+                  const uint4 rr = *reinterpret_cast<const uint4*>(rrow + j);
+                  f[0] += ptx::bf16_lo(rr.x); f[1] += ptx::bf16_hi(rr.x);
+                  f[2] += ptx::bf16_lo(rr.y); f[3] += ptx::bf16_hi(rr.y);
+                  f[4] += ptx::bf16_lo(rr.z); f[5] += ptx::bf16_hi(rr.z);
+                  f[6] += ptx::bf16_lo(rr.w); f[7] += ptx::bf16_hi(rr.w);
+                }
+                *reinterpret_cast<uint4*>(crow + j) = pack8(f);
+              }
+            }
+          }
+        }
+      } else if constexpr (EPI == EPI_SWIGLU) {
+        // columns [128 q, 128 q + 64) of the product are gate features 64 q .., the next 64 the matching up features
+        const int f_total = p.n / 2;
+#pragma unroll 1
+        for (int c0 = 0; c0 < BN / 2; c0 += 32) {
+          const int pair = c0 >> 6, within = c0 & 63;
+          uint32_t g[32], u[32];
+          ptx::tmem_ld_32x32(t_row + pair * 128 + within, g);
+          ptx::tmem_ld_32x32(t_row + pair * 128 + 64 + within, u);
+          ptx::tmem_ld_wait();
+          const int fcol = (tn * (BN / 128) + pair) * 64 + within;
+          if (row < p.m && fcol < f_total) {
+            bf16* crow = p.c + static_cast<size_t>(row) * p.ldc + fcol;
+#pragma unroll
+            for (int j = 0; j < 32; j += 8) {
               float f[8];
 #pragma unroll
-              for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(v[j + e]);
-              if (EPI == EPI_RESIDUAL) {
-                const uint4 rr = *reinterpret_cast<const uint4*>(rrow + j);
-                f[0] += ptx::bf16_lo(rr.x); f[1] += ptx::bf16_hi(rr.x);
-                f[2] += ptx::bf16_lo(rr.y); f[3] += ptx::bf16_hi(rr.y);
-                f[4] += ptx::bf16_lo(rr.z); f[5] += ptx::bf16_hi(rr.z);
-                f[6] += ptx::bf16_lo(rr.w); f[7] += ptx::bf16_hi(rr.w);
+              for (int e = 0; e < 8; ++e) {
+                const float gv = __uint_as_float(g[j + e]);
+                f[e] = gv / (1.f + __expf(-gv)) * __uint_as_float(u[j + e]);
               }
-              uint4 o;
-              o.x = ptx::pack_bf16(f[0], f[1]);
-              o.y = ptx::pack_bf16(f[2], f[3]);
-              o.z = ptx::pack_bf16(f[4], f[5]);
-              o.w = ptx::pack_bf16(f[6], f[7]);
-              *reinterpret_cast<uint4*>(crow + j) = o;
+              *reinterpret_cast<uint4*>(crow + j) = pack8(f);
+            }
+          }
+        }
+      } else {  // EPI_ROPE_KV
+        const RopeEpilogue& rp = p.rope;
+        const int hd = rp.head_dim, half = hd >> 1;
+        int pos = 0, slot = 0;
+        bool row_ok = row < p.m;
+        if (row_ok) {
+          if (rp.cu_seqlens) {
+            int lo = 0, hi = rp.n_req;  // request r with cu[r] <= row < cu[r+1]
+            while (hi - lo > 1) {
+              const int mid = (lo + hi) >> 1;
+              if (rp.cu_seqlens[mid] <= row) lo = mid; else hi = mid;
+            }
+            pos = row - rp.cu_seqlens[lo];
+            slot = rp.slots ? rp.slots[lo] : lo;
+          } else {
+            pos = rp.kv_len[row];
+            slot = row;
+          }
+          if (pos < 0 || pos >= rp.len_cap || pos >= rp.max_pos || slot < 0 || slot >= rp.batch_cap) {
+            if (p.err_word) atomicExch(p.err_word, 2);  // would fall outside the cache or the table: skip the row
+            row_ok = false;
+          }
+        }
+        const int n_heads = rp.n_q_heads + 2 * rp.n_kv_heads;
+        const int heads_per_tile = BN / hd;
+#pragma unroll 1
+        for (int hh = 0; hh < heads_per_tile; ++hh) {
+          const int head = tn * heads_per_tile + hh;
+          if (head >= n_heads) break;  // warp-uniform
+#pragma unroll 1
+          for (int i0 = 0; i0 < half; i0 += 32) {
+            uint32_t lo[32], hi[32];
+            ptx::tmem_ld_32x32(t_row + hh * hd + i0, lo);
+            ptx::tmem_ld_32x32(t_row + hh * hd + half + i0, hi);
+            ptx::tmem_ld_wait();
+            if (!row_ok) continue;
+            bf16* dst;
+            if (head < rp.n_q_heads) {
+              dst = p.c + static_cast<size_t>(row) * p.ldc + head * hd;
+            } else if (head < rp.n_q_heads + rp.n_kv_heads) {
+              dst = rp.k_cache +
+                    ((static_cast<size_t>(slot) * rp.n_kv_heads + (head - rp.n_q_heads)) * rp.len_cap + pos) * hd;
+            } else {
+              dst = rp.v_cache + ((static_cast<size_t>(slot) * rp.n_kv_heads + (head - rp.n_q_heads - rp.n_kv_heads)) *
+                                      rp.len_cap + pos) * hd;
+            }
+            const bool rotate = head < rp.n_q_heads + rp.n_kv_heads;
+            const float4* tab = reinterpret_cast<const float4*>(rp.rope_tab + static_cast<size_t>(pos) * half + i0);
+#pragma unroll
+            for (int j = 0; j < 32; j += 8) {
+              float a[8], b[8];
+#pragma unroll
+              for (int e = 0; e < 8; ++e) { a[e] = __uint_as_float(lo[j + e]); b[e] = __uint_as_float(hi[j + e]); }
+              if (rotate) {
+#pragma unroll
+                for (int e = 0; e < 8; e += 2) {
+                  const float4 cs = tab[(j + e) >> 1];  // (cos, sin) of two consecutive pairs
+                  const float a0 = a[e], b0 = b[e], a1 = a[e + 1], b1 = b[e + 1];
+                  a[e] = a0 * cs.x - b0 * cs.y;      b[e] = b0 * cs.x + a0 * cs.y;
+                  a[e + 1] = a1 * cs.z - b1 * cs.w;  b[e + 1] = b1 * cs.z + a1 * cs.w;
+                }
+              }
+              *reinterpret_cast<uint4*>(dst + i0 + j) = pack8(a);
+              *reinterpret_cast<uint4*>(dst + half + i0 + j) = pack8(b);
             }
           }
         }
@@ -287,11 +386,12 @@ pd_status launch_tc(const GemmArgs& g, cudaStream_t stream) {
   CUtensorMap ta, tb;
   PD_TRY(make_tmap_bf16(&ta, g.a, g.m, g.k, g.lda, BM));
   PD_TRY(make_tmap_bf16(&tb, g.b, g.n, g.k, g.ldb, BN));
-  GemmDev p;
+  GemmDev p{};
   p.c = g.c; p.r = g.r; p.m = g.m; p.n = g.n; p.k = g.k; p.ldc = g.ldc; p.ldr = g.ldr;
   p.tiles_m = (g.m + BM - 1) / BM;
   p.tiles_n = (g.n + BN - 1) / BN;
   p.err_word = g.err_word;
+  if (EPI == EPI_ROPE_KV) p.rope = *g.rope;
   const int tiles = p.tiles_m * p.tiles_n;
   const int grid = tiles < sm_count() ? tiles : sm_count();
   kern<<<grid, GEMM_THREADS, Cfg::SMEM_BYTES, stream>>>(ta, tb, p);
@@ -302,22 +402,33 @@ pd_status launch_tc(const GemmArgs& g, cudaStream_t stream) {
 
 template <int BN>
 pd_status launch_tc_epi(const GemmArgs& g, cudaStream_t stream) {
-  return g.epilogue == EPI_RESIDUAL ? launch_tc<BN, EPI_RESIDUAL>(g, stream) : launch_tc<BN, EPI_STORE>(g, stream);
+  switch (g.epilogue) {
+    case EPI_RESIDUAL: return launch_tc<BN, EPI_RESIDUAL>(g, stream);
+    case EPI_SWIGLU:
+      if constexpr (BN >= 128) return launch_tc<BN, EPI_SWIGLU>(g, stream);
+      return PD_ERR_UNSUPPORTED_SHAPE;
+    case EPI_ROPE_KV:
+      if constexpr (BN >= 128) return launch_tc<BN, EPI_ROPE_KV>(g, stream);
+      return PD_ERR_UNSUPPORTED_SHAPE;
+    default: return launch_tc<BN, EPI_STORE>(g, stream);
+  }
 }
 
 }  // namespace
 
-int gemm_tc_block_n(int m, int n, int k) {
-  (void)k;
-  // Pick the widest tile whose tile count still fills the machine reasonably: cost model =
-  // waves * per-tile time, per-tile time ~ BN (+ a fixed part for the A operand traffic).
+int gemm_block_n(int m, int n, int epilogue) {
+  // Pick the tile width by a small cost model: waves over the SMs times a per-tile time that
+  // grows with the width plus a fixed part for the A operand.  The fused epilogues need whole
+  // heads / gate-up pairs in a tile, so they do not use the 64-wide tile.
   const int sms = sm_count();
   const int tiles_m = (m + BM - 1) / BM;
+  const bool fused = epilogue == EPI_SWIGLU || epilogue == EPI_ROPE_KV;
   int best = 256;
   double best_cost = 1e300;
   const int cands[3] = {256, 128, 64};
   for (int bn : cands) {
-    if (bn > n && bn != 64) continue;
+    if (bn == 64 && fused) continue;
+    if (bn > n && bn != (fused ? 128 : 64)) continue;
     const long long tiles = 1ll * tiles_m * ((n + bn - 1) / bn);
     const long long waves = (tiles + sms - 1) / sms;
     const double cost = static_cast<double>(waves) * (bn + 32.0);
@@ -329,89 +440,21 @@ int gemm_tc_block_n(int m, int n, int k) {
 static pd_status check_gemm_args(const GemmArgs& g) {
   if (!g.a || !g.b || !g.c || g.m < 0 || g.n <= 0 || g.k <= 0) return PD_ERR_INVALID_ARG;
   if (g.epilogue == EPI_RESIDUAL && !g.r) return PD_ERR_INVALID_ARG;
+  if (g.epilogue == EPI_ROPE_KV && !g.rope) return PD_ERR_INVALID_ARG;
   if (g.k % BK != 0 || g.n % 16 != 0) return PD_ERR_UNSUPPORTED_SHAPE;
   if (g.lda % 8 || g.ldb % 8 || g.ldc % 8 || (g.epilogue == EPI_RESIDUAL && g.ldr % 8)) return PD_ERR_UNSUPPORTED_SHAPE;
-  return PD_OK;
-}
-
-pd_status gemm_tc(const GemmArgs& g, cudaStream_t stream) {
-  PD_TRY(check_gemm_args(g));
-  if (g.m == 0) return PD_OK;
-  switch (gemm_tc_block_n(g.m, g.n, g.k)) {
-    case 256: return launch_tc_epi<256>(g, stream);
-    case 128: return launch_tc_epi<128>(g, stream);
-    default: return launch_tc_epi<64>(g, stream);
-  }
-}
-
-// ------------------------------------------------------------- CUDA-core GEMM
-namespace {
-template <int EPI>
-__global__ void __launch_bounds__(256) gemm_simt_kernel(const bf16* __restrict__ a, const bf16* __restrict__ b,
-                                                         bf16* c, const bf16* r, int m, int n, int k, int lda,
-                                                         int ldb, int ldc, int ldr) {
-  // 64 x 64 tile, 16-wide K slices, 4 x 4 outputs per thread.
-  __shared__ float sa[16][64 + 1];
-  __shared__ float sb[16][64 + 1];
-  const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
-  const int row0 = blockIdx.y * 64, col0 = blockIdx.x * 64;
-  float acc[4][4] = {};
-  for (int k0 = 0; k0 < k; k0 += 16) {
-    for (int i = threadIdx.x; i < 64 * 16; i += 256) {
-      const int rr = i >> 4, kk = i & 15;
-      const int gr = row0 + rr, gc = col0 + rr;
-      sa[kk][rr] = (gr < m) ? __bfloat162float(a[static_cast<size_t>(gr) * lda + k0 + kk]) : 0.f;
-      sb[kk][rr] = (gc < n) ? __bfloat162float(b[static_cast<size_t>(gc) * ldb + k0 + kk]) : 0.f;
-    }
-    __syncthreads();
-#pragma unroll
-    for (int kk = 0; kk < 16; ++kk) {
-      float av[4], bv[4];
-#pragma unroll
-      for (int i = 0; i < 4; ++i) { av[i] = sa[kk][ty * 4 + i]; bv[i] = sb[kk][tx * 4 + i]; }
-#pragma unroll
-      for (int i = 0; i < 4; ++i)
-#pragma unroll
-        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
-    }
-    __syncthreads();
-  }
-  for (int i = 0; i < 4; ++i) {
-    const int gr = row0 + ty * 4 + i;
-    if (gr >= m) continue;
-    for (int j = 0; j < 4; ++j) {
-      const int gc = col0 + tx * 4 + j;
-      if (gc >= n) continue;
-      float v = acc[i][j];
-      if (EPI == EPI_RESIDUAL) v += __bfloat162float(r[static_cast<size_t>(gr) * ldr + gc]);
-      c[static_cast<size_t>(gr) * ldc + gc] = __float2bfloat16(v);
-    }
-  }
-}
-}  // namespace
-
-pd_status gemm_simt(const GemmArgs& g, cudaStream_t stream) {
-  PD_TRY(check_gemm_args(g));
-  if (g.m == 0) return PD_OK;
-  dim3 grid((g.n + 63) / 64, (g.m + 63) / 64);
-  if (g.epilogue == EPI_RESIDUAL)
-    gemm_simt_kernel<EPI_RESIDUAL><<<grid, 256, 0, stream>>>(g.a, g.b, g.c, g.r, g.m, g.n, g.k, g.lda, g.ldb,
-                                                            g.ldc, g.ldr);
-  else
-    gemm_simt_kernel<EPI_STORE><<<grid, 256, 0, stream>>>(g.a, g.b, g.c, g.r, g.m, g.n, g.k, g.lda, g.ldb, g.ldc,
-                                                         g.ldr);
-  count_launch();
-  PD_CUDA_TRY(cudaGetLastError());
+  if (g.epilogue == EPI_SWIGLU && g.n % 128 != 0) return PD_ERR_UNSUPPORTED_SHAPE;
   return PD_OK;
 }
 
 pd_status gemm(const GemmArgs& g, cudaStream_t stream) {
-  static int use_simt = -1;
-  if (use_simt < 0) {
-    const char* e = std::getenv("PD_GEMM");
-    use_simt = (e && std::strcmp(e, "simt") == 0) ? 1 : 0;
+  PD_TRY(check_gemm_args(g));
+  if (g.m == 0) return PD_OK;
+  switch (gemm_block_n(g.m, g.n, g.epilogue)) {
+    case 256: return launch_tc_epi<256>(g, stream);
+    case 128: return launch_tc_epi<128>(g, stream);
+    default: return launch_tc_epi<64>(g, stream);
   }
-  return use_simt ? gemm_simt(g, stream) : gemm_tc(g, stream);
 }
 
 }  // namespace pd

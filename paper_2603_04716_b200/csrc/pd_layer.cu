@@ -31,7 +31,7 @@ Workspace carve(const pd_layer_cfg& c, size_t tokens, size_t max_batch, int max_
   w.qkv = take(tokens * nqkv * 2);
   w.attn_o = take(tokens * hq * 2);
   w.resid = take(tokens * d * 2);
-  w.gate_up = take(tokens * 2 * f * 2);
+  w.gate_up = off;  // (unused: SwiGLU is applied in the gate/up GEMM's epilogue)
   w.act = take(tokens * f * 2);
   const int splits = max_batch ? pd::decode_attention_splits(1, c.n_kv_heads, max_kv_len) : 1;  // worst case: B = 1
   w.partial = take(max_batch * c.n_kv_heads * static_cast<size_t>(splits) * (c.n_q_heads / c.n_kv_heads) *
@@ -67,14 +67,12 @@ pd_status mlp_half(pd_layer* L, const bf16* h, bf16* out, int tokens, uint8_t* w
                    cudaStream_t st) {
   const pd_layer_cfg& c = L->cfg;
   bf16* norm = reinterpret_cast<bf16*>(ws + w.norm);
-  bf16* gu = reinterpret_cast<bf16*>(ws + w.gate_up);
   bf16* act = reinterpret_cast<bf16*>(ws + w.act);
   { pd::TraceScope ts(PD_K_RMSNORM, st); PD_TRY(pd::launch_rmsnorm(h, L->g_mlp, norm, tokens, c.d_model, c.rms_eps, st)); }
   pd::GemmArgs g{};
-  g.a = norm; g.b = L->w_gu; g.c = gu; g.m = tokens; g.n = 2 * c.d_ff; g.k = c.d_model;
-  g.lda = c.d_model; g.ldb = c.d_model; g.ldc = 2 * c.d_ff; g.epilogue = pd::EPI_STORE; g.err_word = L->err_word;
+  g.a = norm; g.b = L->w_gu; g.c = act; g.m = tokens; g.n = 2 * c.d_ff; g.k = c.d_model;
+  g.lda = c.d_model; g.ldb = c.d_model; g.ldc = c.d_ff; g.epilogue = pd::EPI_SWIGLU; g.err_word = L->err_word;
   { pd::TraceScope ts(PD_K_GEMM_GATE_UP, st); PD_TRY(pd::gemm(g, st)); }
-  { pd::TraceScope ts(PD_K_SWIGLU, st); PD_TRY(pd::launch_swiglu(gu, act, tokens, c.d_ff, st)); }
   pd::GemmArgs g2{};
   g2.a = act; g2.b = L->w_down; g2.c = out; g2.r = h; g2.m = tokens; g2.n = c.d_model; g2.k = c.d_ff;
   g2.lda = c.d_ff; g2.ldb = c.d_ff; g2.ldc = c.d_model; g2.ldr = c.d_model; g2.epilogue = pd::EPI_RESIDUAL;
@@ -84,7 +82,7 @@ pd_status mlp_half(pd_layer* L, const bf16* h, bf16* out, int tokens, uint8_t* w
 }
 
 // Attention-input half shared by both modes: x -> qkv (q rotated in place, k/v written to the cache).
-pd_status qkv_half(pd_layer* L, const bf16* x, int tokens, const pd::RopeArgs& rope_in, uint8_t* ws,
+pd_status qkv_half(pd_layer* L, const bf16* x, int tokens, const pd::RopeEpilogue& rope, uint8_t* ws,
                    const Workspace& w, cudaStream_t st) {
   const pd_layer_cfg& c = L->cfg;
   bf16* norm = reinterpret_cast<bf16*>(ws + w.norm);
@@ -92,11 +90,9 @@ pd_status qkv_half(pd_layer* L, const bf16* x, int tokens, const pd::RopeArgs& r
   { pd::TraceScope ts(PD_K_RMSNORM, st); PD_TRY(pd::launch_rmsnorm(x, L->g_attn, norm, tokens, c.d_model, c.rms_eps, st)); }
   pd::GemmArgs g{};
   g.a = norm; g.b = L->w_qkv; g.c = qkv; g.m = tokens; g.n = L->n_qkv; g.k = c.d_model;
-  g.lda = c.d_model; g.ldb = c.d_model; g.ldc = L->n_qkv; g.epilogue = pd::EPI_STORE; g.err_word = L->err_word;
+  g.lda = c.d_model; g.ldb = c.d_model; g.ldc = L->n_qkv; g.epilogue = pd::EPI_ROPE_KV; g.rope = &rope;
+  g.err_word = L->err_word;
   { pd::TraceScope ts(PD_K_GEMM_QKV, st); PD_TRY(pd::gemm(g, st)); }
-  pd::RopeArgs r = rope_in;
-  r.qkv = qkv;
-  { pd::TraceScope ts(PD_K_ROPE_KV, st); PD_TRY(pd::launch_rope_scatter(r, st)); }
   return PD_OK;
 }
 
@@ -133,11 +129,11 @@ pd_status prefill_impl(pd_layer* L, const bf16* x, bf16* out, const int32_t* cu_
                        int max_len, const int32_t* slots_dev, const pd_kv_cache* cache, uint8_t* ws,
                        const Workspace& w, cudaStream_t st) {
   const pd_layer_cfg& c = L->cfg;
-  pd::RopeArgs r{};
+  pd::RopeEpilogue r{};
   r.k_cache = static_cast<bf16*>(cache->k); r.v_cache = static_cast<bf16*>(cache->v); r.rope_tab = L->rope_tab;
-  r.cu_seqlens = cu_dev; r.slots = slots_dev; r.kv_len = nullptr; r.n_req = n_req; r.n_tokens = tokens;
+  r.cu_seqlens = cu_dev; r.slots = slots_dev; r.kv_len = nullptr; r.n_req = n_req;
   r.n_q_heads = c.n_q_heads; r.n_kv_heads = c.n_kv_heads; r.head_dim = c.head_dim; r.len_cap = cache->len_cap;
-  r.max_pos = c.max_pos; r.batch_cap = cache->batch_cap; r.err_word = L->err_word;
+  r.max_pos = c.max_pos; r.batch_cap = cache->batch_cap;
   PD_TRY(qkv_half(L, x, tokens, r, ws, w, st));
   pd::PrefillAttnArgs a{};
   a.q = reinterpret_cast<bf16*>(ws + w.qkv); a.ldq = L->n_qkv;
@@ -155,11 +151,11 @@ pd_status prefill_impl(pd_layer* L, const bf16* x, bf16* out, const int32_t* cu_
 pd_status decode_impl(pd_layer* L, const bf16* x, bf16* out, const int32_t* kv_len_dev, int B, int max_kv_len,
                       const pd_kv_cache* cache, uint8_t* ws, const Workspace& w, cudaStream_t st) {
   const pd_layer_cfg& c = L->cfg;
-  pd::RopeArgs r{};
+  pd::RopeEpilogue r{};
   r.k_cache = static_cast<bf16*>(cache->k); r.v_cache = static_cast<bf16*>(cache->v); r.rope_tab = L->rope_tab;
-  r.cu_seqlens = nullptr; r.slots = nullptr; r.kv_len = kv_len_dev; r.n_req = B; r.n_tokens = B;
+  r.cu_seqlens = nullptr; r.slots = nullptr; r.kv_len = kv_len_dev; r.n_req = B;
   r.n_q_heads = c.n_q_heads; r.n_kv_heads = c.n_kv_heads; r.head_dim = c.head_dim; r.len_cap = cache->len_cap;
-  r.max_pos = c.max_pos; r.batch_cap = cache->batch_cap; r.err_word = L->err_word;
+  r.max_pos = c.max_pos; r.batch_cap = cache->batch_cap;
   PD_TRY(qkv_half(L, x, B, r, ws, w, st));
   pd::DecodeAttnArgs a{};
   a.q = reinterpret_cast<bf16*>(ws + w.qkv); a.ldq = L->n_qkv;
@@ -220,9 +216,11 @@ extern "C" pd_status pd_layer_create(const pd_layer_cfg* cfg, const pd_layer_wei
   const cudaMemcpyKind d2d = cudaMemcpyDeviceToDevice;
   if ((e = cudaMemcpyAsync(L->w_qkv, w->w_qkv, L->n_qkv * d * 2, d2d, st)) != cudaSuccess) return fail(e);
   if ((e = cudaMemcpyAsync(L->w_o, w->w_o, d * hq * 2, d2d, st)) != cudaSuccess) return fail(e);
-  // gate rows first, then up rows, so one GEMM produces both halves of the SwiGLU input
-  if ((e = cudaMemcpyAsync(L->w_gu, w->w_gate, f * d * 2, d2d, st)) != cudaSuccess) return fail(e);
-  if ((e = cudaMemcpyAsync(L->w_gu + f * d, w->w_up, f * d * 2, d2d, st)) != cudaSuccess) return fail(e);
+  // 64 gate rows, the matching 64 up rows, and so on: a GEMM tile then holds both halves of its SwiGLU outputs
+  if ((e = cudaMemcpy2DAsync(L->w_gu, 128 * d * 2, w->w_gate, 64 * d * 2, 64 * d * 2, f / 64, d2d, st)) != cudaSuccess)
+    return fail(e);
+  if ((e = cudaMemcpy2DAsync(L->w_gu + 64 * d, 128 * d * 2, w->w_up, 64 * d * 2, 64 * d * 2, f / 64, d2d, st)) != cudaSuccess)
+    return fail(e);
   if ((e = cudaMemcpyAsync(L->w_down, w->w_down, d * f * 2, d2d, st)) != cudaSuccess) return fail(e);
   if ((e = cudaMemcpyAsync(L->g_attn, w->g_attn, d * 2, d2d, st)) != cudaSuccess) return fail(e);
   if ((e = cudaMemcpyAsync(L->g_mlp, w->g_mlp, d * 2, d2d, st)) != cudaSuccess) return fail(e);
@@ -295,6 +293,44 @@ extern "C" pd_status pd_decode_layer(pd_layer* L, const void* x, void* out, cons
   if (reinterpret_cast<uintptr_t>(workspace) & 255u) return PD_ERR_INVALID_ARG;
   return decode_impl(L, static_cast<const bf16*>(x), static_cast<bf16*>(out), kv_len_dev, B, max_kv_len, cache,
                      static_cast<uint8_t*>(workspace), w, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" pd_status pd_decode_attention_workspace_bytes(const pd_layer_cfg* cfg, int32_t B, int32_t max_kv_len,
+                                                         size_t* out_bytes) {
+  PD_TRY(check_cfg(cfg));
+  if (!out_bytes || B < 0 || max_kv_len < 0) return PD_ERR_INVALID_ARG;
+  const int splits = B ? pd::decode_attention_splits(B, cfg->n_kv_heads, max_kv_len) : 1;
+  *out_bytes = pd::align_up(static_cast<size_t>(B) * cfg->n_kv_heads * splits * (cfg->n_q_heads / cfg->n_kv_heads) *
+                                (cfg->head_dim + 2) * 4, 256);
+  return PD_OK;
+}
+
+extern "C" pd_status pd_decode_attention(const pd_layer_cfg* cfg, const void* q, int32_t ldq, void* out,
+                                         const int32_t* kv_len_dev, int32_t B, int32_t max_kv_len,
+                                         const pd_kv_cache* cache, void* workspace, size_t workspace_bytes,
+                                         void* stream) {
+  PD_TRY(check_cfg(cfg));
+  if (B < 0) return PD_ERR_INVALID_ARG;
+  if (B == 0) return PD_OK;
+  PD_TRY(check_cache(nullptr, cache));
+  if (!q || !out || !kv_len_dev || ldq < cfg->n_q_heads * cfg->head_dim || ldq % 8 != 0) return PD_ERR_INVALID_ARG;
+  if (B > cache->batch_cap || max_kv_len <= 0 || max_kv_len > cache->len_cap) return PD_ERR_INVALID_ARG;
+  size_t need = 0;
+  PD_TRY(pd_decode_attention_workspace_bytes(cfg, B, max_kv_len, &need));
+  pd::DecodeAttnArgs a{};
+  a.n_splits = pd::decode_attention_splits(B, cfg->n_kv_heads, max_kv_len);
+  if (a.n_splits > 1) {
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return PD_ERR_INVALID_ARG;
+    if (workspace_bytes < need) return PD_ERR_WORKSPACE_TOO_SMALL;
+  }
+  a.q = static_cast<const bf16*>(q); a.ldq = ldq;
+  a.k_cache = static_cast<const bf16*>(cache->k); a.v_cache = static_cast<const bf16*>(cache->v);
+  a.o = static_cast<bf16*>(out); a.kv_len = kv_len_dev; a.partial = static_cast<float*>(workspace);
+  a.batch = B; a.max_kv_len = max_kv_len;
+  a.n_q_heads = cfg->n_q_heads; a.n_kv_heads = cfg->n_kv_heads; a.head_dim = cfg->head_dim; a.len_cap = cache->len_cap;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  pd::TraceScope ts(PD_K_ATTN_DECODE, st);
+  return pd::launch_decode_attention(a, st);
 }
 
 extern "C" pd_status pd_prefill_stack(pd_layer* const* layers, const pd_kv_cache* caches, int32_t n_layers,
