@@ -133,6 +133,34 @@ pd_status pd_decode_attention(const pd_layer_cfg* cfg, const void* q, int32_t ld
                               const int32_t* kv_len_dev, int32_t B, int32_t max_kv_len, const pd_kv_cache* cache,
                               void* workspace, size_t workspace_bytes, void* stream);
 
+/* pd_decode_attention for callers that may not allocate device memory.  (The paper has no
+ * counterpart of this call; it exists for the library's users.)
+ *
+ * Who needs it: a process whose own memory pool already owns the device, code that runs while
+ * a stream is being captured, or a latency-critical loop that must stay out of the CUDA
+ * allocator.  Such a caller cannot cudaMalloc the scratch that pd_decode_attention wants for
+ * the partial results of its KV-range splits.  Here that scratch is a fixed array of
+ * PD_NOALLOC_SCRATCH_BYTES inside the library image: every GPU that loads the library holds
+ * it from load until the process exits, used or not.  The call itself performs no cudaMalloc,
+ * cudaFree or other allocating routine.
+ *
+ * Arguments and results are those of pd_decode_attention without the workspace pair.
+ * Limits and rules:
+ *   - B * n_q_heads * splits * (head_dim + 2) * 4 bytes must fit the array (splits is chosen
+ *     from B, n_kv_heads and max_kv_len as in pd_decode_attention; batches large enough to
+ *     need no split always fit).  Otherwise the call returns PD_ERR_WORKSPACE_TOO_SMALL and
+ *     launches nothing.
+ *   - The first call on each device looks up the array's device address (that device must be
+ *     current); make this first call before any stream capture begins.
+ *   - All calls on a device share the one array.  It still holds the previous call's partials
+ *     when a call starts; nothing has to be cleared because each call overwrites every entry
+ *     it later reads.  Two calls whose kernels can overlap on the GPU (different streams,
+ *     different host threads) race on it: serialise them on one stream. */
+#define PD_NOALLOC_SCRATCH_BYTES (8u << 20)
+pd_status pd_decode_attention_noalloc(const pd_layer_cfg* cfg, const void* q, int32_t ldq, void* out,
+                                      const int32_t* kv_len_dev, int32_t B, int32_t max_kv_len,
+                                      const pd_kv_cache* cache, void* stream);
+
 /* The same two modes over a stack of n_layers layers run back to back (layer i+1 reads layer
  * i's output), layer i using caches[i % n_caches].  With io_on_host = 0, x/out/cu_seqlens_dev/
  * kv_len are device pointers and the call only enqueues work.  With io_on_host = 1 they are

@@ -35,6 +35,7 @@ EXPORTS = [
     "pd_workspace_bytes", "pd_prefill_layer", "pd_decode_layer", "pd_prefill_stack", "pd_decode_stack",
     "pd_layer_check", "pd_gemm_bf16", "pd_measure", "pd_allocate", "pd_queue_replay",
     "pd_launch_count", "pd_trace_begin", "pd_trace_end", "pd_decode_attention", "pd_decode_attention_workspace_bytes",
+    "pd_decode_attention_noalloc",
 ]
 
 TRACE_CLASSES = ["gemm_qkv", "gemm_o", "gemm_gate_up", "gemm_down", "attn_prefill", "attn_decode", "rmsnorm"]
@@ -129,6 +130,8 @@ _lib.pd_decode_attention_workspace_bytes.argtypes = [C.POINTER(pd_layer_cfg), C.
                                                      C.POINTER(C.c_size_t)]
 _lib.pd_decode_attention.argtypes = [C.POINTER(pd_layer_cfg), _P, C.c_int32, _P, _P, C.c_int32, C.c_int32,
                                      C.POINTER(pd_kv_cache), _P, C.c_size_t, _P]
+_lib.pd_decode_attention_noalloc.argtypes = [C.POINTER(pd_layer_cfg), _P, C.c_int32, _P, _P, C.c_int32, C.c_int32,
+                                             C.POINTER(pd_kv_cache), _P]
 _lib.pd_launch_count.restype = C.c_int64
 _lib.pd_trace_end.argtypes = [C.POINTER(pd_trace_report)]
 for _n in EXPORTS:
@@ -270,6 +273,20 @@ def pd_decode_attention(cfg: LayerConfig, q, ldq: int, out, kv_len_dev, batch: i
     _check(_lib.pd_decode_attention(C.byref(cfg.c_struct()), _ptr(q), ldq, _ptr(out), _ptr(kv_len_dev), batch,
                                     max_kv_len, C.byref(cache), _ptr(workspace), workspace_bytes,
                                     _stream_ptr(stream)), "pd_decode_attention")
+
+
+NOALLOC_SCRATCH_BYTES = 8 << 20
+
+
+def pd_decode_attention_noalloc(cfg: LayerConfig, q, ldq: int, out, kv_len_dev, batch: int, max_kv_len: int,
+                                cache: pd_kv_cache, stream=None):
+    """pd_decode_attention without a workspace argument, for callers that must not allocate
+    device memory: the split partials live in a fixed NOALLOC_SCRATCH_BYTES array inside the
+    library.  Raises PdError(PD_ERR_WORKSPACE_TOO_SMALL) when the problem does not fit it.
+    Calls on one device share that array, so keep them on one stream."""
+    _check(_lib.pd_decode_attention_noalloc(C.byref(cfg.c_struct()), _ptr(q), ldq, _ptr(out), _ptr(kv_len_dev),
+                                            batch, max_kv_len, C.byref(cache), _stream_ptr(stream)),
+           "pd_decode_attention_noalloc")
 
 
 def _layer_array(layers):
