@@ -163,6 +163,8 @@ def main():
     ap.add_argument("--decode-steps", type=int, default=8, help="decode steps per benchmark step")
     ap.add_argument("--layers", type=int, default=N_LAYERS, help="layers actually run (times are scaled to 32)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--skip-sweep", action="store_true",
+                    help="profiling aid: skip the TPOT(B) sweep and decode at the largest batch")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -242,7 +244,7 @@ def main():
     # ---- TPOT(B) curve, measured once (not part of the timed steps)
     sweep_t = [0, L_OUT // 2, L_OUT - 1]
     curve = {}
-    for b in SWEEP:
+    for b in ([] if args.skip_sweep else SWEEP):
         per_t = []
         for t in sweep_t:
             decode_pass(b, t)
@@ -266,6 +268,8 @@ def main():
     e1.record()
     e1.synchronize()
     tp_max_probe = L_IN / (e0.elapsed_time(e1) * 1e-3 * scale)
+    if args.skip_sweep:
+        curve = {b_max: TPOT_SLO}
     alloc = pd.pd_allocate(TP_TOTAL, L_IN, L_OUT, TTFT_SLO, TPOT_SLO, tp_max_probe, list(curve), list(curve.values()))
     b_star = alloc["feasible_batch"] or SWEEP[0]
     dec_ts = [int(round(i * (L_OUT - 1) / max(1, args.decode_steps - 1))) for i in range(args.decode_steps)]
@@ -378,7 +382,7 @@ def main():
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        sample_l = 2048
+        sample_l = L_IN
         dt, threads = oracle_prefill_sample(sample_l)
         cpu = {"value": sample_l / (dt * N_LAYERS), "unit": "tok/s", "cores": threads, "kind": "oracle",
                "sample": f"prefill of {sample_l} tokens through 1 layer ({dt:.1f} s), scaled to {N_LAYERS} layers"}
