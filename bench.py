@@ -165,6 +165,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--skip-sweep", action="store_true",
                     help="profiling aid: skip the TPOT(B) sweep and decode at the largest batch")
+    ap.add_argument("--decode-batch", type=int, default=0,
+                    help="profiling aid: decode at this batch instead of the TPOT-feasible one")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -272,6 +274,8 @@ def main():
         curve = {b_max: TPOT_SLO}
     alloc = pd.pd_allocate(TP_TOTAL, L_IN, L_OUT, TTFT_SLO, TPOT_SLO, tp_max_probe, list(curve), list(curve.values()))
     b_star = alloc["feasible_batch"] or SWEEP[0]
+    if args.decode_batch:
+        b_star = min(b_max, args.decode_batch)
     dec_ts = [int(round(i * (L_OUT - 1) / max(1, args.decode_steps - 1))) for i in range(args.decode_steps)]
 
     rng = np.random.Generator(np.random.Philox(key=99))

@@ -90,6 +90,25 @@ pd_status gemm(const GemmArgs& g, cudaStream_t stream);
 // Tile width (rows of B per tile) the GEMM will use for this problem.
 int gemm_block_n(int m, int n, int epilogue);
 
+// Decode-mode projection: acc[B, N] (fp32) = X[B, K] * W[N, K]^T, weight-streaming, K split over
+// blocks (the buffer is zeroed and accumulated with atomics when it is split).
+struct SkinnyGemmArgs {
+  const bf16* x;  // [B, K], row pitch ldx
+  const bf16* w;  // [N, K] contiguous
+  float* acc;     // [B, N]
+  int batch, n, k, ldx;
+  int* err_word;
+};
+pd_status gemm_skinny(const SkinnyGemmArgs& g, cudaStream_t stream);
+// Row-wise kernels that turn the fp32 sums into the layer's stored tensors.
+pd_status launch_skinny_rope_kv(const float* acc, bf16* qkv, const RopeEpilogue& rp, int batch, int* err_word,
+                                cudaStream_t s);
+// h = x + acc; if n != NULL also n = RMSNorm(h) * gain.
+pd_status launch_skinny_residual(const float* acc, const bf16* x, bf16* h, const bf16* gain, bf16* n, int batch, int d,
+                                 float eps, cudaStream_t s);
+// out[B, F] = silu(gate) * up from acc[B, 2F] whose columns follow the 64/64 interleaved weight rows.
+pd_status launch_skinny_swiglu(const float* acc, bf16* out, int batch, int f, cudaStream_t s);
+
 // ------------------------------------------------------------ elementwise
 pd_status launch_rmsnorm(const bf16* x, const bf16* gain, bf16* y, int rows, int d, float eps, cudaStream_t s);
 

@@ -75,6 +75,7 @@ struct GemmDev {
   int m, n, k;
   int ldc, ldr;
   int tiles_m, tiles_n;
+  int raster_group;  // row tiles that share the column-tile sweep (their A slab stays in L2)
   int* err_word;
   RopeEpilogue rope;  // EPI_ROPE_KV only
 };
@@ -88,10 +89,9 @@ __device__ __forceinline__ uint4 pack8(const float (&f)[8]) {
   return o;
 }
 
-__device__ __forceinline__ void tile_coords(int tile, int tiles_m, int tiles_n, int& tm, int& tn) {
-  // Groups of up to 8 row-tiles share the same column-tiles while they are resident, so
-  // concurrently running blocks hit the same A and B tiles in L2.
-  constexpr int GROUP = 8;
+__device__ __forceinline__ void tile_coords(int tile, int tiles_m, int tiles_n, int GROUP, int& tm, int& tn) {
+  // Groups of row-tiles sweep the column-tiles together, so concurrently running blocks hit the
+  // same A and B tiles in L2 and B is streamed from HBM once per group.
   const int per_group = GROUP * tiles_n;
   const int g = tile / per_group;
   const int first_m = g * GROUP;
@@ -157,7 +157,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       bool ok = true;
       for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
         int tm, tn;
-        tile_coords(tile, p.tiles_m, p.tiles_n, tm, tn);
+        tile_coords(tile, p.tiles_m, p.tiles_n, p.raster_group, tm, tn);
         for (int kb = 0; kb < k_blocks; ++kb) {
           if (!ptx::mbar_wait_bounded(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
           const uint32_t sa = smem_base + stage * Cfg::STAGE_BYTES;
@@ -214,7 +214,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     bool ok = true;
     for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
       int tm, tn;
-      tile_coords(tile, p.tiles_m, p.tiles_n, tm, tn);
+      tile_coords(tile, p.tiles_m, p.tiles_n, p.raster_group, tm, tn);
       // warp-uniform outcome: tcgen05.ld below needs the whole warp
       ok = __all_sync(0xffffffffu, ptx::mbar_wait_bounded(accf_bar(acc), acc_phase, abort_flag));
       if (!ok) break;
@@ -391,6 +391,11 @@ pd_status launch_tc(const GemmArgs& g, cudaStream_t stream) {
   p.tiles_m = (g.m + BM - 1) / BM;
   p.tiles_n = (g.n + BN - 1) / BN;
   p.err_word = g.err_word;
+  {
+    // keep a group's A slab (group x 128 rows x K) within about 40 MB of L2
+    long long grp = (40ll << 20) / (static_cast<long long>(BM) * g.k * 2);
+    p.raster_group = static_cast<int>(grp < 4 ? 4 : (grp > 32 ? 32 : grp));
+  }
   if (EPI == EPI_ROPE_KV) p.rope = *g.rope;
   const int tiles = p.tiles_m * p.tiles_n;
   const int grid = tiles < sm_count() ? tiles : sm_count();
@@ -417,9 +422,11 @@ pd_status launch_tc_epi(const GemmArgs& g, cudaStream_t stream) {
 }  // namespace
 
 int gemm_block_n(int m, int n, int epilogue) {
-  // Pick the tile width by a small cost model: waves over the SMs times a per-tile time that
-  // grows with the width plus a fixed part for the A operand.  The fused epilogues need whole
-  // heads / gate-up pairs in a tile, so they do not use the 64-wide tile.
+  // Pick the tile width by a small cost model: waves over the SMs times a measured relative
+  // per-tile time.  Narrow tiles re-read A from shared memory for fewer columns and keep the
+  // tensor pipe only about 55 % busy against 85 % for the 256-wide tile, so they pay off only
+  // when they remove a mostly idle wave.  The fused epilogues need whole heads / gate-up pairs
+  // in a tile, so they do not use the 64-wide tile.
   const int sms = sm_count();
   const int tiles_m = (m + BM - 1) / BM;
   const bool fused = epilogue == EPI_SWIGLU || epilogue == EPI_ROPE_KV;
@@ -431,7 +438,7 @@ int gemm_block_n(int m, int n, int epilogue) {
     if (bn > n && bn != (fused ? 128 : 64)) continue;
     const long long tiles = 1ll * tiles_m * ((n + bn - 1) / bn);
     const long long waves = (tiles + sms - 1) / sms;
-    const double cost = static_cast<double>(waves) * (bn + 32.0);
+    const double cost = static_cast<double>(waves) * (bn == 256 ? 1.0 : (bn == 128 ? 0.77 : 0.47));
     if (cost < best_cost) { best_cost = cost; best = bn; }
   }
   return best;

@@ -1,0 +1,369 @@
+// Decode-mode projections: Y[B, N] = X[B, K] * W[N, K]^T for a small batch B.
+//
+// With one token per sequence the projections stream every weight once per step and are
+// HBM-bound, so the job is to keep all SMs loading weights.  The roles of the operands are
+// swapped with respect to the prefill GEMM: a tile is 128 weight rows (the M side of
+// tcgen05.mma, so no tensor-core rows are wasted on padding) by the whole batch (the N side,
+// rounded up to 16/32/64/128/256), and the K range is split across blocks until there are
+// about two blocks per SM.  A block accumulates its K slice in tensor memory and adds it into
+// an fp32 [B, N] buffer (red.global.add, L2-resident; plain stores when K is not split).
+// Small row-wise kernels then apply the layer's fused operations to the fp32 sums: RoPE and the
+// KV-cache append, residual add with the following RMSNorm, SwiGLU, residual add.
+#include "pd_common.cuh"
+#include "pd_ptx.cuh"
+
+namespace pd {
+namespace {
+
+constexpr int SK_BM = 128;  // weight rows per tile
+constexpr int SK_BK = 64;
+constexpr int SK_THREADS = 192;
+
+template <int BNB>
+struct SkinnyCfg {
+  static constexpr int W_BYTES = SK_BM * SK_BK * 2;
+  static constexpr int X_BYTES = BNB * SK_BK * 2;
+  static constexpr int STAGE_BYTES = W_BYTES + ((X_BYTES + 1023) / 1024) * 1024;  // keep tiles 1024-byte aligned
+  static constexpr int STAGES = (BNB >= 256) ? 2 : (BNB >= 128 ? 3 : 4);
+  static constexpr int TMEM_COLS = BNB < 32 ? 32 : BNB;
+  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 128;
+};
+
+struct SkinnyDev {
+  float* acc;  // [B, N] fp32
+  int batch, n, k_blocks, splits, tiles_n;
+  int* err_word;
+};
+
+template <int BNB>
+__global__ void __launch_bounds__(SK_THREADS)
+gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_x, SkinnyDev p) {
+  using Cfg = SkinnyCfg<BNB>;
+  constexpr int STAGES = Cfg::STAGES;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem_al = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem_al + STAGES * Cfg::STAGE_BYTES);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 1);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t bar0 = ptx::smem_u32(bars);
+  auto full_bar = [&](int s) { return bar0 + 8u * s; };
+  auto empty_bar = [&](int s) { return bar0 + 8u * (STAGES + s); };
+  const uint32_t acc_bar = bar0 + 8u * (2 * STAGES);
+
+  // work unit: (batch tile, weight-row tile, K slice)
+  int unit = blockIdx.x;
+  const int split = unit % p.splits;
+  unit /= p.splits;
+  const int tn = unit % p.tiles_n;
+  const int tb = unit / p.tiles_n;
+  const int kb0 = static_cast<int>(static_cast<long long>(p.k_blocks) * split / p.splits);
+  const int kb1 = static_cast<int>(static_cast<long long>(p.k_blocks) * (split + 1) / p.splits);
+
+  if (threadIdx.x == 0) {
+    *abort_flag = 0;
+    for (int s = 0; s < STAGES; ++s) {
+      ptx::mbar_init(full_bar(s), 1);
+      ptx::mbar_init(empty_bar(s), 1);
+    }
+    ptx::mbar_init(acc_bar, 1);
+    ptx::fence_barrier_init();
+    ptx::prefetch_tensormap(&tmap_w);
+    ptx::prefetch_tensormap(&tmap_x);
+  }
+  if (warp == 1) {
+    ptx::tmem_alloc(ptx::smem_u32(tmem_slot), Cfg::TMEM_COLS);
+    ptx::tmem_relinquish();
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int kb = kb0; kb < kb1; ++kb) {
+        if (!ptx::mbar_wait_bounded(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
+        const uint32_t sw = smem_base + stage * Cfg::STAGE_BYTES;
+        const uint32_t sx = sw + Cfg::W_BYTES;
+        ptx::mbar_arrive_expect_tx(full_bar(stage), Cfg::W_BYTES + Cfg::X_BYTES);
+        ptx::tma_load_2d(sw, &tmap_w, kb * SK_BK, tn * SK_BM, full_bar(stage));
+        ptx::tma_load_2d(sx, &tmap_x, kb * SK_BK, tb * BNB, full_bar(stage));
+        if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+      }
+      if (!ok) {
+        for (int i = 0; i < 2000; ++i) __nanosleep(1000);  // let loads in flight land before shared memory is released
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      constexpr uint32_t idesc = ptx::umma_idesc_bf16(SK_BM, BNB);
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int kb = kb0; kb < kb1; ++kb) {
+        if (!ptx::mbar_wait_bounded(full_bar(stage), phase, abort_flag)) { ok = false; break; }
+        ptx::tc_fence_after();
+        const uint32_t sw = smem_base + stage * Cfg::STAGE_BYTES;
+        const uint64_t dw = ptx::umma_desc_sw128(sw);
+        const uint64_t dx = ptx::umma_desc_sw128(sw + Cfg::W_BYTES);
+#pragma unroll
+        for (int kk = 0; kk < SK_BK / 16; ++kk)
+          ptx::umma_bf16(tmem_base, dw + 2u * kk, dx + 2u * kk, idesc, (kb > kb0 || kk > 0) ? 1u : 0u);
+        ptx::umma_commit(empty_bar(stage));
+        if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+      }
+      if (ok) ptx::umma_commit(acc_bar);
+    }
+  } else {
+    const int lane_group = warp & 3;
+    const bool ok = __all_sync(0xffffffffu, ptx::mbar_wait_bounded(acc_bar, 0u, abort_flag));
+    if (ok && kb1 > kb0) {
+      ptx::tc_fence_after();
+      const int n = tn * SK_BM + lane_group * 32 + lane;  // output feature of this thread
+      const uint32_t t_row = tmem_base + (static_cast<uint32_t>(lane_group * 32) << 16);
+      constexpr int CH = BNB < 32 ? BNB : 32;
+#pragma unroll 1
+      for (int c0 = 0; c0 < BNB; c0 += CH) {
+        uint32_t v[32];
+        if constexpr (CH == 32) ptx::tmem_ld_32x32(t_row + c0, v);
+        else ptx::tmem_ld_32x16(t_row + c0, v);
+        ptx::tmem_ld_wait();
+        if (n < p.n) {
+#pragma unroll
+          for (int j = 0; j < CH; ++j) {
+            const int b = tb * BNB + c0 + j;
+            if (b < p.batch) {
+              float* dst = p.acc + static_cast<size_t>(b) * p.n + n;  // a warp covers 32 consecutive floats of row b
+              if (p.splits > 1) atomicAdd(dst, __uint_as_float(v[j]));
+              else *dst = __uint_as_float(v[j]);
+            }
+          }
+        }
+      }
+    }
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  if (*abort_flag && threadIdx.x == 0 && p.err_word) atomicExch(p.err_word, 1);
+  if (warp == 1) {
+    __syncwarp();
+    ptx::tc_fence_after();
+    ptx::tmem_dealloc(tmem_base, Cfg::TMEM_COLS);
+  }
+}
+
+template <int BNB>
+pd_status launch_skinny(const SkinnyGemmArgs& g, cudaStream_t stream) {
+  using Cfg = SkinnyCfg<BNB>;
+  static bool attr_set = false;
+  auto kern = gemm_skinny_kernel<BNB>;
+  if (!attr_set) {
+    PD_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES));
+    attr_set = true;
+  }
+  CUtensorMap tw, tx;
+  PD_TRY(make_tmap_bf16(&tw, g.w, g.n, g.k, g.k, SK_BM));
+  PD_TRY(make_tmap_bf16(&tx, g.x, g.batch, g.k, g.ldx, BNB));
+  SkinnyDev p{};
+  p.acc = g.acc; p.batch = g.batch; p.n = g.n; p.k_blocks = g.k / SK_BK;
+  p.tiles_n = (g.n + SK_BM - 1) / SK_BM;
+  const int tiles_b = (g.batch + BNB - 1) / BNB;
+  // about two blocks per SM, each with at least 8 K-blocks
+  const int units = p.tiles_n * tiles_b;
+  int splits = (2 * 148 + units / 2) / units;
+  if (splits > p.k_blocks / 8) splits = p.k_blocks / 8;
+  if (splits < 1) splits = 1;
+  p.splits = splits;
+  p.err_word = g.err_word;
+  if (splits > 1) PD_CUDA_TRY(cudaMemsetAsync(g.acc, 0, static_cast<size_t>(g.batch) * g.n * sizeof(float), stream));
+  kern<<<units * splits, SK_THREADS, Cfg::SMEM_BYTES, stream>>>(tw, tx, p);
+  count_launch();
+  PD_CUDA_TRY(cudaGetLastError());
+  return PD_OK;
+}
+
+// ------------------------------------------------------------ row-wise epilogues
+__device__ __forceinline__ uint4 pack8(const float (&f)[8]) {
+  uint4 o;
+  o.x = ptx::pack_bf16(f[0], f[1]);
+  o.y = ptx::pack_bf16(f[2], f[3]);
+  o.z = ptx::pack_bf16(f[4], f[5]);
+  o.w = ptx::pack_bf16(f[6], f[7]);
+  return o;
+}
+__device__ __forceinline__ void unpack8(const uint4& v, float (&f)[8]) {
+  f[0] = ptx::bf16_lo(v.x); f[1] = ptx::bf16_hi(v.x);
+  f[2] = ptx::bf16_lo(v.y); f[3] = ptx::bf16_hi(v.y);
+  f[4] = ptx::bf16_lo(v.z); f[5] = ptx::bf16_hi(v.z);
+  f[6] = ptx::bf16_lo(v.w); f[7] = ptx::bf16_hi(v.w);
+}
+__device__ __forceinline__ void load8(const float* p, float (&f)[8]) {
+  const float4 a = *reinterpret_cast<const float4*>(p);
+  const float4 b = *reinterpret_cast<const float4*>(p + 4);
+  f[0] = a.x; f[1] = a.y; f[2] = a.z; f[3] = a.w; f[4] = b.x; f[5] = b.y; f[6] = b.z; f[7] = b.w;
+}
+
+// RoPE + KV append for one decode token per block: acc[b, Nqkv] -> q (bf16, in the qkv buffer), cache.
+__global__ void __launch_bounds__(128) skinny_rope_kv_kernel(const float* __restrict__ acc, bf16* qkv, RopeEpilogue rp,
+                                                             int* err_word) {
+  const int b = blockIdx.x;
+  const int pos = rp.kv_len[b], slot = b;
+  if (pos < 0 || pos >= rp.len_cap || pos >= rp.max_pos || slot >= rp.batch_cap) {
+    if (threadIdx.x == 0 && err_word) atomicExch(err_word, 2);
+    return;
+  }
+  const int hd = rp.head_dim, half = hd / 2, per_head = half / 8;
+  const int n_heads = rp.n_q_heads + 2 * rp.n_kv_heads;
+  const int n_qkv = n_heads * hd;
+  const float* row = acc + static_cast<size_t>(b) * n_qkv;
+  const float2* tab = rp.rope_tab + static_cast<size_t>(pos) * half;
+  for (int w = threadIdx.x; w < n_heads * per_head; w += blockDim.x) {
+    const int h = w / per_head, i0 = (w - h * per_head) * 8;
+    float lo[8], hi[8];
+    load8(row + h * hd + i0, lo);
+    load8(row + h * hd + half + i0, hi);
+    bf16* dst;
+    if (h < rp.n_q_heads) {
+      dst = qkv + static_cast<size_t>(b) * n_qkv + h * hd;
+    } else if (h < rp.n_q_heads + rp.n_kv_heads) {
+      dst = rp.k_cache + ((static_cast<size_t>(slot) * rp.n_kv_heads + (h - rp.n_q_heads)) * rp.len_cap + pos) * hd;
+    } else {
+      dst = rp.v_cache +
+            ((static_cast<size_t>(slot) * rp.n_kv_heads + (h - rp.n_q_heads - rp.n_kv_heads)) * rp.len_cap + pos) * hd;
+    }
+    if (h < rp.n_q_heads + rp.n_kv_heads) {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        const float2 cs = tab[i0 + e];
+        const float a = lo[e], c = hi[e];
+        lo[e] = a * cs.x - c * cs.y;
+        hi[e] = c * cs.x + a * cs.y;
+      }
+    }
+    *reinterpret_cast<uint4*>(dst + i0) = pack8(lo);
+    *reinterpret_cast<uint4*>(dst + half + i0) = pack8(hi);
+  }
+}
+
+// h = x + acc (stored bf16); optionally n = RMSNorm(h) * gain computed from the stored h.
+constexpr int RES_THREADS = 256;
+constexpr int RES_MAX_CHUNKS = 8;
+template <bool NORM>
+__global__ void __launch_bounds__(RES_THREADS) skinny_residual_kernel(const float* __restrict__ acc,
+                                                                       const bf16* __restrict__ x, bf16* h,
+                                                                       const bf16* __restrict__ gain, bf16* n, int d,
+                                                                       float eps) {
+  const int b = blockIdx.x;
+  const int chunks = d / 8;
+  uint4 hv[RES_MAX_CHUNKS];
+  float ss = 0.f;
+#pragma unroll
+  for (int i = 0; i < RES_MAX_CHUNKS; ++i) {
+    const int c = threadIdx.x + i * RES_THREADS;
+    if (c < chunks) {
+      float f[8], r[8];
+      load8(acc + static_cast<size_t>(b) * d + c * 8, f);
+      unpack8(*reinterpret_cast<const uint4*>(x + static_cast<size_t>(b) * d + c * 8), r);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) f[e] += r[e];
+      hv[i] = pack8(f);
+      *reinterpret_cast<uint4*>(h + static_cast<size_t>(b) * d + c * 8) = hv[i];
+      if (NORM) {
+        unpack8(hv[i], f);  // the norm sees the stored (rounded) residual stream
+#pragma unroll
+        for (int e = 0; e < 8; ++e) ss = fmaf(f[e], f[e], ss);
+      }
+    }
+  }
+  if constexpr (NORM) {
+  __shared__ float red[RES_THREADS / 32];
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+  __syncthreads();
+  float tot = 0.f;
+#pragma unroll
+  for (int w = 0; w < RES_THREADS / 32; ++w) tot += red[w];
+  const float scale = rsqrtf(tot / static_cast<float>(d) + eps);
+#pragma unroll
+  for (int i = 0; i < RES_MAX_CHUNKS; ++i) {
+    const int c = threadIdx.x + i * RES_THREADS;
+    if (c < chunks) {
+      float f[8], g[8];
+      unpack8(hv[i], f);
+      unpack8(reinterpret_cast<const uint4*>(gain)[c], g);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) f[e] = f[e] * scale * g[e];
+      *reinterpret_cast<uint4*>(n + static_cast<size_t>(b) * d + c * 8) = pack8(f);
+    }
+  }
+  }  // NORM
+}
+
+// a[b, f] = silu(gate) * up with the weight rows interleaved 64 gate / 64 up.
+__global__ void __launch_bounds__(256) skinny_swiglu_kernel(const float* __restrict__ acc, bf16* __restrict__ out,
+                                                             int rows, int f) {
+  const int chunks_per_row = f / 8;
+  const size_t total = static_cast<size_t>(rows) * chunks_per_row;
+  for (size_t idx = blockIdx.x * static_cast<size_t>(blockDim.x) + threadIdx.x; idx < total;
+       idx += static_cast<size_t>(gridDim.x) * blockDim.x) {
+    const size_t r = idx / chunks_per_row;
+    const int c = static_cast<int>(idx - r * chunks_per_row);
+    const int f0 = c * 8;
+    const float* base = acc + r * (2 * static_cast<size_t>(f)) + (f0 >> 6) * 128 + (f0 & 63);
+    float g[8], u[8];
+    load8(base, g);
+    load8(base + 64, u);
+#pragma unroll
+    for (int e = 0; e < 8; ++e) g[e] = g[e] / (1.f + __expf(-g[e])) * u[e];
+    *reinterpret_cast<uint4*>(out + r * f + f0) = pack8(g);
+  }
+}
+
+}  // namespace
+
+pd_status gemm_skinny(const SkinnyGemmArgs& g, cudaStream_t stream) {
+  if (!g.x || !g.w || !g.acc || g.batch <= 0 || g.n <= 0 || g.k <= 0) return PD_ERR_INVALID_ARG;
+  if (g.k % SK_BK != 0 || g.n % 4 != 0 || g.ldx % 8 != 0) return PD_ERR_UNSUPPORTED_SHAPE;
+  if (g.batch <= 16) return launch_skinny<16>(g, stream);
+  if (g.batch <= 32) return launch_skinny<32>(g, stream);
+  if (g.batch <= 64) return launch_skinny<64>(g, stream);
+  if (g.batch <= 128) return launch_skinny<128>(g, stream);
+  return launch_skinny<256>(g, stream);
+}
+
+pd_status launch_skinny_rope_kv(const float* acc, bf16* qkv, const RopeEpilogue& rp, int batch, int* err_word,
+                                cudaStream_t s) {
+  skinny_rope_kv_kernel<<<batch, 128, 0, s>>>(acc, qkv, rp, err_word);
+  count_launch();
+  PD_CUDA_TRY(cudaGetLastError());
+  return PD_OK;
+}
+
+pd_status launch_skinny_residual(const float* acc, const bf16* x, bf16* h, const bf16* gain, bf16* n, int batch, int d,
+                                 float eps, cudaStream_t s) {
+  if (d % 8 != 0 || d > RES_THREADS * RES_MAX_CHUNKS * 8) return PD_ERR_UNSUPPORTED_SHAPE;
+  if (n) skinny_residual_kernel<true><<<batch, RES_THREADS, 0, s>>>(acc, x, h, gain, n, d, eps);
+  else skinny_residual_kernel<false><<<batch, RES_THREADS, 0, s>>>(acc, x, h, nullptr, nullptr, d, eps);
+  count_launch();
+  PD_CUDA_TRY(cudaGetLastError());
+  return PD_OK;
+}
+
+pd_status launch_skinny_swiglu(const float* acc, bf16* out, int batch, int f, cudaStream_t s) {
+  const size_t total = static_cast<size_t>(batch) * (f / 8);
+  size_t blocks = (total + 255) / 256;
+  if (blocks > 148 * 8) blocks = 148 * 8;
+  skinny_swiglu_kernel<<<static_cast<unsigned>(blocks), 256, 0, s>>>(acc, out, batch, f);
+  count_launch();
+  PD_CUDA_TRY(cudaGetLastError());
+  return PD_OK;
+}
+
+}  // namespace pd

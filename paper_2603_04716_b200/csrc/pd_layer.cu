@@ -14,7 +14,7 @@ namespace {
 
 struct Workspace {
   // byte offsets into the caller's workspace
-  size_t norm, qkv, attn_o, resid, gate_up, act, partial, stage_a, stage_b, meta, total;
+  size_t norm, qkv, attn_o, resid, acc, act, partial, stage_a, stage_b, meta, total;
 };
 
 Workspace carve(const pd_layer_cfg& c, size_t tokens, size_t max_batch, int max_kv_len) {
@@ -31,8 +31,12 @@ Workspace carve(const pd_layer_cfg& c, size_t tokens, size_t max_batch, int max_
   w.qkv = take(tokens * nqkv * 2);
   w.attn_o = take(tokens * hq * 2);
   w.resid = take(tokens * d * 2);
-  w.gate_up = off;  // (unused: SwiGLU is applied in the gate/up GEMM's epilogue)
   w.act = take(tokens * f * 2);
+  {  // fp32 sums of the decode-mode projections: [batch, widest projection]
+    size_t widest = nqkv > 2 * f ? nqkv : 2 * f;
+    if (d > widest) widest = d;
+    w.acc = take(max_batch * widest * 4);
+  }
   const int splits = max_batch ? pd::decode_attention_splits(1, c.n_kv_heads, max_kv_len) : 1;  // worst case: B = 1
   w.partial = take(max_batch * c.n_kv_heads * static_cast<size_t>(splits) * (c.n_q_heads / c.n_kv_heads) *
                    (c.head_dim + 2) * 4);
@@ -151,22 +155,54 @@ pd_status prefill_impl(pd_layer* L, const bf16* x, bf16* out, const int32_t* cu_
 pd_status decode_impl(pd_layer* L, const bf16* x, bf16* out, const int32_t* kv_len_dev, int B, int max_kv_len,
                       const pd_kv_cache* cache, uint8_t* ws, const Workspace& w, cudaStream_t st) {
   const pd_layer_cfg& c = L->cfg;
+  const int hq = c.n_q_heads * c.head_dim;
+  bf16* norm = reinterpret_cast<bf16*>(ws + w.norm);
+  bf16* qkv = reinterpret_cast<bf16*>(ws + w.qkv);
+  bf16* attn_o = reinterpret_cast<bf16*>(ws + w.attn_o);
+  bf16* resid = reinterpret_cast<bf16*>(ws + w.resid);
+  bf16* act = reinterpret_cast<bf16*>(ws + w.act);
+  float* acc = reinterpret_cast<float*>(ws + w.acc);
   pd::RopeEpilogue r{};
   r.k_cache = static_cast<bf16*>(cache->k); r.v_cache = static_cast<bf16*>(cache->v); r.rope_tab = L->rope_tab;
   r.cu_seqlens = nullptr; r.slots = nullptr; r.kv_len = kv_len_dev; r.n_req = B;
   r.n_q_heads = c.n_q_heads; r.n_kv_heads = c.n_kv_heads; r.head_dim = c.head_dim; r.len_cap = cache->len_cap;
   r.max_pos = c.max_pos; r.batch_cap = cache->batch_cap;
-  PD_TRY(qkv_half(L, x, B, r, ws, w, st));
+
+  { pd::TraceScope ts(PD_K_RMSNORM, st); PD_TRY(pd::launch_rmsnorm(x, L->g_attn, norm, B, c.d_model, c.rms_eps, st)); }
+  pd::SkinnyGemmArgs g{};
+  g.acc = acc; g.batch = B; g.err_word = L->err_word;
+  {
+    pd::TraceScope ts(PD_K_GEMM_QKV, st);
+    g.x = norm; g.w = L->w_qkv; g.n = L->n_qkv; g.k = c.d_model; g.ldx = c.d_model;
+    PD_TRY(pd::gemm_skinny(g, st));
+    PD_TRY(pd::launch_skinny_rope_kv(acc, qkv, r, B, L->err_word, st));
+  }
   pd::DecodeAttnArgs a{};
-  a.q = reinterpret_cast<bf16*>(ws + w.qkv); a.ldq = L->n_qkv;
+  a.q = qkv; a.ldq = L->n_qkv;
   a.k_cache = static_cast<bf16*>(cache->k); a.v_cache = static_cast<bf16*>(cache->v);
-  a.o = reinterpret_cast<bf16*>(ws + w.attn_o); a.kv_len = kv_len_dev;
+  a.o = attn_o; a.kv_len = kv_len_dev;
   a.partial = reinterpret_cast<float*>(ws + w.partial);
   a.batch = B; a.max_kv_len = max_kv_len; a.n_splits = pd::decode_attention_splits(B, c.n_kv_heads, max_kv_len);
   a.n_q_heads = c.n_q_heads; a.n_kv_heads = c.n_kv_heads; a.head_dim = c.head_dim; a.len_cap = cache->len_cap;
   { pd::TraceScope ts(PD_K_ATTN_DECODE, st); PD_TRY(pd::launch_decode_attention(a, st)); }
-  PD_TRY(oproj(L, x, B, ws, w, st));
-  PD_TRY(mlp_half(L, reinterpret_cast<bf16*>(ws + w.resid), out, B, ws, w, st));
+  {
+    pd::TraceScope ts(PD_K_GEMM_O, st);  // h = x + o W_o^T and n2 = RMSNorm(h) in the same row-wise pass
+    g.x = attn_o; g.w = L->w_o; g.n = c.d_model; g.k = hq; g.ldx = hq;
+    PD_TRY(pd::gemm_skinny(g, st));
+    PD_TRY(pd::launch_skinny_residual(acc, x, resid, L->g_mlp, norm, B, c.d_model, c.rms_eps, st));
+  }
+  {
+    pd::TraceScope ts(PD_K_GEMM_GATE_UP, st);
+    g.x = norm; g.w = L->w_gu; g.n = 2 * c.d_ff; g.k = c.d_model; g.ldx = c.d_model;
+    PD_TRY(pd::gemm_skinny(g, st));
+    PD_TRY(pd::launch_skinny_swiglu(acc, act, B, c.d_ff, st));
+  }
+  {
+    pd::TraceScope ts(PD_K_GEMM_DOWN, st);
+    g.x = act; g.w = L->w_down; g.n = c.d_model; g.k = c.d_ff; g.ldx = c.d_ff;
+    PD_TRY(pd::gemm_skinny(g, st));
+    PD_TRY(pd::launch_skinny_residual(acc, resid, out, nullptr, nullptr, B, c.d_model, c.rms_eps, st));
+  }
   return PD_OK;
 }
 

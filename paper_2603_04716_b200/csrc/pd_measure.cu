@@ -250,8 +250,6 @@ extern "C" pd_status pd_measure(const pd_layer_cfg* cfg_in, const pd_measure_cfg
 
         // the attention kernel alone, over the same caches (q = whatever the last pass left in the workspace)
         pd::DecodeAttnArgs a{};
-        size_t ws_total = 0;
-        (void)ws_total;
         // reuse the library's own carving by running one decode layer first would be circular: place q, o and the
         // partials at the start of the workspace instead (the kernel only needs valid, finite inputs)
         const size_t q_bytes = pd::align_up(static_cast<size_t>(B) * stack.layers[0]->n_qkv * 2, 256);
