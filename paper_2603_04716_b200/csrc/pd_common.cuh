@@ -125,6 +125,8 @@ struct PrefillAttnArgs {
   int n_q_heads, n_kv_heads, head_dim, len_cap, batch_cap;
 };
 pd_status launch_prefill_attention(const PrefillAttnArgs& a, cudaStream_t s);
+// The same operation on tcgen05 / tensor memory (the product path).
+pd_status launch_prefill_attention_tc(const PrefillAttnArgs& a, int* err_word, cudaStream_t s);
 
 struct DecodeAttnArgs {
   const bf16* q;       // [B, ldq]
