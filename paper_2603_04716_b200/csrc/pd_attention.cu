@@ -1,16 +1,11 @@
-// Causal grouped-query attention.
+// Decode attention (the prefill kernel lives in pd_attn_prefill_tc.cu).
 //
-// Prefill: flash-style tiling, one block per (128 query rows, query head, request); K and V
-// tiles of 64 keys stream from the KV cache through a double-buffered cp.async ring; the
-// two contractions run on the tensor cores (warp-level mma, bf16 in, fp32 accumulate) with
-// an online softmax in registers.
-//
-// Decode: memory-bound.  One block per (split of the KV range, KV head, sequence).  The G
-// query heads of the group are the (zero-padded) 16 rows of the MMA, so each K/V row is
-// read from HBM once and used by all G heads.  Every warp streams its own 16-key tiles
-// through a private 3-stage cp.async ring (16-byte loads, no block-wide barrier in the
-// loop), keeps an online softmax per row with warp shuffles, and the warps' and splits'
-// partial (max, sum, output) triples are merged at the end.
+// Memory-bound.  One block per (split of the KV range, KV head, sequence).  The G query heads
+// of the group are the (zero-padded) 16 rows of a warp-level MMA, so each K/V row is read from
+// HBM once and used by all G heads.  Every warp streams its own 16-key tiles through a private
+// 3-stage cp.async ring (16-byte loads, no block-wide barrier in the loop), keeps an online
+// softmax per row with warp shuffles, and the warps' and splits' partial (max, sum, output)
+// triples are merged at the end.
 #include <math_constants.h>
 
 #include "pd_common.cuh"
@@ -26,183 +21,6 @@ constexpr float LOG2E = 1.4426950408889634f;
 template <int HD>
 __device__ __forceinline__ uint32_t tile_off(int r, int c) {
   return static_cast<uint32_t>(r * (HD * 2) + ((c ^ (r & 7)) << 4));
-}
-
-// ================================================================== prefill
-constexpr int PF_BM = 128;      // query rows per block
-constexpr int PF_BN = 64;       // keys per tile
-constexpr int PF_THREADS = 256;  // 8 warps x 16 rows
-
-template <int HD>
-__global__ void __launch_bounds__(PF_THREADS) prefill_attn_kernel(PrefillAttnArgs a) {
-  constexpr int CPR = HD / 8;  // 16-byte chunks per row
-  extern __shared__ __align__(128) uint8_t smem[];
-  const uint32_t s_q = ptx::smem_u32(smem);
-  const uint32_t s_k0 = s_q + PF_BM * HD * 2;
-  const uint32_t s_v0 = s_k0 + 2 * PF_BN * HD * 2;
-
-  const int h = blockIdx.x;
-  const int qt = gridDim.y - 1 - blockIdx.y;  // long (late) tiles first
-  const int req = blockIdx.z;
-  const int start = a.cu_seqlens[req];
-  const int len = a.cu_seqlens[req + 1] - start;
-  const int q0 = qt * PF_BM;
-  if (q0 >= len) return;
-  const int slot = a.slots ? a.slots[req] : req;
-  if (slot < 0 || slot >= a.batch_cap) return;  // reported by the RoPE/KV-write kernel
-  const int group = a.n_q_heads / a.n_kv_heads;
-  const int kvh = h / group;
-  const bf16* kbase = a.k_cache + (static_cast<size_t>(slot) * a.n_kv_heads + kvh) * a.len_cap * HD;
-  const bf16* vbase = a.v_cache + (static_cast<size_t>(slot) * a.n_kv_heads + kvh) * a.len_cap * HD;
-  const bf16* qbase = a.q + static_cast<size_t>(start) * a.ldq + h * HD;
-
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int g = lane >> 2, t4 = lane & 3;
-
-  // Q tile -> shared (rows beyond the request are zero-filled)
-  for (int i = tid; i < PF_BM * CPR; i += PF_THREADS) {
-    const int r = i / CPR, c = i - r * CPR;
-    const bool ok = (q0 + r) < len;
-    const bf16* src = qbase + static_cast<size_t>(ok ? q0 + r : 0) * a.ldq + c * 8;
-    ptx::cp_async_16(s_q + tile_off<HD>(r, c), src, ok);
-  }
-  const int kv_end = min(len, q0 + PF_BM);          // keys this block can see
-  const int n_kt = (kv_end + PF_BN - 1) / PF_BN;
-  auto load_kv = [&](int kt, int stage) {
-    const int k0 = kt * PF_BN;
-    const uint32_t sk = s_k0 + stage * (PF_BN * HD * 2);
-    const uint32_t sv = s_v0 + stage * (PF_BN * HD * 2);
-    for (int i = tid; i < PF_BN * CPR; i += PF_THREADS) {
-      const int r = i / CPR, c = i - r * CPR;
-      const bool ok = (k0 + r) < kv_end;
-      const size_t off = static_cast<size_t>(ok ? k0 + r : 0) * HD + c * 8;
-      ptx::cp_async_16(sk + tile_off<HD>(r, c), kbase + off, ok);
-      ptx::cp_async_16(sv + tile_off<HD>(r, c), vbase + off, ok);
-    }
-  };
-  load_kv(0, 0);
-  ptx::cp_async_commit();
-
-  float o_acc[HD / 8][4];
-#pragma unroll
-  for (int i = 0; i < HD / 8; ++i) o_acc[i][0] = o_acc[i][1] = o_acc[i][2] = o_acc[i][3] = 0.f;
-  float m_row[2] = {-CUDART_INF_F, -CUDART_INF_F};
-  float l_row[2] = {0.f, 0.f};
-  const float sl2 = rsqrtf(static_cast<float>(HD)) * LOG2E;  // scores are kept in log2 units
-  const int row_lo = q0 + warp * 16;                        // this warp's first query position
-  const int my_row[2] = {row_lo + g, row_lo + g + 8};
-
-  for (int kt = 0; kt < n_kt; ++kt) {
-    const int stage = kt & 1;
-    if (kt + 1 < n_kt) {
-      load_kv(kt + 1, stage ^ 1);
-      ptx::cp_async_commit();
-      ptx::cp_async_wait<1>();
-    } else {
-      ptx::cp_async_wait<0>();
-    }
-    __syncthreads();
-    const int k0 = kt * PF_BN;
-    // a warp whose last row precedes the tile's first key has nothing to do in this tile
-    if (k0 <= row_lo + 15) {
-      const uint32_t sk = s_k0 + stage * (PF_BN * HD * 2);
-      const uint32_t sv = s_v0 + stage * (PF_BN * HD * 2);
-      float s_acc[PF_BN / 8][4];
-#pragma unroll
-      for (int i = 0; i < PF_BN / 8; ++i) s_acc[i][0] = s_acc[i][1] = s_acc[i][2] = s_acc[i][3] = 0.f;
-#pragma unroll
-      for (int kk = 0; kk < HD / 16; ++kk) {
-        uint32_t qa[4];
-        ptx::ldmatrix_x4(s_q + tile_off<HD>(warp * 16 + (lane & 7) + ((lane >> 3) & 1) * 8, kk * 2 + (lane >> 4)),
-                         qa[0], qa[1], qa[2], qa[3]);
-#pragma unroll
-        for (int np = 0; np < PF_BN / 16; ++np) {
-          uint32_t b0, b1, b2, b3;
-          ptx::ldmatrix_x4(sk + tile_off<HD>(np * 16 + (lane & 7) + (lane >> 4) * 8, kk * 2 + ((lane >> 3) & 1)),
-                           b0, b1, b2, b3);
-          ptx::mma_bf16_16816(s_acc[2 * np], qa, b0, b1);
-          ptx::mma_bf16_16816(s_acc[2 * np + 1], qa, b2, b3);
-        }
-      }
-      // scale, causal mask (key position <= query position; keys beyond the request are masked too)
-      const bool need_mask = (k0 + PF_BN - 1 > row_lo) || (k0 + PF_BN > kv_end);
-      float tmax[2] = {-CUDART_INF_F, -CUDART_INF_F};
-#pragma unroll
-      for (int nt = 0; nt < PF_BN / 8; ++nt) {
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const int key = k0 + nt * 8 + t4 * 2 + (e & 1);
-          const int rr = e >> 1;
-          float v = s_acc[nt][e] * sl2;
-          if (need_mask && (key > my_row[rr] || key >= kv_end)) v = -CUDART_INF_F;
-          s_acc[nt][e] = v;
-          tmax[rr] = fmaxf(tmax[rr], v);
-        }
-      }
-      float corr[2];
-#pragma unroll
-      for (int rr = 0; rr < 2; ++rr) {
-        tmax[rr] = fmaxf(tmax[rr], __shfl_xor_sync(0xffffffffu, tmax[rr], 1));
-        tmax[rr] = fmaxf(tmax[rr], __shfl_xor_sync(0xffffffffu, tmax[rr], 2));
-        const float m_new = fmaxf(m_row[rr], tmax[rr]);
-        const float m_use = (m_new == -CUDART_INF_F) ? 0.f : m_new;
-        corr[rr] = exp2f(m_row[rr] - m_use);  // 0 when m_row is -inf
-        m_row[rr] = m_new;
-        tmax[rr] = m_use;
-      }
-      float psum[2] = {0.f, 0.f};
-      uint32_t pa[PF_BN / 16][4];
-#pragma unroll
-      for (int nt = 0; nt < PF_BN / 8; ++nt) {
-        const float p0 = exp2f(s_acc[nt][0] - tmax[0]);
-        const float p1 = exp2f(s_acc[nt][1] - tmax[0]);
-        const float p2 = exp2f(s_acc[nt][2] - tmax[1]);
-        const float p3 = exp2f(s_acc[nt][3] - tmax[1]);
-        psum[0] += p0 + p1;
-        psum[1] += p2 + p3;
-        pa[nt >> 1][(nt & 1) * 2 + 0] = ptx::pack_bf16(p0, p1);
-        pa[nt >> 1][(nt & 1) * 2 + 1] = ptx::pack_bf16(p2, p3);
-      }
-      l_row[0] = l_row[0] * corr[0] + psum[0];
-      l_row[1] = l_row[1] * corr[1] + psum[1];
-#pragma unroll
-      for (int i = 0; i < HD / 8; ++i) {
-        o_acc[i][0] *= corr[0]; o_acc[i][1] *= corr[0];
-        o_acc[i][2] *= corr[1]; o_acc[i][3] *= corr[1];
-      }
-#pragma unroll
-      for (int kk = 0; kk < PF_BN / 16; ++kk) {
-#pragma unroll
-        for (int np = 0; np < HD / 16; ++np) {
-          uint32_t b0, b1, b2, b3;
-          ptx::ldmatrix_x4_trans(sv + tile_off<HD>(kk * 16 + (lane & 7) + ((lane >> 3) & 1) * 8, np * 2 + (lane >> 4)),
-                                 b0, b1, b2, b3);
-          ptx::mma_bf16_16816(o_acc[2 * np], pa[kk], b0, b1);
-          ptx::mma_bf16_16816(o_acc[2 * np + 1], pa[kk], b2, b3);
-        }
-      }
-    }
-    __syncthreads();  // the stage is overwritten by the next iteration's loads
-  }
-
-  // finalise: divide by the row sums (summed over the four lanes that share a row) and store
-#pragma unroll
-  for (int rr = 0; rr < 2; ++rr) {
-    l_row[rr] += __shfl_xor_sync(0xffffffffu, l_row[rr], 1);
-    l_row[rr] += __shfl_xor_sync(0xffffffffu, l_row[rr], 2);
-  }
-#pragma unroll
-  for (int rr = 0; rr < 2; ++rr) {
-    if (my_row[rr] < len) {
-      const float inv = 1.f / l_row[rr];
-      bf16* dst = a.o + static_cast<size_t>(start + my_row[rr]) * (a.n_q_heads * HD) + h * HD + t4 * 2;
-#pragma unroll
-      for (int i = 0; i < HD / 8; ++i) {
-        *reinterpret_cast<uint32_t*>(dst + i * 8) =
-            ptx::pack_bf16(o_acc[i][rr * 2] * inv, o_acc[i][rr * 2 + 1] * inv);
-      }
-    }
-  }
 }
 
 // =================================================================== decode
@@ -438,21 +256,6 @@ __global__ void __launch_bounds__(HD) decode_combine_kernel(DecodeAttnArgs a) {
 }
 
 template <int HD>
-pd_status launch_prefill_hd(const PrefillAttnArgs& a, cudaStream_t s) {
-  constexpr int SMEM = (PF_BM + 4 * PF_BN) * HD * 2;
-  static bool attr_set = false;
-  if (!attr_set) {
-    PD_CUDA_TRY(cudaFuncSetAttribute(prefill_attn_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM));
-    attr_set = true;
-  }
-  dim3 grid(a.n_q_heads, (a.max_len + PF_BM - 1) / PF_BM, a.n_req);
-  prefill_attn_kernel<HD><<<grid, PF_THREADS, SMEM, s>>>(a);
-  count_launch();
-  PD_CUDA_TRY(cudaGetLastError());
-  return PD_OK;
-}
-
-template <int HD>
 pd_status launch_decode_hd(const DecodeAttnArgs& a, cudaStream_t s) {
   using SM = DecodeSmem<HD>;
   static bool attr_set = false;
@@ -474,13 +277,6 @@ pd_status launch_decode_hd(const DecodeAttnArgs& a, cudaStream_t s) {
 }
 
 }  // namespace
-
-pd_status launch_prefill_attention(const PrefillAttnArgs& a, cudaStream_t s) {
-  if (a.n_tokens == 0 || a.n_req == 0 || a.max_len == 0) return PD_OK;
-  if (a.head_dim == 128) return launch_prefill_hd<128>(a, s);
-  if (a.head_dim == 64) return launch_prefill_hd<64>(a, s);
-  return PD_ERR_UNSUPPORTED_SHAPE;
-}
 
 int decode_attention_splits(int batch, int n_kv_heads, int max_kv_len) {
   // Aim for a few blocks per SM; a split shorter than 256 keys is not worth its merge.

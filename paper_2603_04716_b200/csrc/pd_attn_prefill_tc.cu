@@ -210,26 +210,35 @@ prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
 #pragma unroll
       for (int c = 0; c < 4; ++c) ptx::tmem_ld_32x32(t_lane + Cfg::S_COL + c * 32, sv[c]);
       ptx::tmem_ld_wait();
-      const bool need_mask = (k0 + TK - 1 > q0 + t * TQ) || (k0 + TK > kv_end);
+      // raw scores stay in registers; the scale is folded into the exponent (scale > 0, so the
+      // maximum can be taken on the raw values)
+      const bool need_mask = (k0 + TK - 1 > q0 + t * TQ) || (k0 + TK > kv_end);  // warp-uniform
       float mx = -CUDART_INF_F;
+      if (need_mask) {
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
+        for (int c = 0; c < 4; ++c) {
 #pragma unroll
-        for (int e = 0; e < 32; ++e) {
-          float v = __uint_as_float(sv[c][e]) * sl2;
-          const int key = k0 + c * 32 + e;
-          if (need_mask && (key > row || key >= kv_end)) v = -CUDART_INF_F;
-          sv[c][e] = __float_as_uint(v);
-          mx = fmaxf(mx, v);
+          for (int e = 0; e < 32; ++e) {
+            const int key = k0 + c * 32 + e;
+            if (key > row || key >= kv_end) sv[c][e] = 0xff800000u;  // -inf
+            mx = fmaxf(mx, __uint_as_float(sv[c][e]));
+          }
+        }
+      } else {
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+#pragma unroll
+          for (int e = 0; e < 32; ++e) mx = fmaxf(mx, __uint_as_float(sv[c][e]));
         }
       }
+      mx *= sl2;
       // lazy maximum: keep the old reference unless this tile exceeds it by more than the threshold
       float factor = 1.f;
       bool grow = false;
       if (j == 0) {
         m_used = mx;  // finite: key 0 is visible to every row
       } else if (mx > m_used + RESCALE_THRESHOLD) {
-        factor = exp2f(m_used - mx);
+        factor = ptx::ex2_approx(m_used - mx);
         m_used = mx;
         grow = true;
       }
@@ -250,7 +259,8 @@ prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
         ptx::tmem_st_wait();
         l_sum *= factor;
       }
-      float psum = 0.f;
+      float psum0 = 0.f, psum1 = 0.f;
+      const float neg_m = -m_used;
 #pragma unroll
       for (int c = 0; c < 2; ++c) {
         uint32_t pk[32];
@@ -258,14 +268,15 @@ prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
         for (int e = 0; e < 32; ++e) {
           // packed column 32 c + e holds keys 2 (32 c + e) and 2 (32 c + e) + 1
           const int k_lo = (c * 32 + e) * 2;
-          const float p0 = exp2f(__uint_as_float(sv[k_lo >> 5][k_lo & 31]) - m_used);
-          const float p1 = exp2f(__uint_as_float(sv[(k_lo + 1) >> 5][(k_lo + 1) & 31]) - m_used);
-          psum += p0 + p1;
+          const float p0 = ptx::ex2_approx(fmaf(__uint_as_float(sv[k_lo >> 5][k_lo & 31]), sl2, neg_m));
+          const float p1 = ptx::ex2_approx(fmaf(__uint_as_float(sv[(k_lo + 1) >> 5][(k_lo + 1) & 31]), sl2, neg_m));
+          psum0 += p0;
+          psum1 += p1;
           pk[e] = ptx::pack_bf16(p0, p1);
         }
         ptx::tmem_st_32x32(t_lane + Cfg::S_COL + c * 32, pk);
       }
-      l_sum += psum;
+      l_sum += psum0 + psum1;
       ptx::tmem_st_wait();
       // the request's last tile may reach past its end: zero those V rows (0 * garbage must stay 0)
       if (k0 + TK > len) {

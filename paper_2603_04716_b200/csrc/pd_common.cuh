@@ -124,8 +124,7 @@ struct PrefillAttnArgs {
   int n_req, n_tokens, max_len;
   int n_q_heads, n_kv_heads, head_dim, len_cap, batch_cap;
 };
-pd_status launch_prefill_attention(const PrefillAttnArgs& a, cudaStream_t s);
-// The same operation on tcgen05 / tensor memory (the product path).
+// Causal GQA attention of a packed ragged batch on tcgen05 / tensor memory.
 pd_status launch_prefill_attention_tc(const PrefillAttnArgs& a, int* err_word, cudaStream_t s);
 
 struct DecodeAttnArgs {

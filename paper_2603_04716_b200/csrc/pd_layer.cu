@@ -3,7 +3,6 @@
 // synchronises except pd_layer_create / pd_layer_destroy / pd_layer_check and the
 // host-I/O variants of the stack calls.
 #include <cmath>
-#include <cstdlib>
 #include <new>
 #include <vector>
 
@@ -149,9 +148,7 @@ pd_status prefill_impl(pd_layer* L, const bf16* x, bf16* out, const int32_t* cu_
   a.batch_cap = cache->batch_cap;
   {
     pd::TraceScope ts(PD_K_ATTN_PREFILL, st);
-    static const bool legacy = std::getenv("PD_ATTN_LEGACY") != nullptr;  // bring-up switch
-    if (legacy) PD_TRY(pd::launch_prefill_attention(a, st));
-    else PD_TRY(pd::launch_prefill_attention_tc(a, L->err_word, st));
+    PD_TRY(pd::launch_prefill_attention_tc(a, L->err_word, st));
   }
   PD_TRY(oproj(L, x, tokens, ws, w, st));
   PD_TRY(mlp_half(L, reinterpret_cast<bf16*>(ws + w.resid), out, tokens, ws, w, st));
