@@ -178,6 +178,7 @@ def main():
     import numpy as np
     import torch
     import paper_2603_04716_b200 as pd
+    from paper_2603_04716_b200.replicas import max_over_ranks
 
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
@@ -326,10 +327,7 @@ def main():
     total_s = g0.elapsed_time(g1) * 1e-3
     pre_s = sum(a.elapsed_time(b) for a, b, _ in timing) * 1e-3
     dec_s = sum(b.elapsed_time(c) for _, b, c in timing) * 1e-3
-    if dist:
-        tt = torch.tensor([total_s, pre_s, dec_s], device=dev, dtype=torch.float64)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        total_s, pre_s, dec_s = tt.tolist()
+    total_s, pre_s, dec_s = max_over_ranks([total_s, pre_s, dec_s], dist, dev)
     pre_model_s = pre_s / args.steps * scale                       # one prefill pass, 32 layers
     tpot_s = dec_s / (args.steps * len(dec_ts)) * scale            # one decode step, 32 layers
     prefill_tok_s = world * L_IN / pre_model_s
@@ -378,10 +376,7 @@ def main():
         e2e_pre.append(t1 - t0)
         e2e_dec.append((t2 - t1) / len(dec_ts))
     e2e_pre_s = statistics.mean(e2e_pre)
-    if dist:
-        tt = torch.tensor([e2e_pre_s], device=dev, dtype=torch.float64)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        e2e_pre_s = tt.item()
+    (e2e_pre_s,) = max_over_ranks([e2e_pre_s], dist, dev)
     e2e_value = world * L_IN / (e2e_pre_s * scale)
 
     cpu = None

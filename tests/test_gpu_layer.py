@@ -112,6 +112,22 @@ def test_tiny_decode_equals_prefill_row_on_gpu(pdlib):
         assert np.all(np.abs(got - out[t]) <= 2e-2 + 2e-2 * np.abs(out[t]))
 
 
+@pytest.mark.parametrize("b", [17, 100, 300])
+def test_tiny_decode_batch_sizes_span_every_skinny_tile(pdlib, b):
+    """Decode batches that fall into the 32-, 128- and (two) 256-wide batch tiles of the projection kernel."""
+    cap = 48
+    ocfg, ow, dl = setup(pdlib, TINY, 64, 0, b, cap)
+    k0, v0 = gen.kv_cache(11, b, 2, cap, 64)
+    k, v, cache = dl.make_cache(b, cap, k0, v0)
+    x = gen.activations(11, b, 512, sub=b)
+    kv_len = [int(v_) for v_ in gen.uniform_lengths(11, b, 0, cap - 1, sub=b)]
+    dout = empty_bf16(b, 512)
+    pdlib.pd_decode_layer(dl.layer, to_dev(x), dout, i32_dev(kv_len), b, max(kv_len) + 1, cache, dl.ws, dl.ws_bytes)
+    pdlib.pd_layer_check(dl.layer)
+    ref = L.decode_layer(ocfg, ow, x, kv_len, k0.astype(np.float64), v0.astype(np.float64))
+    assert_close(from_dev(dout), ref, f"tiny decode B={b}")
+
+
 def test_two_layer_stack_matches_chained_oracle(pdlib):
     import torch
     ocfg, ow0, dl0 = setup(pdlib, TINY, 256, 160, 0, 0, layer=0)
