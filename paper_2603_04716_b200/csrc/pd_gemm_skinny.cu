@@ -4,8 +4,8 @@
 // HBM-bound, so the job is to keep all SMs loading weights.  The roles of the operands are
 // swapped with respect to the prefill GEMM: a tile is 128 weight rows (the M side of
 // tcgen05.mma, so no tensor-core rows are wasted on padding) by the whole batch (the N side,
-// rounded up to 16/32/64/128/256), and the K range is split across blocks until there are
-// about two blocks per SM.  A block accumulates its K slice in tensor memory and adds it into
+// rounded up to 16/32/64/128/256), and the K range is split across blocks until every SM has
+// work (two blocks per SM, so one block's epilogue overlaps another's main loop).  A block accumulates its K slice in tensor memory and adds it into
 // an fp32 [B, N] buffer (red.global.add, L2-resident; plain stores when K is not split).
 // Small row-wise kernels then apply the layer's fused operations to the fp32 sums: RoPE and the
 // KV-cache append, residual add with the following RMSNorm, SwiGLU, residual add.
@@ -19,14 +19,16 @@ constexpr int SK_BM = 128;  // weight rows per tile
 constexpr int SK_BK = 64;
 constexpr int SK_THREADS = 192;
 
-template <int BNB>
+template <int BNB, int MT>
 struct SkinnyCfg {
-  static constexpr int W_BYTES = SK_BM * SK_BK * 2;
+  static constexpr int W_BYTES = MT * SK_BM * SK_BK * 2;
   static constexpr int X_BYTES = BNB * SK_BK * 2;
   static constexpr int STAGE_BYTES = W_BYTES + ((X_BYTES + 1023) / 1024) * 1024;  // keep tiles 1024-byte aligned
-  static constexpr int STAGES = (BNB >= 256) ? 2 : (BNB >= 128 ? 3 : 4);
-  static constexpr int TMEM_COLS = BNB < 32 ? 32 : BNB;
+  static constexpr int STAGES = MT == 2 ? (BNB >= 256 ? 3 : 4) : (BNB >= 256 ? 2 : (BNB >= 128 ? 3 : 4));
+  static constexpr int ACC_COLS = BNB < 32 ? 32 : BNB;   // tensor-memory columns per accumulator
+  static constexpr int TMEM_COLS = MT * ACC_COLS;
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 128;
+  static constexpr int BLOCKS_PER_SM = MT == 2 ? 1 : 2;
 };
 
 struct SkinnyDev {
@@ -35,10 +37,10 @@ struct SkinnyDev {
   int* err_word;
 };
 
-template <int BNB>
+template <int BNB, int MT>
 __global__ void __launch_bounds__(SK_THREADS)
 gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_x, SkinnyDev p) {
-  using Cfg = SkinnyCfg<BNB>;
+  using Cfg = SkinnyCfg<BNB, MT>;
   constexpr int STAGES = Cfg::STAGES;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -92,7 +94,7 @@ gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
         const uint32_t sw = smem_base + stage * Cfg::STAGE_BYTES;
         const uint32_t sx = sw + Cfg::W_BYTES;
         ptx::mbar_arrive_expect_tx(full_bar(stage), Cfg::W_BYTES + Cfg::X_BYTES);
-        ptx::tma_load_2d(sw, &tmap_w, kb * SK_BK, tn * SK_BM, full_bar(stage));
+        ptx::tma_load_2d(sw, &tmap_w, kb * SK_BK, tn * (MT * SK_BM), full_bar(stage));  // box of MT * 128 rows
         ptx::tma_load_2d(sx, &tmap_x, kb * SK_BK, tb * BNB, full_bar(stage));
         if (++stage == STAGES) { stage = 0; phase ^= 1u; }
       }
@@ -113,8 +115,12 @@ gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
         const uint64_t dw = ptx::umma_desc_sw128(sw);
         const uint64_t dx = ptx::umma_desc_sw128(sw + Cfg::W_BYTES);
 #pragma unroll
-        for (int kk = 0; kk < SK_BK / 16; ++kk)
-          ptx::umma_bf16(tmem_base, dw + 2u * kk, dx + 2u * kk, idesc, (kb > kb0 || kk > 0) ? 1u : 0u);
+        for (int mt = 0; mt < MT; ++mt) {
+#pragma unroll
+          for (int kk = 0; kk < SK_BK / 16; ++kk)
+            ptx::umma_bf16(tmem_base + mt * Cfg::ACC_COLS, dw + mt * (SK_BM * SK_BK * 2 / 16) + 2u * kk, dx + 2u * kk, idesc,
+                           (kb > kb0 || kk > 0) ? 1u : 0u);
+        }
         ptx::umma_commit(empty_bar(stage));
         if (++stage == STAGES) { stage = 0; phase ^= 1u; }
       }
@@ -125,9 +131,11 @@ gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
     const bool ok = __all_sync(0xffffffffu, ptx::mbar_wait_bounded(acc_bar, 0u, abort_flag));
     if (ok && kb1 > kb0) {
       ptx::tc_fence_after();
-      const int n = tn * SK_BM + lane_group * 32 + lane;  // output feature of this thread
-      const uint32_t t_row = tmem_base + (static_cast<uint32_t>(lane_group * 32) << 16);
       constexpr int CH = BNB < 32 ? BNB : 32;
+#pragma unroll 1
+      for (int mt = 0; mt < MT; ++mt) {
+      const int n = (tn * MT + mt) * SK_BM + lane_group * 32 + lane;  // output feature of this thread
+      const uint32_t t_row = tmem_base + (static_cast<uint32_t>(lane_group * 32) << 16) + mt * Cfg::ACC_COLS;
 #pragma unroll 1
       for (int c0 = 0; c0 < BNB; c0 += CH) {
         uint32_t v[32];
@@ -146,6 +154,7 @@ gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
           }
         }
       }
+      }
     }
   }
   ptx::tc_fence_before();
@@ -158,25 +167,25 @@ gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
   }
 }
 
-template <int BNB>
+template <int BNB, int MT>
 pd_status launch_skinny(const SkinnyGemmArgs& g, cudaStream_t stream) {
-  using Cfg = SkinnyCfg<BNB>;
+  using Cfg = SkinnyCfg<BNB, MT>;
   static bool attr_set = false;
-  auto kern = gemm_skinny_kernel<BNB>;
+  auto kern = gemm_skinny_kernel<BNB, MT>;
   if (!attr_set) {
     PD_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES));
     attr_set = true;
   }
   CUtensorMap tw, tx;
-  PD_TRY(make_tmap_bf16(&tw, g.w, g.n, g.k, g.k, SK_BM));
+  PD_TRY(make_tmap_bf16(&tw, g.w, g.n, g.k, g.k, MT * SK_BM));
   PD_TRY(make_tmap_bf16(&tx, g.x, g.batch, g.k, g.ldx, BNB));
   SkinnyDev p{};
   p.acc = g.acc; p.batch = g.batch; p.n = g.n; p.k_blocks = g.k / SK_BK;
-  p.tiles_n = (g.n + SK_BM - 1) / SK_BM;
+  p.tiles_n = (g.n + MT * SK_BM - 1) / (MT * SK_BM);
   const int tiles_b = (g.batch + BNB - 1) / BNB;
-  // about two blocks per SM, each with at least 8 K-blocks
+  // fill the resident block slots, each block with at least 8 K-blocks
   const int units = p.tiles_n * tiles_b;
-  int splits = (2 * 148 + units / 2) / units;
+  int splits = (Cfg::BLOCKS_PER_SM * 148 + units / 2) / units;
   if (splits > p.k_blocks / 8) splits = p.k_blocks / 8;
   if (splits < 1) splits = 1;
   p.splits = splits;
@@ -331,11 +340,13 @@ __global__ void __launch_bounds__(256) skinny_swiglu_kernel(const float* __restr
 pd_status gemm_skinny(const SkinnyGemmArgs& g, cudaStream_t stream) {
   if (!g.x || !g.w || !g.acc || g.batch <= 0 || g.n <= 0 || g.k <= 0) return PD_ERR_INVALID_ARG;
   if (g.k % SK_BK != 0 || g.n % 4 != 0 || g.ldx % 8 != 0) return PD_ERR_UNSUPPORTED_SHAPE;
-  if (g.batch <= 16) return launch_skinny<16>(g, stream);
-  if (g.batch <= 32) return launch_skinny<32>(g, stream);
-  if (g.batch <= 64) return launch_skinny<64>(g, stream);
-  if (g.batch <= 128) return launch_skinny<128>(g, stream);
-  return launch_skinny<256>(g, stream);
+  if (g.batch <= 16) return launch_skinny<16, 1>(g, stream);
+  if (g.batch <= 32) return launch_skinny<32, 1>(g, stream);
+  if (g.batch <= 64) return launch_skinny<64, 1>(g, stream);
+  // (two weight sub-tiles per block, MT = 2, measured 10-20 % slower at B = 128..256: one block per SM
+  // loses the overlap of one block's epilogue with another's main loop)
+  if (g.batch <= 128) return launch_skinny<128, 1>(g, stream);
+  return launch_skinny<256, 1>(g, stream);
 }
 
 pd_status launch_skinny_rope_kv(const float* acc, bf16* qkv, const RopeEpilogue& rp, int batch, int* err_word,
