@@ -79,17 +79,18 @@ prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
   const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_al = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem_al + Cfg::BAR_OFF);
-  // 0 q_full | 1,2 k_full | 3,4 v_full | 5,6 kv_empty | 7,8 s_full | 9,10 p_ready | 11,12 o_done
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 13);
+  // 0 q_full | 1,2 k_full | 3,4 v_full | 5,6 v_empty | 7,8 s_full | 9,10 p_ready | 11,12 o_done | 13,14 k_empty
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 15);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   const uint32_t bar0 = ptx::smem_u32(bars);
   auto bar = [&](int i) { return bar0 + 8u * i; };
-  constexpr int B_QFULL = 0, B_KFULL = 1, B_VFULL = 3, B_KVEMPTY = 5, B_SFULL = 7, B_PREADY = 9, B_ODONE = 11;
+  constexpr int B_QFULL = 0, B_KFULL = 1, B_VFULL = 3, B_VEMPTY = 5, B_SFULL = 7, B_PREADY = 9, B_ODONE = 11,
+                B_KEMPTY = 13;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
     *abort_flag = 0;
-    for (int i = 0; i < 13; ++i) ptx::mbar_init(bar(i), (i == B_PREADY || i == B_PREADY + 1) ? 4 : 1);
+    for (int i = 0; i < 15; ++i) ptx::mbar_init(bar(i), (i == B_PREADY || i == B_PREADY + 1) ? 4 : 1);
     ptx::fence_barrier_init();
     ptx::prefetch_tensormap(&tmap_q);
     ptx::prefetch_tensormap(&tmap_k);
@@ -116,12 +117,15 @@ prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
       bool ok = true;
       for (int j = 0; j < n_max && ok; ++j) {
         const int s = j & 1;
-        if (!ptx::mbar_wait_bounded(bar(B_KVEMPTY + s), ((j >> 1) & 1) ^ 1u, abort_flag)) { ok = false; break; }
+        // K and V slots are released separately: K as soon as both tiles' Q K^T have been issued,
+        // V only after the P V products, so the next K tile is on its way while the softmax runs
+        if (!ptx::mbar_wait_bounded(bar(B_KEMPTY + s), ((j >> 1) & 1) ^ 1u, abort_flag)) { ok = false; break; }
         const uint32_t sk = smem_base + Cfg::KV_OFF + s * 2 * Cfg::TILE_BYTES;
         const uint32_t sv = sk + Cfg::TILE_BYTES;
         ptx::mbar_arrive_expect_tx(bar(B_KFULL + s), Cfg::TILE_BYTES);
         for (int c = 0; c < Cfg::SUB; ++c)
           ptx::tma_load_2d(sk + c * Cfg::SUB_BYTES, &tmap_k, c * 64, kv_row0 + j * TK, bar(B_KFULL + s));
+        if (!ptx::mbar_wait_bounded(bar(B_VEMPTY + s), ((j >> 1) & 1) ^ 1u, abort_flag)) { ok = false; break; }
         ptx::mbar_arrive_expect_tx(bar(B_VFULL + s), Cfg::TILE_BYTES);
         for (int c = 0; c < Cfg::SUB; ++c)
           ptx::tma_load_2d(sv + c * Cfg::SUB_BYTES, &tmap_v, c * 64, kv_row0 + j * TK, bar(B_VFULL + s));
@@ -136,7 +140,7 @@ prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
       constexpr uint32_t idesc_qk = ptx::umma_idesc_bf16(TQ, TK);
       constexpr uint32_t idesc_pv = ptx::umma_idesc_bf16_bmn(TQ, HD);
       bool ok = true;
-      auto issue_s = [&](int t, int j) {  // S_t = Q_t K_j^T
+      auto issue_s = [&](int t, int j) {  // S_t = Q_t K_j^T; the last tile to use K_j releases its slot
         const int s = j & 1;
         const uint32_t sq = smem_base + Cfg::Q_OFF + t * Cfg::TILE_BYTES;
         const uint32_t sk = smem_base + Cfg::KV_OFF + s * 2 * Cfg::TILE_BYTES;
@@ -147,6 +151,7 @@ prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
           ptx::umma_bf16(d, ptx::umma_desc_sw128(sq + off), ptx::umma_desc_sw128(sk + off), idesc_qk, kk > 0 ? 1u : 0u);
         }
         ptx::umma_commit(bar(B_SFULL + t));
+        if (t == 1 || j >= n_kv[1]) ptx::umma_commit(bar(B_KEMPTY + s));
       };
       auto issue_pv = [&](int t, int j) {  // O_t += P_t V_j
         const int s = j & 1;
@@ -181,7 +186,7 @@ prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
           ptx::tc_fence_after();
           issue_pv(t, j);
           const bool last_user = (t == 1) || (j >= n_kv[1]);
-          if (last_user) ptx::umma_commit(bar(B_KVEMPTY + s));
+          if (last_user) ptx::umma_commit(bar(B_VEMPTY + s));
           if (j + 1 < n_kv[t]) {
             if (!ptx::mbar_wait_bounded(bar(B_KFULL + (s ^ 1)), ((j + 1) >> 1) & 1, abort_flag)) { ok = false; break; }
             ptx::tc_fence_after();
