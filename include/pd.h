@@ -107,6 +107,18 @@ pd_status pd_prefill_layer(pd_layer* layer, const void* x, void* out, const int3
                            const int32_t* cu_seqlens_host, int32_t n_req, const int32_t* slots_dev,
                            const pd_kv_cache* cache, void* workspace, size_t workspace_bytes, void* stream);
 
+/* Chunked prefill (paper, "Acquire prefill throughput ...": the maximum prefill throughput depends on
+ * the chunked-prefill size, and the M/M/1 model holds when a request is at least one chunk long).
+ * Same as pd_prefill_layer, but request r already has prefix[r] tokens in its cache sequence: its
+ * rows take positions prefix[r], prefix[r]+1, ..., their K/V are appended there, and each row attends
+ * to every cached position up to its own.  `prefix` is given twice like cu_seqlens (device copy read
+ * by the kernels, host copy validated: prefix[r] + len_r must fit the cache and the RoPE table).
+ * prefix = 0 reproduces pd_prefill_layer; one-token chunks reproduce pd_decode_layer. */
+pd_status pd_prefill_chunk_layer(pd_layer* layer, const void* x, void* out, const int32_t* cu_seqlens_dev,
+                                 const int32_t* cu_seqlens_host, int32_t n_req, const int32_t* prefix_dev,
+                                 const int32_t* prefix_host, const int32_t* slots_dev, const pd_kv_cache* cache,
+                                 void* workspace, size_t workspace_bytes, void* stream);
+
 /* Decode mode (paper: the memory-bandwidth-bound phase measured as TPOT versus batch).
  *   x, out        device bf16 [B, d]; out may alias x
  *   kv_len_dev    device int32[B]: tokens already cached for sequence b (= position of the new

@@ -222,6 +222,48 @@ def decode_layer(cfg: LayerConfig, w: LayerWeights, x: np.ndarray, kv_len,
     return _mlp_and_residuals(x, st(o), w, cfg, dt, st)
 
 
+def extend_layer(cfg: LayerConfig, w: LayerWeights, x: np.ndarray, cu_seqlens, prefix_lens,
+                 k_cache: np.ndarray, v_cache: np.ndarray, dtype=np.float64, store=None) -> np.ndarray:
+    """Chunked prefill: one layer over a packed batch of request CHUNKS.
+
+    Request r already has prefix_lens[r] tokens in cache sequence r; its chunk rows
+    cu[r]..cu[r+1]-1 sit at positions prefix_lens[r] + 0, 1, ...  Their K/V are appended
+    IN PLACE at those positions and every row attends to all cached positions up to and
+    including its own.  With prefix_lens = 0 this is prefill_layer; with chunks of one token
+    it is decode_layer.  Caches are [batch, Hkv, len_cap, hd].  Returns out[T, d].
+    """
+    dt = dtype
+    st = store or _identity
+    x = np.asarray(x, dtype=dt)
+    cu = np.asarray(cu_seqlens, dtype=np.int64)
+    pre = np.asarray(prefix_lens, dtype=np.int64)
+    t_total = x.shape[0]
+    assert cu[0] == 0 and cu[-1] == t_total and np.all(np.diff(cu) >= 0) and len(pre) == len(cu) - 1
+    hq, hkv, hd = cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim
+    req = np.repeat(np.arange(len(cu) - 1), np.diff(cu))
+    pos = np.arange(t_total) - cu[req] + pre[req]
+    assert np.all(pos < k_cache.shape[2])
+
+    n1 = st(rmsnorm(x, w.g_attn.astype(dt), cfg.rms_eps))
+    qkv = n1 @ w.w_qkv.astype(dt).T
+    q = st(rope(qkv[:, :hq * hd].reshape(t_total, hq, hd), pos, cfg.rope_theta))
+    k = st(rope(qkv[:, hq * hd:(hq + hkv) * hd].reshape(t_total, hkv, hd), pos, cfg.rope_theta))
+    v = st(qkv[:, (hq + hkv) * hd:].reshape(t_total, hkv, hd))
+
+    o = np.empty((t_total, hq * hd), dtype=dt)
+    for r in range(len(cu) - 1):
+        lo, hi = int(cu[r]), int(cu[r + 1])
+        if hi == lo:
+            continue
+        p0, n = int(pre[r]), hi - lo
+        k_cache[r, :, p0:p0 + n, :] = k[lo:hi].transpose(1, 0, 2)
+        v_cache[r, :, p0:p0 + n, :] = v[lo:hi].transpose(1, 0, 2)
+        keys = np.ascontiguousarray(k_cache[r, :, :p0 + n, :].transpose(1, 0, 2)).astype(dt)
+        vals = np.ascontiguousarray(v_cache[r, :, :p0 + n, :].transpose(1, 0, 2)).astype(dt)
+        o[lo:hi] = _attend(q[lo:hi], keys, vals, pos[lo:hi], np.arange(p0 + n), cfg, None)
+    return _mlp_and_residuals(x, st(o), w, cfg, dt, st)
+
+
 def layer_flops_prefill(cfg: LayerConfig, lens) -> float:
     """Algorithmic flops of one prefill pass (causal half of attention only)."""
     t = float(sum(lens))

@@ -35,7 +35,7 @@ EXPORTS = [
     "pd_workspace_bytes", "pd_prefill_layer", "pd_decode_layer", "pd_prefill_stack", "pd_decode_stack",
     "pd_layer_check", "pd_gemm_bf16", "pd_measure", "pd_allocate", "pd_queue_replay",
     "pd_launch_count", "pd_trace_begin", "pd_trace_end", "pd_decode_attention", "pd_decode_attention_workspace_bytes",
-    "pd_decode_attention_noalloc",
+    "pd_decode_attention_noalloc", "pd_prefill_chunk_layer",
 ]
 
 TRACE_CLASSES = ["gemm_qkv", "gemm_o", "gemm_gate_up", "gemm_down", "attn_prefill", "attn_decode", "rmsnorm"]
@@ -114,6 +114,8 @@ _lib.pd_layer_destroy.argtypes = [_P]
 _lib.pd_workspace_bytes.argtypes = [C.POINTER(pd_layer_cfg), C.c_int32, C.c_int32, C.c_int32, C.POINTER(C.c_size_t)]
 _lib.pd_prefill_layer.argtypes = [_P, _P, _P, _P, C.POINTER(C.c_int32), C.c_int32, _P, C.POINTER(pd_kv_cache), _P,
                                   C.c_size_t, _P]
+_lib.pd_prefill_chunk_layer.argtypes = [_P, _P, _P, _P, C.POINTER(C.c_int32), C.c_int32, _P, C.POINTER(C.c_int32), _P,
+                                        C.POINTER(pd_kv_cache), _P, C.c_size_t, _P]
 _lib.pd_decode_layer.argtypes = [_P, _P, _P, _P, C.c_int32, C.c_int32, C.POINTER(pd_kv_cache), _P, C.c_size_t, _P]
 _lib.pd_prefill_stack.argtypes = [C.POINTER(_P), C.POINTER(pd_kv_cache), C.c_int32, C.c_int32, _P, _P, C.c_int32, _P,
                                   C.POINTER(C.c_int32), C.c_int32, _P, C.c_size_t, _P]
@@ -252,6 +254,16 @@ def pd_prefill_layer(layer: Layer, x, out, cu_seqlens_dev, cu_seqlens_host, cach
     _check(_lib.pd_prefill_layer(layer.handle, _ptr(x), _ptr(out), _ptr(cu_seqlens_dev), cu, len(cu_seqlens_host) - 1,
                                  _ptr(slots_dev), C.byref(cache), _ptr(workspace), workspace_bytes,
                                  _stream_ptr(stream)), "pd_prefill_layer")
+
+
+def pd_prefill_chunk_layer(layer: Layer, x, out, cu_seqlens_dev, cu_seqlens_host, prefix_dev, prefix_host,
+                           cache: pd_kv_cache, workspace, workspace_bytes: int, slots_dev=None, stream=None):
+    cu = _i32_array(cu_seqlens_host)
+    pre = _i32_array(prefix_host)
+    _check(_lib.pd_prefill_chunk_layer(layer.handle, _ptr(x), _ptr(out), _ptr(cu_seqlens_dev), cu,
+                                       len(cu_seqlens_host) - 1, _ptr(prefix_dev), pre, _ptr(slots_dev),
+                                       C.byref(cache), _ptr(workspace), workspace_bytes, _stream_ptr(stream)),
+           "pd_prefill_chunk_layer")
 
 
 def pd_decode_layer(layer: Layer, x, out, kv_len_dev, batch: int, max_kv_len: int, cache: pd_kv_cache, workspace,

@@ -1,6 +1,6 @@
-"""The five benchmark configurations as runnable drivers.
+"""The five benchmark configurations, and the chunked-prefill sweep, as runnable drivers.
 
-    python -m paper_2603_04716_b200.configs <tiny|8b|long_input|decode_heavy|70b> [--quick] [--out FILE]
+    python -m paper_2603_04716_b200.configs <tiny|8b|long_input|decode_heavy|70b|chunked> [--quick] [--out FILE]
 
 Each driver measures what the allocation method needs on the current GPU (maximum prefill
 throughput and the TPOT-versus-batch curve, both through pd_measure), feeds the numbers to
@@ -171,7 +171,68 @@ def run_70b(quick=False):
                                            dm["batch"], dm["tpot_s"])}}
 
 
-RUNNERS = {"tiny": run_tiny, "8b": run_8b, "long_input": run_long_input, "decode_heavy": run_decode_heavy,
+def run_chunked(quick=False):
+    """Maximum prefill throughput versus chunked-prefill size (paper, "Acquire prefill throughput ...": a larger
+    chunk raises the peak prefill throughput until saturation).  One request of L_in tokens is pushed through
+    the layer stack chunk by chunk with pd_prefill_chunk_layer; each chunk attends to the cached prefix."""
+    import statistics
+    import torch
+    peaks = _peaks()
+    l_in = 4096 if quick else 8192
+    nl = 2 if quick else 8
+    cfg = pd.LayerConfig(**SHAPE_8B, max_pos=l_in)
+    dev = torch.device("cuda")
+    d = SHAPE_8B["d_model"]
+
+    def rnd(*shape, std=1.0, mean=0.0):
+        return (torch.randn(*shape, device=dev) * std + mean).to(torch.bfloat16)
+
+    layers, caches, keep = [], [], []
+    for _ in range(nl):
+        w = {"w_qkv": rnd(cfg.n_qkv, d, std=0.02), "w_o": rnd(d, d, std=0.02), "w_gate": rnd(SHAPE_8B["d_ff"], d, std=0.02),
+             "w_up": rnd(SHAPE_8B["d_ff"], d, std=0.02), "w_down": rnd(d, SHAPE_8B["d_ff"], std=0.02),
+             "g_attn": rnd(d, std=0.02, mean=1.0), "g_mlp": rnd(d, std=0.02, mean=1.0)}
+        layers.append(pd.Layer(cfg, w))
+        torch.cuda.synchronize()
+        k = torch.zeros((1, 8, l_in, 128), dtype=torch.bfloat16, device=dev)
+        v = torch.zeros_like(k)
+        keep += [k, v]
+        caches.append(pd.kv_cache_struct(k, v, 1, l_in))
+    ws_bytes = pd.pd_workspace_bytes(cfg, l_in, 0, 0)
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
+    x = rnd(l_in, d)
+    bufs = [torch.empty_like(x), torch.empty_like(x)]
+    out = {}
+    for chunk in ([1024, 4096] if quick else [256, 512, 1024, 2048, 4096, 8192]):
+        metas = []
+        for c0 in range(0, l_in, chunk):
+            n = min(chunk, l_in - c0)
+            metas.append((c0, n, torch.tensor([0, n], dtype=torch.int32, device=dev),
+                          torch.tensor([c0], dtype=torch.int32, device=dev)))
+
+        def one_pass():
+            for c0, n, cu_dev, pre_dev in metas:          # chunk after chunk, each through the whole stack
+                src = x[c0:c0 + n]
+                for i, layer in enumerate(layers):
+                    dst = bufs[i & 1][:n]
+                    pd.pd_prefill_chunk_layer(layer, src, dst, cu_dev, [0, n], pre_dev, [c0], caches[i], ws, ws_bytes)
+                    src = dst
+        one_pass()
+        times = []
+        for _ in range(3 if quick else 5):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            one_pass()
+            e1.record()
+            e1.synchronize()
+            times.append(e0.elapsed_time(e1) * 1e-3)
+        pd.pd_layer_check(layers[0])
+        t = statistics.median(times) * 32 / nl
+        out[str(chunk)] = {"time_s": t, "prefill_max_tok_s": l_in / t}
+    return {"config": "chunked", "l_in": l_in, "layers_run": nl, "chunk_sweep": out}
+
+
+RUNNERS = {"chunked": run_chunked, "tiny": run_tiny, "8b": run_8b, "long_input": run_long_input, "decode_heavy": run_decode_heavy,
            "70b": run_70b}
 
 

@@ -47,6 +47,7 @@ struct AttDev {
   bf16* o;
   const int32_t* cu_seqlens;
   const int32_t* slots;
+  const int32_t* prefix;
   int n_q_heads, n_kv_heads, len_cap, batch_cap;
   int* err_word;
 };
@@ -63,6 +64,8 @@ prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
   if (q0 >= len) return;
   const int slot = p.slots ? p.slots[req] : req;
   if (slot < 0 || slot >= p.batch_cap) return;  // reported by the QKV epilogue
+  const int pre = p.prefix ? p.prefix[req] : 0;  // tokens of this request already in the cache (chunked prefill)
+  const int kv_total = pre + len;                // keys this request has after the chunk
   const int kvh = h / (p.n_q_heads / p.n_kv_heads);
   const int kv_row0 = (slot * p.n_kv_heads + kvh) * p.len_cap;  // first cache row of this (sequence, KV head)
 
@@ -71,7 +74,7 @@ prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
 #pragma unroll
   for (int t = 0; t < 2; ++t) {
     const int r0 = q0 + t * TQ;
-    n_kv[t] = (r0 < len) ? (min(len, r0 + TQ) + TK - 1) / TK : 0;
+    n_kv[t] = (r0 < len) ? (pre + min(len, r0 + TQ) + TK - 1) / TK : 0;
   }
   const int n_max = max(n_kv[0], n_kv[1]);
 
@@ -200,10 +203,11 @@ prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
     const int t = (warp - 2) >> 2;       // row tile of this warpgroup
     const int lane_group = warp & 3;     // tensor-memory lanes this warp may touch
     const int row_in_tile = lane_group * 32 + lane;
-    const int row = q0 + t * TQ + row_in_tile;  // query position inside the request
+    const int row = q0 + t * TQ + row_in_tile;  // row inside the request's chunk
+    const int row_pos = pre + row;              // its position = last key it may see
     const uint32_t t_lane = tmem_base + (static_cast<uint32_t>(lane_group * 32) << 16) + t * Cfg::TILE_COLS;
     const float sl2 = rsqrtf(static_cast<float>(HD)) * LOG2E_F;
-    const int kv_end = min(len, q0 + t * TQ + TQ);
+    const int kv_end = pre + min(len, q0 + t * TQ + TQ);
     float m_used = -CUDART_INF_F, l_sum = 0.f;
     bool ok = true;
     for (int j = 0; j < n_kv[t]; ++j) {
@@ -217,7 +221,7 @@ prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
       ptx::tmem_ld_wait();
       // raw scores stay in registers; the scale is folded into the exponent (scale > 0, so the
       // maximum can be taken on the raw values)
-      const bool need_mask = (k0 + TK - 1 > q0 + t * TQ) || (k0 + TK > kv_end);  // warp-uniform
+      const bool need_mask = (k0 + TK - 1 > pre + q0 + t * TQ) || (k0 + TK > kv_end);  // warp-uniform
       float mx = -CUDART_INF_F;
       if (need_mask) {
 #pragma unroll
@@ -225,7 +229,7 @@ prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
 #pragma unroll
           for (int e = 0; e < 32; ++e) {
             const int key = k0 + c * 32 + e;
-            if (key > row || key >= kv_end) sv[c][e] = 0xff800000u;  // -inf
+            if (key > row_pos || key >= kv_end) sv[c][e] = 0xff800000u;  // -inf
             mx = fmaxf(mx, __uint_as_float(sv[c][e]));
           }
         }
@@ -284,11 +288,11 @@ prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
       l_sum += psum0 + psum1;
       ptx::tmem_st_wait();
       // the request's last tile may reach past its end: zero those V rows (0 * garbage must stay 0)
-      if (k0 + TK > len) {
+      if (k0 + TK > kv_total) {
         // S being ready only proves that K has landed; V has its own barrier
         ok = __all_sync(0xffffffffu, ptx::mbar_wait_bounded(bar(B_VFULL + (j & 1)), (j >> 1) & 1, abort_flag));
         if (!ok) break;
-        if (k0 + row_in_tile >= len) {
+        if (k0 + row_in_tile >= kv_total) {
           const uint32_t svm = smem_base + Cfg::KV_OFF + (j & 1) * 2 * Cfg::TILE_BYTES + Cfg::TILE_BYTES;
 #pragma unroll
           for (int c = 0; c < Cfg::SUB; ++c) {
@@ -355,7 +359,7 @@ pd_status launch_hd(const PrefillAttnArgs& a, int* err_word, cudaStream_t s) {
   PD_TRY(make_tmap_bf16(&tk, a.k_cache, cache_rows, HD, HD, TK));
   PD_TRY(make_tmap_bf16(&tv, a.v_cache, cache_rows, HD, HD, TK));
   AttDev p{};
-  p.o = a.o; p.cu_seqlens = a.cu_seqlens; p.slots = a.slots;
+  p.o = a.o; p.cu_seqlens = a.cu_seqlens; p.slots = a.slots; p.prefix = a.prefix;
   p.n_q_heads = a.n_q_heads; p.n_kv_heads = a.n_kv_heads; p.len_cap = a.len_cap; p.batch_cap = a.batch_cap;
   p.err_word = err_word;
   dim3 grid((a.max_len + 2 * TQ - 1) / (2 * TQ), a.n_q_heads, a.n_req);

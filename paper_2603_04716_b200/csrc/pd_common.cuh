@@ -67,6 +67,7 @@ struct RopeEpilogue {
   const float2* rope_tab;     // [max_pos, hd/2] (cos, sin)
   const int32_t* cu_seqlens;  // prefill: device [n_req + 1]; decode: NULL
   const int32_t* slots;       // prefill: device [n_req] or NULL
+  const int32_t* prefix;      // chunked prefill: device [n_req] tokens already cached per request, or NULL
   const int32_t* kv_len;      // decode: device [B]
   bf16* k_cache;              // [batch_cap, Hkv, len_cap, hd]
   bf16* v_cache;
@@ -121,6 +122,7 @@ struct PrefillAttnArgs {
   bf16* o;             // [T, Hq*hd]
   const int32_t* cu_seqlens;  // device [n_req+1]
   const int32_t* slots;       // device [n_req] or NULL
+  const int32_t* prefix;      // device [n_req] cached tokens before each request's rows, or NULL
   int n_req, n_tokens, max_len;
   int n_q_heads, n_kv_heads, head_dim, len_cap, batch_cap;
 };

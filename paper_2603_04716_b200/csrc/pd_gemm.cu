@@ -287,7 +287,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
               const int mid = (lo + hi) >> 1;
               if (rp.cu_seqlens[mid] <= row) lo = mid; else hi = mid;
             }
-            pos = row - rp.cu_seqlens[lo];
+            pos = row - rp.cu_seqlens[lo] + (rp.prefix ? rp.prefix[lo] : 0);
             slot = rp.slots ? rp.slots[lo] : lo;
           } else {
             pos = rp.kv_len[row];

@@ -112,7 +112,7 @@ pd_status oproj(pd_layer* L, const bf16* x, int tokens, uint8_t* ws, const Works
 }
 
 pd_status validate_prefill(const pd_layer* L, const int32_t* cu_host, int n_req, const pd_kv_cache* cache,
-                           bool default_slots, int* tokens, int* max_len) {
+                           bool default_slots, int* tokens, int* max_len, const int32_t* prefix_host = nullptr) {
   if (!L || !cu_host || n_req < 0 || n_req > 4095) return PD_ERR_INVALID_ARG;
   PD_TRY(check_cache(L, cache));
   if (cu_host[0] != 0) return PD_ERR_INVALID_ARG;
@@ -120,7 +120,8 @@ pd_status validate_prefill(const pd_layer* L, const int32_t* cu_host, int n_req,
   for (int r = 0; r < n_req; ++r) {
     const int len = cu_host[r + 1] - cu_host[r];
     if (len < 0) return PD_ERR_INVALID_ARG;
-    if (len > cache->len_cap || len > L->cfg.max_pos) return PD_ERR_INVALID_ARG;
+    const int pre = prefix_host ? prefix_host[r] : 0;
+    if (pre < 0 || pre > cache->len_cap - len || pre + len > L->cfg.max_pos) return PD_ERR_INVALID_ARG;
     if (len > mx) mx = len;
   }
   if (default_slots && n_req > cache->batch_cap) return PD_ERR_INVALID_ARG;
@@ -131,18 +132,18 @@ pd_status validate_prefill(const pd_layer* L, const int32_t* cu_host, int n_req,
 
 pd_status prefill_impl(pd_layer* L, const bf16* x, bf16* out, const int32_t* cu_dev, int n_req, int tokens,
                        int max_len, const int32_t* slots_dev, const pd_kv_cache* cache, uint8_t* ws,
-                       const Workspace& w, cudaStream_t st) {
+                       const Workspace& w, cudaStream_t st, const int32_t* prefix_dev = nullptr) {
   const pd_layer_cfg& c = L->cfg;
   pd::RopeEpilogue r{};
   r.k_cache = static_cast<bf16*>(cache->k); r.v_cache = static_cast<bf16*>(cache->v); r.rope_tab = L->rope_tab;
-  r.cu_seqlens = cu_dev; r.slots = slots_dev; r.kv_len = nullptr; r.n_req = n_req;
+  r.cu_seqlens = cu_dev; r.slots = slots_dev; r.prefix = prefix_dev; r.kv_len = nullptr; r.n_req = n_req;
   r.n_q_heads = c.n_q_heads; r.n_kv_heads = c.n_kv_heads; r.head_dim = c.head_dim; r.len_cap = cache->len_cap;
   r.max_pos = c.max_pos; r.batch_cap = cache->batch_cap;
   PD_TRY(qkv_half(L, x, tokens, r, ws, w, st));
   pd::PrefillAttnArgs a{};
   a.q = reinterpret_cast<bf16*>(ws + w.qkv); a.ldq = L->n_qkv;
   a.k_cache = static_cast<bf16*>(cache->k); a.v_cache = static_cast<bf16*>(cache->v);
-  a.o = reinterpret_cast<bf16*>(ws + w.attn_o); a.cu_seqlens = cu_dev; a.slots = slots_dev;
+  a.o = reinterpret_cast<bf16*>(ws + w.attn_o); a.cu_seqlens = cu_dev; a.slots = slots_dev; a.prefix = prefix_dev;
   a.n_req = n_req; a.n_tokens = tokens; a.max_len = max_len;
   a.n_q_heads = c.n_q_heads; a.n_kv_heads = c.n_kv_heads; a.head_dim = c.head_dim; a.len_cap = cache->len_cap;
   a.batch_cap = cache->batch_cap;
@@ -316,6 +317,24 @@ extern "C" pd_status pd_prefill_layer(pd_layer* L, const void* x, void* out, con
   if (reinterpret_cast<uintptr_t>(workspace) & 255u) return PD_ERR_INVALID_ARG;
   return prefill_impl(L, static_cast<const bf16*>(x), static_cast<bf16*>(out), cu_dev, n_req, tokens, max_len,
                       slots_dev, cache, static_cast<uint8_t*>(workspace), w, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" pd_status pd_prefill_chunk_layer(pd_layer* L, const void* x, void* out, const int32_t* cu_dev,
+                                            const int32_t* cu_host, int32_t n_req, const int32_t* prefix_dev,
+                                            const int32_t* prefix_host, const int32_t* slots_dev,
+                                            const pd_kv_cache* cache, void* workspace, size_t workspace_bytes,
+                                            void* stream) {
+  if (!prefix_dev || !prefix_host) return PD_ERR_INVALID_ARG;
+  int tokens = 0, max_len = 0;
+  PD_TRY(validate_prefill(L, cu_host, n_req, cache, slots_dev == nullptr, &tokens, &max_len, prefix_host));
+  if (tokens == 0) return PD_OK;
+  if (!x || !out || !cu_dev || !workspace) return PD_ERR_INVALID_ARG;
+  const Workspace w = carve(L->cfg, tokens, 0, 0);
+  if (workspace_bytes < w.total) return PD_ERR_WORKSPACE_TOO_SMALL;
+  if (reinterpret_cast<uintptr_t>(workspace) & 255u) return PD_ERR_INVALID_ARG;
+  return prefill_impl(L, static_cast<const bf16*>(x), static_cast<bf16*>(out), cu_dev, n_req, tokens, max_len,
+                      slots_dev, cache, static_cast<uint8_t*>(workspace), w, static_cast<cudaStream_t>(stream),
+                      prefix_dev);
 }
 
 extern "C" pd_status pd_decode_layer(pd_layer* L, const void* x, void* out, const int32_t* kv_len_dev, int32_t B,

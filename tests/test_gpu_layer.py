@@ -128,6 +128,66 @@ def test_tiny_decode_batch_sizes_span_every_skinny_tile(pdlib, b):
     assert_close(from_dev(dout), ref, f"tiny decode B={b}")
 
 
+def _run_chunks(pd, dl, ocfg, ow, x, lens, bounds, cap, what, parity=None):
+    """Feeds every request in chunks (bounds[r] = chunk boundaries) through pd_prefill_chunk_layer and the
+    oracle's extend_layer, comparing chunk by chunk; returns the GPU output assembled in request order."""
+    import torch
+    cu = np.concatenate([[0], np.cumsum(lens)])
+    n_req = len(lens)
+    k, v, cache = dl.make_cache(n_req, cap)
+    hkv, hd = ocfg.n_kv_heads, ocfg.head_dim
+    ok = np.zeros((n_req, hkv, cap, hd)); ov = np.zeros_like(ok)
+    oks, ovs = ok.copy(), ov.copy()
+    out = np.zeros((int(cu[-1]), ocfg.d_model), dtype=np.float32)
+    for step in range(max(len(b) for b in bounds) - 1):
+        rows, cu_c, pre = [], [0], []
+        for r in range(n_req):
+            b = bounds[r]
+            lo, hi = (b[step], b[step + 1]) if step + 1 < len(b) else (b[-1], b[-1])
+            rows += list(range(int(cu[r]) + lo, int(cu[r]) + hi))
+            cu_c.append(cu_c[-1] + hi - lo)
+            pre.append(lo)
+        if not rows:
+            continue
+        xc = x[rows]
+        dout = empty_bf16(len(rows), ocfg.d_model)
+        pd.pd_prefill_chunk_layer(dl.layer, to_dev(xc), dout, i32_dev(cu_c), cu_c, i32_dev(pre), pre, cache, dl.ws,
+                                  dl.ws_bytes)
+        pd.pd_layer_check(dl.layer)
+        got = from_dev(dout)
+        ref = L.extend_layer(ocfg, ow, xc, cu_c, pre, ok, ov)
+        if parity is None:
+            assert_close(got, ref, f"{what} chunk step {step}")
+        else:
+            ref_s = L.extend_layer(ocfg, ow, xc, cu_c, pre, oks, ovs, store=store_bf16)
+            assert_parity(got, ref, ref_s, f"{what} chunk step {step}")
+        out[rows] = got
+    torch.cuda.synchronize()
+    return out, from_dev(k), from_dev(v), ok, ov
+
+
+def test_tiny_chunked_prefill_matches_oracle_and_full_prefill(pdlib):
+    lens = [300, 129, 40]
+    bounds = [[0, 17, 128, 200, 300], [0, 128, 129], [0, 40]]      # ragged chunks, prefixes off the 128-key tiles
+    ocfg, ow, dl = setup(pdlib, TINY, 512, sum(lens), 0, 0)
+    x = gen.activations(12, sum(lens), 512)
+    out, k, v, ok, ov = _run_chunks(pdlib, dl, ocfg, ow, x, lens, bounds, 320, "tiny")
+    for r, ln in enumerate(lens):
+        assert_close(k[r, :, :ln], ok[r, :, :ln], "K cache after chunks")
+        assert_close(v[r, :, :ln], ov[r, :, :ln], "V cache after chunks")
+    # the whole requests in one go give the same rows (bf16 results of the same math in another order)
+    cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    full, _, _ = run_prefill(pdlib, dl, x, cu, batch_cap=3, len_cap=320)
+    assert np.all(np.abs(out - full) <= 2e-2 + 2e-2 * np.abs(full))
+
+
+def test_8b_chunked_prefill_two_chunks(pdlib):
+    lens = [700]
+    ocfg, ow, dl = setup(pdlib, M8B, 1024, 700, 0, 0, layer=3)
+    x = gen.activations(13, 700, 4096)
+    _run_chunks(pdlib, dl, ocfg, ow, x, lens, [[0, 300, 700]], 768, "8B", parity=True)
+
+
 def test_two_layer_stack_matches_chained_oracle(pdlib):
     import torch
     ocfg, ow0, dl0 = setup(pdlib, TINY, 256, 160, 0, 0, layer=0)

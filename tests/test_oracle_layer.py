@@ -287,3 +287,37 @@ def test_storage_rounding_variant():
     assert len(calls) == 9
     np.testing.assert_array_equal(kc[0, :, 64], gen.bf16_round(kc[0, :, 64].astype(np.float32)))
     np.testing.assert_array_equal(d, gen.bf16_round(d.astype(np.float32)))
+
+
+def test_chunked_prefill_equals_full_prefill_and_decode():
+    """extend_layer over consecutive chunks reproduces prefill_layer row for row (and the cache);
+    one-token chunks reproduce decode_layer."""
+    cfg = TINY
+    w = make_weights(cfg)
+    lens = [70, 33]
+    cu = np.cumsum([0] + lens)
+    x = gen.activations(9, sum(lens), cfg.d_model)
+    full, k, v = L.prefill_layer(cfg, w, x, cu)
+    kc = np.zeros((2, cfg.n_kv_heads, 80, cfg.head_dim)); vc = np.zeros_like(kc)
+    out = np.zeros_like(full)
+    splits = [[0, 17, 64, 70], [0, 1, 33]]          # chunk boundaries per request (ragged, not tile aligned)
+    for step in range(3):
+        rows, cu_c, pre = [], [0], []
+        for r in range(2):
+            b = splits[r]
+            lo, hi = (b[step], b[step + 1]) if step + 1 < len(b) else (b[-1], b[-1])
+            rows += list(range(int(cu[r]) + lo, int(cu[r]) + hi))
+            cu_c.append(cu_c[-1] + hi - lo)
+            pre.append(lo)
+        if rows:
+            out[rows] = L.extend_layer(cfg, w, x[rows], cu_c, pre, kc, vc)
+    np.testing.assert_allclose(out, full, rtol=1e-10, atol=1e-11)
+    np.testing.assert_allclose(kc[0, :, :70], k[:70].transpose(1, 0, 2), rtol=1e-12, atol=1e-13)
+    np.testing.assert_allclose(vc[1, :, :33], v[70:].transpose(1, 0, 2), rtol=1e-12, atol=1e-13)
+    # one-token chunk == decode step
+    kd, vd = kc.copy(), vc.copy()
+    xs = gen.activations(9, 2, cfg.d_model, sub=1)
+    dec = L.decode_layer(cfg, w, xs, [70, 33], kd, vd)
+    ext = L.extend_layer(cfg, w, xs, [0, 1, 2], [70, 33], kc, vc)
+    np.testing.assert_allclose(ext, dec, rtol=1e-12, atol=1e-13)
+    np.testing.assert_array_equal(kc, kd)
