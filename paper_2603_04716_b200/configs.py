@@ -54,6 +54,34 @@ def _prefill_time_grid(cfg, lengths, n_layers_run, n_layers_model, reps, peaks):
     return out
 
 
+def refine_feasible_batch(measure_tpot, batch, tpot_s, tpot_slo_s, max_probes=8):
+    """Integer refinement of the TPOT-feasible batch (paper, "Acquire decode throughput ...": determine the batch
+    size that satisfies the target TPOT).  The sweep gives the largest feasible sweep point B_lo and the first
+    infeasible one B_hi; TPOT is measured at midpoints until the largest feasible integer is bracketed.
+    `measure_tpot(b)` returns the measured TPOT of batch b in seconds.  Returns (batch, tpot_s, probes)."""
+    pts = sorted(zip(batch, tpot_s))
+    lo = None
+    hi = None
+    for b, t in pts:
+        if t <= tpot_slo_s:
+            lo = (b, t)
+        else:
+            hi = (b, t)
+            break
+    if lo is None or hi is None:
+        return (lo[0], lo[1], []) if lo else (0, float("nan"), [])
+    probes = []
+    while hi[0] - lo[0] > 1 and len(probes) < max_probes:
+        mid = (lo[0] + hi[0]) // 2
+        t = measure_tpot(mid)
+        probes.append((mid, t))
+        if t <= tpot_slo_s:
+            lo = (mid, t)
+        else:
+            hi = (mid, t)
+    return lo[0], lo[1], probes
+
+
 def run_tiny(quick=False):
     peaks = _peaks()
     cfg = pd.LayerConfig(**SHAPE_TINY, max_pos=256)
@@ -132,9 +160,23 @@ def run_decode_heavy(quick=False):
     d = pd.pd_measure(cfg, n_layers_run=nl, n_layers_model=32, warmup=1, reps=3, seed=0, batch_sizes=sweep,
                       kv_len_start=512, n_steps=2048, step_stride=1024 if quick else 256,
                       peak_bf16_flops=peaks[0], peak_hbm_bytes_s=peaks[1])
+    def tpot_at(b):
+        m = pd.pd_measure(cfg, n_layers_run=nl, n_layers_model=32, warmup=1, reps=3, seed=0, batch_sizes=[int(b)],
+                          kv_len_start=512, n_steps=2048, step_stride=1024 if quick else 256,
+                          peak_bf16_flops=peaks[0], peak_hbm_bytes_s=peaks[1])
+        return m["tpot_s"][0]
+
     per_slo = {}
     for slo_ms in (20, 35, 50, 75, 100):
-        per_slo[str(slo_ms)] = _alloc(5e5, 512, 2048, 2.0, slo_ms * 1e-3, p["prefill_tok_s"], d["batch"], d["tpot_s"])
+        a = _alloc(5e5, 512, 2048, 2.0, slo_ms * 1e-3, p["prefill_tok_s"], d["batch"], d["tpot_s"])
+        if a["status"] == 0 and not a["sweep_capped"]:
+            # the SLO binds between two sweep points: bracket the largest feasible integer batch by measurement
+            b_ref, t_ref, probes = refine_feasible_batch(tpot_at, d["batch"], d["tpot_s"], slo_ms * 1e-3,
+                                                         max_probes=3 if quick else 8)
+            a["refined"] = _alloc(5e5, 512, 2048, 2.0, slo_ms * 1e-3, p["prefill_tok_s"],
+                                  d["batch"] + [b_ref], d["tpot_s"] + [t_ref])
+            a["refined"]["probes"] = probes
+        per_slo[str(slo_ms)] = a
     return {"config": "decode_heavy", "layers_run": nl, "ttft_slo_s": 2.0, "prefill": p, "decode": d,
             "allocation_per_tpot_slo_ms": per_slo}
 
