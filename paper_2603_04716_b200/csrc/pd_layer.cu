@@ -14,7 +14,7 @@ namespace {
 
 struct Workspace {
   // byte offsets into the caller's workspace
-  size_t norm, qkv, attn_o, resid, acc, act, partial, stage_a, stage_b, meta, total;
+  size_t norm, qkv, attn_o, resid, acc, act, partial, stage_a, stage_b, meta, splitk, total;
 };
 
 Workspace carve(const pd_layer_cfg& c, size_t tokens, size_t max_batch, int max_kv_len) {
@@ -43,6 +43,7 @@ Workspace carve(const pd_layer_cfg& c, size_t tokens, size_t max_batch, int max_
   w.stage_a = take(tokens * d * 2);  // activations between layers of a stack / staged host input
   w.stage_b = take(tokens * d * 2);
   w.meta = take(4096 * 4);           // staged cu_seqlens / kv_len of the host-I/O stack calls
+  w.splitk = take(tokens > 256 ? pd::kSplitScratchBytes : 0);  // partial tiles of K-split GEMM tails (prefill only)
   w.total = off;
   return w;
 }
@@ -66,6 +67,15 @@ pd_status check_cache(const pd_layer* L, const pd_kv_cache* c) {
   return PD_OK;
 }
 
+// Lets a prefill GEMM cut the tiles of its last partial wave in two along K.
+void enable_tail_split(pd_layer* L, pd::GemmArgs& g, uint8_t* ws, const Workspace& w, size_t tokens) {
+  if (tokens <= 256) return;
+  g.split_scratch = reinterpret_cast<float*>(ws + w.splitk);
+  g.split_scratch_bytes = pd::kSplitScratchBytes;
+  g.split_flags = L->split_flags;
+  g.split_epoch = ++L->split_epoch;
+}
+
 // MLP half shared by both modes: h (residual stream after attention) -> out.
 pd_status mlp_half(pd_layer* L, const bf16* h, bf16* out, int tokens, uint8_t* ws, const Workspace& w,
                    cudaStream_t st) {
@@ -81,6 +91,7 @@ pd_status mlp_half(pd_layer* L, const bf16* h, bf16* out, int tokens, uint8_t* w
   g2.a = act; g2.b = L->w_down; g2.c = out; g2.r = h; g2.m = tokens; g2.n = c.d_model; g2.k = c.d_ff;
   g2.lda = c.d_ff; g2.ldb = c.d_ff; g2.ldc = c.d_model; g2.ldr = c.d_model; g2.epilogue = pd::EPI_RESIDUAL;
   g2.err_word = L->err_word;
+  enable_tail_split(L, g2, ws, w, tokens);
   { pd::TraceScope ts(PD_K_GEMM_DOWN, st); PD_TRY(pd::gemm(g2, st)); }
   return PD_OK;
 }
@@ -96,6 +107,7 @@ pd_status qkv_half(pd_layer* L, const bf16* x, int tokens, const pd::RopeEpilogu
   g.a = norm; g.b = L->w_qkv; g.c = qkv; g.m = tokens; g.n = L->n_qkv; g.k = c.d_model;
   g.lda = c.d_model; g.ldb = c.d_model; g.ldc = L->n_qkv; g.epilogue = pd::EPI_ROPE_KV; g.rope = &rope;
   g.err_word = L->err_word;
+  enable_tail_split(L, g, ws, w, tokens);
   { pd::TraceScope ts(PD_K_GEMM_QKV, st); PD_TRY(pd::gemm(g, st)); }
   return PD_OK;
 }
@@ -107,6 +119,7 @@ pd_status oproj(pd_layer* L, const bf16* x, int tokens, uint8_t* ws, const Works
   g.a = reinterpret_cast<bf16*>(ws + w.attn_o); g.b = L->w_o; g.c = reinterpret_cast<bf16*>(ws + w.resid); g.r = x;
   g.m = tokens; g.n = c.d_model; g.k = hq; g.lda = hq; g.ldb = hq; g.ldc = c.d_model; g.ldr = c.d_model;
   g.epilogue = pd::EPI_RESIDUAL; g.err_word = L->err_word;
+  enable_tail_split(L, g, ws, w, tokens);
   pd::TraceScope ts(PD_K_GEMM_O, st);
   return pd::gemm(g, st);
 }
@@ -253,6 +266,9 @@ extern "C" pd_status pd_layer_create(const pd_layer_cfg* cfg, const pd_layer_wei
   if ((e = cudaMalloc(&L->rope_tab, static_cast<size_t>(cfg->max_pos) * half * sizeof(float2))) != cudaSuccess)
     return fail(e);
   if ((e = cudaMalloc(&L->err_word, sizeof(int))) != cudaSuccess) return fail(e);
+  if ((e = cudaMalloc(&L->split_flags, pd::kSplitMaxTiles * 4 * sizeof(int))) != cudaSuccess) return fail(e);
+  if ((e = cudaMemsetAsync(L->split_flags, 0, pd::kSplitMaxTiles * 4 * sizeof(int), st)) != cudaSuccess) return fail(e);
+  L->split_epoch = 0;
   const cudaMemcpyKind d2d = cudaMemcpyDeviceToDevice;
   if ((e = cudaMemcpyAsync(L->w_qkv, w->w_qkv, L->n_qkv * d * 2, d2d, st)) != cudaSuccess) return fail(e);
   if ((e = cudaMemcpyAsync(L->w_o, w->w_o, d * hq * 2, d2d, st)) != cudaSuccess) return fail(e);
@@ -286,7 +302,7 @@ extern "C" pd_status pd_layer_create(const pd_layer_cfg* cfg, const pd_layer_wei
 extern "C" pd_status pd_layer_destroy(pd_layer* L) {
   if (!L) return PD_OK;
   cudaFree(L->w_qkv); cudaFree(L->w_o); cudaFree(L->w_gu); cudaFree(L->w_down);
-  cudaFree(L->g_attn); cudaFree(L->g_mlp); cudaFree(L->rope_tab); cudaFree(L->err_word);
+  cudaFree(L->g_attn); cudaFree(L->g_mlp); cudaFree(L->rope_tab); cudaFree(L->err_word); cudaFree(L->split_flags);
   delete L;
   return PD_OK;
 }
