@@ -80,6 +80,7 @@ struct GemmDev {
   // blocks; the first writes its fp32 partial tile to `split_scratch` and raises a flag per 32-row group,
   // the second adds it before the epilogue.  n_units = main_tiles + 2 * (tiles - main_tiles) when enabled.
   int n_units, main_tiles;
+  int tail_halves;       // 1: instead, tail tiles are cut in two along N (two 128-column halves, no hand-over)
   float* split_scratch;  // [tail tile][128][BN] fp32
   int* split_flags;      // [tail tile][4] epoch of the last partial written
   int split_epoch;       // > 0 enables the split
@@ -110,19 +111,25 @@ __device__ __forceinline__ void tile_coords(int tile, int tiles_m, int tiles_n, 
 
 // Work unit -> tile, K-block range and role (0 whole tile, 1 first K half: writes a partial, 2 second K half:
 // adds the partner's partial and runs the epilogue).
+// role 3: the unit is the 128-column half `n_half` of its tile (whole K, independent of the other half).
 struct UnitInfo {
-  int tile, kb_lo, kb_hi, role;
+  int tile, kb_lo, kb_hi, role, n_half;
 };
-__device__ __forceinline__ UnitInfo unit_info(int unit, int main_tiles, int k_blocks) {
+__device__ __forceinline__ UnitInfo unit_info(int unit, int main_tiles, int k_blocks, int tail_halves) {
   UnitInfo u;
+  u.n_half = 0;
   if (unit < main_tiles) {
     u.tile = unit; u.kb_lo = 0; u.kb_hi = k_blocks; u.role = 0;
   } else {
     const int v = unit - main_tiles;
     u.tile = main_tiles + (v >> 1);
-    const int kh = k_blocks >> 1;
-    if (v & 1) { u.kb_lo = kh; u.kb_hi = k_blocks; u.role = 2; }
-    else { u.kb_lo = 0; u.kb_hi = kh; u.role = 1; }
+    if (tail_halves) {
+      u.kb_lo = 0; u.kb_hi = k_blocks; u.role = 3; u.n_half = v & 1;
+    } else {
+      const int kh = k_blocks >> 1;
+      if (v & 1) { u.kb_lo = kh; u.kb_hi = k_blocks; u.role = 2; }
+      else { u.kb_lo = 0; u.kb_hi = kh; u.role = 1; }
+    }
   }
   return u;
 }
@@ -182,7 +189,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       uint32_t phase = 0;
       bool ok = true;
       for (int unit = blockIdx.x; unit < n_units && ok; unit += gridDim.x) {
-        const UnitInfo ui = unit_info(unit, p.main_tiles, k_blocks);
+        const UnitInfo ui = unit_info(unit, p.main_tiles, k_blocks, p.tail_halves);
         int tm, tn;
         tile_coords(ui.tile, p.tiles_m, p.tiles_n, p.raster_group, tm, tn);
         for (int kb = ui.kb_lo; kb < ui.kb_hi; ++kb) {
@@ -210,7 +217,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       uint32_t acc_phase = 0;
       bool ok = true;
       for (int unit = blockIdx.x; unit < n_units && ok; unit += gridDim.x) {
-        const UnitInfo ui = unit_info(unit, p.main_tiles, k_blocks);
+        const UnitInfo ui = unit_info(unit, p.main_tiles, k_blocks, p.tail_halves);
         if (!ptx::mbar_wait_bounded(acce_bar(acc), acc_phase ^ 1u, abort_flag)) { ok = false; break; }
         ptx::tc_fence_after();
         const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * Cfg::ACC_COLS);
@@ -220,11 +227,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
           const uint32_t sa = smem_base + stage * Cfg::STAGE_BYTES;
           const uint32_t sb = sa + Cfg::A_BYTES;
           const uint64_t da = ptx::umma_desc_sw128(sa);
-          const uint64_t db = ptx::umma_desc_sw128(sb);
+          // a half-width unit multiplies by rows 128 n_half .. of the B tile only (128 rows = 16 KB further on)
+          const uint64_t db = ptx::umma_desc_sw128(sb + ui.n_half * (128 * BK * 2));
+          const uint32_t idesc_u = (ui.role == 3) ? ptx::umma_idesc_bf16(BM, 128) : idesc;
 #pragma unroll
           for (int kk = 0; kk < BK / 16; ++kk) {
             // 16 bf16 = 32 bytes along K inside the 128-byte swizzled row: +2 in 16-byte units
-            ptx::umma_bf16(d_tmem, da + 2u * kk, db + 2u * kk, idesc, (kb > ui.kb_lo || kk > 0) ? 1u : 0u);
+            ptx::umma_bf16(d_tmem, da + 2u * kk, db + 2u * kk, idesc_u, (kb > ui.kb_lo || kk > 0) ? 1u : 0u);
           }
           ptx::umma_commit(empty_bar(stage));  // stage is free once these MMAs have read it
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
@@ -241,7 +250,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     uint32_t acc_phase = 0;
     bool ok = true;
     for (int unit = blockIdx.x; unit < n_units && ok; unit += gridDim.x) {
-      const UnitInfo ui = unit_info(unit, p.main_tiles, k_blocks);
+      const UnitInfo ui = unit_info(unit, p.main_tiles, k_blocks, p.tail_halves);
       int tm, tn;
       tile_coords(ui.tile, p.tiles_m, p.tiles_n, p.raster_group, tm, tn);
       // warp-uniform outcome: tcgen05.ld below needs the whole warp
@@ -253,7 +262,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                              static_cast<uint32_t>(acc * Cfg::ACC_COLS);
       // partner data of a K-split tile: this thread's row of the fp32 partial tile
       float* part_row = nullptr;
-      if (ui.role != 0) {
+      if (ui.role == 1 || ui.role == 2) {
         const int slot = ui.tile - p.main_tiles;
         part_row = p.split_scratch + (static_cast<size_t>(slot) * BM + lane_group * 32 + lane) * BN;
         int* flag = p.split_flags + slot * 4 + lane_group;
@@ -304,14 +313,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
           }
         }
       };
+      // a half-width unit holds columns [128 n_half, 128 n_half + 128) of its tile in accumulator columns 0..127
+      const int acc_cols = (ui.role == 3) ? 128 : BN;
+      const int col_base = tn * BN + ui.n_half * 128;
       if (ui.role == 1 || !ok) {
         // nothing more to do for this unit
       } else if constexpr (EPI == EPI_STORE || EPI == EPI_RESIDUAL) {
 #pragma unroll 1
-        for (int c0 = 0; c0 < BN; c0 += 32) {
+        for (int c0 = 0; c0 < acc_cols; c0 += 32) {
           uint32_t v[32];
           load_acc(c0, v);
-          const int col = tn * BN + c0;
+          const int col = col_base + c0;
           if (row < p.m) {
             bf16* crow = p.c + static_cast<size_t>(row) * p.ldc + col;
             const bf16* rrow = (EPI == EPI_RESIDUAL) ? p.r + static_cast<size_t>(row) * p.ldr + col : nullptr;
@@ -337,12 +349,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         // columns [128 q, 128 q + 64) of the product are gate features 64 q .., the next 64 the matching up features
         const int f_total = p.n / 2;
 #pragma unroll 1
-        for (int c0 = 0; c0 < BN / 2; c0 += 32) {
+        for (int c0 = 0; c0 < acc_cols / 2; c0 += 32) {
           const int pair = c0 >> 6, within = c0 & 63;
           uint32_t g[32], u[32];
           load_acc(pair * 128 + within, g);
           load_acc(pair * 128 + 64 + within, u);
-          const int fcol = (tn * (BN / 128) + pair) * 64 + within;
+          const int fcol = (tn * (BN / 128) + ui.n_half + pair) * 64 + within;
           if (row < p.m && fcol < f_total) {
             bf16* crow = p.c + static_cast<size_t>(row) * p.ldc + fcol;
 #pragma unroll
@@ -381,10 +393,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
           }
         }
         const int n_heads = rp.n_q_heads + 2 * rp.n_kv_heads;
-        const int heads_per_tile = BN / hd;
+        const int heads_per_tile = acc_cols / hd;
 #pragma unroll 1
         for (int hh = 0; hh < heads_per_tile; ++hh) {
-          const int head = tn * heads_per_tile + hh;
+          const int head = col_base / hd + hh;
           if (head >= n_heads) break;  // warp-uniform
 #pragma unroll 1
           for (int i0 = 0; i0 < half; i0 += 32) {
@@ -483,6 +495,7 @@ pd_status launch_tc(const GemmArgs& g, cudaStream_t stream) {
   p.n_units = tiles;
   p.main_tiles = tiles;
   p.split_scratch = nullptr; p.split_flags = nullptr; p.split_epoch = 0;
+  p.tail_halves = 0;
   {
     // last wave holds `tail` tiles: if they occupy at most half of the SMs, cut each in two along K
     const int tail = tiles % sms;
@@ -494,6 +507,11 @@ pd_status launch_tc(const GemmArgs& g, cudaStream_t stream) {
       p.main_tiles = tiles - tail;
       p.n_units = tiles + tail;
       p.split_scratch = g.split_scratch; p.split_flags = g.split_flags; p.split_epoch = g.split_epoch;
+    } else if (BN == 256 && tail > 0 && 2 * tail <= sms && g.n % 256 == 0) {
+      // otherwise give the two 128-column halves of every tail tile to different blocks
+      p.main_tiles = tiles - tail;
+      p.n_units = tiles + tail;
+      p.tail_halves = 1;
     }
   }
   const int grid = p.n_units < sms ? p.n_units : sms;
