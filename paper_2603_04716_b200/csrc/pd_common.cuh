@@ -85,12 +85,11 @@ struct GemmArgs {
   const RopeEpilogue* rope;   // EPI_ROPE_KV
   int* err_word;              // device int32: 1 = a bounded wait gave up, 2 = a position or slot was out of range
   // Optional K split of the last partial wave (see gemm_tc_kernel): fp32 scratch of at least
-  // kSplitMaxTiles * 128 * 256 * 4 bytes, kSplitMaxTiles * 4 zero-initialised flags that only ever receive
-  // increasing epochs, and this launch's epoch (> 0).  Launches sharing flags must be ordered on one stream.
+  // kSplitMaxTiles * 128 * 256 * 4 bytes and kSplitMaxTiles * 4 flags that are zero between launches.
+  // Launches sharing flags must be ordered on one stream.
   float* split_scratch;
   size_t split_scratch_bytes;
   int* split_flags;
-  int split_epoch;
 };
 constexpr int kSplitMaxTiles = 74;
 constexpr size_t kSplitScratchBytes = static_cast<size_t>(kSplitMaxTiles) * 128 * 256 * 4;
@@ -167,5 +166,4 @@ struct pd_layer {
   float2* rope_tab;                        // [max_pos, hd/2]
   int* err_word;                           // device int32
   int* split_flags;                        // device int32[kSplitMaxTiles * 4], see GemmArgs
-  int split_epoch;                         // host counter, one per K-split GEMM launch of this layer
 };

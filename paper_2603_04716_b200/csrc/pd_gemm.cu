@@ -78,12 +78,13 @@ struct GemmDev {
   int raster_group;  // row tiles that share the column-tile sweep (their A slab stays in L2)
   // Tail split: the tiles of the last, partly filled wave are each cut in two along K and given to two
   // blocks; the first writes its fp32 partial tile to `split_scratch` and raises a flag per 32-row group,
-  // the second adds it before the epilogue.  n_units = main_tiles + 2 * (tiles - main_tiles) when enabled.
+  // the second adds it before the epilogue and lowers the flag again (so the flags are zero between
+  // launches and a captured launch can be replayed).  n_units = main_tiles + 2 * (tiles - main_tiles).
   int n_units, main_tiles;
   int tail_halves;       // 1: instead, tail tiles are cut in two along N (two 128-column halves, no hand-over)
   float* split_scratch;  // [tail tile][128][BN] fp32
-  int* split_flags;      // [tail tile][4] epoch of the last partial written
-  int split_epoch;       // > 0 enables the split
+  int* split_flags;      // [tail tile][4], 1 while a partial waits to be consumed
+  int split_enable;
   int* err_word;
   RopeEpilogue rope;  // EPI_ROPE_KV only
 };
@@ -279,14 +280,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
           }
           __threadfence();
           __syncwarp();
-          if (lane == 0) *reinterpret_cast<volatile int*>(flag) = p.split_epoch;
+          if (lane == 0) *reinterpret_cast<volatile int*>(flag) = 1;
         } else {
           // second K half: wait (bounded) for the partner's rows of this warp
           bool seen = true;
           if (lane == 0) {
             const uint64_t t0 = ptx::globaltimer_ns();
             uint32_t spins = 0;
-            while (*reinterpret_cast<volatile int*>(flag) != p.split_epoch) {
+            while (*reinterpret_cast<volatile int*>(flag) != 1) {
               if ((++spins & 1023u) == 0u && (*abort_flag || ptx::globaltimer_ns() - t0 > 4000000000ull)) {
                 *abort_flag = 1;
                 seen = false;
@@ -439,6 +440,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       // all of this warp's reads of the accumulator are complete: hand the buffer back
       ptx::tc_fence_before();
       __syncwarp();
+      if (ui.role == 2 && lane == 0) {
+        // the partner's partial has been consumed: lower the flag for the next launch
+        __threadfence();
+        *reinterpret_cast<volatile int*>(p.split_flags + (ui.tile - p.main_tiles) * 4 + lane_group) = 0;
+      }
       if (lane == 0) ptx::mbar_arrive(acce_bar(acc));
       if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
     }
@@ -494,7 +500,7 @@ pd_status launch_tc(const GemmArgs& g, cudaStream_t stream) {
   const int sms = sm_count();
   p.n_units = tiles;
   p.main_tiles = tiles;
-  p.split_scratch = nullptr; p.split_flags = nullptr; p.split_epoch = 0;
+  p.split_scratch = nullptr; p.split_flags = nullptr; p.split_enable = 0;
   p.tail_halves = 0;
   {
     // last wave holds `tail` tiles: if they occupy at most half of the SMs, cut each in two along K
@@ -502,11 +508,11 @@ pd_status launch_tc(const GemmArgs& g, cudaStream_t stream) {
     const size_t need = static_cast<size_t>(tail) * BM * BN * sizeof(float);
     // (pays only for long K: with K = 4096 the parked partial tile and the hand-over cost as much as the
     // half tile they save; measured -6 % on the K = 14336 down projection, +5 % on the K = 4096 ones)
-    if (tail > 0 && 2 * tail <= sms && g.k / BK >= 128 && g.split_scratch && g.split_flags && g.split_epoch > 0 &&
+    if (tail > 0 && 2 * tail <= sms && g.k / BK >= 128 && g.split_scratch && g.split_flags &&
         need <= g.split_scratch_bytes && tail <= kSplitMaxTiles) {
       p.main_tiles = tiles - tail;
       p.n_units = tiles + tail;
-      p.split_scratch = g.split_scratch; p.split_flags = g.split_flags; p.split_epoch = g.split_epoch;
+      p.split_scratch = g.split_scratch; p.split_flags = g.split_flags; p.split_enable = 1;
     } else if (BN == 256 && tail > 0 && 2 * tail <= sms && g.n % 256 == 0) {
       // otherwise give the two 128-column halves of every tail tile to different blocks
       p.main_tiles = tiles - tail;

@@ -73,7 +73,6 @@ void enable_tail_split(pd_layer* L, pd::GemmArgs& g, uint8_t* ws, const Workspac
   g.split_scratch = reinterpret_cast<float*>(ws + w.splitk);
   g.split_scratch_bytes = pd::kSplitScratchBytes;
   g.split_flags = L->split_flags;
-  g.split_epoch = ++L->split_epoch;
 }
 
 // MLP half shared by both modes: h (residual stream after attention) -> out.
@@ -296,7 +295,6 @@ extern "C" pd_status pd_layer_create(const pd_layer_cfg* cfg, const pd_layer_wei
   if ((e = cudaMalloc(&L->err_word, sizeof(int))) != cudaSuccess) return fail(e);
   if ((e = cudaMalloc(&L->split_flags, pd::kSplitMaxTiles * 4 * sizeof(int))) != cudaSuccess) return fail(e);
   if ((e = cudaMemsetAsync(L->split_flags, 0, pd::kSplitMaxTiles * 4 * sizeof(int), st)) != cudaSuccess) return fail(e);
-  L->split_epoch = 0;
   const cudaMemcpyKind d2d = cudaMemcpyDeviceToDevice;
   if ((e = cudaMemcpyAsync(L->w_qkv, w->w_qkv, L->n_qkv * d * 2, d2d, st)) != cudaSuccess) return fail(e);
   if ((e = cudaMemcpyAsync(L->w_o, w->w_o, d * hq * 2, d2d, st)) != cudaSuccess) return fail(e);
@@ -343,6 +341,8 @@ extern "C" pd_status pd_layer_check(pd_layer* L, void* stream) {
   PD_CUDA_TRY(cudaStreamSynchronize(st));
   if (word != 0) {
     PD_CUDA_TRY(cudaMemsetAsync(L->err_word, 0, sizeof(int), st));
+    // an aborted K-split GEMM may have left a hand-over flag raised
+    PD_CUDA_TRY(cudaMemsetAsync(L->split_flags, 0, pd::kSplitMaxTiles * 4 * sizeof(int), st));
     return word == 2 ? PD_ERR_INVALID_ARG : PD_ERR_DEVICE_TIMEOUT;
   }
   return PD_OK;

@@ -28,6 +28,45 @@ struct Events {
   ~Events() { if (a) cudaEventDestroy(a); if (b) cudaEventDestroy(b); }
 };
 
+// Times work that `enqueue` puts on stream `st` (no allocation, no synchronisation inside).  After one
+// eager run the work is captured into a CUDA graph and the graph is replayed for the warm-up and timed
+// repetitions, which removes most of the per-kernel launch gaps of the ~13 small kernels per decode
+// layer; if capture is not possible the repetitions are launched eagerly.  `launches` receives the number
+// of kernels of one run.
+template <class F>
+pd_status time_enqueued(F&& enqueue, cudaStream_t st, Events& ev, int warmup, int reps, std::vector<double>* times,
+                        long long* launches) {
+  const long long l0 = pd::g_launch_count;
+  PD_TRY(enqueue());
+  *launches = pd::g_launch_count - l0;
+  PD_CUDA_TRY(cudaStreamSynchronize(st));
+  cudaGraph_t graph = nullptr;
+  cudaGraphExec_t exec = nullptr;
+  if (cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal) == cudaSuccess) {
+    const pd_status s = enqueue();
+    const cudaError_t e = cudaStreamEndCapture(st, &graph);
+    if (s != PD_OK || e != cudaSuccess || cudaGraphInstantiate(&exec, graph, 0) != cudaSuccess) exec = nullptr;
+  }
+  (void)cudaGetLastError();  // a failed capture leaves a sticky-free error behind
+  pd_status result = PD_OK;
+  for (int it = 0; it < warmup + reps && result == PD_OK; ++it) {
+    cudaError_t e = cudaEventRecord(ev.a, st);
+    if (e == cudaSuccess) {
+      if (exec) e = cudaGraphLaunch(exec, st);
+      else result = enqueue();
+    }
+    if (e == cudaSuccess) e = cudaEventRecord(ev.b, st);
+    if (e == cudaSuccess) e = cudaEventSynchronize(ev.b);
+    float ms = 0.f;
+    if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, ev.a, ev.b);
+    if (e != cudaSuccess) result = pd::cuda_fail(e);
+    else if (it >= warmup) times->push_back(ms * 1e-3);
+  }
+  if (exec) cudaGraphExecDestroy(exec);
+  if (graph) cudaGraphDestroy(graph);
+  return result;
+}
+
 double median(std::vector<double> v) {
   std::sort(v.begin(), v.end());
   const size_t n = v.size();
@@ -149,20 +188,14 @@ extern "C" pd_status pd_measure(const pd_layer_cfg* cfg_in, const pd_measure_cfg
       PD_CUDA_TRY(cudaMemcpyAsync(cu_dev.p, cu.data(), cu.size() * 4, cudaMemcpyHostToDevice, st));
       PD_TRY(pd::launch_fill_normal(static_cast<bf16*>(x.p), tokens * d, m->seed, 1000, 0.f, 1.f, st));
       std::vector<double> times;
-      for (int it = 0; it < m->warmup + m->reps; ++it) {
-        const long long l0 = pd::g_launch_count;
-        PD_CUDA_TRY(cudaEventRecord(ev.a, st));
-        PD_TRY(pd_prefill_stack(stack.layers.data(), caches.data(), nl, ring, x.p, y.p, 0,
-                                static_cast<const int32_t*>(cu_dev.p), cu.data(), m->n_req, ws.p, ws_bytes, st));
-        PD_CUDA_TRY(cudaEventRecord(ev.b, st));
-        PD_CUDA_TRY(cudaEventSynchronize(ev.b));
-        float ms = 0.f;
-        PD_CUDA_TRY(cudaEventElapsedTime(&ms, ev.a, ev.b));
-        if (it >= m->warmup) {
-          times.push_back(ms * 1e-3);
-          timed_launches += pd::g_launch_count - l0;
-        }
-      }
+      long long per_run = 0;
+      PD_TRY(time_enqueued(
+          [&] {
+            return pd_prefill_stack(stack.layers.data(), caches.data(), nl, ring, x.p, y.p, 0,
+                                    static_cast<const int32_t*>(cu_dev.p), cu.data(), m->n_req, ws.p, ws_bytes, st);
+          },
+          st, ev, m->warmup, m->reps, &times, &per_run));
+      timed_launches += per_run * m->reps;
       PD_TRY(pd_layer_check(stack.layers[0], st));
       out->prefill_time_s = median(times) * scale_layers;
       out->prefill_tok_s = tokens / out->prefill_time_s;
@@ -232,20 +265,14 @@ extern "C" pd_status pd_measure(const pd_layer_cfg* cfg_in, const pd_measure_cfg
         int max_kv = 0;
         for (int b = 0; b < B; ++b) max_kv = std::max(max_kv, kv_host[si * B + b] + 1);
         std::vector<double> times;
-        for (int it = 0; it < m->warmup + m->reps; ++it) {
-          const long long l0 = pd::g_launch_count;
-          PD_CUDA_TRY(cudaEventRecord(ev.a, st));
-          PD_TRY(pd_decode_stack(stack.layers.data(), caches.data(), nl, ring, x.p, y.p, 0, kvp, B, max_kv, ws.p,
-                                 ws_bytes, st));
-          PD_CUDA_TRY(cudaEventRecord(ev.b, st));
-          PD_CUDA_TRY(cudaEventSynchronize(ev.b));
-          float ms = 0.f;
-          PD_CUDA_TRY(cudaEventElapsedTime(&ms, ev.a, ev.b));
-          if (it >= m->warmup) {
-            times.push_back(ms * 1e-3);
-            timed_launches += pd::g_launch_count - l0;
-          }
-        }
+        long long per_run = 0;
+        PD_TRY(time_enqueued(
+            [&] {
+              return pd_decode_stack(stack.layers.data(), caches.data(), nl, ring, x.p, y.p, 0, kvp, B, max_kv, ws.p,
+                                     ws_bytes, st);
+            },
+            st, ev, m->warmup, m->reps, &times, &per_run));
+        timed_launches += per_run * m->reps;
         step_time_sum += median(times);
 
         // the attention kernel alone, over the same caches (q = whatever the last pass left in the workspace)
