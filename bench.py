@@ -35,6 +35,15 @@ KV_START = 2048
 L_OUT = 256
 SWEEP = [1, 2, 4, 8, 16, 32, 64, 128, 256]
 TTFT_SLO, TPOT_SLO, TP_TOTAL = 2.0, 0.050, 2e5
+# DRAM traffic per launch from ncu (dram__bytes_read.sum + dram__bytes_write.sum), captured on the same shapes with
+# one layer (profiles/gemm_tc_prefill_8b_ncu_full.md, profiles/prefill_attn_tc_and_decode_kernels_ncu_full.md).
+# Set an entry to None whenever the kernel changes after the capture.
+NCU_TRAFFIC = {
+    "gemm_tc_kernel": {"bytes_per_launch": 328.5e6, "algorithmic_bytes_per_launch": 238.8e6,
+                       "note": "mean over the four prefill projections of a layer (1313.8 MB / 4)"},
+    "decode_attn_kernel": {"bytes_per_launch": 2.1563e9, "algorithmic_bytes_per_launch": 2.1485e9,
+                           "note": "B = 256 at KV length 2049; grows in proportion to the KV length"},
+}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -445,12 +454,15 @@ def main():
                          "bound": "tensor", "achieved": gemm_tf, "peak": peak_tf, "unit": "TFLOP/s",
                          "frac": gemm_tf / peak_tf, "frac_of_burst_peak": gemm_tf / peaks["bf16_tflops"],
                          "peak_source": peaks["source"] + " (sustained bf16)", "launches": gemm_n,
-                         "avg_launch_ms": gemm_s / max(1, gemm_n) * 1e3, "traffic": None,
+                         "avg_launch_ms": gemm_s / max(1, gemm_n) * 1e3, "traffic": NCU_TRAFFIC["gemm_tc_kernel"]["bytes_per_launch"], "traffic_unit": "DRAM bytes per launch (ncu)",
+                         "traffic_detail": NCU_TRAFFIC["gemm_tc_kernel"],
                          "timing": "CUDA events around each launch in a separate traced pass of the same step"},
             "roofline_decode_attention": {"kernel": "decode_attn_kernel", "bound": "hbm", "achieved": attn_gbs,
                                           "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": attn_gbs / peaks["hbm_gbs"],
                                           "launches": attn_dec_n, "avg_launch_ms": attn_dec_s / max(1, attn_dec_n) * 1e3,
-                                          "traffic": None},
+                                          "traffic": NCU_TRAFFIC["decode_attn_kernel"]["bytes_per_launch"],
+                                          "traffic_unit": "DRAM bytes per launch (ncu)",
+                                          "traffic_detail": NCU_TRAFFIC["decode_attn_kernel"]},
             "kernel_time_ms": {"prefill": {k: v[0] * 1e3 for k, v in tr_pre.items() if v[1]},
                                "decode": {k: v[0] * 1e3 / len(dec_ts) for k, v in tr_dec.items() if v[1]}},
             "e2e": {"value": e2e_value, "unit": "tok/s", "h2d_bytes_per_step": xh.numel() * 2 + 8,
