@@ -12,6 +12,7 @@ import numpy as np
 # stream ids (tensor kinds)
 S_WQKV, S_WO, S_WGATE, S_WUP, S_WDOWN, S_GATTN, S_GMLP = range(7)
 S_X, S_KCACHE, S_VCACHE, S_XSTEP, S_LENGTHS, S_ARRIVALS, S_SERVICE, S_ROWS = range(16, 24)
+S_EMBED, S_LMHEAD, S_GFINAL, S_TOKENS = range(32, 36)
 
 
 def _rng(seed: int, stream: int, sub: int = 0) -> np.random.Generator:
@@ -60,6 +61,21 @@ def layer_weights(d_model: int, n_q_heads: int, n_kv_heads: int, head_dim: int, 
         "g_attn": normal_bf16(seed, S_GATTN, (d_model,), std, mean=1.0, sub=layer),
         "g_mlp": normal_bf16(seed, S_GMLP, (d_model,), std, mean=1.0, sub=layer),
     }
+
+
+def model_head_weights(vocab: int, d_model: int, seed: int = 0, std: float = 0.02) -> dict:
+    """Embedding table ~N(0, 1) (the scale the layer inputs are drawn with), LM head ~N(0, std),
+    final gain 1 + N(0, std); bf16 values as float32."""
+    return {
+        "embed": normal_bf16(seed, S_EMBED, (vocab, d_model), 1.0),
+        "g_final": normal_bf16(seed, S_GFINAL, (d_model,), std, mean=1.0),
+        "lm_head": normal_bf16(seed, S_LMHEAD, (vocab, d_model), std),
+    }
+
+
+def token_ids(seed: int, n: int, vocab: int, sub: int = 0) -> np.ndarray:
+    """n token ids uniform in [0, vocab)."""
+    return _rng(seed, S_TOKENS, sub).integers(0, vocab, size=n, dtype=np.int64).astype(np.int32)
 
 
 def activations(seed: int, n_tokens: int, d_model: int, sub: int = 0, stream: int = S_X) -> np.ndarray:
