@@ -192,6 +192,64 @@ pd_status pd_decode_stack(pd_layer* const* layers, const pd_kv_cache* caches, in
  * a kernel gave up).  Synchronises `stream`.  PD_OK or PD_ERR_DEVICE_TIMEOUT. */
 pd_status pd_layer_check(pd_layer* layer, void* stream);
 
+/* ------------------------------------------------------------ whole model */
+
+/* A whole-model step: token embedding, the layer stack, final RMSNorm, LM-head projection,
+ * greedy sampling.  The paper's TTFT runs to the first output token and its TPOT from one
+ * output token to the next ("Acquire prefill throughput under TTFT constraints", "Acquire
+ * decode throughput under TPOT constraints"), so a measured step ends with a token id; the
+ * paper does not define the network around the layers, this is the standard one:
+ *   x = E[token];  h = layers(x);  n = RMSNorm(h_last) * g_final;  logits = n W_lm^T (fp32);
+ *   next = argmax logits, the lowest index among equal maxima.
+ * Prefill takes the last row of every request, decode every row. */
+typedef struct pd_model pd_model;
+
+/* Device pointers, bf16, row-major; copied at creation.  vocab must be a multiple of 4. */
+typedef struct {
+  uint32_t struct_size;
+  int32_t vocab;
+  const void* embed;   /* [vocab, d_model] */
+  const void* g_final; /* [d_model] */
+  const void* lm_head; /* [vocab, d_model] */
+} pd_model_weights;
+
+/* The layers (all of one shape) are borrowed: they must outlive the model.  The copies are
+ * enqueued on `stream`. */
+pd_status pd_model_create(pd_layer* const* layers, int32_t n_layers, const pd_model_weights* w, void* stream,
+                          pd_model** out);
+pd_status pd_model_destroy(pd_model* model);
+
+/* Workspace for prefill passes of up to max_tokens tokens in max_requests requests and decode
+ * steps of up to max_batch sequences over max_kv_len cached tokens (includes fp32 logits for
+ * the case that the caller passes no logits buffer). */
+pd_status pd_model_workspace_bytes(const pd_model* model, int32_t max_tokens, int32_t max_requests,
+                                   int32_t max_batch, int32_t max_kv_len, size_t* out_bytes);
+
+/* Prefill of a packed ragged batch of prompts up to the first output token.
+ *   tokens_dev  device int32[T] token ids (T = cu_seqlens[n_req]); an id outside [0, vocab)
+ *               gives a zero embedding row and makes pd_model_check return PD_ERR_INVALID_ARG
+ *   cu_seqlens  as for pd_prefill_layer; request r is written to cache sequence r of
+ *               caches[i % n_caches] for layer i
+ *   next_dev    device int32[n_req]: the greedy token after each prompt, -1 for an empty one
+ *   logits_dev  optional device fp32[n_req, vocab] (16-byte aligned); NULL keeps the logits
+ *               in the workspace
+ * Only enqueues work on `stream`; allocates nothing. */
+pd_status pd_model_prefill(pd_model* model, const int32_t* tokens_dev, const int32_t* cu_seqlens_dev,
+                           const int32_t* cu_seqlens_host, int32_t n_req, const pd_kv_cache* caches,
+                           int32_t n_caches, int32_t* next_dev, float* logits_dev, void* workspace,
+                           size_t workspace_bytes, void* stream);
+
+/* One decode step: tokens_dev[b] is the newest token of sequence b whose kv_len_dev[b] earlier
+ * tokens are cached; its K/V are appended in every layer and next_dev[b] receives the greedy
+ * next token.  Captured in a CUDA graph this is the whole-model decode step. */
+pd_status pd_model_decode_step(pd_model* model, const int32_t* tokens_dev, const int32_t* kv_len_dev, int32_t B,
+                               int32_t max_kv_len, const pd_kv_cache* caches, int32_t n_caches, int32_t* next_dev,
+                               float* logits_dev, void* workspace, size_t workspace_bytes, void* stream);
+
+/* pd_layer_check over every layer plus the model's own error word (bad token id).
+ * Synchronises `stream`. */
+pd_status pd_model_check(pd_model* model, void* stream);
+
 /* Plain C[M,N] = A[M,K] * B[N,K]^T in bf16 with fp32 accumulation on the tensor cores
  * (the contraction every projection of the layer uses), exposed for unit tests and
  * roofline measurement.  A, B, C device bf16 row-major; K a multiple of 64, N of 16.
@@ -210,7 +268,7 @@ int64_t pd_launch_count(void);
 #define PD_TRACE_CLASSES 16
 enum {
   PD_K_GEMM_QKV = 0, PD_K_GEMM_O = 1, PD_K_GEMM_GATE_UP = 2, PD_K_GEMM_DOWN = 3, PD_K_ATTN_PREFILL = 4,
-  PD_K_ATTN_DECODE = 5, PD_K_RMSNORM = 6
+  PD_K_ATTN_DECODE = 5, PD_K_RMSNORM = 6, PD_K_EMBED = 7, PD_K_LM_HEAD = 8, PD_K_SAMPLE = 9
 };
 typedef struct {
   uint32_t struct_size;

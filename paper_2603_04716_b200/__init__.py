@@ -36,9 +36,12 @@ EXPORTS = [
     "pd_layer_check", "pd_gemm_bf16", "pd_measure", "pd_allocate", "pd_queue_replay",
     "pd_launch_count", "pd_trace_begin", "pd_trace_end", "pd_decode_attention", "pd_decode_attention_workspace_bytes",
     "pd_decode_attention_noalloc", "pd_prefill_chunk_layer",
+    "pd_model_create", "pd_model_destroy", "pd_model_workspace_bytes", "pd_model_prefill", "pd_model_decode_step",
+    "pd_model_check",
 ]
 
-TRACE_CLASSES = ["gemm_qkv", "gemm_o", "gemm_gate_up", "gemm_down", "attn_prefill", "attn_decode", "rmsnorm"]
+TRACE_CLASSES = ["gemm_qkv", "gemm_o", "gemm_gate_up", "gemm_down", "attn_prefill", "attn_decode", "rmsnorm",
+                 "embed", "lm_head", "sample"]
 
 
 class PdError(RuntimeError):
@@ -59,6 +62,11 @@ class pd_layer_cfg(C.Structure):
 class pd_layer_weights(C.Structure):
     _fields_ = [("struct_size", C.c_uint32)] + [(n, C.c_void_p) for n in
                 ("w_qkv", "w_o", "w_gate", "w_up", "w_down", "g_attn", "g_mlp")]
+
+
+class pd_model_weights(C.Structure):
+    _fields_ = [("struct_size", C.c_uint32), ("vocab", C.c_int32), ("embed", C.c_void_p), ("g_final", C.c_void_p),
+                ("lm_head", C.c_void_p)]
 
 
 class pd_kv_cache(C.Structure):
@@ -134,6 +142,14 @@ _lib.pd_decode_attention.argtypes = [C.POINTER(pd_layer_cfg), _P, C.c_int32, _P,
                                      C.POINTER(pd_kv_cache), _P, C.c_size_t, _P]
 _lib.pd_decode_attention_noalloc.argtypes = [C.POINTER(pd_layer_cfg), _P, C.c_int32, _P, _P, C.c_int32, C.c_int32,
                                              C.POINTER(pd_kv_cache), _P]
+_lib.pd_model_create.argtypes = [C.POINTER(_P), C.c_int32, C.POINTER(pd_model_weights), _P, C.POINTER(_P)]
+_lib.pd_model_destroy.argtypes = [_P]
+_lib.pd_model_check.argtypes = [_P, _P]
+_lib.pd_model_workspace_bytes.argtypes = [_P, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.POINTER(C.c_size_t)]
+_lib.pd_model_prefill.argtypes = [_P, _P, _P, C.POINTER(C.c_int32), C.c_int32, C.POINTER(pd_kv_cache), C.c_int32, _P,
+                                  _P, _P, C.c_size_t, _P]
+_lib.pd_model_decode_step.argtypes = [_P, _P, _P, C.c_int32, C.c_int32, C.POINTER(pd_kv_cache), C.c_int32, _P, _P, _P,
+                                      C.c_size_t, _P]
 _lib.pd_launch_count.restype = C.c_int64
 _lib.pd_trace_end.argtypes = [C.POINTER(pd_trace_report)]
 for _n in EXPORTS:
@@ -322,6 +338,57 @@ def pd_decode_stack(layers, caches, x, out, io_on_host: bool, kv_len, batch: int
     _check(_lib.pd_decode_stack(_layer_array(layers), _cache_array(caches), len(layers), len(caches), _ptr(x),
                                 _ptr(out), int(io_on_host), _ptr(kv_len), batch, max_kv_len, _ptr(workspace),
                                 workspace_bytes, _stream_ptr(stream)), "pd_decode_stack")
+
+
+class Model:
+    """Owns a pd_model handle (embedding, final norm gain, LM head) over borrowed layers."""
+
+    def __init__(self, layers, vocab: int, embed, g_final, lm_head, stream=None):
+        self.layers = list(layers)          # keeps the borrowed layers alive
+        self.vocab = vocab
+        w = pd_model_weights(C.sizeof(pd_model_weights), vocab, _ptr(embed), _ptr(g_final), _ptr(lm_head))
+        h = _P()
+        _check(_lib.pd_model_create(_layer_array(self.layers), len(self.layers), C.byref(w), _stream_ptr(stream),
+                                    C.byref(h)), "pd_model_create")
+        self.handle = h
+
+    def close(self):
+        if getattr(self, "handle", None):
+            _lib.pd_model_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def pd_model_workspace_bytes(model: Model, max_tokens: int, max_requests: int, max_batch: int,
+                             max_kv_len: int) -> int:
+    out = C.c_size_t(0)
+    _check(_lib.pd_model_workspace_bytes(model.handle, max_tokens, max_requests, max_batch, max_kv_len,
+                                         C.byref(out)), "pd_model_workspace_bytes")
+    return out.value
+
+
+def pd_model_prefill(model: Model, tokens_dev, cu_seqlens_dev, cu_seqlens_host, caches, next_dev, workspace,
+                     workspace_bytes: int, logits_dev=None, stream=None):
+    cu = _i32_array(cu_seqlens_host)
+    _check(_lib.pd_model_prefill(model.handle, _ptr(tokens_dev), _ptr(cu_seqlens_dev), cu, len(cu_seqlens_host) - 1,
+                                 _cache_array(caches), len(caches), _ptr(next_dev), _ptr(logits_dev),
+                                 _ptr(workspace), workspace_bytes, _stream_ptr(stream)), "pd_model_prefill")
+
+
+def pd_model_decode_step(model: Model, tokens_dev, kv_len_dev, batch: int, max_kv_len: int, caches, next_dev,
+                         workspace, workspace_bytes: int, logits_dev=None, stream=None):
+    _check(_lib.pd_model_decode_step(model.handle, _ptr(tokens_dev), _ptr(kv_len_dev), batch, max_kv_len,
+                                     _cache_array(caches), len(caches), _ptr(next_dev), _ptr(logits_dev),
+                                     _ptr(workspace), workspace_bytes, _stream_ptr(stream)), "pd_model_decode_step")
+
+
+def pd_model_check(model: Model, stream=None):
+    _check(_lib.pd_model_check(model.handle, _stream_ptr(stream)), "pd_model_check")
 
 
 def pd_layer_check(layer: Layer, stream=None):

@@ -118,6 +118,13 @@ pd_status launch_skinny_residual(const float* acc, const bf16* x, bf16* h, const
 // out[B, F] = silu(gate) * up from acc[B, 2F] whose columns follow the 64/64 interleaved weight rows.
 pd_status launch_skinny_swiglu(const float* acc, bf16* out, int batch, int f, cudaStream_t s);
 
+// ------------------------------------------------------------ whole model
+// Pieces of the whole-model step around the layer stack (the measurement harness times them alone).
+pd_status model_embed(pd_model* m, const int32_t* tokens_dev, int n, bf16* x, cudaStream_t st);
+// h -> logits -> greedy tokens; cu_dev != NULL selects the last row of each request first (into sel).
+pd_status model_head(pd_model* m, const bf16* h, const int32_t* cu_dev, int rows, bf16* sel, bf16* norm,
+                     float* logits, int32_t* next_dev, cudaStream_t st);
+
 // ------------------------------------------------------------ elementwise
 pd_status launch_rmsnorm(const bf16* x, const bf16* gain, bf16* y, int rows, int d, float eps, cudaStream_t s);
 
