@@ -419,6 +419,61 @@ def main():
     (e2e_pre_s,) = max_over_ranks([e2e_pre_s], dist, dev)
     e2e_value = world * L_IN / (e2e_pre_s * scale)
 
+    # ---- whole-model step over the same layers: token ids in, greedy token out (embedding, final norm,
+    # LM head over a 128256-entry vocabulary and the sampler added to the stack)
+    vocab = 128256
+    model = pd.Model(layers, vocab, randn_bf16(vocab, d), randn_bf16(d, std=0.02, mean=1.0),
+                     randn_bf16(vocab, d, std=0.02))
+    mws_bytes = pd.pd_model_workspace_bytes(model, L_IN, 1, b_max, cap)
+    mws = torch.empty(mws_bytes, dtype=torch.uint8, device=dev)
+    tok_pre = torch.randint(0, vocab, (L_IN,), dtype=torch.int32, device=dev, generator=gen_t)
+    tok_dec = torch.randint(0, vocab, (b_max,), dtype=torch.int32, device=dev, generator=gen_t)
+    next_pre = torch.zeros(1, dtype=torch.int32, device=dev)
+    next_dec = torch.zeros(b_max, dtype=torch.int32, device=dev)
+    t_mid = dec_ts[len(dec_ts) // 2]
+
+    def timed(fn, reps=3):
+        fn()
+        out_s = []
+        for _ in range(reps):
+            a, b = ev(), ev()
+            a.record()
+            fn()
+            b.record()
+            b.synchronize()
+            out_s.append(a.elapsed_time(b) * 1e-3)
+        return statistics.median(out_s)
+
+    def model_prefill():
+        pd.pd_model_prefill(model, tok_pre, cu_dev, cu_host, pre_caches, next_pre, mws, mws_bytes)
+
+    def model_decode():
+        pd.pd_model_decode_step(model, tok_dec, kv_lens[t_mid], b_star, KV_START + t_mid + 1, dec_caches, next_dec,
+                                mws, mws_bytes)
+
+    wm_pre = timed(runner("model_prefill", model_prefill)[0])
+    wm_dec = timed(runner("model_decode", model_decode)[0])
+    pd.pd_model_check(model)
+
+    def head_time(fn):
+        """Embedding + LM head + sampler kernels of one traced (eager) pass, by their CUDA events."""
+        pd.pd_trace_begin()
+        fn()
+        tr = pd.pd_trace_end()
+        return sum(tr[k][0] for k in ("embed", "lm_head", "sample"))
+
+    head_pre, head_dec = head_time(model_prefill), head_time(model_decode)
+    # whole-model time at 32 layers: the measured pass with its layer-stack part scaled up
+    wm_pre_s, wm_dec_s = (wm_pre - head_pre) * scale + head_pre, (wm_dec - head_dec) * scale + head_dec
+    wm_pre_s, wm_dec_s = max_over_ranks([wm_pre_s, wm_dec_s], dist, dev)
+    whole_model = {"vocab": vocab, "ttft_compute_ms": wm_pre_s * 1e3, "prefill_tok_s": world * L_IN / wm_pre_s,
+                   "tpot_ms": wm_dec_s * 1e3, "decode_tok_s": world * b_star / wm_dec_s,
+                   "head_ms_prefill": head_pre * 1e3, "head_ms_decode": head_dec * 1e3,
+                   "lm_head_gbs_decode": vocab * d * 2 / head_dec / 1e9 if head_dec > 0 else None,
+                   "first_token": int(next_pre.item()),
+                   "note": "graph replay of pd_model_prefill / pd_model_decode_step; head = embedding + LM head + "
+                           "sampler kernels by CUDA events in a traced pass"}
+
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         sample_l = L_IN
@@ -468,6 +523,7 @@ def main():
             "e2e": {"value": e2e_value, "unit": "tok/s", "h2d_bytes_per_step": xh.numel() * 2 + 8,
                     "d2h_bytes_per_step": yh.numel() * 2,
                     "decode_tok_s": world * b_star / (statistics.mean(e2e_dec) * scale)},
+            "whole_model": whole_model,
             "gpu_launches": launches, "clocks": clocks, "wall_s_timed_region": t_wall,
         }
         if cpu:

@@ -287,7 +287,11 @@ pd_status pd_trace_end(pd_trace_report* out);
  * Decode (paper, "Acquire decode throughput ..."): for every batch size, steps t = 0,
  * step_stride, ... < n_steps (and the last step) run the stack at kv_len = kv_len_start + t;
  * TPOT(B) is the mean step time scaled to n_layers_model layers.
- * Either part is skipped when its count (n_req / n_batch_sizes) is 0. */
+ * Either part is skipped when its count (n_req / n_batch_sizes) is 0.
+ * With vocab > 0 the step is the whole-model step: the time of the token embedding, the final
+ * RMSNorm, the LM head over a vocabulary of that size and the greedy sampling (once per step,
+ * not per layer; timed on their own, median of `reps`) is added to prefill_time_s and TPOT(B)
+ * and reported in prefill_head_s / decode_head_s. */
 typedef struct {
   uint32_t struct_size;
   int32_t n_layers_run, n_layers_model;
@@ -299,6 +303,7 @@ typedef struct {
   int32_t n_batch_sizes;
   int32_t kv_len_start, n_steps, step_stride;
   const int32_t* kv_len_mix; /* optional host int32[max batch]: per-sequence start lengths (ragged); NULL = kv_len_start */
+  int32_t vocab;             /* 0: layer stack only; > 0 (a multiple of 4): whole-model step */
 } pd_measure_cfg;
 
 typedef struct {
@@ -315,6 +320,8 @@ typedef struct {
   double attn_time_s[32];           /* decode-attention kernel alone, per layer, mean over the steps */
   double attn_frac_hbm_peak[32];
   int32_t gpu_launches;             /* kernels launched inside the timed regions */
+  double prefill_head_s;            /* embedding + final norm + LM head + sampling of the prefill pass (vocab > 0) */
+  double decode_head_s[32];         /* the same for one decode step at batch[i] */
 } pd_measurement;
 
 pd_status pd_measure(const pd_layer_cfg* cfg, const pd_measure_cfg* mcfg, double peak_bf16_flops,

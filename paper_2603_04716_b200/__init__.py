@@ -80,7 +80,7 @@ class pd_measure_cfg(C.Structure):
                 ("l_in", C.POINTER(C.c_int32)), ("n_req", C.c_int32),
                 ("batch_sizes", C.POINTER(C.c_int32)), ("n_batch_sizes", C.c_int32),
                 ("kv_len_start", C.c_int32), ("n_steps", C.c_int32), ("step_stride", C.c_int32),
-                ("kv_len_mix", C.POINTER(C.c_int32))]
+                ("kv_len_mix", C.POINTER(C.c_int32)), ("vocab", C.c_int32)]
 
 
 class pd_measurement(C.Structure):
@@ -89,7 +89,7 @@ class pd_measurement(C.Structure):
                 ("n_points", C.c_int32), ("batch", C.c_int32 * 32), ("tpot_s", C.c_double * 32),
                 ("decode_bytes", C.c_double * 32), ("decode_frac_hbm_peak", C.c_double * 32),
                 ("attn_time_s", C.c_double * 32), ("attn_frac_hbm_peak", C.c_double * 32),
-                ("gpu_launches", C.c_int32)]
+                ("gpu_launches", C.c_int32), ("prefill_head_s", C.c_double), ("decode_head_s", C.c_double * 32)]
 
 
 class pd_trace_report(C.Structure):
@@ -402,12 +402,14 @@ def pd_gemm_bf16(a, b, c, m: int, n: int, k: int, err_word=None, stream=None):
 def pd_measure(cfg: LayerConfig, *, n_layers_run: int, n_layers_model: int, warmup: int = 3, reps: int = 10,
                seed: int = 0, l_in=(), batch_sizes=(), kv_len_start: int = 0, n_steps: int = 1,
                step_stride: int = 1, kv_len_mix=None, peak_bf16_flops: float = 0.0,
-               peak_hbm_bytes_s: float = 0.0) -> dict:
+               peak_hbm_bytes_s: float = 0.0, vocab: int = 0) -> dict:
+    """vocab > 0 measures the whole-model step (embedding, final norm, LM head and greedy sampling added
+    to the prefill time and to every TPOT)."""
     l_arr = _i32_array(l_in) if len(l_in) else None
     b_arr = _i32_array(batch_sizes) if len(batch_sizes) else None
     mix = _i32_array(kv_len_mix) if kv_len_mix is not None else None
     m = pd_measure_cfg(C.sizeof(pd_measure_cfg), n_layers_run, n_layers_model, warmup, reps, seed,
-                       l_arr, len(l_in), b_arr, len(batch_sizes), kv_len_start, n_steps, step_stride, mix)
+                       l_arr, len(l_in), b_arr, len(batch_sizes), kv_len_start, n_steps, step_stride, mix, vocab)
     out = pd_measurement()
     _check(_lib.pd_measure(C.byref(cfg.c_struct()), C.byref(m), peak_bf16_flops, peak_hbm_bytes_s, C.byref(out)),
            "pd_measure")
@@ -419,6 +421,7 @@ def pd_measure(cfg: LayerConfig, *, n_layers_run: int, n_layers_model: int, warm
         "decode_bytes": list(out.decode_bytes[:n]), "decode_frac_hbm_peak": list(out.decode_frac_hbm_peak[:n]),
         "attn_time_s": list(out.attn_time_s[:n]), "attn_frac_hbm_peak": list(out.attn_frac_hbm_peak[:n]),
         "gpu_launches": out.gpu_launches,
+        "prefill_head_s": out.prefill_head_s, "decode_head_s": list(out.decode_head_s[:n]),
     }
 
 

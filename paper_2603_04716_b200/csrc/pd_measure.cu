@@ -23,6 +23,11 @@ struct Stack {
   ~Stack() { for (pd_layer* l : layers) pd_layer_destroy(l); }
 };
 
+struct ModelGuard {
+  pd_model* m = nullptr;
+  ~ModelGuard() { pd_model_destroy(m); }
+};
+
 struct Events {
   cudaEvent_t a = nullptr, b = nullptr;
   ~Events() { if (a) cudaEventDestroy(a); if (b) cudaEventDestroy(b); }
@@ -109,6 +114,37 @@ pd_status build_stack(const pd_layer_cfg& cfg, int n_layers, uint64_t seed, cuda
   return PD_OK;
 }
 
+// Synthetic embedding table, final gain and LM head over the stack's layers.
+pd_status build_model(const pd_layer_cfg& cfg, Stack& stack, int vocab, uint64_t seed, cudaStream_t st, ModelGuard* out) {
+  const size_t table = static_cast<size_t>(vocab) * cfg.d_model;
+  DevBuf e, h, g;
+  PD_CUDA_TRY(e.alloc(table * 2));
+  PD_CUDA_TRY(h.alloc(table * 2));
+  PD_CUDA_TRY(g.alloc(static_cast<size_t>(cfg.d_model) * 2));
+  PD_TRY(pd::launch_fill_normal(static_cast<bf16*>(e.p), table, seed, 5000, 0.f, 1.f, st));
+  PD_TRY(pd::launch_fill_normal(static_cast<bf16*>(h.p), table, seed, 5001, 0.f, 0.02f, st));
+  PD_TRY(pd::launch_fill_normal(static_cast<bf16*>(g.p), cfg.d_model, seed, 5002, 1.f, 0.02f, st));
+  pd_model_weights w{};
+  w.struct_size = sizeof(w);
+  w.vocab = vocab; w.embed = e.p; w.g_final = g.p; w.lm_head = h.p;
+  PD_TRY(pd_model_create(stack.layers.data(), static_cast<int>(stack.layers.size()), &w, st, &out->m));
+  PD_CUDA_TRY(cudaStreamSynchronize(st));  // the temporaries die here
+  return PD_OK;
+}
+
+// Uniform token ids from a counter hash (host side; the values only steer which embedding rows are read).
+std::vector<int32_t> synthetic_tokens(size_t n, int vocab, uint64_t seed) {
+  std::vector<int32_t> t(n);
+  for (size_t i = 0; i < n; ++i) {
+    uint64_t z = seed * 0x9E3779B97F4A7C15ull + i + 0x7F4A7C15ull;
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+    z ^= z >> 31;
+    t[i] = static_cast<int32_t>(z % static_cast<uint64_t>(vocab));
+  }
+  return t;
+}
+
 // Number of KV buffers to cycle through: one per layer if memory allows, otherwise as many as
 // fit in 70 % of the free memory (still far larger than L2 in total).
 int cache_ring(size_t bytes_per_cache, int n_layers) {
@@ -127,7 +163,7 @@ extern "C" pd_status pd_measure(const pd_layer_cfg* cfg_in, const pd_measure_cfg
   if (!cfg_in || !m || !out || m->struct_size != sizeof(pd_measure_cfg) || cfg_in->struct_size != sizeof(pd_layer_cfg))
     return PD_ERR_INVALID_ARG;
   if (m->n_layers_run <= 0 || m->n_layers_model <= 0 || m->warmup < 0 || m->reps <= 0) return PD_ERR_INVALID_ARG;
-  if (m->n_req < 0 || m->n_batch_sizes < 0 || m->n_batch_sizes > 32) return PD_ERR_INVALID_ARG;
+  if (m->n_req < 0 || m->n_batch_sizes < 0 || m->n_batch_sizes > 32 || m->vocab < 0) return PD_ERR_INVALID_ARG;
   if ((m->n_req > 0 && !m->l_in) || (m->n_batch_sizes > 0 && (!m->batch_sizes || m->n_steps <= 0 || m->kv_len_start < 0)))
     return PD_ERR_INVALID_ARG;
   std::memset(out, 0, sizeof(*out));
@@ -147,6 +183,8 @@ extern "C" pd_status pd_measure(const pd_layer_cfg* cfg_in, const pd_measure_cfg
 
   Stack stack;
   PD_TRY(build_stack(cfg, nl, m->seed, st, &stack));
+  ModelGuard model;
+  if (m->vocab > 0) PD_TRY(build_model(cfg, stack, m->vocab, m->seed, st, &model));
   const long long launches_before = pd::g_launch_count;
   long long timed_launches = 0;
 
@@ -198,6 +236,31 @@ extern "C" pd_status pd_measure(const pd_layer_cfg* cfg_in, const pd_measure_cfg
       timed_launches += per_run * m->reps;
       PD_TRY(pd_layer_check(stack.layers[0], st));
       out->prefill_time_s = median(times) * scale_layers;
+      if (model.m) {  // embedding in front, final norm + LM head + sampling behind: once per pass
+        const std::vector<int32_t> tok = synthetic_tokens(tokens, m->vocab, m->seed);
+        DevBuf tok_dev, sel, norm, logits, next;
+        PD_CUDA_TRY(tok_dev.alloc(tok.size() * 4));
+        PD_CUDA_TRY(sel.alloc(m->n_req * d * 2));
+        PD_CUDA_TRY(norm.alloc(m->n_req * d * 2));
+        PD_CUDA_TRY(logits.alloc(static_cast<size_t>(m->n_req) * m->vocab * 4));
+        PD_CUDA_TRY(next.alloc(m->n_req * 4));
+        PD_CUDA_TRY(cudaMemcpyAsync(tok_dev.p, tok.data(), tok.size() * 4, cudaMemcpyHostToDevice, st));
+        std::vector<double> htimes;
+        long long hrun = 0;
+        PD_TRY(time_enqueued(
+            [&] {
+              PD_TRY(pd::model_embed(model.m, static_cast<const int32_t*>(tok_dev.p), tokens, static_cast<bf16*>(x.p), st));
+              return pd::model_head(model.m, static_cast<const bf16*>(y.p), static_cast<const int32_t*>(cu_dev.p),
+                                    m->n_req, static_cast<bf16*>(sel.p), static_cast<bf16*>(norm.p),
+                                    static_cast<float*>(logits.p), static_cast<int32_t*>(next.p), st);
+            },
+            st, ev, m->warmup, m->reps, &htimes, &hrun));
+        timed_launches += hrun * m->reps;
+        PD_TRY(pd_model_check(model.m, st));
+        out->prefill_head_s = median(htimes);
+        out->prefill_time_s += out->prefill_head_s;
+        out->prefill_flops += 2.0 * m->n_req * static_cast<double>(m->vocab) * d;
+      }
       out->prefill_tok_s = tokens / out->prefill_time_s;
       if (peak_bf16_flops > 0) out->prefill_frac_bf16_peak = out->prefill_flops / out->prefill_time_s / peak_bf16_flops;
     }
@@ -306,14 +369,40 @@ extern "C" pd_status pd_measure(const pd_layer_cfg* cfg_in, const pd_measure_cfg
         attn_time_sum += median(atimes);
       }
       PD_TRY(pd_layer_check(stack.layers[0], st));
+      double head_time = 0.0;
+      if (model.m) {
+        const std::vector<int32_t> tok = synthetic_tokens(B, m->vocab, m->seed + bi);
+        DevBuf tok_dev, norm, logits, next;
+        PD_CUDA_TRY(tok_dev.alloc(tok.size() * 4));
+        PD_CUDA_TRY(norm.alloc(B * d * 2));
+        PD_CUDA_TRY(logits.alloc(static_cast<size_t>(B) * m->vocab * 4));
+        PD_CUDA_TRY(next.alloc(B * 4));
+        PD_CUDA_TRY(cudaMemcpyAsync(tok_dev.p, tok.data(), tok.size() * 4, cudaMemcpyHostToDevice, st));
+        std::vector<double> htimes;
+        long long hrun = 0;
+        PD_TRY(time_enqueued(
+            [&] {
+              PD_TRY(pd::model_embed(model.m, static_cast<const int32_t*>(tok_dev.p), B, static_cast<bf16*>(x.p), st));
+              return pd::model_head(model.m, static_cast<const bf16*>(y.p), nullptr, B, nullptr,
+                                    static_cast<bf16*>(norm.p), static_cast<float*>(logits.p),
+                                    static_cast<int32_t*>(next.p), st);
+            },
+            st, ev, m->warmup, m->reps, &htimes, &hrun));
+        timed_launches += hrun * m->reps;
+        PD_TRY(pd_model_check(model.m, st));
+        head_time = median(htimes);
+      }
       const double step_time = step_time_sum / steps.size();  // n_layers_run layers
       const double attn_time = attn_time_sum / steps.size();  // one layer
       const double kv_bytes_layer = kv_tokens_mean * 2.0 * kv_row;
       const double bytes_layer = static_cast<double>(params_bytes) + kv_bytes_layer + B * 2.0 * kv_row + 2.0 * B * d * 2;
       const int pi = out->n_points++;
       out->batch[pi] = B;
-      out->tpot_s[pi] = step_time * scale_layers;
+      out->tpot_s[pi] = step_time * scale_layers + head_time;
+      out->decode_head_s[pi] = head_time;
       out->decode_bytes[pi] = bytes_layer * m->n_layers_model;
+      if (model.m)  // LM head once, embedding rows, logits written and read back by the sampler
+        out->decode_bytes[pi] += static_cast<double>(m->vocab) * d * 2 + 2.0 * B * d * 2 + 2.0 * B * m->vocab * 4.0;
       out->attn_time_s[pi] = attn_time;
       if (peak_hbm_bytes_s > 0) {
         out->decode_frac_hbm_peak[pi] = out->decode_bytes[pi] / out->tpot_s[pi] / peak_hbm_bytes_s;

@@ -49,6 +49,26 @@ def test_measure_8b_shape_two_layers_scaled(pdlib):
     assert m["decode_bytes"][2] > m["decode_bytes"][0]
 
 
+def test_measure_whole_model_step_adds_the_head(pdlib):
+    """vocab > 0: the prefill time and every TPOT contain the embedding + final norm + LM head + sampling
+    time, which is also reported on its own; the LM head alone must stream the table at a plausible rate."""
+    shape = dict(d_model=4096, n_q_heads=32, n_kv_heads=8, head_dim=128, d_ff=14336)
+    cfg = pdlib.LayerConfig(**shape, max_pos=1024)
+    vocab = 128256
+    m = pdlib.pd_measure(cfg, n_layers_run=1, n_layers_model=32, warmup=2, reps=5, seed=2, l_in=[512, 100],
+                         batch_sizes=[1, 64], kv_len_start=256, n_steps=2, step_stride=1,
+                         peak_bf16_flops=1.4e15, peak_hbm_bytes_s=6.4e12, vocab=vocab)
+    table_bytes = vocab * 4096 * 2
+    assert 0 < m["prefill_head_s"] < m["prefill_time_s"]
+    for tpot, head in zip(m["tpot_s"], m["decode_head_s"]):
+        assert 0 < head < tpot
+        assert 0.3e12 < table_bytes / head < 8e12          # between 5 % of and just above the HBM rate
+    plain = pdlib.pd_measure(cfg, n_layers_run=1, n_layers_model=32, warmup=2, reps=5, seed=2, l_in=[512, 100],
+                             batch_sizes=[1, 64], kv_len_start=256, n_steps=2, step_stride=1)
+    assert plain["prefill_head_s"] == 0.0 and plain["decode_head_s"] == [0.0, 0.0]
+    assert m["prefill_flops"] > plain["prefill_flops"]
+
+
 def test_trace_reports_every_kernel_class(pdlib):
     import torch
     import pd_inputs as gen

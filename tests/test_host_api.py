@@ -32,7 +32,7 @@ def test_struct_sizes_match_c_layout(pdlib):
     assert ctypes.sizeof(pdlib.pd_kv_cache) == 32
     assert ctypes.sizeof(pdlib.pd_alloc_in) == 8 + 7 * 8 + 8 + 16
     assert ctypes.sizeof(pdlib.pd_alloc_out) == 8 + 5 * 8 + 8 + 3 * 8 + 16 + 8
-    assert ctypes.sizeof(pdlib.pd_measurement) == 8 + 4 * 8 + 8 + 32 * 4 + 5 * 32 * 8 + 8
+    assert ctypes.sizeof(pdlib.pd_measurement) == 8 + 4 * 8 + 8 + 32 * 4 + 5 * 32 * 8 + 8 + 8 + 32 * 8
 
 
 def _same(a, b):
