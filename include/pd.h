@@ -360,6 +360,18 @@ typedef struct {
  * Fields that can still be computed are filled; the others are NaN / 0. */
 pd_status pd_allocate(const pd_alloc_in* in, pd_alloc_out* out);
 
+/* pd_allocate with the two extensions the paper names but does not work out ("Acquire prefill
+ * throughput under TTFT constraints"):
+ *   prefix_hit_frac in [0, 1): prefix caching; the input length is replaced, everywhere in
+ *     Eq. 1-13, by the part that misses the cache, l_in * (1 - prefix_hit_frac), so the
+ *     throughputs count computed tokens;
+ *   dp_groups >= 1: data-parallel prefill; each of the G groups of an instance is its own
+ *     M/M/1 queue with 1/G of prefill_max_tok_s, so Eq. 13 reads
+ *     TP_prefill = TP_max - G * L_in / (TTFT - T_overhead); mu, lambda and rho in the result
+ *     describe one group, everything else one instance.
+ * (0, 1) gives pd_allocate's result bit for bit.  PD_ERR_INVALID_ARG outside those ranges. */
+pd_status pd_allocate_ext(const pd_alloc_in* in, double prefix_hit_frac, int32_t dp_groups, pd_alloc_out* out);
+
 /* FIFO single-server replay of n requests (host): request i arrives gaps[i] after request
  * i-1 and needs service[i] seconds.  Outputs the mean sojourn time (what Eq. 12 predicts as
  * 1/(mu - lambda)) and the mean waiting time. */

@@ -13,7 +13,13 @@ Readings where the paper is silent:
     ceiling is returned alongside as the SLO-safe count;
   * the TPOT-feasible batch is the largest sweep point such that every sweep point
     up to and including it meets the SLO (no interpolation);
-  * T_overhead is an explicit input.
+  * T_overhead is an explicit input;
+  * prefix caching ("Acquire prefill throughput under TTFT constraints", closing remark): the
+    input length is replaced, everywhere it occurs in Eq. 1-13, by the length that misses
+    the cache, L_in (1 - hit fraction); throughputs then count computed tokens;
+  * prefill data parallelism (same section): each of the G groups of an instance is its own
+    M/M/1 queue with 1/G of the instance's maximum throughput, so Eq. 13 becomes
+    TP_prefill = TP_max - G L_in / (TTFT - T_overhead); G = 1 is the paper's case.
 """
 from __future__ import annotations
 
@@ -139,6 +145,49 @@ def allocate(tp_total, l_in, l_out, ttft_slo, tpot_slo, prefill_max_tok_s,
     a.n_decode_ceil = ceil_count(a.n_decode_frac)
     a.achieved_total_tok_s = achieved_total_throughput(
         a.n_prefill, a.n_decode, a.tp_prefill_eff, a.tp_decode_eff, l_in, l_out)
+    return a
+
+
+def allocate_ext(tp_total, l_in, l_out, ttft_slo, tpot_slo, prefill_max_tok_s, batch, tpot,
+                 t_overhead=0.0, prefix_hit_frac=0.0, dp_groups=1) -> Allocation:
+    """`allocate` with a prefix-cache hit fraction and G data-parallel prefill groups.
+
+    mu, lam, rho describe ONE group: mu = (TP_max / G) / L, lam = (TP_prefill / G) / L with
+    L the non-cached input length; everything else is per instance.
+    """
+    if not (0.0 <= prefix_hit_frac < 1.0) or dp_groups < 1:
+        raise ValueError("hit fraction in [0, 1), at least one group")
+    l_eff = l_in * (1.0 - prefix_hit_frac)
+    g = float(dp_groups)
+    a = Allocation(status="ok")
+    a.mu = (prefill_max_tok_s / g) / l_eff                             # Eq. 9 for one group
+    budget = ttft_slo - t_overhead
+    if budget > 0.0:
+        a.tp_prefill_eff = prefill_max_tok_s - (g * l_eff) / budget    # Eq. 13, G queues
+    if not (budget > 0.0 and a.tp_prefill_eff > 0.0):
+        a.status = "infeasible_ttft"
+    else:
+        a.lam = (a.tp_prefill_eff / g) / l_eff
+        a.rho = a.lam / a.mu
+    idx, b_star, capped = feasible_batch(batch, tpot, tpot_slo)
+    if idx < 0:
+        if a.status == "ok":
+            a.status = "infeasible_tpot"
+    else:
+        a.feasible_batch = b_star
+        a.sweep_capped = capped
+        a.tp_decode_eff = b_star / tpot[idx]
+    if a.status != "ok":
+        return a
+    a.n_prefill_frac = (tp_total * l_eff) / ((l_eff + l_out) * a.tp_prefill_eff)
+    a.n_decode_frac = (tp_total * l_out) / ((l_eff + l_out) * a.tp_decode_eff)
+    a.ratio_pd = (l_eff * a.tp_decode_eff) / (l_out * a.tp_prefill_eff)
+    a.n_prefill = round_count(a.n_prefill_frac)
+    a.n_decode = round_count(a.n_decode_frac)
+    a.n_prefill_ceil = ceil_count(a.n_prefill_frac)
+    a.n_decode_ceil = ceil_count(a.n_decode_frac)
+    a.achieved_total_tok_s = achieved_total_throughput(
+        a.n_prefill, a.n_decode, a.tp_prefill_eff, a.tp_decode_eff, l_eff, l_out)
     return a
 
 

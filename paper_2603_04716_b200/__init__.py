@@ -37,7 +37,7 @@ EXPORTS = [
     "pd_launch_count", "pd_trace_begin", "pd_trace_end", "pd_decode_attention", "pd_decode_attention_workspace_bytes",
     "pd_decode_attention_noalloc", "pd_prefill_chunk_layer",
     "pd_model_create", "pd_model_destroy", "pd_model_workspace_bytes", "pd_model_prefill", "pd_model_decode_step",
-    "pd_model_check",
+    "pd_model_check", "pd_allocate_ext",
 ]
 
 TRACE_CLASSES = ["gemm_qkv", "gemm_o", "gemm_gate_up", "gemm_down", "attn_prefill", "attn_decode", "rmsnorm",
@@ -134,6 +134,7 @@ _lib.pd_gemm_bf16.argtypes = [_P, _P, _P, C.c_int32, C.c_int32, C.c_int32, _P, _
 _lib.pd_measure.argtypes = [C.POINTER(pd_layer_cfg), C.POINTER(pd_measure_cfg), C.c_double, C.c_double,
                             C.POINTER(pd_measurement)]
 _lib.pd_allocate.argtypes = [C.POINTER(pd_alloc_in), C.POINTER(pd_alloc_out)]
+_lib.pd_allocate_ext.argtypes = [C.POINTER(pd_alloc_in), C.c_double, C.c_int32, C.POINTER(pd_alloc_out)]
 _lib.pd_queue_replay.argtypes = [C.POINTER(C.c_double), C.POINTER(C.c_double), C.c_int64, C.POINTER(C.c_double),
                                  C.POINTER(C.c_double)]
 _lib.pd_decode_attention_workspace_bytes.argtypes = [C.POINTER(pd_layer_cfg), C.c_int32, C.c_int32,
@@ -435,6 +436,23 @@ def pd_allocate(tp_total_tok_s: float, l_in: float, l_out: float, ttft_slo_s: fl
                       prefill_max_tok_s, n, b, t)
     out = pd_alloc_out()
     st = _check(_lib.pd_allocate(C.byref(inp), C.byref(out)), "pd_allocate",
+                allow=(PD_ERR_INFEASIBLE_TTFT, PD_ERR_INFEASIBLE_TPOT))
+    res = {name: getattr(out, name) for name, _ in pd_alloc_out._fields_ if name != "struct_size"}
+    res["status"] = st
+    return res
+
+
+def pd_allocate_ext(tp_total_tok_s: float, l_in: float, l_out: float, ttft_slo_s: float, tpot_slo_s: float,
+                    prefill_max_tok_s: float, batch, tpot_s, t_overhead_s: float = 0.0, prefix_hit_frac: float = 0.0,
+                    dp_groups: int = 1) -> dict:
+    """pd_allocate with a prefix-cache hit fraction and data-parallel prefill groups (mu, lam, rho per group)."""
+    n = len(batch)
+    b = _i32_array(batch) if n else None
+    t = (C.c_double * n)(*[float(v) for v in tpot_s]) if n else None
+    inp = pd_alloc_in(C.sizeof(pd_alloc_in), tp_total_tok_s, l_in, l_out, ttft_slo_s, tpot_slo_s, t_overhead_s,
+                      prefill_max_tok_s, n, b, t)
+    out = pd_alloc_out()
+    st = _check(_lib.pd_allocate_ext(C.byref(inp), prefix_hit_frac, dp_groups, C.byref(out)), "pd_allocate_ext",
                 allow=(PD_ERR_INFEASIBLE_TTFT, PD_ERR_INFEASIBLE_TPOT))
     res = {name: getattr(out, name) for name, _ in pd_alloc_out._fields_ if name != "struct_size"}
     res["status"] = st

@@ -45,7 +45,25 @@ extern "C" const char* pd_status_str(pd_status s) {
 
 extern "C" int pd_version(void) { return 1; }
 
+namespace {
+pd_status allocate_impl(const pd_alloc_in* in, double prefix_hit_frac, int32_t dp_groups, pd_alloc_out* out);
+}
+
 extern "C" pd_status pd_allocate(const pd_alloc_in* in, pd_alloc_out* out) {
+  return allocate_impl(in, 0.0, 1, out);
+}
+
+extern "C" pd_status pd_allocate_ext(const pd_alloc_in* in, double prefix_hit_frac, int32_t dp_groups,
+                                     pd_alloc_out* out) {
+  if (!(prefix_hit_frac >= 0.0) || !(prefix_hit_frac < 1.0) || dp_groups < 1) return PD_ERR_INVALID_ARG;
+  return allocate_impl(in, prefix_hit_frac, dp_groups, out);
+}
+
+namespace {
+// L_in is the input length that misses the prefix cache; the G data-parallel groups of a prefill instance
+// are G M/M/1 queues with 1/G of its maximum throughput each (hit fraction 0 and G = 1: the paper's case,
+// where the two extra factors are exact no-ops in IEEE arithmetic).
+pd_status allocate_impl(const pd_alloc_in* in, double prefix_hit_frac, int32_t dp_groups, pd_alloc_out* out) {
   if (!in || !out || in->struct_size != sizeof(pd_alloc_in)) return PD_ERR_INVALID_ARG;
   const double nan = std::numeric_limits<double>::quiet_NaN();
   std::memset(out, 0, sizeof(*out));
@@ -53,8 +71,9 @@ extern "C" pd_status pd_allocate(const pd_alloc_in* in, pd_alloc_out* out) {
   out->tp_prefill_eff = out->tp_decode_eff = out->mu = out->lambda = out->rho = nan;
   out->n_prefill_frac = out->n_decode_frac = out->ratio_pd = out->achieved_total_tok_s = nan;
 
-  const double L_in = in->l_in, L_out = in->l_out;
-  if (!(in->tp_total_tok_s > 0.0) || !(L_in > 0.0) || !(L_out > 0.0) || !(in->prefill_max_tok_s > 0.0) ||
+  const double L_in = in->l_in * (1.0 - prefix_hit_frac), L_out = in->l_out;
+  const double G = static_cast<double>(dp_groups);
+  if (!(in->tp_total_tok_s > 0.0) || !(in->l_in > 0.0) || !(L_out > 0.0) || !(in->prefill_max_tok_s > 0.0) ||
       !(in->tpot_slo_s > 0.0) || !(in->t_overhead_s >= 0.0) || in->n_points < 0 ||
       (in->n_points > 0 && (!in->batch || !in->tpot_s)))
     return PD_ERR_INVALID_ARG;
@@ -64,15 +83,15 @@ extern "C" pd_status pd_allocate(const pd_alloc_in* in, pd_alloc_out* out) {
   pd_status status = PD_OK;
 
   // Prefill side: service rate (Eq. 9), TTFT budget (Eq. 8, 12), effective throughput (Eq. 13).
-  out->mu = in->prefill_max_tok_s / L_in;
+  out->mu = (in->prefill_max_tok_s / G) / L_in;  // one group
   const double budget = in->ttft_slo_s - in->t_overhead_s;
   bool prefill_ok = false;
   if (budget > 0.0) {
-    out->tp_prefill_eff = in->prefill_max_tok_s - L_in / budget;
+    out->tp_prefill_eff = in->prefill_max_tok_s - (G * L_in) / budget;
     prefill_ok = out->tp_prefill_eff > 0.0;
   }
   if (prefill_ok) {
-    out->lambda = out->tp_prefill_eff / L_in;  // Eq. 11 solved for lambda with Eq. 10
+    out->lambda = (out->tp_prefill_eff / G) / L_in;  // Eq. 11 solved for lambda with Eq. 10, one group
     out->rho = out->lambda / out->mu;           // Eq. 10
   } else {
     status = PD_ERR_INFEASIBLE_TTFT;
@@ -109,6 +128,7 @@ extern "C" pd_status pd_allocate(const pd_alloc_in* in, pd_alloc_out* out) {
   out->achieved_total_tok_s = side_p < side_d ? side_p : side_d;
   return PD_OK;
 }
+}  // namespace
 
 extern "C" pd_status pd_queue_replay(const double* gaps, const double* service, int64_t n, double* mean_sojourn_s,
                                      double* mean_wait_s) {

@@ -72,6 +72,39 @@ def test_allocate_matches_oracle_bit_for_bit(pdlib):
     assert seen == {"ok", "infeasible_ttft", "infeasible_tpot"}
 
 
+def test_allocate_ext_matches_oracle_bit_for_bit(pdlib):
+    """Prefix-cache hit fraction and data-parallel prefill groups: every field against the oracle."""
+    rnd = random.Random(23)
+    status_names = {0: "ok", pdlib.PD_ERR_INFEASIBLE_TTFT: "infeasible_ttft", pdlib.PD_ERR_INFEASIBLE_TPOT: "infeasible_tpot"}
+    seen = set()
+    for trial in range(1500):
+        n = rnd.randint(1, 8)
+        batch = sorted(rnd.sample(range(1, 1024), n))
+        tpot = sorted(rnd.uniform(0.002, 0.12) for _ in range(n))
+        hit = rnd.choice([0.0, 0.5, rnd.uniform(0.0, 0.95)])
+        groups = rnd.choice([1, 1, 2, 4, 8, 16])
+        args = (rnd.uniform(1e3, 1e6), float(rnd.randint(16, 32768)), float(rnd.randint(1, 4096)), rnd.uniform(0.05, 8.0),
+                rnd.uniform(0.001, 0.13), rnd.uniform(5e3, 2e5), batch, tpot, rnd.choice([0.0, 0.1]))
+        o = A.allocate_ext(*args, prefix_hit_frac=hit, dp_groups=groups)
+        p = pdlib.pd_allocate_ext(*args, prefix_hit_frac=hit, dp_groups=groups)
+        assert status_names[p["status"]] == o.status
+        seen.add(o.status)
+        assert (p["feasible_batch"], p["n_prefill"], p["n_decode"], p["n_prefill_ceil"], p["n_decode_ceil"]) == \
+               (o.feasible_batch, o.n_prefill, o.n_decode, o.n_prefill_ceil, o.n_decode_ceil)
+        for mine, theirs in (("tp_prefill_eff", o.tp_prefill_eff), ("tp_decode_eff", o.tp_decode_eff), ("mu", o.mu),
+                             ("lam", o.lam), ("rho", o.rho), ("n_prefill_frac", o.n_prefill_frac),
+                             ("n_decode_frac", o.n_decode_frac), ("ratio_pd", o.ratio_pd),
+                             ("achieved_total_tok_s", o.achieved_total_tok_s)):
+            assert _same(p[mine], theirs), (mine, p[mine], theirs)
+        if hit == 0.0 and groups == 1:
+            q = pdlib.pd_allocate(*args)
+            assert all(_same(q[k], p[k]) if isinstance(q[k], float) else q[k] == p[k] for k in q)
+    assert seen == {"ok", "infeasible_ttft", "infeasible_tpot"}
+    for bad in (dict(prefix_hit_frac=1.0), dict(prefix_hit_frac=-0.1), dict(dp_groups=0)):
+        with pytest.raises(pdlib.PdError):
+            pdlib.pd_allocate_ext(1e4, 10, 10, 1, 0.05, 1e4, [1], [0.01], **bad)
+
+
 def test_allocate_worked_example(pdlib, worked_example):
     g = worked_example
     b = 34

@@ -146,3 +146,58 @@ def test_queue_replay_hand_case():
     # idle server: no waiting
     soj, wait = A.queue_replay([0.0, 10.0, 10.0], [3.0, 1.0, 2.0])
     assert wait == 0.0 and soj == pytest.approx(2.0)
+
+
+# ------------------------------------------------ prefix cache and data-parallel prefill groups
+def test_allocate_ext_defaults_equal_the_paper_case_bit_for_bit():
+    rnd = random.Random(5)
+    for _ in range(200):
+        args = (rnd.uniform(1e3, 1e6), rnd.uniform(16, 30000), rnd.uniform(1, 4000), rnd.uniform(0.2, 8.0),
+                rnd.uniform(0.005, 0.2), rnd.uniform(1e3, 2e5), [1, 2, 4, 8], [rnd.uniform(0.004, 0.3) for _ in range(4)])
+        a, b = A.allocate(*args), A.allocate_ext(*args)
+        for f in a.__dataclass_fields__:
+            x, y = getattr(a, f), getattr(b, f)
+            assert x == y or (isinstance(x, float) and math.isnan(x) and math.isnan(y)), f
+
+
+def test_dp_groups_are_independent_mm1_queues():
+    """G groups, each with 1/G of the instance's maximum throughput and 1/G of its arrivals: every group's
+    M/M/1 sojourn time is the TTFT budget, and a replay of ONE group's queue (exponential gaps at lam,
+    exponential service at mu) reproduces it."""
+    tp_max, l_in, ttft, over = 80_000.0, 2048.0, 1.5, 0.1
+    one = A.allocate_ext(2e5, l_in, 256.0, ttft, 0.05, tp_max, [8], [0.02], over)
+    rng = np.random.Generator(np.random.Philox(key=11))
+    for g in (1, 2, 4, 8):
+        a = A.allocate_ext(2e5, l_in, 256.0, ttft, 0.05, tp_max, [8], [0.02], over, dp_groups=g)
+        assert a.status == "ok"
+        assert 1.0 / (a.mu - a.lam) == pytest.approx(ttft - over, rel=1e-12)          # Eq. 12 per group
+        assert a.mu == pytest.approx(tp_max / g / l_in, rel=1e-15)
+        # the instance loses the same L_in / budget per group: linear in G
+        assert tp_max - a.tp_prefill_eff == pytest.approx(g * (tp_max - one.tp_prefill_eff), rel=1e-12)
+        assert a.n_prefill_frac >= one.n_prefill_frac
+        n = 300_000
+        soj, _ = A.queue_replay(rng.exponential(1.0 / a.lam, size=n).tolist(), rng.exponential(1.0 / a.mu, size=n).tolist())
+        assert soj == pytest.approx(ttft - over, rel=0.06)
+    # so many groups that a lone request already misses the budget
+    assert A.allocate_ext(2e5, l_in, 256.0, ttft, 0.05, tp_max, [8], [0.02], over, dp_groups=64).status == "infeasible_ttft"
+
+
+def test_prefix_cache_hits_shorten_the_effective_input():
+    base = dict(tp_total=2e5, l_in=4096.0, l_out=256.0, ttft_slo=2.0, tpot_slo=0.05, prefill_max_tok_s=8e4,
+                batch=[64, 128], tpot=[0.03, 0.045])
+    prev = None
+    for hit in (0.0, 0.25, 0.5, 0.9):
+        a = A.allocate_ext(**base, prefix_hit_frac=hit)
+        # the service rate of Eq. 9 rises as 1 / (1 - hit): only the missed tokens are computed
+        assert a.mu * (1.0 - hit) == pytest.approx(8e4 / 4096.0, rel=1e-12)
+        # with hit fraction h the method sees a workload of input length L_in (1 - h)
+        b = A.allocate(2e5, 4096.0 * (1.0 - hit), 256.0, 2.0, 0.05, 8e4, [64, 128], [0.03, 0.045])
+        assert (a.n_prefill, a.n_decode, a.feasible_batch) == (b.n_prefill, b.n_decode, b.feasible_batch)
+        if prev is not None:
+            assert a.tp_prefill_eff > prev.tp_prefill_eff          # Eq. 13: a shorter input costs less queueing
+            assert a.ratio_pd < prev.ratio_pd                      # Eq. 7: fewer prefill instances per decode instance
+        prev = a
+    with pytest.raises(ValueError):
+        A.allocate_ext(**base, prefix_hit_frac=1.0)
+    with pytest.raises(ValueError):
+        A.allocate_ext(**base, dp_groups=0)
