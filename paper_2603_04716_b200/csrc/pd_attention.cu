@@ -47,6 +47,9 @@ __global__ void __launch_bounds__(DC_THREADS) decode_attn_kernel(DecodeAttnArgs 
   const int group = a.n_q_heads / a.n_kv_heads;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int g = lane >> 2, t4 = lane & 3;
+  // q and the newest K/V row come from the kernel before this one
+  ptx::grid_launch_dependents();
+  ptx::grid_dependency_wait();
 
   const int total = min(a.kv_len[b] + 1, a.len_cap);
   // split the key range into n_splits runs whose length is a multiple of the block's 64-key step
@@ -240,6 +243,8 @@ __global__ void __launch_bounds__(HD) decode_combine_kernel(DecodeAttnArgs a) {
   const int b = blockIdx.y, hq = blockIdx.x, d = threadIdx.x;
   const int group = a.n_q_heads / a.n_kv_heads;
   const int kvh = hq / group, r = hq - kvh * group;
+  ptx::grid_launch_dependents();
+  ptx::grid_dependency_wait();
   const float* base = a.partial + ((static_cast<size_t>(b) * a.n_kv_heads + kvh) * a.n_splits) * group * RS;
   float m = -CUDART_INF_F;
   for (int s = 0; s < a.n_splits; ++s) m = fmaxf(m, base[(s * group + r) * RS + HD]);
@@ -264,14 +269,12 @@ pd_status launch_decode_hd(const DecodeAttnArgs& a, cudaStream_t s) {
     attr_set = true;
   }
   dim3 grid(a.n_splits, a.n_kv_heads, a.batch);
-  decode_attn_kernel<HD><<<grid, DC_THREADS, SM::BYTES, s>>>(a);
+  PD_CUDA_TRY(launch_pdl(decode_attn_kernel<HD>, grid, dim3(DC_THREADS), SM::BYTES, s, a));
   count_launch();
-  PD_CUDA_TRY(cudaGetLastError());
   if (a.n_splits > 1) {
     dim3 cgrid(a.n_q_heads, a.batch);
-    decode_combine_kernel<HD><<<cgrid, HD, 0, s>>>(a);
+    PD_CUDA_TRY(launch_pdl(decode_combine_kernel<HD>, cgrid, dim3(HD), 0, s, a));
     count_launch();
-    PD_CUDA_TRY(cudaGetLastError());
   }
   return PD_OK;
 }

@@ -32,6 +32,23 @@ inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 extern thread_local long long g_launch_count;
 inline void count_launch(int n = 1) { g_launch_count += n; }
 
+// Launches `kern` so that it may begin while the previous kernel of `st` is still running (programmatic
+// dependent launch).  Such a kernel must call ptx::grid_dependency_wait() before it touches anything an
+// earlier kernel writes or still reads; everything before that call overlaps the predecessor's tail.
+// PD_DISABLE_PDL=1 in the environment launches normally instead (for A/B timing).
+bool pdl_enabled();
+template <class... KArgs, class... Args>
+cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl_enabled() ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+}
+
 // Brackets the kernels launched in its scope with CUDA events while a trace is active
 // (pd_trace_begin .. pd_trace_end); free otherwise.
 class TraceScope {
@@ -107,16 +124,22 @@ struct SkinnyGemmArgs {
   float* acc;     // [B, N]
   int batch, n, k, ldx;
   int* err_word;
+  bool acc_zeroed;  // the caller guarantees acc is zero when the kernel's epilogue runs (no memset is enqueued)
 };
 pd_status gemm_skinny(const SkinnyGemmArgs& g, cudaStream_t stream);
+// Number of K slices gemm_skinny will use (1: plain stores, acc need not be zero).
+int gemm_skinny_splits(int batch, int n, int k);
 // Row-wise kernels that turn the fp32 sums into the layer's stored tensors.
+// Every row-wise kernel can also clear the fp32 sums of a LATER projection (zero_ptr[batch, zero_cols], NULL to
+// skip): the buffer is idle while the kernel runs, and the projection then needs no memset of its own.
 pd_status launch_skinny_rope_kv(const float* acc, bf16* qkv, const RopeEpilogue& rp, int batch, int* err_word,
-                                cudaStream_t s);
+                                float* zero_ptr, int zero_cols, cudaStream_t s);
 // h = x + acc; if n != NULL also n = RMSNorm(h) * gain.
 pd_status launch_skinny_residual(const float* acc, const bf16* x, bf16* h, const bf16* gain, bf16* n, int batch, int d,
-                                 float eps, cudaStream_t s);
+                                 float eps, float* zero_ptr, int zero_cols, cudaStream_t s);
 // out[B, F] = silu(gate) * up from acc[B, 2F] whose columns follow the 64/64 interleaved weight rows.
-pd_status launch_skinny_swiglu(const float* acc, bf16* out, int batch, int f, cudaStream_t s);
+pd_status launch_skinny_swiglu(const float* acc, bf16* out, int batch, int f, float* zero_ptr, int zero_cols,
+                               cudaStream_t s);
 
 // ------------------------------------------------------------ whole model
 // Pieces of the whole-model step around the layer stack (the measurement harness times them alone).
@@ -127,6 +150,10 @@ pd_status model_head(pd_model* m, const bf16* h, const int32_t* cu_dev, int rows
 
 // ------------------------------------------------------------ elementwise
 pd_status launch_rmsnorm(const bf16* x, const bf16* gain, bf16* y, int rows, int d, float eps, cudaStream_t s);
+// The same as the first kernel of a decode layer: launched with programmatic serialization, and clears
+// zero_ptr[rows, zero_cols] (fp32, NULL to skip) for a later projection.
+pd_status launch_rmsnorm_decode(const bf16* x, const bf16* gain, bf16* y, int rows, int d, float eps, float* zero_ptr,
+                                int zero_cols, cudaStream_t s);
 
 // -------------------------------------------------------------- attention
 struct PrefillAttnArgs {

@@ -28,8 +28,14 @@ constexpr int RMS_MAX_CHUNKS = 8;  // 8 chunks * 8 elements * 256 threads = d up
 
 __global__ void __launch_bounds__(RMS_THREADS) rmsnorm_kernel(const bf16* __restrict__ x,
                                                                const bf16* __restrict__ gain, bf16* __restrict__ y,
-                                                               int d, float eps) {
+                                                               int d, float eps, float* zero_ptr, int zero_cols) {
   const int row = blockIdx.x;
+  ptx::grid_launch_dependents();
+  ptx::grid_dependency_wait();
+  if (zero_ptr) {  // fp32 sums of a later decode projection, idle while this kernel runs
+    float4* q = reinterpret_cast<float4*>(zero_ptr + static_cast<size_t>(row) * zero_cols);
+    for (int i = threadIdx.x; i < zero_cols / 4; i += RMS_THREADS) q[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+  }
   const uint4* xr = reinterpret_cast<const uint4*>(x + static_cast<size_t>(row) * d);
   const uint4* gr = reinterpret_cast<const uint4*>(gain);
   uint4* yr = reinterpret_cast<uint4*>(y + static_cast<size_t>(row) * d);
@@ -99,9 +105,18 @@ __global__ void __launch_bounds__(256) fill_normal_kernel(bf16* dst, size_t n, u
 pd_status launch_rmsnorm(const bf16* x, const bf16* gain, bf16* y, int rows, int d, float eps, cudaStream_t s) {
   if (rows == 0) return PD_OK;
   if (d % 8 != 0 || d > RMS_THREADS * RMS_MAX_CHUNKS * 8) return PD_ERR_UNSUPPORTED_SHAPE;
-  rmsnorm_kernel<<<rows, RMS_THREADS, 0, s>>>(x, gain, y, d, eps);
+  rmsnorm_kernel<<<rows, RMS_THREADS, 0, s>>>(x, gain, y, d, eps, nullptr, 0);
   count_launch();
   PD_CUDA_TRY(cudaGetLastError());
+  return PD_OK;
+}
+
+pd_status launch_rmsnorm_decode(const bf16* x, const bf16* gain, bf16* y, int rows, int d, float eps, float* zero_ptr,
+                                int zero_cols, cudaStream_t s) {
+  if (rows == 0) return PD_OK;
+  if (d % 8 != 0 || d > RMS_THREADS * RMS_MAX_CHUNKS * 8 || (zero_ptr && zero_cols % 4 != 0)) return PD_ERR_UNSUPPORTED_SHAPE;
+  PD_CUDA_TRY(launch_pdl(rmsnorm_kernel, dim3(rows), dim3(RMS_THREADS), 0, s, x, gain, y, d, eps, zero_ptr, zero_cols));
+  count_launch();
   return PD_OK;
 }
 

@@ -9,6 +9,13 @@
 // an fp32 [B, N] buffer (red.global.add, L2-resident; plain stores when K is not split).
 // Small row-wise kernels then apply the layer's fused operations to the fp32 sums: RoPE and the
 // KV-cache append, residual add with the following RMSNorm, SwiGLU, residual add.
+//
+// The chain of a decode layer is launched with programmatic serialization.  Weights do not depend on
+// earlier kernels, so a block fills its whole TMA ring with weight tiles BEFORE it waits for the previous
+// kernel; only the activation tiles and the accumulation into the fp32 buffer come after the wait.  The
+// weight stream therefore keeps running across kernel boundaries.  (Pulling further weight tiles into L2
+// before the wait was measured too: no gain, the ring already covers the gap.)  The fp32 buffer of a K-split
+// projection is cleared by a row-wise kernel earlier in the chain instead of a memset.
 #include "pd_common.cuh"
 #include "pd_ptx.cuh"
 
@@ -84,12 +91,28 @@ gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
+  ptx::grid_launch_dependents();
   if (warp == 0) {
     if (lane == 0) {
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (int kb = kb0; kb < kb1; ++kb) {
+      // ring prologue: weight tiles first (they depend on no earlier kernel), then the dependency wait,
+      // then the activation tiles of the same stages
+      const int pre = min(STAGES, kb1 - kb0);
+      for (int i = 0; i < pre; ++i) {
+        const uint32_t sw = smem_base + i * Cfg::STAGE_BYTES;
+        ptx::mbar_arrive_expect_tx(full_bar(i), Cfg::W_BYTES + Cfg::X_BYTES);
+        ptx::tma_load_2d(sw, &tmap_w, (kb0 + i) * SK_BK, tn * (MT * SK_BM), full_bar(i));
+      }
+      ptx::grid_dependency_wait();
+      for (int i = 0; i < pre; ++i) {
+        const uint32_t sx = smem_base + i * Cfg::STAGE_BYTES + Cfg::W_BYTES;
+        ptx::tma_load_2d(sx, &tmap_x, (kb0 + i) * SK_BK, tb * BNB, full_bar(i));
+      }
+      if (pre == STAGES) phase = 1u;  // the ring has wrapped once
+      else stage = pre;
+      for (int kb = kb0 + pre; kb < kb1; ++kb) {
         if (!ptx::mbar_wait_bounded(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
         const uint32_t sw = smem_base + stage * Cfg::STAGE_BYTES;
         const uint32_t sx = sw + Cfg::W_BYTES;
@@ -129,6 +152,7 @@ gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
   } else {
     const int lane_group = warp & 3;
     const bool ok = __all_sync(0xffffffffu, ptx::mbar_wait_bounded(acc_bar, 0u, abort_flag));
+    ptx::grid_dependency_wait();  // (long since satisfied) orders the sums after the kernel that cleared the buffer
     if (ok && kb1 > kb0) {
       ptx::tc_fence_after();
       constexpr int CH = BNB < 32 ? BNB : 32;
@@ -167,6 +191,15 @@ gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
   }
 }
 
+// K slices per (weight tile, batch tile) unit: fill the resident block slots, each block with at least 8 K-blocks.
+int skinny_splits(int units, int k_blocks, int blocks_per_sm) {
+  int splits = (blocks_per_sm * 148 + units / 2) / units;
+  if (splits > k_blocks / 8) splits = k_blocks / 8;
+  return splits < 1 ? 1 : splits;
+}
+
+int skinny_bnb(int batch) { return batch <= 16 ? 16 : batch <= 32 ? 32 : batch <= 64 ? 64 : batch <= 128 ? 128 : 256; }
+
 template <int BNB, int MT>
 pd_status launch_skinny(const SkinnyGemmArgs& g, cudaStream_t stream) {
   using Cfg = SkinnyCfg<BNB, MT>;
@@ -183,17 +216,14 @@ pd_status launch_skinny(const SkinnyGemmArgs& g, cudaStream_t stream) {
   p.acc = g.acc; p.batch = g.batch; p.n = g.n; p.k_blocks = g.k / SK_BK;
   p.tiles_n = (g.n + MT * SK_BM - 1) / (MT * SK_BM);
   const int tiles_b = (g.batch + BNB - 1) / BNB;
-  // fill the resident block slots, each block with at least 8 K-blocks
   const int units = p.tiles_n * tiles_b;
-  int splits = (Cfg::BLOCKS_PER_SM * 148 + units / 2) / units;
-  if (splits > p.k_blocks / 8) splits = p.k_blocks / 8;
-  if (splits < 1) splits = 1;
+  const int splits = skinny_splits(units, p.k_blocks, Cfg::BLOCKS_PER_SM);
   p.splits = splits;
   p.err_word = g.err_word;
-  if (splits > 1) PD_CUDA_TRY(cudaMemsetAsync(g.acc, 0, static_cast<size_t>(g.batch) * g.n * sizeof(float), stream));
-  kern<<<units * splits, SK_THREADS, Cfg::SMEM_BYTES, stream>>>(tw, tx, p);
+  if (splits > 1 && !g.acc_zeroed)
+    PD_CUDA_TRY(cudaMemsetAsync(g.acc, 0, static_cast<size_t>(g.batch) * g.n * sizeof(float), stream));
+  PD_CUDA_TRY(launch_pdl(kern, dim3(units * splits), dim3(SK_THREADS), Cfg::SMEM_BYTES, stream, tw, tx, p));
   count_launch();
-  PD_CUDA_TRY(cudaGetLastError());
   return PD_OK;
 }
 
@@ -218,10 +248,19 @@ __device__ __forceinline__ void load8(const float* p, float (&f)[8]) {
   f[0] = a.x; f[1] = a.y; f[2] = a.z; f[3] = a.w; f[4] = b.x; f[5] = b.y; f[6] = b.z; f[7] = b.w;
 }
 
+// Clears n floats at p with the threads of one block (p 16-byte aligned, n a multiple of 4).
+__device__ __forceinline__ void zero_row(float* p, int n) {
+  float4* q = reinterpret_cast<float4*>(p);
+  for (int i = threadIdx.x; i < n / 4; i += blockDim.x) q[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+}
+
 // RoPE + KV append for one decode token per block: acc[b, Nqkv] -> q (bf16, in the qkv buffer), cache.
 __global__ void __launch_bounds__(128) skinny_rope_kv_kernel(const float* __restrict__ acc, bf16* qkv, RopeEpilogue rp,
-                                                             int* err_word) {
+                                                             int* err_word, float* zero_ptr, int zero_cols) {
   const int b = blockIdx.x;
+  ptx::grid_launch_dependents();
+  ptx::grid_dependency_wait();
+  if (zero_ptr) zero_row(zero_ptr + static_cast<size_t>(b) * zero_cols, zero_cols);
   const int pos = rp.kv_len[b], slot = b;
   if (pos < 0 || pos >= rp.len_cap || pos >= rp.max_pos || slot >= rp.batch_cap) {
     if (threadIdx.x == 0 && err_word) atomicExch(err_word, 2);
@@ -267,9 +306,12 @@ template <bool NORM>
 __global__ void __launch_bounds__(RES_THREADS) skinny_residual_kernel(const float* __restrict__ acc,
                                                                        const bf16* __restrict__ x, bf16* h,
                                                                        const bf16* __restrict__ gain, bf16* n, int d,
-                                                                       float eps) {
+                                                                       float eps, float* zero_ptr, int zero_cols) {
   const int b = blockIdx.x;
   const int chunks = d / 8;
+  ptx::grid_launch_dependents();
+  ptx::grid_dependency_wait();
+  if (zero_ptr) zero_row(zero_ptr + static_cast<size_t>(b) * zero_cols, zero_cols);
   uint4 hv[RES_MAX_CHUNKS];
   float ss = 0.f;
 #pragma unroll
@@ -317,9 +359,18 @@ __global__ void __launch_bounds__(RES_THREADS) skinny_residual_kernel(const floa
 
 // a[b, f] = silu(gate) * up with the weight rows interleaved 64 gate / 64 up.
 __global__ void __launch_bounds__(256) skinny_swiglu_kernel(const float* __restrict__ acc, bf16* __restrict__ out,
-                                                             int rows, int f) {
+                                                             int rows, int f, float* zero_ptr, int zero_cols) {
   const int chunks_per_row = f / 8;
   const size_t total = static_cast<size_t>(rows) * chunks_per_row;
+  ptx::grid_launch_dependents();
+  ptx::grid_dependency_wait();
+  if (zero_ptr) {
+    float4* q = reinterpret_cast<float4*>(zero_ptr);
+    const size_t quads = static_cast<size_t>(rows) * zero_cols / 4;
+    for (size_t i = blockIdx.x * static_cast<size_t>(blockDim.x) + threadIdx.x; i < quads;
+         i += static_cast<size_t>(gridDim.x) * blockDim.x)
+      q[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+  }
   for (size_t idx = blockIdx.x * static_cast<size_t>(blockDim.x) + threadIdx.x; idx < total;
        idx += static_cast<size_t>(gridDim.x) * blockDim.x) {
     const size_t r = idx / chunks_per_row;
@@ -337,6 +388,12 @@ __global__ void __launch_bounds__(256) skinny_swiglu_kernel(const float* __restr
 
 }  // namespace
 
+int gemm_skinny_splits(int batch, int n, int k) {
+  const int bnb = skinny_bnb(batch);
+  const int units = ((n + SK_BM - 1) / SK_BM) * ((batch + bnb - 1) / bnb);
+  return skinny_splits(units, k / SK_BK, 2);
+}
+
 pd_status gemm_skinny(const SkinnyGemmArgs& g, cudaStream_t stream) {
   if (!g.x || !g.w || !g.acc || g.batch <= 0 || g.n <= 0 || g.k <= 0) return PD_ERR_INVALID_ARG;
   if (g.k % SK_BK != 0 || g.n % 4 != 0 || g.ldx % 8 != 0) return PD_ERR_UNSUPPORTED_SHAPE;
@@ -350,30 +407,38 @@ pd_status gemm_skinny(const SkinnyGemmArgs& g, cudaStream_t stream) {
 }
 
 pd_status launch_skinny_rope_kv(const float* acc, bf16* qkv, const RopeEpilogue& rp, int batch, int* err_word,
-                                cudaStream_t s) {
-  skinny_rope_kv_kernel<<<batch, 128, 0, s>>>(acc, qkv, rp, err_word);
+                                float* zero_ptr, int zero_cols, cudaStream_t s) {
+  if (zero_ptr && zero_cols % 4 != 0) return PD_ERR_UNSUPPORTED_SHAPE;
+  PD_CUDA_TRY(launch_pdl(skinny_rope_kv_kernel, dim3(batch), dim3(128), 0, s, acc, qkv, rp, err_word, zero_ptr, zero_cols));
   count_launch();
-  PD_CUDA_TRY(cudaGetLastError());
   return PD_OK;
 }
 
 pd_status launch_skinny_residual(const float* acc, const bf16* x, bf16* h, const bf16* gain, bf16* n, int batch, int d,
-                                 float eps, cudaStream_t s) {
+                                 float eps, float* zero_ptr, int zero_cols, cudaStream_t s) {
   if (d % 8 != 0 || d > RES_THREADS * RES_MAX_CHUNKS * 8) return PD_ERR_UNSUPPORTED_SHAPE;
-  if (n) skinny_residual_kernel<true><<<batch, RES_THREADS, 0, s>>>(acc, x, h, gain, n, d, eps);
-  else skinny_residual_kernel<false><<<batch, RES_THREADS, 0, s>>>(acc, x, h, nullptr, nullptr, d, eps);
+  if (zero_ptr && zero_cols % 4 != 0) return PD_ERR_UNSUPPORTED_SHAPE;
+  const bf16* no_gain = nullptr;
+  bf16* no_out = nullptr;
+  if (n)
+    PD_CUDA_TRY(launch_pdl(skinny_residual_kernel<true>, dim3(batch), dim3(RES_THREADS), 0, s, acc, x, h, gain, n, d, eps,
+                           zero_ptr, zero_cols));
+  else
+    PD_CUDA_TRY(launch_pdl(skinny_residual_kernel<false>, dim3(batch), dim3(RES_THREADS), 0, s, acc, x, h, no_gain, no_out,
+                           d, eps, zero_ptr, zero_cols));
   count_launch();
-  PD_CUDA_TRY(cudaGetLastError());
   return PD_OK;
 }
 
-pd_status launch_skinny_swiglu(const float* acc, bf16* out, int batch, int f, cudaStream_t s) {
+pd_status launch_skinny_swiglu(const float* acc, bf16* out, int batch, int f, float* zero_ptr, int zero_cols,
+                               cudaStream_t s) {
+  if (zero_ptr && zero_cols % 4 != 0) return PD_ERR_UNSUPPORTED_SHAPE;
   const size_t total = static_cast<size_t>(batch) * (f / 8);
   size_t blocks = (total + 255) / 256;
-  if (blocks > 148 * 8) blocks = 148 * 8;
-  skinny_swiglu_kernel<<<static_cast<unsigned>(blocks), 256, 0, s>>>(acc, out, batch, f);
+  if (blocks > 148 * 4) blocks = 148 * 4;  // all resident beside the projection blocks they wait for
+  PD_CUDA_TRY(launch_pdl(skinny_swiglu_kernel, dim3(static_cast<unsigned>(blocks)), dim3(256), 0, s, acc, out, batch, f,
+                         zero_ptr, zero_cols));
   count_launch();
-  PD_CUDA_TRY(cudaGetLastError());
   return PD_OK;
 }
 

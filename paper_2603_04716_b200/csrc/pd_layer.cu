@@ -12,9 +12,14 @@ using pd::bf16;
 
 namespace {
 
+// Batches beyond one 256-wide batch tile run the projections on the prefill GEMM (fused epilogues, tail
+// tiles split): the weight-streaming kernel would read every weight once per batch tile (measured per
+// 8B-shaped layer: 327 -> 242 us at B = 384, 352 -> 275 us at B = 512; at B = 256 the two paths tie).
+constexpr int kWideDecodeBatch = 257;
+
 struct Workspace {
   // byte offsets into the caller's workspace
-  size_t norm, qkv, attn_o, resid, acc, act, partial, stage_a, stage_b, meta, splitk, total;
+  size_t norm, qkv, attn_o, resid, acc_qkv, acc_o, acc_gu, acc_down, act, partial, stage_a, stage_b, meta, splitk, total;
 };
 
 Workspace carve(const pd_layer_cfg& c, size_t tokens, size_t max_batch, int max_kv_len) {
@@ -32,10 +37,13 @@ Workspace carve(const pd_layer_cfg& c, size_t tokens, size_t max_batch, int max_
   w.attn_o = take(tokens * hq * 2);
   w.resid = take(tokens * d * 2);
   w.act = take(tokens * f * 2);
-  {  // fp32 sums of the decode-mode projections: [batch, widest projection]
-    size_t widest = nqkv > 2 * f ? nqkv : 2 * f;
-    if (d > widest) widest = d;
-    w.acc = take(max_batch * widest * 4);
+  {  // fp32 sums of the four decode-mode projections, one buffer each (a buffer is cleared by a row-wise kernel
+     // earlier in the chain while another one is in use); batches beyond the weight-streaming path need none
+    const size_t rows = max_batch < static_cast<size_t>(kWideDecodeBatch) ? max_batch : 0;
+    w.acc_qkv = take(rows * nqkv * 4);
+    w.acc_o = take(rows * d * 4);
+    w.acc_gu = take(rows * 2 * f * 4);
+    w.acc_down = take(rows * d * 4);
   }
   const int splits = max_batch ? pd::decode_attention_splits(1, c.n_kv_heads, max_kv_len) : 1;  // worst case: B = 1
   w.partial = take(max_batch * c.n_kv_heads * static_cast<size_t>(splits) * (c.n_q_heads / c.n_kv_heads) *
@@ -168,10 +176,6 @@ pd_status prefill_impl(pd_layer* L, const bf16* x, bf16* out, const int32_t* cu_
   return PD_OK;
 }
 
-// Batches beyond one 256-wide batch tile run the projections on the prefill GEMM (fused epilogues, tail
-// tiles split): the weight-streaming kernel would read every weight once per batch tile (measured per
-// 8B-shaped layer: 327 -> 242 us at B = 384, 352 -> 275 us at B = 512; at B = 256 the two paths tie).
-constexpr int kWideDecodeBatch = 257;
 
 pd_status decode_impl_wide(pd_layer* L, const bf16* x, bf16* out, const int32_t* kv_len_dev, int B, int max_kv_len,
                            const pd_kv_cache* cache, uint8_t* ws, const Workspace& w, cudaStream_t st) {
@@ -205,21 +209,36 @@ pd_status decode_impl(pd_layer* L, const bf16* x, bf16* out, const int32_t* kv_l
   bf16* attn_o = reinterpret_cast<bf16*>(ws + w.attn_o);
   bf16* resid = reinterpret_cast<bf16*>(ws + w.resid);
   bf16* act = reinterpret_cast<bf16*>(ws + w.act);
-  float* acc = reinterpret_cast<float*>(ws + w.acc);
+  float* acc_qkv = reinterpret_cast<float*>(ws + w.acc_qkv);
+  float* acc_o = reinterpret_cast<float*>(ws + w.acc_o);
+  float* acc_gu = reinterpret_cast<float*>(ws + w.acc_gu);
+  float* acc_down = reinterpret_cast<float*>(ws + w.acc_down);
   pd::RopeEpilogue r{};
   r.k_cache = static_cast<bf16*>(cache->k); r.v_cache = static_cast<bf16*>(cache->v); r.rope_tab = L->rope_tab;
   r.cu_seqlens = nullptr; r.slots = nullptr; r.kv_len = kv_len_dev; r.n_req = B;
   r.n_q_heads = c.n_q_heads; r.n_kv_heads = c.n_kv_heads; r.head_dim = c.head_dim; r.len_cap = cache->len_cap;
   r.max_pos = c.max_pos; r.batch_cap = cache->batch_cap;
 
-  { pd::TraceScope ts(PD_K_RMSNORM, st); PD_TRY(pd::launch_rmsnorm(x, L->g_attn, norm, B, c.d_model, c.rms_eps, st)); }
+  // The whole chain is launched with programmatic serialization (each kernel waits for its predecessor
+  // only where it first needs it).  A K-split projection adds into its fp32 buffer; that buffer is cleared
+  // by a row-wise kernel two or more launches earlier, never by a memset between the kernels.
+  const int n_gu = 2 * c.d_ff;
+  float* z_qkv = pd::gemm_skinny_splits(B, L->n_qkv, c.d_model) > 1 ? acc_qkv : nullptr;
+  float* z_o = pd::gemm_skinny_splits(B, c.d_model, hq) > 1 ? acc_o : nullptr;
+  float* z_gu = pd::gemm_skinny_splits(B, n_gu, c.d_model) > 1 ? acc_gu : nullptr;
+  float* z_down = pd::gemm_skinny_splits(B, c.d_model, c.d_ff) > 1 ? acc_down : nullptr;
+
+  {
+    pd::TraceScope ts(PD_K_RMSNORM, st);
+    PD_TRY(pd::launch_rmsnorm_decode(x, L->g_attn, norm, B, c.d_model, c.rms_eps, z_qkv, L->n_qkv, st));
+  }
   pd::SkinnyGemmArgs g{};
-  g.acc = acc; g.batch = B; g.err_word = L->err_word;
+  g.batch = B; g.err_word = L->err_word; g.acc_zeroed = true;
   {
     pd::TraceScope ts(PD_K_GEMM_QKV, st);
-    g.x = norm; g.w = L->w_qkv; g.n = L->n_qkv; g.k = c.d_model; g.ldx = c.d_model;
+    g.x = norm; g.w = L->w_qkv; g.acc = acc_qkv; g.n = L->n_qkv; g.k = c.d_model; g.ldx = c.d_model;
     PD_TRY(pd::gemm_skinny(g, st));
-    PD_TRY(pd::launch_skinny_rope_kv(acc, qkv, r, B, L->err_word, st));
+    PD_TRY(pd::launch_skinny_rope_kv(acc_qkv, qkv, r, B, L->err_word, z_o, c.d_model, st));
   }
   pd::DecodeAttnArgs a{};
   a.q = qkv; a.ldq = L->n_qkv;
@@ -231,21 +250,21 @@ pd_status decode_impl(pd_layer* L, const bf16* x, bf16* out, const int32_t* kv_l
   { pd::TraceScope ts(PD_K_ATTN_DECODE, st); PD_TRY(pd::launch_decode_attention(a, st)); }
   {
     pd::TraceScope ts(PD_K_GEMM_O, st);  // h = x + o W_o^T and n2 = RMSNorm(h) in the same row-wise pass
-    g.x = attn_o; g.w = L->w_o; g.n = c.d_model; g.k = hq; g.ldx = hq;
+    g.x = attn_o; g.w = L->w_o; g.acc = acc_o; g.n = c.d_model; g.k = hq; g.ldx = hq;
     PD_TRY(pd::gemm_skinny(g, st));
-    PD_TRY(pd::launch_skinny_residual(acc, x, resid, L->g_mlp, norm, B, c.d_model, c.rms_eps, st));
+    PD_TRY(pd::launch_skinny_residual(acc_o, x, resid, L->g_mlp, norm, B, c.d_model, c.rms_eps, z_gu, n_gu, st));
   }
   {
     pd::TraceScope ts(PD_K_GEMM_GATE_UP, st);
-    g.x = norm; g.w = L->w_gu; g.n = 2 * c.d_ff; g.k = c.d_model; g.ldx = c.d_model;
+    g.x = norm; g.w = L->w_gu; g.acc = acc_gu; g.n = n_gu; g.k = c.d_model; g.ldx = c.d_model;
     PD_TRY(pd::gemm_skinny(g, st));
-    PD_TRY(pd::launch_skinny_swiglu(acc, act, B, c.d_ff, st));
+    PD_TRY(pd::launch_skinny_swiglu(acc_gu, act, B, c.d_ff, z_down, c.d_model, st));
   }
   {
     pd::TraceScope ts(PD_K_GEMM_DOWN, st);
-    g.x = act; g.w = L->w_down; g.n = c.d_model; g.k = c.d_ff; g.ldx = c.d_ff;
+    g.x = act; g.w = L->w_down; g.acc = acc_down; g.n = c.d_model; g.k = c.d_ff; g.ldx = c.d_ff;
     PD_TRY(pd::gemm_skinny(g, st));
-    PD_TRY(pd::launch_skinny_residual(acc, resid, out, nullptr, nullptr, B, c.d_model, c.rms_eps, st));
+    PD_TRY(pd::launch_skinny_residual(acc_down, resid, out, nullptr, nullptr, B, c.d_model, c.rms_eps, nullptr, 0, st));
   }
   return PD_OK;
 }

@@ -163,7 +163,7 @@ pd_status model_head(pd_model* m, const bf16* h, const int32_t* cu_dev, int rows
   { TraceScope ts(PD_K_RMSNORM, st); PD_TRY(launch_rmsnorm(src, m->g_final, norm, rows, d, m->cfg.rms_eps, st)); }
   SkinnyGemmArgs g{};
   g.x = norm; g.w = m->lm_head; g.acc = logits; g.batch = rows; g.n = m->vocab; g.k = d; g.ldx = d;
-  g.err_word = m->err_word;
+  g.err_word = m->err_word; g.acc_zeroed = false;
   { TraceScope ts(PD_K_LM_HEAD, st); PD_TRY(gemm_skinny(g, st)); }
   {
     TraceScope ts(PD_K_SAMPLE, st);

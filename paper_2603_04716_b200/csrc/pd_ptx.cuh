@@ -79,6 +79,14 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity,
   }
 }
 
+// ------------------------------------------------- programmatic dependent launch
+// A kernel launched with the programmatic-serialization attribute may start while the previous
+// kernel of its stream is still running.  grid_dependency_wait blocks until every grid this one
+// depends on has completed and its writes are visible (it returns at once in a normally launched
+// kernel); grid_launch_dependents lets the next kernel start its own prologue.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ----------------------------------------------------------------------- TMA
 __device__ __forceinline__ void prefetch_tensormap(const void* tmap) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(tmap)) : "memory");

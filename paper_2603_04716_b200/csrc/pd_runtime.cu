@@ -1,5 +1,6 @@
 // Process-level plumbing of the library: last CUDA error, launch counter and the
 // optional per-kernel-class CUDA-event trace used for roofline reporting.
+#include <cstdlib>
 #include <vector>
 
 #include "pd_common.cuh"
@@ -8,6 +9,14 @@ namespace pd {
 
 thread_local int g_last_cuda_error = 0;
 thread_local long long g_launch_count = 0;
+
+bool pdl_enabled() {
+  static const bool on = [] {
+    const char* v = std::getenv("PD_DISABLE_PDL");
+    return !(v && v[0] == '1');
+  }();
+  return on;
+}
 
 pd_status cuda_fail(cudaError_t e) {
   g_last_cuda_error = static_cast<int>(e);
