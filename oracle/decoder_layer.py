@@ -33,6 +33,11 @@ points and nowhere else (no rounding inside a contraction, the softmax or SwiGLU
 "the kernels compute the right function" (tight, against the rounded variant) from
 "bf16 storage costs this much accuracy" (against the exact variant).
 
+Projections.  ``proj=None`` (default) evaluates every projection as the plain product
+x @ W^T.  A callable ``proj(x, name, lo, hi)`` replaces it (rows lo..hi of weight ``name``);
+oracle/fp8.py provides the FP8 variant.  It changes how the five projections are evaluated
+and nothing else.
+
 Parity pins (see tests/test_oracle_layer.py): softmax rows sum to one, decode
 step t equals prefill row t, zero-weight and single-token special cases,
 rotation invariants of RoPE, permutation invariance over packed requests, a
@@ -138,16 +143,28 @@ def _identity(a: np.ndarray) -> np.ndarray:
     return a
 
 
+class _ExactProjector:
+    """Default projection: x @ W[name][lo:hi]^T in the working precision."""
+
+    def __init__(self, w: LayerWeights, dt):
+        self.w, self.dt, self.cast = w, dt, {}
+
+    def __call__(self, x, name, lo=None, hi=None):
+        if name not in self.cast:
+            self.cast[name] = getattr(self.w, name).astype(self.dt)
+        return x @ self.cast[name][lo:hi].T
+
+
 def _mlp_and_residuals(x_rows: np.ndarray, o_rows: np.ndarray, w: LayerWeights,
-                       cfg: LayerConfig, dt, st) -> np.ndarray:
-    h = st(x_rows + o_rows @ w.w_o.astype(dt).T)
+                       cfg: LayerConfig, dt, st, pj) -> np.ndarray:
+    h = st(x_rows + pj(o_rows, "w_o"))
     n2 = st(rmsnorm(h, w.g_mlp.astype(dt), cfg.rms_eps))
-    a = st(silu(n2 @ w.w_gate.astype(dt).T) * (n2 @ w.w_up.astype(dt).T))
-    return st(h + a @ w.w_down.astype(dt).T)
+    a = st(silu(pj(n2, "w_gate")) * pj(n2, "w_up"))
+    return st(h + pj(a, "w_down"))
 
 
 def prefill_layer(cfg: LayerConfig, w: LayerWeights, x: np.ndarray, cu_seqlens,
-                  rows=None, dtype=np.float64, probs_out: list | None = None, store=None):
+                  rows=None, dtype=np.float64, probs_out: list | None = None, store=None, proj=None):
     """One layer over a packed ragged batch of requests.
 
     ``cu_seqlens`` has n_req + 1 entries; request r owns rows cu[r]..cu[r+1]-1 at
@@ -167,14 +184,13 @@ def prefill_layer(cfg: LayerConfig, w: LayerWeights, x: np.ndarray, cu_seqlens,
     req = np.repeat(np.arange(len(cu) - 1), np.diff(cu))
     pos = np.arange(t_total) - cu[req]
 
+    pj = proj or _ExactProjector(w, dt)
     n1 = st(rmsnorm(x, w.g_attn.astype(dt), cfg.rms_eps))
-    w_qkv = w.w_qkv.astype(dt)
-    w_q, w_k, w_v = w_qkv[:hq * hd], w_qkv[hq * hd:(hq + hkv) * hd], w_qkv[(hq + hkv) * hd:]
-    k = st(rope((n1 @ w_k.T).reshape(t_total, hkv, hd), pos, cfg.rope_theta))
-    v = st((n1 @ w_v.T).reshape(t_total, hkv, hd))
+    k = st(rope(pj(n1, "w_qkv", hq * hd, (hq + hkv) * hd).reshape(t_total, hkv, hd), pos, cfg.rope_theta))
+    v = st(pj(n1, "w_qkv", (hq + hkv) * hd, (hq + 2 * hkv) * hd).reshape(t_total, hkv, hd))
 
     sel = np.arange(t_total) if rows is None else np.asarray(rows, dtype=np.int64)
-    q = st(rope((n1[sel] @ w_q.T).reshape(len(sel), hq, hd), pos[sel], cfg.rope_theta))
+    q = st(rope(pj(n1[sel], "w_qkv", 0, hq * hd).reshape(len(sel), hq, hd), pos[sel], cfg.rope_theta))
 
     o = np.empty((len(sel), hq * hd), dtype=dt)
     for r in range(len(cu) - 1):
@@ -183,13 +199,13 @@ def prefill_layer(cfg: LayerConfig, w: LayerWeights, x: np.ndarray, cu_seqlens,
             continue
         lo, hi = cu[r], cu[r + 1]
         o[mine] = _attend(q[mine], k[lo:hi], v[lo:hi], pos[sel][mine], pos[lo:hi], cfg, probs_out)
-    out = _mlp_and_residuals(x[sel], st(o), w, cfg, dt, st)
+    out = _mlp_and_residuals(x[sel], st(o), w, cfg, dt, st, pj)
     return out, k, v
 
 
 def decode_layer(cfg: LayerConfig, w: LayerWeights, x: np.ndarray, kv_len,
                  k_cache: np.ndarray, v_cache: np.ndarray, dtype=np.float64,
-                 probs_out: list | None = None, store=None) -> np.ndarray:
+                 probs_out: list | None = None, store=None, proj=None) -> np.ndarray:
     """One decode step for a batch of B sequences, one new token each.
 
     kv_len[b] tokens are already cached for sequence b; the new token has
@@ -205,8 +221,9 @@ def decode_layer(cfg: LayerConfig, w: LayerWeights, x: np.ndarray, kv_len,
     hq, hkv, hd = cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim
     assert np.all(kv_len < k_cache.shape[2])
 
+    pj = proj or _ExactProjector(w, dt)
     n1 = st(rmsnorm(x, w.g_attn.astype(dt), cfg.rms_eps))
-    qkv = n1 @ w.w_qkv.astype(dt).T
+    qkv = pj(n1, "w_qkv")
     q = st(rope(qkv[:, :hq * hd].reshape(b_sz, hq, hd), kv_len, cfg.rope_theta))
     k = st(rope(qkv[:, hq * hd:(hq + hkv) * hd].reshape(b_sz, hkv, hd), kv_len, cfg.rope_theta))
     v = st(qkv[:, (hq + hkv) * hd:].reshape(b_sz, hkv, hd))
@@ -219,11 +236,11 @@ def decode_layer(cfg: LayerConfig, w: LayerWeights, x: np.ndarray, kv_len,
         keys = np.ascontiguousarray(k_cache[b, :, :n + 1, :].transpose(1, 0, 2)).astype(dt)
         vals = np.ascontiguousarray(v_cache[b, :, :n + 1, :].transpose(1, 0, 2)).astype(dt)
         o[b:b + 1] = _attend(q[b:b + 1], keys, vals, kv_len[b:b + 1], np.arange(n + 1), cfg, probs_out)
-    return _mlp_and_residuals(x, st(o), w, cfg, dt, st)
+    return _mlp_and_residuals(x, st(o), w, cfg, dt, st, pj)
 
 
 def extend_layer(cfg: LayerConfig, w: LayerWeights, x: np.ndarray, cu_seqlens, prefix_lens,
-                 k_cache: np.ndarray, v_cache: np.ndarray, dtype=np.float64, store=None) -> np.ndarray:
+                 k_cache: np.ndarray, v_cache: np.ndarray, dtype=np.float64, store=None, proj=None) -> np.ndarray:
     """Chunked prefill: one layer over a packed batch of request CHUNKS.
 
     Request r already has prefix_lens[r] tokens in cache sequence r; its chunk rows
@@ -244,8 +261,9 @@ def extend_layer(cfg: LayerConfig, w: LayerWeights, x: np.ndarray, cu_seqlens, p
     pos = np.arange(t_total) - cu[req] + pre[req]
     assert np.all(pos < k_cache.shape[2])
 
+    pj = proj or _ExactProjector(w, dt)
     n1 = st(rmsnorm(x, w.g_attn.astype(dt), cfg.rms_eps))
-    qkv = n1 @ w.w_qkv.astype(dt).T
+    qkv = pj(n1, "w_qkv")
     q = st(rope(qkv[:, :hq * hd].reshape(t_total, hq, hd), pos, cfg.rope_theta))
     k = st(rope(qkv[:, hq * hd:(hq + hkv) * hd].reshape(t_total, hkv, hd), pos, cfg.rope_theta))
     v = st(qkv[:, (hq + hkv) * hd:].reshape(t_total, hkv, hd))
@@ -261,7 +279,7 @@ def extend_layer(cfg: LayerConfig, w: LayerWeights, x: np.ndarray, cu_seqlens, p
         keys = np.ascontiguousarray(k_cache[r, :, :p0 + n, :].transpose(1, 0, 2)).astype(dt)
         vals = np.ascontiguousarray(v_cache[r, :, :p0 + n, :].transpose(1, 0, 2)).astype(dt)
         o[lo:hi] = _attend(q[lo:hi], keys, vals, pos[lo:hi], np.arange(p0 + n), cfg, None)
-    return _mlp_and_residuals(x, st(o), w, cfg, dt, st)
+    return _mlp_and_residuals(x, st(o), w, cfg, dt, st, pj)
 
 
 def layer_flops_prefill(cfg: LayerConfig, lens) -> float:
