@@ -257,6 +257,22 @@ pd_status pd_model_check(pd_model* model, void* stream);
 pd_status pd_gemm_bf16(const void* a, const void* b, void* c, int32_t m, int32_t n, int32_t k,
                        int32_t* err_word, void* stream);
 
+/* FP8 projections.  The paper's TTFT validation (Figure 1 experiment) runs an FP8 checkpoint but gives
+ * neither the number format nor the scaling; the reading built here is OCP E4M3 codes with one fp32 scale
+ * per row: a weight matrix is quantised per output channel, an activation matrix per token.
+ *
+ * pd_quantize_fp8_rows: x device bf16 [rows, k] with row pitch ldx elements -> codes device uint8
+ * [rows, k] (contiguous), scales device fp32 [rows].  scale = max|row| / 448 (1 for an all-zero row),
+ * code = E4M3(x / scale), both in fp32, round to nearest even, saturating.  k a multiple of 16.
+ *
+ * pd_gemm_fp8: C[M,N] (device bf16) = (dec(A)[M,K] * dec(B)[N,K]^T) * a_scales[m] * b_scales[n] with fp32
+ * accumulation on the tensor cores (tcgen05 kind::f8f6f4).  Codes contiguous row-major, 16-byte aligned;
+ * K a multiple of 128, N of 16.  `err_word` as in pd_gemm_bf16.  Both calls only enqueue work. */
+pd_status pd_quantize_fp8_rows(const void* x, int32_t ldx, int32_t rows, int32_t k, void* codes, float* scales,
+                               void* stream);
+pd_status pd_gemm_fp8(const void* a_codes, const float* a_scales, const void* b_codes, const float* b_scales,
+                      void* c, int32_t m, int32_t n, int32_t k, int32_t* err_word, void* stream);
+
 /* Kernels launched so far by the calling thread through this library. */
 int64_t pd_launch_count(void);
 

@@ -37,7 +37,7 @@ EXPORTS = [
     "pd_launch_count", "pd_trace_begin", "pd_trace_end", "pd_decode_attention", "pd_decode_attention_workspace_bytes",
     "pd_decode_attention_noalloc", "pd_prefill_chunk_layer",
     "pd_model_create", "pd_model_destroy", "pd_model_workspace_bytes", "pd_model_prefill", "pd_model_decode_step",
-    "pd_model_check", "pd_allocate_ext",
+    "pd_model_check", "pd_allocate_ext", "pd_quantize_fp8_rows", "pd_gemm_fp8",
 ]
 
 TRACE_CLASSES = ["gemm_qkv", "gemm_o", "gemm_gate_up", "gemm_down", "attn_prefill", "attn_decode", "rmsnorm",
@@ -131,6 +131,8 @@ _lib.pd_decode_stack.argtypes = [C.POINTER(_P), C.POINTER(pd_kv_cache), C.c_int3
                                  C.c_int32, C.c_int32, _P, C.c_size_t, _P]
 _lib.pd_layer_check.argtypes = [_P, _P]
 _lib.pd_gemm_bf16.argtypes = [_P, _P, _P, C.c_int32, C.c_int32, C.c_int32, _P, _P]
+_lib.pd_quantize_fp8_rows.argtypes = [_P, C.c_int32, C.c_int32, C.c_int32, _P, _P, _P]
+_lib.pd_gemm_fp8.argtypes = [_P, _P, _P, _P, _P, C.c_int32, C.c_int32, C.c_int32, _P, _P]
 _lib.pd_measure.argtypes = [C.POINTER(pd_layer_cfg), C.POINTER(pd_measure_cfg), C.c_double, C.c_double,
                             C.POINTER(pd_measurement)]
 _lib.pd_allocate.argtypes = [C.POINTER(pd_alloc_in), C.POINTER(pd_alloc_out)]
@@ -398,6 +400,17 @@ def pd_layer_check(layer: Layer, stream=None):
 
 def pd_gemm_bf16(a, b, c, m: int, n: int, k: int, err_word=None, stream=None):
     _check(_lib.pd_gemm_bf16(_ptr(a), _ptr(b), _ptr(c), m, n, k, _ptr(err_word), _stream_ptr(stream)), "pd_gemm_bf16")
+
+
+def pd_quantize_fp8_rows(x, rows: int, k: int, codes, scales, ldx: int = 0, stream=None):
+    """x: device bf16 [rows, k] (row pitch ldx, default k) -> codes: device uint8 [rows, k], scales: device fp32 [rows]."""
+    _check(_lib.pd_quantize_fp8_rows(_ptr(x), ldx or k, rows, k, _ptr(codes), _ptr(scales), _stream_ptr(stream)),
+           "pd_quantize_fp8_rows")
+
+
+def pd_gemm_fp8(a_codes, a_scales, b_codes, b_scales, c, m: int, n: int, k: int, err_word=None, stream=None):
+    _check(_lib.pd_gemm_fp8(_ptr(a_codes), _ptr(a_scales), _ptr(b_codes), _ptr(b_scales), _ptr(c), m, n, k,
+                            _ptr(err_word), _stream_ptr(stream)), "pd_gemm_fp8")
 
 
 def pd_measure(cfg: LayerConfig, *, n_layers_run: int, n_layers_model: int, warmup: int = 3, reps: int = 10,

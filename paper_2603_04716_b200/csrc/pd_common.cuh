@@ -69,6 +69,10 @@ class TraceScope {
 pd_status make_tmap_bf16(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint64_t ld,
                          uint32_t box_rows);
 
+// The same for one-byte elements (FP8 codes): boxes of box_rows x 128 columns.
+pd_status make_tmap_u8(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint64_t ld,
+                       uint32_t box_rows);
+
 // ------------------------------------------------------------------ GEMM
 enum GemmEpilogue : int {
   EPI_STORE = 0,     // C = acc
@@ -92,13 +96,16 @@ struct RopeEpilogue {
 };
 
 struct GemmArgs {
-  const bf16* a;  // [M, K], row pitch lda
+  const bf16* a;  // [M, K], row pitch lda (FP8 operands: E4M3 codes, one byte per element, behind the same pointers)
   const bf16* b;  // [N, K], row pitch ldb
   bf16* c;        // [M, N] (EPI_SWIGLU: [M, N/2]; EPI_ROPE_KV: q heads only), row pitch ldc
   const bf16* r;  // residual [M, N], row pitch ldr (EPI_RESIDUAL); may alias c
   int m, n, k;
   int lda, ldb, ldc, ldr;
   int epilogue;
+  int fp8;                    // 1: A and B hold E4M3 codes; the product is scaled by scale_a[row] * scale_b[column]
+  const float* scale_a;       // [M]
+  const float* scale_b;       // [N]
   const RopeEpilogue* rope;   // EPI_ROPE_KV
   int* err_word;              // device int32: 1 = a bounded wait gave up, 2 = a position or slot was out of range
   // Optional K split of the last partial wave (see gemm_tc_kernel): fp32 scratch of at least
@@ -184,6 +191,11 @@ struct DecodeAttnArgs {
 };
 int decode_attention_splits(int batch, int n_kv_heads, int max_kv_len);
 pd_status launch_decode_attention(const DecodeAttnArgs& a, cudaStream_t s);
+
+// Per-row dynamic FP8 quantisation: scale[r] = max|x[r, :]| / 448 (1 for an all-zero row),
+// codes[r, k] = E4M3(x[r, k] / scale[r]), round to nearest even, saturating.  k a multiple of 16.
+pd_status launch_quantize_rows_fp8(const bf16* x, int ldx, int rows, int k, uint8_t* codes, int ldq, float* scale,
+                                   cudaStream_t s);
 
 // Seeded N(mean, std) fill in bf16 (counter-based; value i depends only on seed, stream, i).
 pd_status launch_fill_normal(bf16* dst, size_t n, uint64_t seed, uint64_t stream_id, float mean, float std,

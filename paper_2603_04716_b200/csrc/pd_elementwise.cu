@@ -21,6 +21,50 @@ __device__ __forceinline__ uint4 pack8(const float (&f)[8]) {
   return o;
 }
 
+// ------------------------------------------------------- FP8 row quantisation
+// One block per row: pass 1 finds max|x|, pass 2 (the row is still in L1/L2) divides by
+// scale = max / 448 in fp32 (IEEE division, the precision in which the codes are defined) and
+// converts with round-to-nearest-even, saturating.  An all-zero row gets scale 1.
+constexpr int QNT_THREADS = 256;
+
+__global__ void __launch_bounds__(QNT_THREADS) quantize_rows_fp8_kernel(const bf16* __restrict__ x, int ldx, int k,
+                                                                         uint8_t* __restrict__ codes, int ldq,
+                                                                         float* __restrict__ scale_out) {
+  const int row = blockIdx.x;
+  ptx::grid_launch_dependents();
+  ptx::grid_dependency_wait();
+  const uint4* xr = reinterpret_cast<const uint4*>(x + static_cast<size_t>(row) * ldx);
+  const int chunks = k / 8;
+  float amax = 0.f;
+  for (int c = threadIdx.x; c < chunks; c += QNT_THREADS) {
+    float f[8];
+    unpack8(xr[c], f);
+#pragma unroll
+    for (int e = 0; e < 8; ++e) amax = fmaxf(amax, fabsf(f[e]));
+  }
+  __shared__ float red[QNT_THREADS / 32];
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = amax;
+  __syncthreads();
+  float tot = 0.f;
+#pragma unroll
+  for (int w = 0; w < QNT_THREADS / 32; ++w) tot = fmaxf(tot, red[w]);
+  const float scale = tot > 0.f ? __fdiv_rn(tot, 448.f) : 1.f;
+  if (threadIdx.x == 0) scale_out[row] = scale;
+  uint2* qr = reinterpret_cast<uint2*>(codes + static_cast<size_t>(row) * ldq);
+  for (int c = threadIdx.x; c < chunks; c += QNT_THREADS) {
+    float f[8];
+    unpack8(xr[c], f);
+#pragma unroll
+    for (int e = 0; e < 8; ++e) f[e] = __fdiv_rn(f[e], scale);
+    uint2 o;
+    o.x = ptx::cvt_e4m3x2(f[0], f[1]) | (ptx::cvt_e4m3x2(f[2], f[3]) << 16);
+    o.y = ptx::cvt_e4m3x2(f[4], f[5]) | (ptx::cvt_e4m3x2(f[6], f[7]) << 16);
+    qr[c] = o;
+  }
+}
+
 // ------------------------------------------------------------------- RMSNorm
 // y = x * rsqrt(mean(x^2) + eps) * g; one block per row, row kept in registers.
 constexpr int RMS_THREADS = 256;
@@ -120,6 +164,16 @@ pd_status launch_rmsnorm_decode(const bf16* x, const bf16* gain, bf16* y, int ro
   return PD_OK;
 }
 
+pd_status launch_quantize_rows_fp8(const bf16* x, int ldx, int rows, int k, uint8_t* codes, int ldq, float* scale,
+                                   cudaStream_t s) {
+  if (rows == 0) return PD_OK;
+  if (!x || !codes || !scale || rows < 0 || k <= 0) return PD_ERR_INVALID_ARG;
+  if (k % 16 != 0 || ldx % 8 != 0 || ldq % 16 != 0 || ldx < k || ldq < k) return PD_ERR_UNSUPPORTED_SHAPE;
+  PD_CUDA_TRY(launch_pdl(quantize_rows_fp8_kernel, dim3(rows), dim3(QNT_THREADS), 0, s, x, ldx, k, codes, ldq, scale));
+  count_launch();
+  return PD_OK;
+}
+
 pd_status launch_fill_normal(bf16* dst, size_t n, uint64_t seed, uint64_t stream_id, float mean, float std,
                              cudaStream_t s) {
   if (n == 0) return PD_OK;
@@ -130,3 +184,9 @@ pd_status launch_fill_normal(bf16* dst, size_t n, uint64_t seed, uint64_t stream
 }
 
 }  // namespace pd
+
+extern "C" pd_status pd_quantize_fp8_rows(const void* x, int32_t ldx, int32_t rows, int32_t k, void* codes,
+                                          float* scales, void* stream) {
+  return pd::launch_quantize_rows_fp8(static_cast<const pd::bf16*>(x), ldx, rows, k, static_cast<uint8_t*>(codes), k,
+                                      scales, static_cast<cudaStream_t>(stream));
+}

@@ -1,4 +1,7 @@
-// C[M,N] = A[M,K] * B[N,K]^T (+ residual), bf16 operands, fp32 accumulation.
+// C[M,N] = A[M,K] * B[N,K]^T (+ residual), bf16 or FP8 (E4M3) operands, fp32 accumulation.
+// With FP8 operands a shared-memory row of 128 bytes holds 128 K elements instead of 64, the
+// instruction is tcgen05.mma.kind::f8f6f4 (32 K elements each) and the accumulator is multiplied by
+// the row scale of A and the row scale of B before the epilogue proper.
 //
 // A persistent, warp-specialised kernel.  One thread issues TMA tile
 // loads of A (128 x 64) and B (BN x 64) into a ring of shared-memory stages; one thread
@@ -51,11 +54,28 @@ pd_status make_tmap_bf16(CUtensorMap* out, const void* base, uint64_t rows, uint
   return r == CUDA_SUCCESS ? PD_OK : PD_ERR_INVALID_ARG;
 }
 
+pd_status make_tmap_u8(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint64_t ld,
+                       uint32_t box_rows) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return PD_ERR_CUDA;
+  if ((reinterpret_cast<uintptr_t>(base) & 15u) || ld % 16 != 0 || box_rows == 0 || box_rows > 256)
+    return PD_ERR_INVALID_ARG;
+  cuuint64_t dims[2] = {cols, rows};
+  cuuint64_t strides[1] = {ld};
+  cuuint32_t box[2] = {128, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? PD_OK : PD_ERR_INVALID_ARG;
+}
+
 // ---------------------------------------------------------------- tcgen05 GEMM
 namespace {
 
 constexpr int BM = 128;
-constexpr int BK = 64;
+constexpr int BK = 64;        // K elements of a bf16 stage (128 bytes per row)
+constexpr int BK_F8 = 128;    // K elements of an FP8 stage (the same 128 bytes per row)
 constexpr int GEMM_THREADS = 192;  // warp 0: TMA, warp 1: MMA, warps 2-5: epilogue
 constexpr int TMEM_COLS = 512;
 
@@ -86,6 +106,8 @@ struct GemmDev {
   int* split_flags;      // [tail tile][4], 1 while a partial waits to be consumed
   int split_enable;
   int* err_word;
+  const float* scale_a;  // FP8 operands: per-row scale of A [M] and of B [N]
+  const float* scale_b;
   RopeEpilogue rope;  // EPI_ROPE_KV only
 };
 
@@ -135,7 +157,7 @@ __device__ __forceinline__ UnitInfo unit_info(int unit, int main_tiles, int k_bl
   return u;
 }
 
-template <int BN, int EPI>
+template <int BN, int EPI, bool F8>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b, GemmDev p) {
   using Cfg = GemmCfg<BN>;
@@ -180,8 +202,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
+  constexpr int KE = F8 ? BK_F8 : BK;  // K elements per stage
   const int n_units = p.n_units;
-  const int k_blocks = p.k / BK;
+  const int k_blocks = p.k / KE;
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
@@ -198,8 +221,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
           const uint32_t sa = smem_base + stage * Cfg::STAGE_BYTES;
           const uint32_t sb = sa + Cfg::A_BYTES;
           ptx::mbar_arrive_expect_tx(full_bar(stage), Cfg::STAGE_BYTES);
-          ptx::tma_load_2d(sa, &tmap_a, kb * BK, tm * BM, full_bar(stage));
-          ptx::tma_load_2d(sb, &tmap_b, kb * BK, tn * BN, full_bar(stage));
+          ptx::tma_load_2d(sa, &tmap_a, kb * KE, tm * BM, full_bar(stage));
+          ptx::tma_load_2d(sb, &tmap_b, kb * KE, tn * BN, full_bar(stage));
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
       }
@@ -211,7 +234,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
   } else if (warp == 1) {
     // -------------------------------------------------------------- MMA issuer
     if (lane == 0) {
-      constexpr uint32_t idesc = ptx::umma_idesc_bf16(BM, BN);
+      constexpr uint32_t idesc = F8 ? ptx::umma_idesc_e4m3(BM, BN) : ptx::umma_idesc_bf16(BM, BN);
+      constexpr uint32_t idesc_half = F8 ? ptx::umma_idesc_e4m3(BM, 128) : ptx::umma_idesc_bf16(BM, 128);
       int stage = 0;
       uint32_t phase = 0;
       int acc = 0;
@@ -229,12 +253,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
           const uint32_t sb = sa + Cfg::A_BYTES;
           const uint64_t da = ptx::umma_desc_sw128(sa);
           // a half-width unit multiplies by rows 128 n_half .. of the B tile only (128 rows = 16 KB further on)
-          const uint64_t db = ptx::umma_desc_sw128(sb + ui.n_half * (128 * BK * 2));
-          const uint32_t idesc_u = (ui.role == 3) ? ptx::umma_idesc_bf16(BM, 128) : idesc;
+          const uint64_t db = ptx::umma_desc_sw128(sb + ui.n_half * (128 * 128));
+          const uint32_t idesc_u = (ui.role == 3) ? idesc_half : idesc;
 #pragma unroll
-          for (int kk = 0; kk < BK / 16; ++kk) {
-            // 16 bf16 = 32 bytes along K inside the 128-byte swizzled row: +2 in 16-byte units
-            ptx::umma_bf16(d_tmem, da + 2u * kk, db + 2u * kk, idesc_u, (kb > ui.kb_lo || kk > 0) ? 1u : 0u);
+          for (int kk = 0; kk < 4; ++kk) {
+            // one instruction covers 32 bytes along K (16 bf16 or 32 FP8) of the 128-byte swizzled row:
+            // +2 in 16-byte units
+            const uint32_t accum = (kb > ui.kb_lo || kk > 0) ? 1u : 0u;
+            if constexpr (F8) ptx::umma_f8(d_tmem, da + 2u * kk, db + 2u * kk, idesc_u, accum);
+            else ptx::umma_bf16(d_tmem, da + 2u * kk, db + 2u * kk, idesc_u, accum);
           }
           ptx::umma_commit(empty_bar(stage));  // stage is free once these MMAs have read it
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
@@ -299,7 +326,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
           __threadfence();
         }
       }
-      // accumulator chunk -> registers (+ the partner's partial for a K-split tile)
+      // a half-width unit holds columns [128 n_half, 128 n_half + 128) of its tile in accumulator columns 0..127
+      const int acc_cols = (ui.role == 3) ? 128 : BN;
+      const int col_base = tn * BN + ui.n_half * 128;
+      float row_scale = 1.f;
+      if constexpr (F8) row_scale = row < p.m ? p.scale_a[row] : 0.f;
+      // accumulator chunk -> registers (+ the partner's partial for a K-split tile; x the operand scales for FP8)
       auto load_acc = [&](int col_off, uint32_t (&v)[32]) {
         ptx::tmem_ld_32x32(t_row + col_off, v);
         ptx::tmem_ld_wait();
@@ -313,10 +345,19 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             v[j + 3] = __float_as_uint(__uint_as_float(v[j + 3]) + q.w);
           }
         }
+        if constexpr (F8) {
+          const int col = col_base + col_off;  // row of B = column of the product (a multiple of 32)
+#pragma unroll
+          for (int j = 0; j < 32; j += 4) {
+            float4 sb = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (col + j < p.n) sb = __ldg(reinterpret_cast<const float4*>(p.scale_b + col + j));
+            v[j] = __float_as_uint(__uint_as_float(v[j]) * (row_scale * sb.x));
+            v[j + 1] = __float_as_uint(__uint_as_float(v[j + 1]) * (row_scale * sb.y));
+            v[j + 2] = __float_as_uint(__uint_as_float(v[j + 2]) * (row_scale * sb.z));
+            v[j + 3] = __float_as_uint(__uint_as_float(v[j + 3]) * (row_scale * sb.w));
+          }
+        }
       };
-      // a half-width unit holds columns [128 n_half, 128 n_half + 128) of its tile in accumulator columns 0..127
-      const int acc_cols = (ui.role == 3) ? 128 : BN;
-      const int col_base = tn * BN + ui.n_half * 128;
       if (ui.role == 1 || !ok) {
         // nothing more to do for this unit
       } else if constexpr (EPI == EPI_STORE || EPI == EPI_RESIDUAL) {
@@ -473,19 +514,25 @@ int sm_count() {
   return g_sm_count;
 }
 
-template <int BN, int EPI>
+template <int BN, int EPI, bool F8>
 pd_status launch_tc(const GemmArgs& g, cudaStream_t stream) {
   using Cfg = GemmCfg<BN>;
   static bool attr_set = false;
-  auto kern = gemm_tc_kernel<BN, EPI>;
+  auto kern = gemm_tc_kernel<BN, EPI, F8>;
   if (!attr_set) {
     PD_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES));
     attr_set = true;
   }
   CUtensorMap ta, tb;
-  PD_TRY(make_tmap_bf16(&ta, g.a, g.m, g.k, g.lda, BM));
-  PD_TRY(make_tmap_bf16(&tb, g.b, g.n, g.k, g.ldb, BN));
+  if (F8) {
+    PD_TRY(make_tmap_u8(&ta, g.a, g.m, g.k, g.lda, BM));
+    PD_TRY(make_tmap_u8(&tb, g.b, g.n, g.k, g.ldb, BN));
+  } else {
+    PD_TRY(make_tmap_bf16(&ta, g.a, g.m, g.k, g.lda, BM));
+    PD_TRY(make_tmap_bf16(&tb, g.b, g.n, g.k, g.ldb, BN));
+  }
   GemmDev p{};
+  p.scale_a = g.scale_a; p.scale_b = g.scale_b;
   p.c = g.c; p.r = g.r; p.m = g.m; p.n = g.n; p.k = g.k; p.ldc = g.ldc; p.ldr = g.ldr;
   p.tiles_m = (g.m + BM - 1) / BM;
   p.tiles_n = (g.n + BN - 1) / BN;
@@ -508,7 +555,7 @@ pd_status launch_tc(const GemmArgs& g, cudaStream_t stream) {
     const size_t need = static_cast<size_t>(tail) * BM * BN * sizeof(float);
     // (pays only for long K: with K = 4096 the parked partial tile and the hand-over cost as much as the
     // half tile they save; measured -6 % on the K = 14336 down projection, +5 % on the K = 4096 ones)
-    if (tail > 0 && 2 * tail <= sms && g.k / BK >= 128 && g.split_scratch && g.split_flags &&
+    if (tail > 0 && 2 * tail <= sms && g.k / (F8 ? BK_F8 : BK) >= 128 && g.split_scratch && g.split_flags &&
         need <= g.split_scratch_bytes && tail <= kSplitMaxTiles) {
       p.main_tiles = tiles - tail;
       p.n_units = tiles + tail;
@@ -527,17 +574,17 @@ pd_status launch_tc(const GemmArgs& g, cudaStream_t stream) {
   return PD_OK;
 }
 
-template <int BN>
+template <int BN, bool F8>
 pd_status launch_tc_epi(const GemmArgs& g, cudaStream_t stream) {
   switch (g.epilogue) {
-    case EPI_RESIDUAL: return launch_tc<BN, EPI_RESIDUAL>(g, stream);
+    case EPI_RESIDUAL: return launch_tc<BN, EPI_RESIDUAL, F8>(g, stream);
     case EPI_SWIGLU:
-      if constexpr (BN >= 128) return launch_tc<BN, EPI_SWIGLU>(g, stream);
+      if constexpr (BN >= 128) return launch_tc<BN, EPI_SWIGLU, F8>(g, stream);
       return PD_ERR_UNSUPPORTED_SHAPE;
     case EPI_ROPE_KV:
-      if constexpr (BN >= 128) return launch_tc<BN, EPI_ROPE_KV>(g, stream);
+      if constexpr (BN >= 128) return launch_tc<BN, EPI_ROPE_KV, F8>(g, stream);
       return PD_ERR_UNSUPPORTED_SHAPE;
-    default: return launch_tc<BN, EPI_STORE>(g, stream);
+    default: return launch_tc<BN, EPI_STORE, F8>(g, stream);
   }
 }
 
@@ -570,8 +617,10 @@ static pd_status check_gemm_args(const GemmArgs& g) {
   if (!g.a || !g.b || !g.c || g.m < 0 || g.n <= 0 || g.k <= 0) return PD_ERR_INVALID_ARG;
   if (g.epilogue == EPI_RESIDUAL && !g.r) return PD_ERR_INVALID_ARG;
   if (g.epilogue == EPI_ROPE_KV && !g.rope) return PD_ERR_INVALID_ARG;
-  if (g.k % BK != 0 || g.n % 16 != 0) return PD_ERR_UNSUPPORTED_SHAPE;
-  if (g.lda % 8 || g.ldb % 8 || g.ldc % 8 || (g.epilogue == EPI_RESIDUAL && g.ldr % 8)) return PD_ERR_UNSUPPORTED_SHAPE;
+  if (g.fp8 && (!g.scale_a || !g.scale_b)) return PD_ERR_INVALID_ARG;
+  if (g.k % (g.fp8 ? BK_F8 : BK) != 0 || g.n % 16 != 0) return PD_ERR_UNSUPPORTED_SHAPE;
+  const int opa = g.fp8 ? 16 : 8;  // operand row pitches: multiples of 16 bytes
+  if (g.lda % opa || g.ldb % opa || g.ldc % 8 || (g.epilogue == EPI_RESIDUAL && g.ldr % 8)) return PD_ERR_UNSUPPORTED_SHAPE;
   if (g.epilogue == EPI_SWIGLU && g.n % 128 != 0) return PD_ERR_UNSUPPORTED_SHAPE;
   return PD_OK;
 }
@@ -579,10 +628,18 @@ static pd_status check_gemm_args(const GemmArgs& g) {
 pd_status gemm(const GemmArgs& g, cudaStream_t stream) {
   PD_TRY(check_gemm_args(g));
   if (g.m == 0) return PD_OK;
-  switch (gemm_block_n(g.m, g.n, g.epilogue)) {
-    case 256: return launch_tc_epi<256>(g, stream);
-    case 128: return launch_tc_epi<128>(g, stream);
-    default: return launch_tc_epi<64>(g, stream);
+  const int bn = gemm_block_n(g.m, g.n, g.epilogue);
+  if (g.fp8) {
+    switch (bn) {
+      case 256: return launch_tc_epi<256, true>(g, stream);
+      case 128: return launch_tc_epi<128, true>(g, stream);
+      default: return launch_tc_epi<64, true>(g, stream);
+    }
+  }
+  switch (bn) {
+    case 256: return launch_tc_epi<256, false>(g, stream);
+    case 128: return launch_tc_epi<128, false>(g, stream);
+    default: return launch_tc_epi<64, false>(g, stream);
   }
 }
 
@@ -598,6 +655,20 @@ extern "C" pd_status pd_gemm_bf16(const void* a, const void* b, void* c, int32_t
   g.m = m; g.n = n; g.k = k;
   g.lda = k; g.ldb = k; g.ldc = n; g.ldr = 0;
   g.epilogue = pd::EPI_STORE;
+  g.err_word = err_word;
+  return pd::gemm(g, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" pd_status pd_gemm_fp8(const void* a_codes, const float* a_scales, const void* b_codes, const float* b_scales,
+                                 void* c, int32_t m, int32_t n, int32_t k, int32_t* err_word, void* stream) {
+  pd::GemmArgs g{};
+  g.a = static_cast<const pd::bf16*>(a_codes);
+  g.b = static_cast<const pd::bf16*>(b_codes);
+  g.c = static_cast<pd::bf16*>(c);
+  g.m = m; g.n = n; g.k = k;
+  g.lda = k; g.ldb = k; g.ldc = n; g.ldr = 0;
+  g.epilogue = pd::EPI_STORE;
+  g.fp8 = 1; g.scale_a = a_scales; g.scale_b = b_scales;
   g.err_word = err_word;
   return pd::gemm(g, static_cast<cudaStream_t>(stream));
 }
