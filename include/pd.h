@@ -50,12 +50,17 @@ int pd_version(void);
 
 /* Shape of one decoder layer.  Supported: head_dim 64 or 128, n_q_heads a multiple
  * of n_kv_heads with group size <= 16, d_model and d_ff multiples of 64,
- * max_pos = largest token position + 1 ever used (RoPE table length). */
+ * max_pos = largest token position + 1 ever used (RoPE table length).
+ * fp8_projections = 1 runs the five projections in FP8 (see pd_gemm_fp8 for the reading of the paper's
+ * FP8 checkpoint): pd_layer_create quantises every weight matrix per output channel to E4M3 and keeps
+ * only the codes and scales; each pass quantises the projection inputs per token.  Attention, norms,
+ * residual stream and KV cache stay bf16.  Needs d_model, d_ff and n_q_heads * head_dim multiples of 128. */
 typedef struct {
   uint32_t struct_size;
   int32_t d_model, n_q_heads, n_kv_heads, head_dim, d_ff;
   float rms_eps, rope_theta;
   int32_t max_pos;
+  int32_t fp8_projections;
 } pd_layer_cfg;
 
 /* Caller's weights: device pointers, bf16, row-major [out_features, in_features]. */
@@ -256,6 +261,19 @@ pd_status pd_model_check(pd_model* model, void* stream);
  * `err_word` device int32 (may be NULL), set non-zero if a bounded wait gave up. */
 pd_status pd_gemm_bf16(const void* a, const void* b, void* c, int32_t m, int32_t n, int32_t k,
                        int32_t* err_word, void* stream);
+
+/* Where a layer pass leaves its intermediates.  Byte offsets, inside the workspace handed to
+ * pd_prefill_layer / pd_prefill_chunk_layer over `tokens` rows (or pd_decode_layer with B = tokens), of the
+ * bf16 tensors that are still there when the pass has finished: norm = RMSNorm output that fed the MLP
+ * [tokens, d]; qkv = [tokens, Nqkv] of which the q columns (after RoPE) are written; attn_o = attention output
+ * [tokens, Hq*hd]; resid = residual stream after the attention half [tokens, d]; act = SwiGLU output
+ * [tokens, F].  For inspection and stage-by-stage parity checks (the layer is the unit the paper's benchmarks
+ * time; the stages are this library's).  Host only. */
+typedef struct {
+  uint32_t struct_size;
+  uint64_t norm, qkv, attn_o, resid, act;
+} pd_workspace_layout;
+pd_status pd_workspace_offsets(const pd_layer_cfg* cfg, int32_t tokens, pd_workspace_layout* out);
 
 /* FP8 projections.  The paper's TTFT validation (Figure 1 experiment) runs an FP8 checkpoint but gives
  * neither the number format nor the scaling; the reading built here is OCP E4M3 codes with one fp32 scale

@@ -37,7 +37,7 @@ EXPORTS = [
     "pd_launch_count", "pd_trace_begin", "pd_trace_end", "pd_decode_attention", "pd_decode_attention_workspace_bytes",
     "pd_decode_attention_noalloc", "pd_prefill_chunk_layer",
     "pd_model_create", "pd_model_destroy", "pd_model_workspace_bytes", "pd_model_prefill", "pd_model_decode_step",
-    "pd_model_check", "pd_allocate_ext", "pd_quantize_fp8_rows", "pd_gemm_fp8",
+    "pd_model_check", "pd_allocate_ext", "pd_quantize_fp8_rows", "pd_gemm_fp8", "pd_workspace_offsets",
 ]
 
 TRACE_CLASSES = ["gemm_qkv", "gemm_o", "gemm_gate_up", "gemm_down", "attn_prefill", "attn_decode", "rmsnorm",
@@ -56,7 +56,12 @@ class PdError(RuntimeError):
 class pd_layer_cfg(C.Structure):
     _fields_ = [("struct_size", C.c_uint32), ("d_model", C.c_int32), ("n_q_heads", C.c_int32),
                 ("n_kv_heads", C.c_int32), ("head_dim", C.c_int32), ("d_ff", C.c_int32),
-                ("rms_eps", C.c_float), ("rope_theta", C.c_float), ("max_pos", C.c_int32)]
+                ("rms_eps", C.c_float), ("rope_theta", C.c_float), ("max_pos", C.c_int32),
+                ("fp8_projections", C.c_int32)]
+
+
+class pd_workspace_layout(C.Structure):
+    _fields_ = [("struct_size", C.c_uint32)] + [(n, C.c_uint64) for n in ("norm", "qkv", "attn_o", "resid", "act")]
 
 
 class pd_layer_weights(C.Structure):
@@ -131,6 +136,7 @@ _lib.pd_decode_stack.argtypes = [C.POINTER(_P), C.POINTER(pd_kv_cache), C.c_int3
                                  C.c_int32, C.c_int32, _P, C.c_size_t, _P]
 _lib.pd_layer_check.argtypes = [_P, _P]
 _lib.pd_gemm_bf16.argtypes = [_P, _P, _P, C.c_int32, C.c_int32, C.c_int32, _P, _P]
+_lib.pd_workspace_offsets.argtypes = [C.POINTER(pd_layer_cfg), C.c_int32, C.POINTER(pd_workspace_layout)]
 _lib.pd_quantize_fp8_rows.argtypes = [_P, C.c_int32, C.c_int32, C.c_int32, _P, _P, _P]
 _lib.pd_gemm_fp8.argtypes = [_P, _P, _P, _P, _P, C.c_int32, C.c_int32, C.c_int32, _P, _P]
 _lib.pd_measure.argtypes = [C.POINTER(pd_layer_cfg), C.POINTER(pd_measure_cfg), C.c_double, C.c_double,
@@ -203,10 +209,11 @@ class LayerConfig:
     rms_eps: float = 1e-6
     rope_theta: float = 1e4
     max_pos: int = 4096
+    fp8_projections: bool = False
 
     def c_struct(self) -> pd_layer_cfg:
         return pd_layer_cfg(C.sizeof(pd_layer_cfg), self.d_model, self.n_q_heads, self.n_kv_heads, self.head_dim,
-                            self.d_ff, self.rms_eps, self.rope_theta, self.max_pos)
+                            self.d_ff, self.rms_eps, self.rope_theta, self.max_pos, int(self.fp8_projections))
 
     @property
     def n_qkv(self) -> int:
@@ -400,6 +407,13 @@ def pd_layer_check(layer: Layer, stream=None):
 
 def pd_gemm_bf16(a, b, c, m: int, n: int, k: int, err_word=None, stream=None):
     _check(_lib.pd_gemm_bf16(_ptr(a), _ptr(b), _ptr(c), m, n, k, _ptr(err_word), _stream_ptr(stream)), "pd_gemm_bf16")
+
+
+def pd_workspace_offsets(cfg: LayerConfig, tokens: int) -> dict:
+    """Byte offsets of the intermediates a layer pass over `tokens` rows leaves in its workspace."""
+    out = pd_workspace_layout(C.sizeof(pd_workspace_layout))
+    _check(_lib.pd_workspace_offsets(C.byref(cfg.c_struct()), tokens, C.byref(out)), "pd_workspace_offsets")
+    return {n: int(getattr(out, n)) for n in ("norm", "qkv", "attn_o", "resid", "act")}
 
 
 def pd_quantize_fp8_rows(x, rows: int, k: int, codes, scales, ldx: int = 0, stream=None):

@@ -132,10 +132,13 @@ struct SkinnyGemmArgs {
   int batch, n, k, ldx;
   int* err_word;
   bool acc_zeroed;  // the caller guarantees acc is zero when the kernel's epilogue runs (no memset is enqueued)
+  int fp8;                 // 1: x and w hold E4M3 codes (one byte per element); sums are scaled by scale_x[b] * scale_w[n]
+  const float* scale_x;    // [B]
+  const float* scale_w;    // [N]
 };
 pd_status gemm_skinny(const SkinnyGemmArgs& g, cudaStream_t stream);
 // Number of K slices gemm_skinny will use (1: plain stores, acc need not be zero).
-int gemm_skinny_splits(int batch, int n, int k);
+int gemm_skinny_splits(int batch, int n, int k, bool fp8 = false);
 // Row-wise kernels that turn the fp32 sums into the layer's stored tensors.
 // Every row-wise kernel can also clear the fp32 sums of a LATER projection (zero_ptr[batch, zero_cols], NULL to
 // skip): the buffer is idle while the kernel runs, and the projection then needs no memset of its own.
@@ -208,6 +211,9 @@ struct pd_layer {
   pd_layer_cfg cfg;
   int n_qkv;
   pd::bf16 *w_qkv, *w_o, *w_gu, *w_down;  // owned copies; w_gu = [2F, d]: 64 gate rows, 64 up rows, alternating
+                                           // (released after quantisation when cfg.fp8_projections is set)
+  uint8_t *q_qkv, *q_o, *q_gu, *q_down;    // FP8 mode: E4M3 codes in the same layouts
+  float *s_qkv, *s_o, *s_gu, *s_down;      // FP8 mode: one scale per weight row
   pd::bf16 *g_attn, *g_mlp;
   float2* rope_tab;                        // [max_pos, hd/2]
   int* err_word;                           // device int32

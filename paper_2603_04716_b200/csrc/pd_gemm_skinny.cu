@@ -42,13 +42,18 @@ struct SkinnyDev {
   float* acc;  // [B, N] fp32
   int batch, n, k_blocks, splits, tiles_n;
   int* err_word;
+  const float* scale_x;  // FP8 operands: per-row scales of X [B] and of W [N]
+  const float* scale_w;
 };
 
-template <int BNB, int MT>
+// F8: both operands are E4M3 codes (a 128-byte shared-memory row then holds 128 K elements, one MMA covers 32)
+// and every partial sum is multiplied by scale_x[b] * scale_w[n] on its way out.
+template <int BNB, int MT, bool F8>
 __global__ void __launch_bounds__(SK_THREADS)
 gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_x, SkinnyDev p) {
   using Cfg = SkinnyCfg<BNB, MT>;
   constexpr int STAGES = Cfg::STAGES;
+  constexpr int KE = F8 ? 2 * SK_BK : SK_BK;  // K elements per stage (128 bytes per row either way)
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_al = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
@@ -103,12 +108,12 @@ gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
       for (int i = 0; i < pre; ++i) {
         const uint32_t sw = smem_base + i * Cfg::STAGE_BYTES;
         ptx::mbar_arrive_expect_tx(full_bar(i), Cfg::W_BYTES + Cfg::X_BYTES);
-        ptx::tma_load_2d(sw, &tmap_w, (kb0 + i) * SK_BK, tn * (MT * SK_BM), full_bar(i));
+        ptx::tma_load_2d(sw, &tmap_w, (kb0 + i) * KE, tn * (MT * SK_BM), full_bar(i));
       }
       ptx::grid_dependency_wait();
       for (int i = 0; i < pre; ++i) {
         const uint32_t sx = smem_base + i * Cfg::STAGE_BYTES + Cfg::W_BYTES;
-        ptx::tma_load_2d(sx, &tmap_x, (kb0 + i) * SK_BK, tb * BNB, full_bar(i));
+        ptx::tma_load_2d(sx, &tmap_x, (kb0 + i) * KE, tb * BNB, full_bar(i));
       }
       if (pre == STAGES) phase = 1u;  // the ring has wrapped once
       else stage = pre;
@@ -117,8 +122,8 @@ gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
         const uint32_t sw = smem_base + stage * Cfg::STAGE_BYTES;
         const uint32_t sx = sw + Cfg::W_BYTES;
         ptx::mbar_arrive_expect_tx(full_bar(stage), Cfg::W_BYTES + Cfg::X_BYTES);
-        ptx::tma_load_2d(sw, &tmap_w, kb * SK_BK, tn * (MT * SK_BM), full_bar(stage));  // box of MT * 128 rows
-        ptx::tma_load_2d(sx, &tmap_x, kb * SK_BK, tb * BNB, full_bar(stage));
+        ptx::tma_load_2d(sw, &tmap_w, kb * KE, tn * (MT * SK_BM), full_bar(stage));  // box of MT * 128 rows
+        ptx::tma_load_2d(sx, &tmap_x, kb * KE, tb * BNB, full_bar(stage));
         if (++stage == STAGES) { stage = 0; phase ^= 1u; }
       }
       if (!ok) {
@@ -127,7 +132,7 @@ gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
     }
   } else if (warp == 1) {
     if (lane == 0) {
-      constexpr uint32_t idesc = ptx::umma_idesc_bf16(SK_BM, BNB);
+      constexpr uint32_t idesc = F8 ? ptx::umma_idesc_e4m3(SK_BM, BNB) : ptx::umma_idesc_bf16(SK_BM, BNB);
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
@@ -140,9 +145,14 @@ gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
 #pragma unroll
         for (int mt = 0; mt < MT; ++mt) {
 #pragma unroll
-          for (int kk = 0; kk < SK_BK / 16; ++kk)
-            ptx::umma_bf16(tmem_base + mt * Cfg::ACC_COLS, dw + mt * (SK_BM * SK_BK * 2 / 16) + 2u * kk, dx + 2u * kk, idesc,
-                           (kb > kb0 || kk > 0) ? 1u : 0u);
+          for (int kk = 0; kk < 4; ++kk) {  // 32 bytes along K per instruction
+            const uint32_t accum = (kb > kb0 || kk > 0) ? 1u : 0u;
+            if constexpr (F8)
+              ptx::umma_f8(tmem_base + mt * Cfg::ACC_COLS, dw + mt * (SK_BM * 128 / 16) + 2u * kk, dx + 2u * kk, idesc, accum);
+            else
+              ptx::umma_bf16(tmem_base + mt * Cfg::ACC_COLS, dw + mt * (SK_BM * 128 / 16) + 2u * kk, dx + 2u * kk, idesc,
+                             accum);
+          }
         }
         ptx::umma_commit(empty_bar(stage));
         if (++stage == STAGES) { stage = 0; phase ^= 1u; }
@@ -188,10 +198,19 @@ gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
         }
         const int n4 = n - r4;  // first of this lane's four features (n is a multiple of 4 per group of lanes)
         if (n4 < p.n) {
+          float4 sw4 = make_float4(1.f, 1.f, 1.f, 1.f);
+          if constexpr (F8) sw4 = __ldg(reinterpret_cast<const float4*>(p.scale_w + n4));
 #pragma unroll
           for (int m = 0; m < CH; m += 4) {
             const int b = tb * BNB + c0 + m + r4;
             if (b < p.batch) {
+              if constexpr (F8) {
+                const float sx = __ldg(p.scale_x + b);
+                v[m] = __float_as_uint(__uint_as_float(v[m]) * (sx * sw4.x));
+                v[m + 1] = __float_as_uint(__uint_as_float(v[m + 1]) * (sx * sw4.y));
+                v[m + 2] = __float_as_uint(__uint_as_float(v[m + 2]) * (sx * sw4.z));
+                v[m + 3] = __float_as_uint(__uint_as_float(v[m + 3]) * (sx * sw4.w));
+              }
               float* dst = p.acc + static_cast<size_t>(b) * p.n + n4;
               if (p.splits > 1) ptx::red_add_v4_f32(dst, v[m], v[m + 1], v[m + 2], v[m + 3]);
               else *reinterpret_cast<uint4*>(dst) = make_uint4(v[m], v[m + 1], v[m + 2], v[m + 3]);
@@ -221,24 +240,30 @@ int skinny_splits(int units, int k_blocks, int blocks_per_sm) {
 
 int skinny_bnb(int batch) { return batch <= 16 ? 16 : batch <= 32 ? 32 : batch <= 64 ? 64 : batch <= 128 ? 128 : 256; }
 
-template <int BNB, int MT>
+template <int BNB, int MT, bool F8>
 pd_status launch_skinny(const SkinnyGemmArgs& g, cudaStream_t stream) {
   using Cfg = SkinnyCfg<BNB, MT>;
   static bool attr_set = false;
-  auto kern = gemm_skinny_kernel<BNB, MT>;
+  auto kern = gemm_skinny_kernel<BNB, MT, F8>;
   if (!attr_set) {
     PD_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES));
     attr_set = true;
   }
   CUtensorMap tw, tx;
-  PD_TRY(make_tmap_bf16(&tw, g.w, g.n, g.k, g.k, MT * SK_BM));
-  PD_TRY(make_tmap_bf16(&tx, g.x, g.batch, g.k, g.ldx, BNB));
+  if (F8) {
+    PD_TRY(make_tmap_u8(&tw, g.w, g.n, g.k, g.k, MT * SK_BM));
+    PD_TRY(make_tmap_u8(&tx, g.x, g.batch, g.k, g.ldx, BNB));
+  } else {
+    PD_TRY(make_tmap_bf16(&tw, g.w, g.n, g.k, g.k, MT * SK_BM));
+    PD_TRY(make_tmap_bf16(&tx, g.x, g.batch, g.k, g.ldx, BNB));
+  }
   SkinnyDev p{};
-  p.acc = g.acc; p.batch = g.batch; p.n = g.n; p.k_blocks = g.k / SK_BK;
+  p.scale_x = g.scale_x; p.scale_w = g.scale_w;
+  p.acc = g.acc; p.batch = g.batch; p.n = g.n; p.k_blocks = g.k / (F8 ? 2 * SK_BK : SK_BK);
   p.tiles_n = (g.n + MT * SK_BM - 1) / (MT * SK_BM);
   const int tiles_b = (g.batch + BNB - 1) / BNB;
   const int units = p.tiles_n * tiles_b;
-  const int splits = skinny_splits(units, p.k_blocks, Cfg::BLOCKS_PER_SM);
+  const int splits = skinny_splits(units, p.k_blocks, Cfg::BLOCKS_PER_SM);  // (k_blocks already counts FP8 stages)
   p.splits = splits;
   p.err_word = g.err_word;
   if (splits > 1 && !g.acc_zeroed)
@@ -409,22 +434,31 @@ __global__ void __launch_bounds__(256) skinny_swiglu_kernel(const float* __restr
 
 }  // namespace
 
-int gemm_skinny_splits(int batch, int n, int k) {
+int gemm_skinny_splits(int batch, int n, int k, bool fp8) {
   const int bnb = skinny_bnb(batch);
   const int units = ((n + SK_BM - 1) / SK_BM) * ((batch + bnb - 1) / bnb);
-  return skinny_splits(units, k / SK_BK, 2);
+  return skinny_splits(units, k / (fp8 ? 2 * SK_BK : SK_BK), 2);
 }
 
 pd_status gemm_skinny(const SkinnyGemmArgs& g, cudaStream_t stream) {
   if (!g.x || !g.w || !g.acc || g.batch <= 0 || g.n <= 0 || g.k <= 0) return PD_ERR_INVALID_ARG;
+  if (g.fp8) {
+    if (!g.scale_x || !g.scale_w) return PD_ERR_INVALID_ARG;
+    if (g.k % (2 * SK_BK) != 0 || g.n % 4 != 0 || g.ldx % 16 != 0) return PD_ERR_UNSUPPORTED_SHAPE;
+    if (g.batch <= 16) return launch_skinny<16, 1, true>(g, stream);
+    if (g.batch <= 32) return launch_skinny<32, 1, true>(g, stream);
+    if (g.batch <= 64) return launch_skinny<64, 1, true>(g, stream);
+    if (g.batch <= 128) return launch_skinny<128, 1, true>(g, stream);
+    return launch_skinny<256, 1, true>(g, stream);
+  }
   if (g.k % SK_BK != 0 || g.n % 4 != 0 || g.ldx % 8 != 0) return PD_ERR_UNSUPPORTED_SHAPE;
-  if (g.batch <= 16) return launch_skinny<16, 1>(g, stream);
-  if (g.batch <= 32) return launch_skinny<32, 1>(g, stream);
-  if (g.batch <= 64) return launch_skinny<64, 1>(g, stream);
+  if (g.batch <= 16) return launch_skinny<16, 1, false>(g, stream);
+  if (g.batch <= 32) return launch_skinny<32, 1, false>(g, stream);
+  if (g.batch <= 64) return launch_skinny<64, 1, false>(g, stream);
   // (two weight sub-tiles per block, MT = 2, measured 10-20 % slower at B = 128..256: one block per SM
   // loses the overlap of one block's epilogue with another's main loop)
-  if (g.batch <= 128) return launch_skinny<128, 1>(g, stream);
-  return launch_skinny<256, 1>(g, stream);
+  if (g.batch <= 128) return launch_skinny<128, 1, false>(g, stream);
+  return launch_skinny<256, 1, false>(g, stream);
 }
 
 pd_status launch_skinny_rope_kv(const float* acc, bf16* qkv, const RopeEpilogue& rp, int batch, int* err_word,

@@ -19,7 +19,9 @@ constexpr int kWideDecodeBatch = 257;
 
 struct Workspace {
   // byte offsets into the caller's workspace
-  size_t norm, qkv, attn_o, resid, acc_qkv, acc_o, acc_gu, acc_down, act, partial, stage_a, stage_b, meta, splitk, total;
+  size_t norm, qkv, attn_o, resid, acc_qkv, acc_o, acc_gu, acc_down, act, partial, stage_a, stage_b, meta, splitk;
+  size_t q_act, s_act;  // FP8 mode: codes and per-row scales of the activation matrix a projection is about to read
+  size_t total;
 };
 
 Workspace carve(const pd_layer_cfg& c, size_t tokens, size_t max_batch, int max_kv_len) {
@@ -52,6 +54,9 @@ Workspace carve(const pd_layer_cfg& c, size_t tokens, size_t max_batch, int max_
   w.stage_b = take(tokens * d * 2);
   w.meta = take(4096 * 4);           // staged cu_seqlens / kv_len of the host-I/O stack calls
   w.splitk = take(tokens > 256 ? pd::kSplitScratchBytes : 0);  // partial tiles of K-split GEMM tails (prefill only)
+  const size_t widest = f > hq ? (f > d ? f : d) : (hq > d ? hq : d);
+  w.q_act = take(c.fp8_projections ? tokens * widest : 0);
+  w.s_act = take(c.fp8_projections ? tokens * 4 : 0);
   w.total = off;
   return w;
 }
@@ -64,6 +69,24 @@ pd_status check_cfg(const pd_layer_cfg* c) {
   if (c->head_dim != 64 && c->head_dim != 128) return PD_ERR_UNSUPPORTED_SHAPE;
   if (c->n_q_heads % c->n_kv_heads != 0 || c->n_q_heads / c->n_kv_heads > 16) return PD_ERR_UNSUPPORTED_SHAPE;
   if (c->d_model % 64 != 0 || c->d_ff % 64 != 0 || c->d_model > 16384) return PD_ERR_UNSUPPORTED_SHAPE;
+  if (c->fp8_projections != 0 && c->fp8_projections != 1) return PD_ERR_INVALID_ARG;
+  if (c->fp8_projections && (c->d_model % 128 != 0 || c->d_ff % 128 != 0 || (c->n_q_heads * c->head_dim) % 128 != 0))
+    return PD_ERR_UNSUPPORTED_SHAPE;
+  return PD_OK;
+}
+
+// FP8 mode: quantises the rows of `a` (the matrix a projection is about to read) into the workspace and points
+// the GEMM at the codes and scales of both operands.
+pd_status use_fp8(pd_layer* L, pd::GemmArgs& g, const uint8_t* w_codes, const float* w_scales, uint8_t* ws,
+                  const Workspace& w, cudaStream_t st) {
+  uint8_t* q = ws + w.q_act;
+  float* sc = reinterpret_cast<float*>(ws + w.s_act);
+  PD_TRY(pd::launch_quantize_rows_fp8(g.a, g.lda, g.m, g.k, q, g.k, sc, st));
+  g.a = reinterpret_cast<const bf16*>(q);
+  g.lda = g.k;
+  g.b = reinterpret_cast<const bf16*>(w_codes);
+  g.fp8 = 1; g.scale_a = sc; g.scale_b = w_scales;
+  (void)L;
   return PD_OK;
 }
 
@@ -93,13 +116,21 @@ pd_status mlp_half(pd_layer* L, const bf16* h, bf16* out, int tokens, uint8_t* w
   pd::GemmArgs g{};
   g.a = norm; g.b = L->w_gu; g.c = act; g.m = tokens; g.n = 2 * c.d_ff; g.k = c.d_model;
   g.lda = c.d_model; g.ldb = c.d_model; g.ldc = c.d_ff; g.epilogue = pd::EPI_SWIGLU; g.err_word = L->err_word;
-  { pd::TraceScope ts(PD_K_GEMM_GATE_UP, st); PD_TRY(pd::gemm(g, st)); }
+  {
+    pd::TraceScope ts(PD_K_GEMM_GATE_UP, st);
+    if (c.fp8_projections) PD_TRY(use_fp8(L, g, L->q_gu, L->s_gu, ws, w, st));
+    PD_TRY(pd::gemm(g, st));
+  }
   pd::GemmArgs g2{};
   g2.a = act; g2.b = L->w_down; g2.c = out; g2.r = h; g2.m = tokens; g2.n = c.d_model; g2.k = c.d_ff;
   g2.lda = c.d_ff; g2.ldb = c.d_ff; g2.ldc = c.d_model; g2.ldr = c.d_model; g2.epilogue = pd::EPI_RESIDUAL;
   g2.err_word = L->err_word;
   enable_tail_split(L, g2, ws, w, tokens);
-  { pd::TraceScope ts(PD_K_GEMM_DOWN, st); PD_TRY(pd::gemm(g2, st)); }
+  {
+    pd::TraceScope ts(PD_K_GEMM_DOWN, st);
+    if (c.fp8_projections) PD_TRY(use_fp8(L, g2, L->q_down, L->s_down, ws, w, st));
+    PD_TRY(pd::gemm(g2, st));
+  }
   return PD_OK;
 }
 
@@ -115,7 +146,11 @@ pd_status qkv_half(pd_layer* L, const bf16* x, int tokens, const pd::RopeEpilogu
   g.lda = c.d_model; g.ldb = c.d_model; g.ldc = L->n_qkv; g.epilogue = pd::EPI_ROPE_KV; g.rope = &rope;
   g.err_word = L->err_word;
   enable_tail_split(L, g, ws, w, tokens);
-  { pd::TraceScope ts(PD_K_GEMM_QKV, st); PD_TRY(pd::gemm(g, st)); }
+  {
+    pd::TraceScope ts(PD_K_GEMM_QKV, st);
+    if (c.fp8_projections) PD_TRY(use_fp8(L, g, L->q_qkv, L->s_qkv, ws, w, st));
+    PD_TRY(pd::gemm(g, st));
+  }
   return PD_OK;
 }
 
@@ -128,6 +163,7 @@ pd_status oproj(pd_layer* L, const bf16* x, int tokens, uint8_t* ws, const Works
   g.epilogue = pd::EPI_RESIDUAL; g.err_word = L->err_word;
   enable_tail_split(L, g, ws, w, tokens);
   pd::TraceScope ts(PD_K_GEMM_O, st);
+  if (c.fp8_projections) PD_TRY(use_fp8(L, g, L->q_o, L->s_o, ws, w, st));
   return pd::gemm(g, st);
 }
 
@@ -223,10 +259,22 @@ pd_status decode_impl(pd_layer* L, const bf16* x, bf16* out, const int32_t* kv_l
   // only where it first needs it).  A K-split projection adds into its fp32 buffer; that buffer is cleared
   // by a row-wise kernel two or more launches earlier, never by a memset between the kernels.
   const int n_gu = 2 * c.d_ff;
-  float* z_qkv = pd::gemm_skinny_splits(B, L->n_qkv, c.d_model) > 1 ? acc_qkv : nullptr;
-  float* z_o = pd::gemm_skinny_splits(B, c.d_model, hq) > 1 ? acc_o : nullptr;
-  float* z_gu = pd::gemm_skinny_splits(B, n_gu, c.d_model) > 1 ? acc_gu : nullptr;
-  float* z_down = pd::gemm_skinny_splits(B, c.d_model, c.d_ff) > 1 ? acc_down : nullptr;
+  const bool f8 = c.fp8_projections != 0;
+  float* z_qkv = pd::gemm_skinny_splits(B, L->n_qkv, c.d_model, f8) > 1 ? acc_qkv : nullptr;
+  float* z_o = pd::gemm_skinny_splits(B, c.d_model, hq, f8) > 1 ? acc_o : nullptr;
+  float* z_gu = pd::gemm_skinny_splits(B, n_gu, c.d_model, f8) > 1 ? acc_gu : nullptr;
+  float* z_down = pd::gemm_skinny_splits(B, c.d_model, c.d_ff, f8) > 1 ? acc_down : nullptr;
+  // FP8 mode: a row-wise quantiser in front of every projection (same programmatic-serialization chain)
+  uint8_t* q_act = ws + w.q_act;
+  float* s_act = reinterpret_cast<float*>(ws + w.s_act);
+  auto fp8_in = [&](pd::SkinnyGemmArgs& a, const uint8_t* w_codes, const float* w_scales) -> pd_status {
+    if (!f8) return PD_OK;
+    PD_TRY(pd::launch_quantize_rows_fp8(a.x, a.ldx, B, a.k, q_act, a.k, s_act, st));
+    a.x = reinterpret_cast<const bf16*>(q_act); a.ldx = a.k;
+    a.w = reinterpret_cast<const bf16*>(w_codes);
+    a.fp8 = 1; a.scale_x = s_act; a.scale_w = w_scales;
+    return PD_OK;
+  };
 
   {
     pd::TraceScope ts(PD_K_RMSNORM, st);
@@ -237,6 +285,7 @@ pd_status decode_impl(pd_layer* L, const bf16* x, bf16* out, const int32_t* kv_l
   {
     pd::TraceScope ts(PD_K_GEMM_QKV, st);
     g.x = norm; g.w = L->w_qkv; g.acc = acc_qkv; g.n = L->n_qkv; g.k = c.d_model; g.ldx = c.d_model;
+    PD_TRY(fp8_in(g, L->q_qkv, L->s_qkv));
     PD_TRY(pd::gemm_skinny(g, st));
     PD_TRY(pd::launch_skinny_rope_kv(acc_qkv, qkv, r, B, L->err_word, z_o, c.d_model, st));
   }
@@ -251,18 +300,21 @@ pd_status decode_impl(pd_layer* L, const bf16* x, bf16* out, const int32_t* kv_l
   {
     pd::TraceScope ts(PD_K_GEMM_O, st);  // h = x + o W_o^T and n2 = RMSNorm(h) in the same row-wise pass
     g.x = attn_o; g.w = L->w_o; g.acc = acc_o; g.n = c.d_model; g.k = hq; g.ldx = hq;
+    PD_TRY(fp8_in(g, L->q_o, L->s_o));
     PD_TRY(pd::gemm_skinny(g, st));
     PD_TRY(pd::launch_skinny_residual(acc_o, x, resid, L->g_mlp, norm, B, c.d_model, c.rms_eps, z_gu, n_gu, st));
   }
   {
     pd::TraceScope ts(PD_K_GEMM_GATE_UP, st);
     g.x = norm; g.w = L->w_gu; g.acc = acc_gu; g.n = n_gu; g.k = c.d_model; g.ldx = c.d_model;
+    PD_TRY(fp8_in(g, L->q_gu, L->s_gu));
     PD_TRY(pd::gemm_skinny(g, st));
     PD_TRY(pd::launch_skinny_swiglu(acc_gu, act, B, c.d_ff, z_down, c.d_model, st));
   }
   {
     pd::TraceScope ts(PD_K_GEMM_DOWN, st);
     g.x = act; g.w = L->w_down; g.acc = acc_down; g.n = c.d_model; g.k = c.d_ff; g.ldx = c.d_ff;
+    PD_TRY(fp8_in(g, L->q_down, L->s_down));
     PD_TRY(pd::gemm_skinny(g, st));
     PD_TRY(pd::launch_skinny_residual(acc_down, resid, out, nullptr, nullptr, B, c.d_model, c.rms_eps, nullptr, 0, st));
   }
@@ -277,6 +329,14 @@ extern "C" pd_status pd_workspace_bytes(const pd_layer_cfg* cfg, int32_t max_tok
   if (!out_bytes || max_tokens < 0 || max_batch < 0 || max_kv_len < 0) return PD_ERR_INVALID_ARG;
   const size_t tokens = static_cast<size_t>(max_tokens > max_batch ? max_tokens : max_batch);
   *out_bytes = carve(*cfg, tokens, static_cast<size_t>(max_batch), max_kv_len).total;
+  return PD_OK;
+}
+
+extern "C" pd_status pd_workspace_offsets(const pd_layer_cfg* cfg, int32_t tokens, pd_workspace_layout* out) {
+  PD_TRY(check_cfg(cfg));
+  if (!out || out->struct_size != sizeof(pd_workspace_layout) || tokens < 0) return PD_ERR_INVALID_ARG;
+  const Workspace w = carve(*cfg, static_cast<size_t>(tokens), 0, 0);  // these five do not depend on the decode sizes
+  out->norm = w.norm; out->qkv = w.qkv; out->attn_o = w.attn_o; out->resid = w.resid; out->act = w.act;
   return PD_OK;
 }
 
@@ -327,6 +387,23 @@ extern "C" pd_status pd_layer_create(const pd_layer_cfg* cfg, const pd_layer_wei
   if ((e = cudaMemcpyAsync(L->g_mlp, w->g_mlp, d * 2, d2d, st)) != cudaSuccess) return fail(e);
   if ((e = cudaMemsetAsync(L->err_word, 0, sizeof(int), st)) != cudaSuccess) return fail(e);
 
+  if (cfg->fp8_projections) {
+    // per-output-channel E4M3 codes and scales of the four (repacked) matrices; the bf16 copies are then released
+    struct Q { bf16** src; uint8_t** codes; float** scales; size_t rows, k; } qs[4] = {
+        {&L->w_qkv, &L->q_qkv, &L->s_qkv, static_cast<size_t>(L->n_qkv), d}, {&L->w_o, &L->q_o, &L->s_o, d, hq},
+        {&L->w_gu, &L->q_gu, &L->s_gu, 2 * f, d}, {&L->w_down, &L->q_down, &L->s_down, d, f}};
+    for (auto& q : qs) {
+      if ((e = cudaMalloc(q.codes, q.rows * q.k)) != cudaSuccess) return fail(e);
+      if ((e = cudaMalloc(q.scales, q.rows * sizeof(float))) != cudaSuccess) return fail(e);
+      const pd_status qs_st = pd::launch_quantize_rows_fp8(*q.src, static_cast<int>(q.k), static_cast<int>(q.rows),
+                                                           static_cast<int>(q.k), *q.codes, static_cast<int>(q.k),
+                                                           *q.scales, st);
+      if (qs_st != PD_OK) { pd_layer_destroy(L); return qs_st; }
+    }
+    if ((e = cudaStreamSynchronize(st)) != cudaSuccess) return fail(e);
+    for (auto& q : qs) { cudaFree(*q.src); *q.src = nullptr; }
+  }
+
   // RoPE table in double on the host: (cos, sin)(pos * theta^(-2i/hd))
   std::vector<float2> tab(static_cast<size_t>(cfg->max_pos) * half);
   std::vector<double> inv_freq(half);
@@ -347,6 +424,8 @@ extern "C" pd_status pd_layer_create(const pd_layer_cfg* cfg, const pd_layer_wei
 extern "C" pd_status pd_layer_destroy(pd_layer* L) {
   if (!L) return PD_OK;
   cudaFree(L->w_qkv); cudaFree(L->w_o); cudaFree(L->w_gu); cudaFree(L->w_down);
+  cudaFree(L->q_qkv); cudaFree(L->q_o); cudaFree(L->q_gu); cudaFree(L->q_down);
+  cudaFree(L->s_qkv); cudaFree(L->s_o); cudaFree(L->s_gu); cudaFree(L->s_down);
   cudaFree(L->g_attn); cudaFree(L->g_mlp); cudaFree(L->rope_tab); cudaFree(L->err_word); cudaFree(L->split_flags);
   delete L;
   return PD_OK;

@@ -27,7 +27,8 @@ def test_library_exports_every_declared_symbol(pdlib):
 
 def test_struct_sizes_match_c_layout(pdlib):
     # natural C layout: checked against hand-computed sizes of include/pd.h
-    assert ctypes.sizeof(pdlib.pd_layer_cfg) == 36
+    assert ctypes.sizeof(pdlib.pd_layer_cfg) == 40
+    assert ctypes.sizeof(pdlib.pd_workspace_layout) == 8 + 5 * 8
     assert ctypes.sizeof(pdlib.pd_layer_weights) == 8 + 7 * 8
     assert ctypes.sizeof(pdlib.pd_kv_cache) == 32
     assert ctypes.sizeof(pdlib.pd_alloc_in) == 8 + 7 * 8 + 8 + 16
