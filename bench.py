@@ -176,6 +176,7 @@ def main():
     ap.add_argument("--skip-sweep", action="store_true",
                     help="profiling aid: skip the TPOT(B) sweep and decode at the largest batch")
     ap.add_argument("--no-graphs", action="store_true", help="launch the layer stacks eagerly instead of replaying CUDA graphs")
+    ap.add_argument("--no-fp8", action="store_true", help="skip the FP8-projection section")
     ap.add_argument("--decode-batch", type=int, default=0,
                     help="profiling aid: decode at this batch instead of the TPOT-feasible one")
     args = ap.parse_args()
@@ -474,6 +475,53 @@ def main():
                    "note": "graph replay of pd_model_prefill / pd_model_decode_step; head = embedding + LM head + "
                            "sampler kernels by CUDA events in a traced pass"}
 
+    # ---- the same stack with FP8 (E4M3) projections: a separate precision, reported beside the bf16 headline
+    fp8_out = None
+    if not args.no_fp8:
+        del model, mws
+        cfg8 = pd.LayerConfig(**SHAPE, max_pos=max(L_IN, KV_START + L_OUT), fp8_projections=True)
+        layers8 = []
+        for _ in range(n_layers):
+            w = {"w_qkv": randn_bf16(nqkv, d, std=0.02), "w_o": randn_bf16(d, SHAPE["n_q_heads"] * SHAPE["head_dim"], std=0.02),
+                 "w_gate": randn_bf16(SHAPE["d_ff"], d, std=0.02), "w_up": randn_bf16(SHAPE["d_ff"], d, std=0.02),
+                 "w_down": randn_bf16(d, SHAPE["d_ff"], std=0.02), "g_attn": randn_bf16(d, std=0.02, mean=1.0),
+                 "g_mlp": randn_bf16(d, std=0.02, mean=1.0)}
+            layers8.append(pd.Layer(cfg8, w))
+            torch.cuda.synchronize()
+            del w
+        ws8_bytes = pd.pd_workspace_bytes(cfg8, L_IN, b_max, cap)
+        ws8 = torch.empty(ws8_bytes, dtype=torch.uint8, device=dev)
+
+        def prefill8():
+            pd.pd_prefill_stack(layers8, pre_caches, x_pre, y_pre, False, cu_dev, cu_host, ws8, ws8_bytes)
+
+        def decode8(batch):
+            pd.pd_decode_stack(layers8, dec_caches, x_dec, y_dec, False, kv_lens[t_mid], batch, KV_START + t_mid + 1,
+                               ws8, ws8_bytes)
+
+        pre8_s = timed(runner("prefill_fp8", prefill8)[0], reps=5) * scale
+        dec8 = {}
+        for b in sorted({1, 64, b_star}):
+            dec8[b] = timed(runner(("decode_fp8", b), lambda b=b: decode8(b))[0], reps=5) * scale
+        pd.pd_layer_check(layers8[0])
+        pd.pd_trace_begin()
+        prefill8()
+        tr8 = pd.pd_trace_end()
+        gemm8_s = sum(tr8[k][0] for k in ("gemm_qkv", "gemm_o", "gemm_gate_up", "gemm_down"))
+        (pre8_s,) = max_over_ranks([pre8_s], dist, dev)
+        peak8 = 2.0 * peaks["bf16_tflops"]      # dense FP8 runs at twice the bf16 rate (nominal ratio x measured bf16 burst)
+        fp8_out = {"prefill_tok_s": world * L_IN / pre8_s, "prefill_ms_per_pass": pre8_s * 1e3,
+                   "prefill_tflops": flops_all * scale / pre8_s / 1e12,
+                   "gemm_tflops_incl_quantisers": flops_gemm / gemm8_s / 1e12,
+                   "gemm_frac_of_fp8_peak": flops_gemm / gemm8_s / 1e12 / peak8, "fp8_peak_tflops": peak8,
+                   "peak_source": "2 x measured bf16 burst (nominal FP8 : bf16 ratio)",
+                   "tpot_ms": {str(b): v * 1e3 for b, v in dec8.items()},
+                   "decode_tok_s": world * b_star / dec8[b_star],
+                   "kernel_time_ms_prefill": {k: v[0] * 1e3 for k, v in tr8.items() if v[1]},
+                   "note": "E4M3 weights per output channel, activations per token; attention, norms, residual stream "
+                           "and KV cache stay bf16; not part of `value`"}
+        del layers8, ws8
+
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         sample_l = L_IN
@@ -524,6 +572,7 @@ def main():
                     "d2h_bytes_per_step": yh.numel() * 2,
                     "decode_tok_s": world * b_star / (statistics.mean(e2e_dec) * scale)},
             "whole_model": whole_model,
+            "fp8_projections": fp8_out,
             "gpu_launches": launches, "clocks": clocks, "wall_s_timed_region": t_wall,
         }
         if cpu:
