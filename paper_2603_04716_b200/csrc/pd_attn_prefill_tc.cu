@@ -222,7 +222,6 @@ prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
       // raw scores stay in registers; the scale is folded into the exponent (scale > 0, so the
       // maximum can be taken on the raw values)
       const bool need_mask = (k0 + TK - 1 > pre + q0 + t * TQ) || (k0 + TK > kv_end);  // warp-uniform
-      float mx = -CUDART_INF_F;
       if (need_mask) {
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
@@ -230,16 +229,19 @@ prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
           for (int e = 0; e < 32; ++e) {
             const int key = k0 + c * 32 + e;
             if (key > row_pos || key >= kv_end) sv[c][e] = 0xff800000u;  // -inf
-            mx = fmaxf(mx, __uint_as_float(sv[c][e]));
           }
         }
-      } else {
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-#pragma unroll
-          for (int e = 0; e < 32; ++e) mx = fmaxf(mx, __uint_as_float(sv[c][e]));
-        }
       }
+      // row maximum: four independent chains of three-input maxima (the softmax warps set the pace of the
+      // kernel, so their instruction count and dependency depth are what is being minimised here)
+      float mx4[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F};
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+#pragma unroll
+        for (int e = 0; e < 32; e += 2)
+          mx4[(e >> 1) & 3] = ptx::fmax3(mx4[(e >> 1) & 3], __uint_as_float(sv[c][e]), __uint_as_float(sv[c][e + 1]));
+      }
+      float mx = ptx::fmax3(fmaxf(mx4[0], mx4[1]), mx4[2], mx4[3]);
       mx *= sl2;
       // lazy maximum: keep the old reference unless this tile exceeds it by more than the threshold
       float factor = 1.f;
@@ -268,8 +270,13 @@ prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
         ptx::tmem_st_wait();
         l_sum *= factor;
       }
-      float psum0 = 0.f, psum1 = 0.f;
-      const float neg_m = -m_used;
+      // p = 2^(s * scale - m) for a pair of keys at a time: one packed FMA, two exponentials, one packed add.
+      // (Evaluating a share of the exponentials with a polynomial on the FMA pipe was measured slower, 300 us
+      // against 199 us at L_in 4096: the two row tiles alternate, so a scheduler mostly runs one softmax warp at
+      // a time and the polynomial's dependent chain is exposed.)
+      const uint64_t sl2_2 = ptx::pack_f32x2(sl2, sl2);
+      const uint64_t negm_2 = ptx::pack_f32x2(-m_used, -m_used);
+      uint64_t ps[4] = {0ull, 0ull, 0ull, 0ull};
 #pragma unroll
       for (int c = 0; c < 2; ++c) {
         uint32_t pk[32];
@@ -277,15 +284,21 @@ prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
         for (int e = 0; e < 32; ++e) {
           // packed column 32 c + e holds keys 2 (32 c + e) and 2 (32 c + e) + 1
           const int k_lo = (c * 32 + e) * 2;
-          const float p0 = ptx::ex2_approx(fmaf(__uint_as_float(sv[k_lo >> 5][k_lo & 31]), sl2, neg_m));
-          const float p1 = ptx::ex2_approx(fmaf(__uint_as_float(sv[(k_lo + 1) >> 5][(k_lo + 1) & 31]), sl2, neg_m));
-          psum0 += p0;
-          psum1 += p1;
+          const uint64_t x2 = ptx::pack_f32x2(__uint_as_float(sv[k_lo >> 5][k_lo & 31]),
+                                              __uint_as_float(sv[k_lo >> 5][(k_lo & 31) + 1]));
+          float y0, y1;
+          ptx::unpack_f32x2(ptx::fma_f32x2(x2, sl2_2, negm_2), y0, y1);
+          const float p0 = ptx::ex2_approx(y0), p1 = ptx::ex2_approx(y1);
+          ps[e & 3] = ptx::add_f32x2(ps[e & 3], ptx::pack_f32x2(p0, p1));
           pk[e] = ptx::pack_bf16(p0, p1);
         }
         ptx::tmem_st_32x32(t_lane + Cfg::S_COL + c * 32, pk);
       }
-      l_sum += psum0 + psum1;
+      {
+        float a0, a1;
+        ptx::unpack_f32x2(ptx::add_f32x2(ptx::add_f32x2(ps[0], ps[1]), ptx::add_f32x2(ps[2], ps[3])), a0, a1);
+        l_sum += a0 + a1;
+      }
       ptx::tmem_st_wait();
       // the request's last tile may reach past its end: zero those V rows (0 * garbage must stay 0)
       if (k0 + TK > kv_total) {
