@@ -144,9 +144,10 @@ int gemm_skinny_splits(int batch, int n, int k, bool fp8 = false);
 // skip): the buffer is idle while the kernel runs, and the projection then needs no memset of its own.
 pd_status launch_skinny_rope_kv(const float* acc, bf16* qkv, const RopeEpilogue& rp, int batch, int* err_word,
                                 float* zero_ptr, int zero_cols, cudaStream_t s);
-// h = x + acc; if n != NULL also n = RMSNorm(h) * gain.
+// h = x + acc; if n != NULL also n = RMSNorm(h) * gain (and, with q_out / s_out, the E4M3 codes and scales of n).
 pd_status launch_skinny_residual(const float* acc, const bf16* x, bf16* h, const bf16* gain, bf16* n, int batch, int d,
-                                 float eps, float* zero_ptr, int zero_cols, cudaStream_t s);
+                                 float eps, float* zero_ptr, int zero_cols, cudaStream_t s, uint8_t* q_out = nullptr,
+                                 float* s_out = nullptr);
 // out[B, F] = silu(gate) * up from acc[B, 2F] whose columns follow the 64/64 interleaved weight rows.
 pd_status launch_skinny_swiglu(const float* acc, bf16* out, int batch, int f, float* zero_ptr, int zero_cols,
                                cudaStream_t s);
@@ -159,11 +160,14 @@ pd_status model_head(pd_model* m, const bf16* h, const int32_t* cu_dev, int rows
                      float* logits, int32_t* next_dev, cudaStream_t st);
 
 // ------------------------------------------------------------ elementwise
-pd_status launch_rmsnorm(const bf16* x, const bf16* gain, bf16* y, int rows, int d, float eps, cudaStream_t s);
+// q_out / s_out (both or neither): also emit the E4M3 codes [rows, d] and per-row scales of the stored result,
+// identical to running launch_quantize_rows_fp8 on y.
+pd_status launch_rmsnorm(const bf16* x, const bf16* gain, bf16* y, int rows, int d, float eps, cudaStream_t s,
+                         uint8_t* q_out = nullptr, float* s_out = nullptr);
 // The same as the first kernel of a decode layer: launched with programmatic serialization, and clears
 // zero_ptr[rows, zero_cols] (fp32, NULL to skip) for a later projection.
 pd_status launch_rmsnorm_decode(const bf16* x, const bf16* gain, bf16* y, int rows, int d, float eps, float* zero_ptr,
-                                int zero_cols, cudaStream_t s);
+                                int zero_cols, cudaStream_t s, uint8_t* q_out = nullptr, float* s_out = nullptr);
 
 // -------------------------------------------------------------- attention
 struct PrefillAttnArgs {

@@ -70,9 +70,12 @@ __global__ void __launch_bounds__(QNT_THREADS) quantize_rows_fp8_kernel(const bf
 constexpr int RMS_THREADS = 256;
 constexpr int RMS_MAX_CHUNKS = 8;  // 8 chunks * 8 elements * 256 threads = d up to 16384
 
+// With q_out != NULL the row is also quantised to E4M3 exactly as quantize_rows_fp8_kernel would quantise the
+// stored bf16 row (the maximum and the quotients are taken on the bf16-rounded values).
 __global__ void __launch_bounds__(RMS_THREADS) rmsnorm_kernel(const bf16* __restrict__ x,
                                                                const bf16* __restrict__ gain, bf16* __restrict__ y,
-                                                               int d, float eps, float* zero_ptr, int zero_cols) {
+                                                               int d, float eps, float* zero_ptr, int zero_cols,
+                                                               uint8_t* __restrict__ q_out, float* __restrict__ s_out) {
   const int row = blockIdx.x;
   ptx::grid_launch_dependents();
   ptx::grid_dependency_wait();
@@ -106,6 +109,7 @@ __global__ void __launch_bounds__(RMS_THREADS) rmsnorm_kernel(const bf16* __rest
 #pragma unroll
   for (int w = 0; w < RMS_THREADS / 32; ++w) tot += red[w];
   const float scale = rsqrtf(tot / static_cast<float>(d) + eps);
+  float amax = 0.f;
 #pragma unroll
   for (int i = 0; i < RMS_MAX_CHUNKS; ++i) {
     const int c = threadIdx.x + i * RMS_THREADS;
@@ -115,7 +119,40 @@ __global__ void __launch_bounds__(RMS_THREADS) rmsnorm_kernel(const bf16* __rest
       unpack8(gr[c], g);
 #pragma unroll
       for (int e = 0; e < 8; ++e) f[e] = f[e] * scale * g[e];
-      yr[c] = pack8(f);
+      v[i] = pack8(f);
+      yr[c] = v[i];
+      if (q_out) {
+        unpack8(v[i], f);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) amax = fmaxf(amax, fabsf(f[e]));
+      }
+    }
+  }
+  if (q_out) {  // block-uniform
+    __syncthreads();  // everyone has read red[]
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = amax;
+    __syncthreads();
+    float mx = 0.f;
+#pragma unroll
+    for (int w = 0; w < RMS_THREADS / 32; ++w) mx = fmaxf(mx, red[w]);
+    const float qs = mx > 0.f ? __fdiv_rn(mx, 448.f) : 1.f;
+    if (threadIdx.x == 0) s_out[row] = qs;
+    uint2* qr = reinterpret_cast<uint2*>(q_out + static_cast<size_t>(row) * d);
+#pragma unroll
+    for (int i = 0; i < RMS_MAX_CHUNKS; ++i) {
+      const int c = threadIdx.x + i * RMS_THREADS;
+      if (c < chunks) {
+        float f[8];
+        unpack8(v[i], f);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) f[e] = __fdiv_rn(f[e], qs);
+        uint2 o;
+        o.x = ptx::cvt_e4m3x2(f[0], f[1]) | (ptx::cvt_e4m3x2(f[2], f[3]) << 16);
+        o.y = ptx::cvt_e4m3x2(f[4], f[5]) | (ptx::cvt_e4m3x2(f[6], f[7]) << 16);
+        qr[c] = o;
+      }
     }
   }
 }
@@ -146,20 +183,23 @@ __global__ void __launch_bounds__(256) fill_normal_kernel(bf16* dst, size_t n, u
 
 }  // namespace
 
-pd_status launch_rmsnorm(const bf16* x, const bf16* gain, bf16* y, int rows, int d, float eps, cudaStream_t s) {
+pd_status launch_rmsnorm(const bf16* x, const bf16* gain, bf16* y, int rows, int d, float eps, cudaStream_t s,
+                         uint8_t* q_out, float* s_out) {
   if (rows == 0) return PD_OK;
-  if (d % 8 != 0 || d > RMS_THREADS * RMS_MAX_CHUNKS * 8) return PD_ERR_UNSUPPORTED_SHAPE;
-  rmsnorm_kernel<<<rows, RMS_THREADS, 0, s>>>(x, gain, y, d, eps, nullptr, 0);
+  if (d % 8 != 0 || d > RMS_THREADS * RMS_MAX_CHUNKS * 8 || (q_out && !s_out)) return PD_ERR_UNSUPPORTED_SHAPE;
+  rmsnorm_kernel<<<rows, RMS_THREADS, 0, s>>>(x, gain, y, d, eps, nullptr, 0, q_out, s_out);
   count_launch();
   PD_CUDA_TRY(cudaGetLastError());
   return PD_OK;
 }
 
 pd_status launch_rmsnorm_decode(const bf16* x, const bf16* gain, bf16* y, int rows, int d, float eps, float* zero_ptr,
-                                int zero_cols, cudaStream_t s) {
+                                int zero_cols, cudaStream_t s, uint8_t* q_out, float* s_out) {
   if (rows == 0) return PD_OK;
-  if (d % 8 != 0 || d > RMS_THREADS * RMS_MAX_CHUNKS * 8 || (zero_ptr && zero_cols % 4 != 0)) return PD_ERR_UNSUPPORTED_SHAPE;
-  PD_CUDA_TRY(launch_pdl(rmsnorm_kernel, dim3(rows), dim3(RMS_THREADS), 0, s, x, gain, y, d, eps, zero_ptr, zero_cols));
+  if (d % 8 != 0 || d > RMS_THREADS * RMS_MAX_CHUNKS * 8 || (zero_ptr && zero_cols % 4 != 0) || (q_out && !s_out))
+    return PD_ERR_UNSUPPORTED_SHAPE;
+  PD_CUDA_TRY(launch_pdl(rmsnorm_kernel, dim3(rows), dim3(RMS_THREADS), 0, s, x, gain, y, d, eps, zero_ptr, zero_cols,
+                         q_out, s_out));
   count_launch();
   return PD_OK;
 }

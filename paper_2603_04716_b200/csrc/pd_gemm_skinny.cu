@@ -352,7 +352,9 @@ template <bool NORM>
 __global__ void __launch_bounds__(RES_THREADS) skinny_residual_kernel(const float* __restrict__ acc,
                                                                        const bf16* __restrict__ x, bf16* h,
                                                                        const bf16* __restrict__ gain, bf16* n, int d,
-                                                                       float eps, float* zero_ptr, int zero_cols) {
+                                                                       float eps, float* zero_ptr, int zero_cols,
+                                                                       uint8_t* __restrict__ q_out,
+                                                                       float* __restrict__ s_out) {
   const int b = blockIdx.x;
   const int chunks = d / 8;
   ptx::grid_launch_dependents();
@@ -388,6 +390,7 @@ __global__ void __launch_bounds__(RES_THREADS) skinny_residual_kernel(const floa
 #pragma unroll
   for (int w = 0; w < RES_THREADS / 32; ++w) tot += red[w];
   const float scale = rsqrtf(tot / static_cast<float>(d) + eps);
+  float amax = 0.f;
 #pragma unroll
   for (int i = 0; i < RES_MAX_CHUNKS; ++i) {
     const int c = threadIdx.x + i * RES_THREADS;
@@ -397,7 +400,39 @@ __global__ void __launch_bounds__(RES_THREADS) skinny_residual_kernel(const floa
       unpack8(reinterpret_cast<const uint4*>(gain)[c], g);
 #pragma unroll
       for (int e = 0; e < 8; ++e) f[e] = f[e] * scale * g[e];
-      *reinterpret_cast<uint4*>(n + static_cast<size_t>(b) * d + c * 8) = pack8(f);
+      hv[i] = pack8(f);
+      *reinterpret_cast<uint4*>(n + static_cast<size_t>(b) * d + c * 8) = hv[i];
+      if (q_out) {
+        unpack8(hv[i], f);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) amax = fmaxf(amax, fabsf(f[e]));
+      }
+    }
+  }
+  if (q_out) {  // block-uniform: E4M3 codes and scale of the stored n, as the row quantiser would produce them
+    __syncthreads();
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = amax;
+    __syncthreads();
+    float mx = 0.f;
+#pragma unroll
+    for (int w = 0; w < RES_THREADS / 32; ++w) mx = fmaxf(mx, red[w]);
+    const float qs = mx > 0.f ? __fdiv_rn(mx, 448.f) : 1.f;
+    if (threadIdx.x == 0) s_out[b] = qs;
+#pragma unroll
+    for (int i = 0; i < RES_MAX_CHUNKS; ++i) {
+      const int c = threadIdx.x + i * RES_THREADS;
+      if (c < chunks) {
+        float f[8];
+        unpack8(hv[i], f);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) f[e] = __fdiv_rn(f[e], qs);
+        uint2 o;
+        o.x = ptx::cvt_e4m3x2(f[0], f[1]) | (ptx::cvt_e4m3x2(f[2], f[3]) << 16);
+        o.y = ptx::cvt_e4m3x2(f[4], f[5]) | (ptx::cvt_e4m3x2(f[6], f[7]) << 16);
+        *reinterpret_cast<uint2*>(q_out + static_cast<size_t>(b) * d + c * 8) = o;
+      }
     }
   }
   }  // NORM
@@ -470,17 +505,17 @@ pd_status launch_skinny_rope_kv(const float* acc, bf16* qkv, const RopeEpilogue&
 }
 
 pd_status launch_skinny_residual(const float* acc, const bf16* x, bf16* h, const bf16* gain, bf16* n, int batch, int d,
-                                 float eps, float* zero_ptr, int zero_cols, cudaStream_t s) {
-  if (d % 8 != 0 || d > RES_THREADS * RES_MAX_CHUNKS * 8) return PD_ERR_UNSUPPORTED_SHAPE;
+                                 float eps, float* zero_ptr, int zero_cols, cudaStream_t s, uint8_t* q_out, float* s_out) {
+  if (d % 8 != 0 || d > RES_THREADS * RES_MAX_CHUNKS * 8 || (q_out && (!s_out || !n))) return PD_ERR_UNSUPPORTED_SHAPE;
   if (zero_ptr && zero_cols % 4 != 0) return PD_ERR_UNSUPPORTED_SHAPE;
   const bf16* no_gain = nullptr;
   bf16* no_out = nullptr;
   if (n)
     PD_CUDA_TRY(launch_pdl(skinny_residual_kernel<true>, dim3(batch), dim3(RES_THREADS), 0, s, acc, x, h, gain, n, d, eps,
-                           zero_ptr, zero_cols));
+                           zero_ptr, zero_cols, q_out, s_out));
   else
     PD_CUDA_TRY(launch_pdl(skinny_residual_kernel<false>, dim3(batch), dim3(RES_THREADS), 0, s, acc, x, h, no_gain, no_out,
-                           d, eps, zero_ptr, zero_cols));
+                           d, eps, zero_ptr, zero_cols, q_out, s_out));
   count_launch();
   return PD_OK;
 }

@@ -77,11 +77,12 @@ pd_status check_cfg(const pd_layer_cfg* c) {
 
 // FP8 mode: quantises the rows of `a` (the matrix a projection is about to read) into the workspace and points
 // the GEMM at the codes and scales of both operands.
+// (`quantised`: the producer of `a` has already left its codes and scales there.)
 pd_status use_fp8(pd_layer* L, pd::GemmArgs& g, const uint8_t* w_codes, const float* w_scales, uint8_t* ws,
-                  const Workspace& w, cudaStream_t st) {
+                  const Workspace& w, cudaStream_t st, bool quantised = false) {
   uint8_t* q = ws + w.q_act;
   float* sc = reinterpret_cast<float*>(ws + w.s_act);
-  PD_TRY(pd::launch_quantize_rows_fp8(g.a, g.lda, g.m, g.k, q, g.k, sc, st));
+  if (!quantised) PD_TRY(pd::launch_quantize_rows_fp8(g.a, g.lda, g.m, g.k, q, g.k, sc, st));
   g.a = reinterpret_cast<const bf16*>(q);
   g.lda = g.k;
   g.b = reinterpret_cast<const bf16*>(w_codes);
@@ -112,13 +113,18 @@ pd_status mlp_half(pd_layer* L, const bf16* h, bf16* out, int tokens, uint8_t* w
   const pd_layer_cfg& c = L->cfg;
   bf16* norm = reinterpret_cast<bf16*>(ws + w.norm);
   bf16* act = reinterpret_cast<bf16*>(ws + w.act);
-  { pd::TraceScope ts(PD_K_RMSNORM, st); PD_TRY(pd::launch_rmsnorm(h, L->g_mlp, norm, tokens, c.d_model, c.rms_eps, st)); }
+  const bool f8 = c.fp8_projections != 0;  // the norm then also emits the codes and scales the projection reads
+  {
+    pd::TraceScope ts(PD_K_RMSNORM, st);
+    PD_TRY(pd::launch_rmsnorm(h, L->g_mlp, norm, tokens, c.d_model, c.rms_eps, st, f8 ? ws + w.q_act : nullptr,
+                              f8 ? reinterpret_cast<float*>(ws + w.s_act) : nullptr));
+  }
   pd::GemmArgs g{};
   g.a = norm; g.b = L->w_gu; g.c = act; g.m = tokens; g.n = 2 * c.d_ff; g.k = c.d_model;
   g.lda = c.d_model; g.ldb = c.d_model; g.ldc = c.d_ff; g.epilogue = pd::EPI_SWIGLU; g.err_word = L->err_word;
   {
     pd::TraceScope ts(PD_K_GEMM_GATE_UP, st);
-    if (c.fp8_projections) PD_TRY(use_fp8(L, g, L->q_gu, L->s_gu, ws, w, st));
+    if (f8) PD_TRY(use_fp8(L, g, L->q_gu, L->s_gu, ws, w, st, true));
     PD_TRY(pd::gemm(g, st));
   }
   pd::GemmArgs g2{};
@@ -140,7 +146,12 @@ pd_status qkv_half(pd_layer* L, const bf16* x, int tokens, const pd::RopeEpilogu
   const pd_layer_cfg& c = L->cfg;
   bf16* norm = reinterpret_cast<bf16*>(ws + w.norm);
   bf16* qkv = reinterpret_cast<bf16*>(ws + w.qkv);
-  { pd::TraceScope ts(PD_K_RMSNORM, st); PD_TRY(pd::launch_rmsnorm(x, L->g_attn, norm, tokens, c.d_model, c.rms_eps, st)); }
+  const bool f8 = c.fp8_projections != 0;
+  {
+    pd::TraceScope ts(PD_K_RMSNORM, st);
+    PD_TRY(pd::launch_rmsnorm(x, L->g_attn, norm, tokens, c.d_model, c.rms_eps, st, f8 ? ws + w.q_act : nullptr,
+                              f8 ? reinterpret_cast<float*>(ws + w.s_act) : nullptr));
+  }
   pd::GemmArgs g{};
   g.a = norm; g.b = L->w_qkv; g.c = qkv; g.m = tokens; g.n = L->n_qkv; g.k = c.d_model;
   g.lda = c.d_model; g.ldb = c.d_model; g.ldc = L->n_qkv; g.epilogue = pd::EPI_ROPE_KV; g.rope = &rope;
@@ -148,7 +159,7 @@ pd_status qkv_half(pd_layer* L, const bf16* x, int tokens, const pd::RopeEpilogu
   enable_tail_split(L, g, ws, w, tokens);
   {
     pd::TraceScope ts(PD_K_GEMM_QKV, st);
-    if (c.fp8_projections) PD_TRY(use_fp8(L, g, L->q_qkv, L->s_qkv, ws, w, st));
+    if (f8) PD_TRY(use_fp8(L, g, L->q_qkv, L->s_qkv, ws, w, st, true));
     PD_TRY(pd::gemm(g, st));
   }
   return PD_OK;
@@ -267,9 +278,9 @@ pd_status decode_impl(pd_layer* L, const bf16* x, bf16* out, const int32_t* kv_l
   // FP8 mode: a row-wise quantiser in front of every projection (same programmatic-serialization chain)
   uint8_t* q_act = ws + w.q_act;
   float* s_act = reinterpret_cast<float*>(ws + w.s_act);
-  auto fp8_in = [&](pd::SkinnyGemmArgs& a, const uint8_t* w_codes, const float* w_scales) -> pd_status {
+  auto fp8_in = [&](pd::SkinnyGemmArgs& a, const uint8_t* w_codes, const float* w_scales, bool quantised) -> pd_status {
     if (!f8) return PD_OK;
-    PD_TRY(pd::launch_quantize_rows_fp8(a.x, a.ldx, B, a.k, q_act, a.k, s_act, st));
+    if (!quantised) PD_TRY(pd::launch_quantize_rows_fp8(a.x, a.ldx, B, a.k, q_act, a.k, s_act, st));
     a.x = reinterpret_cast<const bf16*>(q_act); a.ldx = a.k;
     a.w = reinterpret_cast<const bf16*>(w_codes);
     a.fp8 = 1; a.scale_x = s_act; a.scale_w = w_scales;
@@ -278,14 +289,15 @@ pd_status decode_impl(pd_layer* L, const bf16* x, bf16* out, const int32_t* kv_l
 
   {
     pd::TraceScope ts(PD_K_RMSNORM, st);
-    PD_TRY(pd::launch_rmsnorm_decode(x, L->g_attn, norm, B, c.d_model, c.rms_eps, z_qkv, L->n_qkv, st));
+    PD_TRY(pd::launch_rmsnorm_decode(x, L->g_attn, norm, B, c.d_model, c.rms_eps, z_qkv, L->n_qkv, st,
+                                     f8 ? q_act : nullptr, f8 ? s_act : nullptr));
   }
   pd::SkinnyGemmArgs g{};
   g.batch = B; g.err_word = L->err_word; g.acc_zeroed = true;
   {
     pd::TraceScope ts(PD_K_GEMM_QKV, st);
     g.x = norm; g.w = L->w_qkv; g.acc = acc_qkv; g.n = L->n_qkv; g.k = c.d_model; g.ldx = c.d_model;
-    PD_TRY(fp8_in(g, L->q_qkv, L->s_qkv));
+    PD_TRY(fp8_in(g, L->q_qkv, L->s_qkv, true));
     PD_TRY(pd::gemm_skinny(g, st));
     PD_TRY(pd::launch_skinny_rope_kv(acc_qkv, qkv, r, B, L->err_word, z_o, c.d_model, st));
   }
@@ -300,21 +312,22 @@ pd_status decode_impl(pd_layer* L, const bf16* x, bf16* out, const int32_t* kv_l
   {
     pd::TraceScope ts(PD_K_GEMM_O, st);  // h = x + o W_o^T and n2 = RMSNorm(h) in the same row-wise pass
     g.x = attn_o; g.w = L->w_o; g.acc = acc_o; g.n = c.d_model; g.k = hq; g.ldx = hq;
-    PD_TRY(fp8_in(g, L->q_o, L->s_o));
+    PD_TRY(fp8_in(g, L->q_o, L->s_o, false));
     PD_TRY(pd::gemm_skinny(g, st));
-    PD_TRY(pd::launch_skinny_residual(acc_o, x, resid, L->g_mlp, norm, B, c.d_model, c.rms_eps, z_gu, n_gu, st));
+    PD_TRY(pd::launch_skinny_residual(acc_o, x, resid, L->g_mlp, norm, B, c.d_model, c.rms_eps, z_gu, n_gu, st,
+                                      f8 ? q_act : nullptr, f8 ? s_act : nullptr));
   }
   {
     pd::TraceScope ts(PD_K_GEMM_GATE_UP, st);
     g.x = norm; g.w = L->w_gu; g.acc = acc_gu; g.n = n_gu; g.k = c.d_model; g.ldx = c.d_model;
-    PD_TRY(fp8_in(g, L->q_gu, L->s_gu));
+    PD_TRY(fp8_in(g, L->q_gu, L->s_gu, true));
     PD_TRY(pd::gemm_skinny(g, st));
     PD_TRY(pd::launch_skinny_swiglu(acc_gu, act, B, c.d_ff, z_down, c.d_model, st));
   }
   {
     pd::TraceScope ts(PD_K_GEMM_DOWN, st);
     g.x = act; g.w = L->w_down; g.acc = acc_down; g.n = c.d_model; g.k = c.d_ff; g.ldx = c.d_ff;
-    PD_TRY(fp8_in(g, L->q_down, L->s_down));
+    PD_TRY(fp8_in(g, L->q_down, L->s_down, false));
     PD_TRY(pd::gemm_skinny(g, st));
     PD_TRY(pd::launch_skinny_residual(acc_down, resid, out, nullptr, nullptr, B, c.d_model, c.rms_eps, nullptr, 0, st));
   }
