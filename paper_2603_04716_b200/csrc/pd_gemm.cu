@@ -13,6 +13,7 @@
 // and the KV cache (a tile holds whole heads).
 // Every barrier wait is wall-clock bounded; on a timeout the block raises a shared abort
 // flag, records an error word in global memory and leaves through the normal teardown.
+#include <cstdlib>
 #include <mutex>
 
 #include "pd_common.cuh"
@@ -155,6 +156,167 @@ __device__ __forceinline__ UnitInfo unit_info(int unit, int main_tiles, int k_bl
     }
   }
   return u;
+}
+
+// Epilogue of one accumulator tile for the thread that owns row `row` (tensor-memory lane of t_row): reads the
+// accumulator in chunks of 32 columns and applies the epilogue EPI.  role / n_half as in UnitInfo; part_row is the
+// thread's row of the partner's fp32 partial (roles 1 and 2); ok = false skips the work (an aborted wait).
+template <int BN, int EPI, bool F8>
+__device__ __forceinline__ void epilogue_tile(const GemmDev& p, int role, int n_half, int tm, int tn, int row,
+                                              uint32_t t_row, const float* part_row, bool ok) {
+  (void)tm;
+  // a half-width unit holds columns [128 n_half, 128 n_half + 128) of its tile in accumulator columns 0..127
+  const int acc_cols = (role == 3) ? 128 : BN;
+  const int col_base = tn * BN + n_half * 128;
+  float row_scale = 1.f;
+  if constexpr (F8) row_scale = row < p.m ? p.scale_a[row] : 0.f;
+  // accumulator chunk -> registers (+ the partner's partial for a K-split tile; x the operand scales for FP8)
+  auto load_acc = [&](int col_off, uint32_t (&v)[32]) {
+    ptx::tmem_ld_32x32(t_row + col_off, v);
+    ptx::tmem_ld_wait();
+    if (role == 2) {
+#pragma unroll
+      for (int j = 0; j < 32; j += 4) {
+        const float4 q = __ldcg(reinterpret_cast<const float4*>(part_row + col_off + j));
+        v[j] = __float_as_uint(__uint_as_float(v[j]) + q.x);
+        v[j + 1] = __float_as_uint(__uint_as_float(v[j + 1]) + q.y);
+        v[j + 2] = __float_as_uint(__uint_as_float(v[j + 2]) + q.z);
+        v[j + 3] = __float_as_uint(__uint_as_float(v[j + 3]) + q.w);
+      }
+    }
+    if constexpr (F8) {
+      const int col = col_base + col_off;  // row of B = column of the product (a multiple of 32)
+#pragma unroll
+      for (int j = 0; j < 32; j += 4) {
+        float4 sb = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (col + j < p.n) sb = __ldg(reinterpret_cast<const float4*>(p.scale_b + col + j));
+        v[j] = __float_as_uint(__uint_as_float(v[j]) * (row_scale * sb.x));
+        v[j + 1] = __float_as_uint(__uint_as_float(v[j + 1]) * (row_scale * sb.y));
+        v[j + 2] = __float_as_uint(__uint_as_float(v[j + 2]) * (row_scale * sb.z));
+        v[j + 3] = __float_as_uint(__uint_as_float(v[j + 3]) * (row_scale * sb.w));
+      }
+    }
+  };
+  if (role == 1 || !ok) {
+    // nothing more to do for this unit
+  } else if constexpr (EPI == EPI_STORE || EPI == EPI_RESIDUAL) {
+#pragma unroll 1
+    for (int c0 = 0; c0 < acc_cols; c0 += 32) {
+      uint32_t v[32];
+      load_acc(c0, v);
+      const int col = col_base + c0;
+      if (row < p.m) {
+        bf16* crow = p.c + static_cast<size_t>(row) * p.ldc + col;
+        const bf16* rrow = (EPI == EPI_RESIDUAL) ? p.r + static_cast<size_t>(row) * p.ldr + col : nullptr;
+#pragma unroll
+        for (int j = 0; j < 32; j += 8) {
+          if (col + j < p.n) {
+            float f[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(v[j + e]);
+            if (EPI == EPI_RESIDUAL) {
+              const uint4 rr = *reinterpret_cast<const uint4*>(rrow + j);
+              f[0] += ptx::bf16_lo(rr.x); f[1] += ptx::bf16_hi(rr.x);
+              f[2] += ptx::bf16_lo(rr.y); f[3] += ptx::bf16_hi(rr.y);
+              f[4] += ptx::bf16_lo(rr.z); f[5] += ptx::bf16_hi(rr.z);
+              f[6] += ptx::bf16_lo(rr.w); f[7] += ptx::bf16_hi(rr.w);
+            }
+            *reinterpret_cast<uint4*>(crow + j) = pack8(f);
+          }
+        }
+      }
+    }
+  } else if constexpr (EPI == EPI_SWIGLU) {
+    // columns [128 q, 128 q + 64) of the product are gate features 64 q .., the next 64 the matching up features
+    const int f_total = p.n / 2;
+#pragma unroll 1
+    for (int c0 = 0; c0 < acc_cols / 2; c0 += 32) {
+      const int pair = c0 >> 6, within = c0 & 63;
+      uint32_t g[32], u[32];
+      load_acc(pair * 128 + within, g);
+      load_acc(pair * 128 + 64 + within, u);
+      const int fcol = (tn * (BN / 128) + n_half + pair) * 64 + within;
+      if (row < p.m && fcol < f_total) {
+        bf16* crow = p.c + static_cast<size_t>(row) * p.ldc + fcol;
+#pragma unroll
+        for (int j = 0; j < 32; j += 8) {
+          float f[8];
+#pragma unroll
+          for (int e = 0; e < 8; ++e) {
+            const float gv = __uint_as_float(g[j + e]);
+            f[e] = gv / (1.f + __expf(-gv)) * __uint_as_float(u[j + e]);
+          }
+          *reinterpret_cast<uint4*>(crow + j) = pack8(f);
+        }
+      }
+    }
+  } else {  // EPI_ROPE_KV
+    const RopeEpilogue& rp = p.rope;
+    const int hd = rp.head_dim, half = hd >> 1;
+    int pos = 0, slot = 0;
+    bool row_ok = row < p.m;
+    if (row_ok) {
+      if (rp.cu_seqlens) {
+        int lo = 0, hi = rp.n_req;  // request r with cu[r] <= row < cu[r+1]
+        while (hi - lo > 1) {
+          const int mid = (lo + hi) >> 1;
+          if (rp.cu_seqlens[mid] <= row) lo = mid; else hi = mid;
+        }
+        pos = row - rp.cu_seqlens[lo] + (rp.prefix ? rp.prefix[lo] : 0);
+        slot = rp.slots ? rp.slots[lo] : lo;
+      } else {
+        pos = rp.kv_len[row];
+        slot = row;
+      }
+      if (pos < 0 || pos >= rp.len_cap || pos >= rp.max_pos || slot < 0 || slot >= rp.batch_cap) {
+        if (p.err_word) atomicExch(p.err_word, 2);  // would fall outside the cache or the table: skip the row
+        row_ok = false;
+      }
+    }
+    const int n_heads = rp.n_q_heads + 2 * rp.n_kv_heads;
+    const int heads_per_tile = acc_cols / hd;
+#pragma unroll 1
+    for (int hh = 0; hh < heads_per_tile; ++hh) {
+      const int head = col_base / hd + hh;
+      if (head >= n_heads) break;  // warp-uniform
+#pragma unroll 1
+      for (int i0 = 0; i0 < half; i0 += 32) {
+        uint32_t lo[32], hi[32];
+        load_acc(hh * hd + i0, lo);
+        load_acc(hh * hd + half + i0, hi);
+        if (!row_ok) continue;
+        bf16* dst;
+        if (head < rp.n_q_heads) {
+          dst = p.c + static_cast<size_t>(row) * p.ldc + head * hd;
+        } else if (head < rp.n_q_heads + rp.n_kv_heads) {
+          dst = rp.k_cache +
+                ((static_cast<size_t>(slot) * rp.n_kv_heads + (head - rp.n_q_heads)) * rp.len_cap + pos) * hd;
+        } else {
+          dst = rp.v_cache + ((static_cast<size_t>(slot) * rp.n_kv_heads + (head - rp.n_q_heads - rp.n_kv_heads)) *
+                                  rp.len_cap + pos) * hd;
+        }
+        const bool rotate = head < rp.n_q_heads + rp.n_kv_heads;
+        const float4* tab = reinterpret_cast<const float4*>(rp.rope_tab + static_cast<size_t>(pos) * half + i0);
+#pragma unroll
+        for (int j = 0; j < 32; j += 8) {
+          float a[8], b[8];
+#pragma unroll
+          for (int e = 0; e < 8; ++e) { a[e] = __uint_as_float(lo[j + e]); b[e] = __uint_as_float(hi[j + e]); }
+          if (rotate) {
+#pragma unroll
+            for (int e = 0; e < 8; e += 2) {
+              const float4 cs = tab[(j + e) >> 1];  // (cos, sin) of two consecutive pairs
+              const float a0 = a[e], b0 = b[e], a1 = a[e + 1], b1 = b[e + 1];
+              a[e] = a0 * cs.x - b0 * cs.y;      b[e] = b0 * cs.x + a0 * cs.y;
+              a[e + 1] = a1 * cs.z - b1 * cs.w;  b[e + 1] = b1 * cs.z + a1 * cs.w;
+            }
+          }
+          *reinterpret_cast<uint4*>(dst + i0 + j) = pack8(a);
+          *reinterpret_cast<uint4*>(dst + half + i0 + j) = pack8(b);
+        }
+      }
+    }
+  }
 }
 
 template <int BN, int EPI, bool F8>
@@ -326,158 +488,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
           __threadfence();
         }
       }
-      // a half-width unit holds columns [128 n_half, 128 n_half + 128) of its tile in accumulator columns 0..127
-      const int acc_cols = (ui.role == 3) ? 128 : BN;
-      const int col_base = tn * BN + ui.n_half * 128;
-      float row_scale = 1.f;
-      if constexpr (F8) row_scale = row < p.m ? p.scale_a[row] : 0.f;
-      // accumulator chunk -> registers (+ the partner's partial for a K-split tile; x the operand scales for FP8)
-      auto load_acc = [&](int col_off, uint32_t (&v)[32]) {
-        ptx::tmem_ld_32x32(t_row + col_off, v);
-        ptx::tmem_ld_wait();
-        if (ui.role == 2) {
-#pragma unroll
-          for (int j = 0; j < 32; j += 4) {
-            const float4 q = __ldcg(reinterpret_cast<const float4*>(part_row + col_off + j));
-            v[j] = __float_as_uint(__uint_as_float(v[j]) + q.x);
-            v[j + 1] = __float_as_uint(__uint_as_float(v[j + 1]) + q.y);
-            v[j + 2] = __float_as_uint(__uint_as_float(v[j + 2]) + q.z);
-            v[j + 3] = __float_as_uint(__uint_as_float(v[j + 3]) + q.w);
-          }
-        }
-        if constexpr (F8) {
-          const int col = col_base + col_off;  // row of B = column of the product (a multiple of 32)
-#pragma unroll
-          for (int j = 0; j < 32; j += 4) {
-            float4 sb = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (col + j < p.n) sb = __ldg(reinterpret_cast<const float4*>(p.scale_b + col + j));
-            v[j] = __float_as_uint(__uint_as_float(v[j]) * (row_scale * sb.x));
-            v[j + 1] = __float_as_uint(__uint_as_float(v[j + 1]) * (row_scale * sb.y));
-            v[j + 2] = __float_as_uint(__uint_as_float(v[j + 2]) * (row_scale * sb.z));
-            v[j + 3] = __float_as_uint(__uint_as_float(v[j + 3]) * (row_scale * sb.w));
-          }
-        }
-      };
-      if (ui.role == 1 || !ok) {
-        // nothing more to do for this unit
-      } else if constexpr (EPI == EPI_STORE || EPI == EPI_RESIDUAL) {
-#pragma unroll 1
-        for (int c0 = 0; c0 < acc_cols; c0 += 32) {
-          uint32_t v[32];
-          load_acc(c0, v);
-          const int col = col_base + c0;
-          if (row < p.m) {
-            bf16* crow = p.c + static_cast<size_t>(row) * p.ldc + col;
-            const bf16* rrow = (EPI == EPI_RESIDUAL) ? p.r + static_cast<size_t>(row) * p.ldr + col : nullptr;
-#pragma unroll
-            for (int j = 0; j < 32; j += 8) {
-              if (col + j < p.n) {
-                float f[8];
-#pragma unroll
-                for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(v[j + e]);
-                if (EPI == EPI_RESIDUAL) {
-                  const uint4 rr = *reinterpret_cast<const uint4*>(rrow + j);
-                  f[0] += ptx::bf16_lo(rr.x); f[1] += ptx::bf16_hi(rr.x);
-                  f[2] += ptx::bf16_lo(rr.y); f[3] += ptx::bf16_hi(rr.y);
-                  f[4] += ptx::bf16_lo(rr.z); f[5] += ptx::bf16_hi(rr.z);
-                  f[6] += ptx::bf16_lo(rr.w); f[7] += ptx::bf16_hi(rr.w);
-                }
-                *reinterpret_cast<uint4*>(crow + j) = pack8(f);
-              }
-            }
-          }
-        }
-      } else if constexpr (EPI == EPI_SWIGLU) {
-        // columns [128 q, 128 q + 64) of the product are gate features 64 q .., the next 64 the matching up features
-        const int f_total = p.n / 2;
-#pragma unroll 1
-        for (int c0 = 0; c0 < acc_cols / 2; c0 += 32) {
-          const int pair = c0 >> 6, within = c0 & 63;
-          uint32_t g[32], u[32];
-          load_acc(pair * 128 + within, g);
-          load_acc(pair * 128 + 64 + within, u);
-          const int fcol = (tn * (BN / 128) + ui.n_half + pair) * 64 + within;
-          if (row < p.m && fcol < f_total) {
-            bf16* crow = p.c + static_cast<size_t>(row) * p.ldc + fcol;
-#pragma unroll
-            for (int j = 0; j < 32; j += 8) {
-              float f[8];
-#pragma unroll
-              for (int e = 0; e < 8; ++e) {
-                const float gv = __uint_as_float(g[j + e]);
-                f[e] = gv / (1.f + __expf(-gv)) * __uint_as_float(u[j + e]);
-              }
-              *reinterpret_cast<uint4*>(crow + j) = pack8(f);
-            }
-          }
-        }
-      } else {  // EPI_ROPE_KV
-        const RopeEpilogue& rp = p.rope;
-        const int hd = rp.head_dim, half = hd >> 1;
-        int pos = 0, slot = 0;
-        bool row_ok = row < p.m;
-        if (row_ok) {
-          if (rp.cu_seqlens) {
-            int lo = 0, hi = rp.n_req;  // request r with cu[r] <= row < cu[r+1]
-            while (hi - lo > 1) {
-              const int mid = (lo + hi) >> 1;
-              if (rp.cu_seqlens[mid] <= row) lo = mid; else hi = mid;
-            }
-            pos = row - rp.cu_seqlens[lo] + (rp.prefix ? rp.prefix[lo] : 0);
-            slot = rp.slots ? rp.slots[lo] : lo;
-          } else {
-            pos = rp.kv_len[row];
-            slot = row;
-          }
-          if (pos < 0 || pos >= rp.len_cap || pos >= rp.max_pos || slot < 0 || slot >= rp.batch_cap) {
-            if (p.err_word) atomicExch(p.err_word, 2);  // would fall outside the cache or the table: skip the row
-            row_ok = false;
-          }
-        }
-        const int n_heads = rp.n_q_heads + 2 * rp.n_kv_heads;
-        const int heads_per_tile = acc_cols / hd;
-#pragma unroll 1
-        for (int hh = 0; hh < heads_per_tile; ++hh) {
-          const int head = col_base / hd + hh;
-          if (head >= n_heads) break;  // warp-uniform
-#pragma unroll 1
-          for (int i0 = 0; i0 < half; i0 += 32) {
-            uint32_t lo[32], hi[32];
-            load_acc(hh * hd + i0, lo);
-            load_acc(hh * hd + half + i0, hi);
-            if (!row_ok) continue;
-            bf16* dst;
-            if (head < rp.n_q_heads) {
-              dst = p.c + static_cast<size_t>(row) * p.ldc + head * hd;
-            } else if (head < rp.n_q_heads + rp.n_kv_heads) {
-              dst = rp.k_cache +
-                    ((static_cast<size_t>(slot) * rp.n_kv_heads + (head - rp.n_q_heads)) * rp.len_cap + pos) * hd;
-            } else {
-              dst = rp.v_cache + ((static_cast<size_t>(slot) * rp.n_kv_heads + (head - rp.n_q_heads - rp.n_kv_heads)) *
-                                      rp.len_cap + pos) * hd;
-            }
-            const bool rotate = head < rp.n_q_heads + rp.n_kv_heads;
-            const float4* tab = reinterpret_cast<const float4*>(rp.rope_tab + static_cast<size_t>(pos) * half + i0);
-#pragma unroll
-            for (int j = 0; j < 32; j += 8) {
-              float a[8], b[8];
-#pragma unroll
-              for (int e = 0; e < 8; ++e) { a[e] = __uint_as_float(lo[j + e]); b[e] = __uint_as_float(hi[j + e]); }
-              if (rotate) {
-#pragma unroll
-                for (int e = 0; e < 8; e += 2) {
-                  const float4 cs = tab[(j + e) >> 1];  // (cos, sin) of two consecutive pairs
-                  const float a0 = a[e], b0 = b[e], a1 = a[e + 1], b1 = b[e + 1];
-                  a[e] = a0 * cs.x - b0 * cs.y;      b[e] = b0 * cs.x + a0 * cs.y;
-                  a[e + 1] = a1 * cs.z - b1 * cs.w;  b[e + 1] = b1 * cs.z + a1 * cs.w;
-                }
-              }
-              *reinterpret_cast<uint4*>(dst + i0 + j) = pack8(a);
-              *reinterpret_cast<uint4*>(dst + half + i0 + j) = pack8(b);
-            }
-          }
-        }
-      }
+      epilogue_tile<BN, EPI, F8>(p, ui.role, ui.n_half, tm, tn, row, t_row, part_row, ok);
       // all of this warp's reads of the accumulator are complete: hand the buffer back
       ptx::tc_fence_before();
       __syncwarp();
@@ -498,6 +509,154 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     __syncwarp();
     ptx::tc_fence_after();
     ptx::tmem_dealloc(tmem_base, TMEM_COLS);
+  }
+}
+
+// ------------------------------------------------------------- CTA-pair variant
+// The same GEMM on pairs of CTAs (cluster of two on one TPC): a pair owns a 256 x 256 tile.  Each CTA loads its
+// 128 rows of A and 128 of the tile's 256 rows of B (so a stage is 32 KB per CTA instead of 48 KB and every byte of
+// B is read from shared memory once for both SMs), the even CTA's MMA thread issues tcgen05.mma.cta_group::2 for
+// both, and each CTA drains its own 128 accumulator rows through the common epilogue.
+// Barriers: `full` lives in the even CTA and counts the bytes of both CTAs' loads; `empty` and `accumulator full`
+// exist in both CTAs and are signalled together by a multicast commit; `accumulator empty` lives in the even CTA
+// and collects the epilogue warps of both.  A CTA only ever WAITS on its own barriers, always bounded.
+constexpr int P2_STAGE_BYTES = 2 * BM * 128;  // A rows + B rows of this CTA, 16 KB each
+constexpr int P2_STAGES = 6;
+constexpr int P2_SMEM_BYTES = P2_STAGES * P2_STAGE_BYTES + 1024 + 256;
+
+template <int EPI, bool F8>
+__global__ void __launch_bounds__(GEMM_THREADS, 1)
+gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b, GemmDev p) {
+  constexpr int BN = 256;
+  constexpr int STAGES = P2_STAGES;
+  constexpr int KE = F8 ? BK_F8 : BK;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem_al = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem_al + STAGES * P2_STAGE_BYTES);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const uint32_t rank = ptx::cluster_ctarank();
+  const uint32_t bar0 = ptx::smem_u32(bars);
+  auto full_bar = [&](int s) { return bar0 + 8u * s; };
+  auto empty_bar = [&](int s) { return bar0 + 8u * (STAGES + s); };
+  auto accf_bar = [&](int a) { return bar0 + 8u * (2 * STAGES + a); };
+  auto acce_bar = [&](int a) { return bar0 + 8u * (2 * STAGES + 2 + a); };
+
+  if (threadIdx.x == 0) {
+    *abort_flag = 0;
+    for (int s = 0; s < STAGES; ++s) {
+      ptx::mbar_init(full_bar(s), 1);
+      ptx::mbar_init(empty_bar(s), 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      ptx::mbar_init(accf_bar(a), 1);
+      ptx::mbar_init(acce_bar(a), 8);  // four epilogue warps of each CTA
+    }
+    ptx::fence_barrier_init();
+    ptx::prefetch_tensormap(&tmap_a);
+    ptx::prefetch_tensormap(&tmap_b);
+  }
+  if (warp == 1) {
+    ptx::tmem_alloc_pair(ptx::smem_u32(tmem_slot), TMEM_COLS);
+    ptx::tmem_relinquish_pair();
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::cluster_sync_all();  // both CTAs' barriers are initialised before either CTA signals the other
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  const int k_blocks = p.k / KE;
+  const int pair_id = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+  const int tiles_m2 = (p.tiles_m + 1) >> 1;  // 256-row tiles
+  const int n_units = tiles_m2 * p.tiles_n;
+  const int group2 = max(1, p.raster_group >> 1);
+
+  if (warp == 0) {
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int unit = pair_id; unit < n_units && ok; unit += n_pairs) {
+        int tm2, tn;
+        tile_coords(unit, tiles_m2, p.tiles_n, group2, tm2, tn);
+        for (int kb = 0; kb < k_blocks; ++kb) {
+          if (!ptx::mbar_wait_bounded(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
+          const uint32_t sa = smem_base + stage * P2_STAGE_BYTES;
+          const uint32_t sb = sa + BM * 128;
+          const uint32_t lead_full = ptx::map_to_cta(full_bar(stage), 0);
+          if (rank == 0) ptx::mbar_arrive_expect_tx(full_bar(stage), 2 * P2_STAGE_BYTES);
+          ptx::tma_load_2d_pair(sa, &tmap_a, kb * KE, (2 * tm2 + static_cast<int>(rank)) * BM, lead_full);
+          ptx::tma_load_2d_pair(sb, &tmap_b, kb * KE, tn * BN + static_cast<int>(rank) * 128, lead_full);
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+      }
+      if (!ok) {
+        for (int i = 0; i < 2000; ++i) __nanosleep(1000);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0 && rank == 0) {
+      constexpr uint32_t idesc = F8 ? ptx::umma_idesc_e4m3(2 * BM, BN) : ptx::umma_idesc_bf16(2 * BM, BN);
+      int stage = 0, acc = 0;
+      uint32_t phase = 0, acc_phase = 0;
+      bool ok = true;
+      for (int unit = pair_id; unit < n_units && ok; unit += n_pairs) {
+        if (!ptx::mbar_wait_bounded(acce_bar(acc), acc_phase ^ 1u, abort_flag)) break;
+        ptx::tc_fence_after();
+        const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * BN);
+        for (int kb = 0; kb < k_blocks; ++kb) {
+          if (!ptx::mbar_wait_bounded(full_bar(stage), phase, abort_flag)) { ok = false; break; }
+          ptx::tc_fence_after();
+          const uint32_t sa = smem_base + stage * P2_STAGE_BYTES;
+          const uint64_t da = ptx::umma_desc_sw128(sa);
+          const uint64_t db = ptx::umma_desc_sw128(sa + BM * 128);
+#pragma unroll
+          for (int kk = 0; kk < 4; ++kk) {
+            const uint32_t accum = (kb > 0 || kk > 0) ? 1u : 0u;
+            if constexpr (F8) ptx::umma_f8_pair(d_tmem, da + 2u * kk, db + 2u * kk, idesc, accum);
+            else ptx::umma_bf16_pair(d_tmem, da + 2u * kk, db + 2u * kk, idesc, accum);
+          }
+          ptx::umma_commit_pair(empty_bar(stage), 3);  // the stage is free in both CTAs
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        ptx::umma_commit_pair(accf_bar(acc), 3);
+        if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+      }
+    }
+  } else {
+    const int lane_group = warp & 3;
+    int acc = 0;
+    uint32_t acc_phase = 0;
+    for (int unit = pair_id; unit < n_units; unit += n_pairs) {
+      int tm2, tn;
+      tile_coords(unit, tiles_m2, p.tiles_n, group2, tm2, tn);
+      const int tm = 2 * tm2 + static_cast<int>(rank);
+      if (!__all_sync(0xffffffffu, ptx::mbar_wait_bounded(accf_bar(acc), acc_phase, abort_flag))) break;
+      ptx::tc_fence_after();
+      const int row = tm * BM + lane_group * 32 + lane;
+      const uint32_t t_row = tmem_base + (static_cast<uint32_t>(lane_group * 32) << 16) + static_cast<uint32_t>(acc * BN);
+      epilogue_tile<BN, EPI, F8>(p, 0, 0, tm, tn, row, t_row, nullptr, true);
+      ptx::tc_fence_before();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive_cluster(ptx::map_to_cta(acce_bar(acc), 0));
+      if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+    }
+  }
+
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::cluster_sync_all();  // neither CTA leaves (or frees tensor memory) while its peer may still signal it
+  if (*abort_flag && threadIdx.x == 0 && p.err_word) atomicExch(p.err_word, 1);
+  if (warp == 1) {
+    __syncwarp();
+    ptx::tc_fence_after();
+    ptx::tmem_dealloc_pair(tmem_base, TMEM_COLS);
   }
 }
 
@@ -574,6 +733,79 @@ pd_status launch_tc(const GemmArgs& g, cudaStream_t stream) {
   return PD_OK;
 }
 
+// CTA pairs resident at once for the pair kernel (0: clusters of two cannot be placed).
+template <int EPI, bool F8>
+int pair_capacity() {
+  static int cap = -1;
+  if (cap >= 0) return cap;
+  auto kern = gemm_tc_pair_kernel<EPI, F8>;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, P2_SMEM_BYTES) != cudaSuccess) return cap = 0;
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(2 * sm_count());
+  cfg.blockDim = dim3(GEMM_THREADS);
+  cfg.dynamicSmemBytes = P2_SMEM_BYTES;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  int n = 0;
+  if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess) { cudaGetLastError(); n = 0; }
+  return cap = n;
+}
+
+template <int EPI, bool F8>
+pd_status launch_tc_pair(const GemmArgs& g, cudaStream_t stream) {
+  auto kern = gemm_tc_pair_kernel<EPI, F8>;
+  const int cap = pair_capacity<EPI, F8>();
+  if (cap <= 0) return PD_ERR_UNSUPPORTED_SHAPE;
+  CUtensorMap ta, tb;
+  if (F8) {
+    PD_TRY(make_tmap_u8(&ta, g.a, g.m, g.k, g.lda, BM));
+    PD_TRY(make_tmap_u8(&tb, g.b, g.n, g.k, g.ldb, 128));
+  } else {
+    PD_TRY(make_tmap_bf16(&ta, g.a, g.m, g.k, g.lda, BM));
+    PD_TRY(make_tmap_bf16(&tb, g.b, g.n, g.k, g.ldb, 128));
+  }
+  GemmDev p{};
+  p.scale_a = g.scale_a; p.scale_b = g.scale_b;
+  p.c = g.c; p.r = g.r; p.m = g.m; p.n = g.n; p.k = g.k; p.ldc = g.ldc; p.ldr = g.ldr;
+  p.tiles_m = (g.m + BM - 1) / BM;
+  p.tiles_n = g.n / 256;
+  p.err_word = g.err_word;
+  {
+    long long grp = (40ll << 20) / (static_cast<long long>(BM) * g.k * (F8 ? 1 : 2));
+    p.raster_group = static_cast<int>(grp < 4 ? 4 : (grp > 32 ? 32 : grp));
+  }
+  if (EPI == EPI_ROPE_KV) p.rope = *g.rope;
+  const int units = ((p.tiles_m + 1) / 2) * p.tiles_n;
+  p.n_units = units; p.main_tiles = units;
+  const int pairs = units < cap ? units : cap;
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(2 * pairs);
+  cfg.blockDim = dim3(GEMM_THREADS);
+  cfg.dynamicSmemBytes = P2_SMEM_BYTES;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  PD_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, ta, tb, p));
+  count_launch();
+  return PD_OK;
+}
+
+template <bool F8>
+pd_status launch_tc_pair_epi(const GemmArgs& g, cudaStream_t stream) {
+  switch (g.epilogue) {
+    case EPI_RESIDUAL: return launch_tc_pair<EPI_RESIDUAL, F8>(g, stream);
+    case EPI_SWIGLU: return launch_tc_pair<EPI_SWIGLU, F8>(g, stream);
+    case EPI_ROPE_KV: return launch_tc_pair<EPI_ROPE_KV, F8>(g, stream);
+    default: return launch_tc_pair<EPI_STORE, F8>(g, stream);
+  }
+}
+
 template <int BN, bool F8>
 pd_status launch_tc_epi(const GemmArgs& g, cudaStream_t stream) {
   switch (g.epilogue) {
@@ -613,6 +845,16 @@ int gemm_block_n(int m, int n, int epilogue) {
   return best;
 }
 
+// Eligible problems (256-wide tiles, N a multiple of 256, more than one row tile) run on the CTA-pair kernel;
+// PD_GEMM_PAIRS=0 in the environment keeps them on the single-CTA kernel (for A/B timing).
+static int pair_mode() {
+  static const int mode = [] {
+    const char* v = std::getenv("PD_GEMM_PAIRS");
+    return (v && v[0] == '0') ? 0 : 1;
+  }();
+  return mode;
+}
+
 static pd_status check_gemm_args(const GemmArgs& g) {
   if (!g.a || !g.b || !g.c || g.m < 0 || g.n <= 0 || g.k <= 0) return PD_ERR_INVALID_ARG;
   if (g.epilogue == EPI_RESIDUAL && !g.r) return PD_ERR_INVALID_ARG;
@@ -629,6 +871,10 @@ pd_status gemm(const GemmArgs& g, cudaStream_t stream) {
   PD_TRY(check_gemm_args(g));
   if (g.m == 0) return PD_OK;
   const int bn = gemm_block_n(g.m, g.n, g.epilogue);
+  if (bn == 256 && g.n % 256 == 0 && g.m > BM && pair_mode() != 0) {
+    const pd_status st = g.fp8 ? launch_tc_pair_epi<true>(g, stream) : launch_tc_pair_epi<false>(g, stream);
+    if (st != PD_ERR_UNSUPPORTED_SHAPE) return st;  // (clusters of two could not be placed: single-CTA kernel)
+  }
   if (g.fp8) {
     switch (bn) {
       case 256: return launch_tc_epi<256, true>(g, stream);
