@@ -521,12 +521,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
 // exist in both CTAs and are signalled together by a multicast commit; `accumulator empty` lives in the even CTA
 // and collects the epilogue warps of both.  A CTA only ever WAITS on its own barriers, always bounded.
 constexpr int P2_STAGE_BYTES = 2 * BM * 128;  // A rows + B rows of this CTA, 16 KB each
-constexpr int P2_STAGES = 6;
+constexpr int P2_STAGES = 7;
 constexpr int P2_SMEM_BYTES = P2_STAGES * P2_STAGE_BYTES + 1024 + 256;
 
 template <int EPI, bool F8>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
-gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b, GemmDev p) {
+gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
+                    const __grid_constant__ CUtensorMap tmap_b_half, GemmDev p) {
   constexpr int BN = 256;
   constexpr int STAGES = P2_STAGES;
   constexpr int KE = F8 ? BK_F8 : BK;
@@ -559,6 +560,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
     ptx::fence_barrier_init();
     ptx::prefetch_tensormap(&tmap_a);
     ptx::prefetch_tensormap(&tmap_b);
+    ptx::prefetch_tensormap(&tmap_b_half);
   }
   if (warp == 1) {
     ptx::tmem_alloc_pair(ptx::smem_u32(tmem_slot), TMEM_COLS);
@@ -573,7 +575,8 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
   const int k_blocks = p.k / KE;
   const int pair_id = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
   const int tiles_m2 = (p.tiles_m + 1) >> 1;  // 256-row tiles
-  const int n_units = tiles_m2 * p.tiles_n;
+  const int n_units = p.n_units;  // whole tiles [0, main_tiles), then the tiles of the last partial wave as two
+                                  // independent 128-column halves each (tail_halves), see unit_info
   const int group2 = max(1, p.raster_group >> 1);
 
   if (warp == 0) {
@@ -582,16 +585,21 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
       uint32_t phase = 0;
       bool ok = true;
       for (int unit = pair_id; unit < n_units && ok; unit += n_pairs) {
+        const UnitInfo ui = unit_info(unit, p.main_tiles, k_blocks, 1);
         int tm2, tn;
-        tile_coords(unit, tiles_m2, p.tiles_n, group2, tm2, tn);
+        tile_coords(ui.tile, tiles_m2, p.tiles_n, group2, tm2, tn);
+        const bool half = ui.role == 3;  // this CTA then supplies 64 of the half tile's 128 rows of B
         for (int kb = 0; kb < k_blocks; ++kb) {
           if (!ptx::mbar_wait_bounded(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
           const uint32_t sa = smem_base + stage * P2_STAGE_BYTES;
           const uint32_t sb = sa + BM * 128;
           const uint32_t lead_full = ptx::map_to_cta(full_bar(stage), 0);
-          if (rank == 0) ptx::mbar_arrive_expect_tx(full_bar(stage), 2 * P2_STAGE_BYTES);
+          if (rank == 0) ptx::mbar_arrive_expect_tx(full_bar(stage), half ? 2 * (BM + 64) * 128 : 2 * P2_STAGE_BYTES);
           ptx::tma_load_2d_pair(sa, &tmap_a, kb * KE, (2 * tm2 + static_cast<int>(rank)) * BM, lead_full);
-          ptx::tma_load_2d_pair(sb, &tmap_b, kb * KE, tn * BN + static_cast<int>(rank) * 128, lead_full);
+          if (half)
+            ptx::tma_load_2d_pair(sb, &tmap_b_half, kb * KE, tn * BN + ui.n_half * 128 + static_cast<int>(rank) * 64, lead_full);
+          else
+            ptx::tma_load_2d_pair(sb, &tmap_b, kb * KE, tn * BN + static_cast<int>(rank) * 128, lead_full);
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
       }
@@ -601,11 +609,13 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
     }
   } else if (warp == 1) {
     if (lane == 0 && rank == 0) {
-      constexpr uint32_t idesc = F8 ? ptx::umma_idesc_e4m3(2 * BM, BN) : ptx::umma_idesc_bf16(2 * BM, BN);
+      constexpr uint32_t idesc_full = F8 ? ptx::umma_idesc_e4m3(2 * BM, BN) : ptx::umma_idesc_bf16(2 * BM, BN);
+      constexpr uint32_t idesc_half = F8 ? ptx::umma_idesc_e4m3(2 * BM, 128) : ptx::umma_idesc_bf16(2 * BM, 128);
       int stage = 0, acc = 0;
       uint32_t phase = 0, acc_phase = 0;
       bool ok = true;
       for (int unit = pair_id; unit < n_units && ok; unit += n_pairs) {
+        const uint32_t idesc = unit < p.main_tiles ? idesc_full : idesc_half;
         if (!ptx::mbar_wait_bounded(acce_bar(acc), acc_phase ^ 1u, abort_flag)) break;
         ptx::tc_fence_after();
         const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * BN);
@@ -634,14 +644,15 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
     int acc = 0;
     uint32_t acc_phase = 0;
     for (int unit = pair_id; unit < n_units; unit += n_pairs) {
+      const UnitInfo ui = unit_info(unit, p.main_tiles, k_blocks, 1);
       int tm2, tn;
-      tile_coords(unit, tiles_m2, p.tiles_n, group2, tm2, tn);
+      tile_coords(ui.tile, tiles_m2, p.tiles_n, group2, tm2, tn);
       const int tm = 2 * tm2 + static_cast<int>(rank);
       if (!__all_sync(0xffffffffu, ptx::mbar_wait_bounded(accf_bar(acc), acc_phase, abort_flag))) break;
       ptx::tc_fence_after();
       const int row = tm * BM + lane_group * 32 + lane;
       const uint32_t t_row = tmem_base + (static_cast<uint32_t>(lane_group * 32) << 16) + static_cast<uint32_t>(acc * BN);
-      epilogue_tile<BN, EPI, F8>(p, 0, 0, tm, tn, row, t_row, nullptr, true);
+      epilogue_tile<BN, EPI, F8>(p, ui.role, ui.n_half, tm, tn, row, t_row, nullptr, true);
       ptx::tc_fence_before();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive_cluster(ptx::map_to_cta(acce_bar(acc), 0));
@@ -759,13 +770,15 @@ pd_status launch_tc_pair(const GemmArgs& g, cudaStream_t stream) {
   auto kern = gemm_tc_pair_kernel<EPI, F8>;
   const int cap = pair_capacity<EPI, F8>();
   if (cap <= 0) return PD_ERR_UNSUPPORTED_SHAPE;
-  CUtensorMap ta, tb;
+  CUtensorMap ta, tb, tbh;
   if (F8) {
     PD_TRY(make_tmap_u8(&ta, g.a, g.m, g.k, g.lda, BM));
     PD_TRY(make_tmap_u8(&tb, g.b, g.n, g.k, g.ldb, 128));
+    PD_TRY(make_tmap_u8(&tbh, g.b, g.n, g.k, g.ldb, 64));
   } else {
     PD_TRY(make_tmap_bf16(&ta, g.a, g.m, g.k, g.lda, BM));
     PD_TRY(make_tmap_bf16(&tb, g.b, g.n, g.k, g.ldb, 128));
+    PD_TRY(make_tmap_bf16(&tbh, g.b, g.n, g.k, g.ldb, 64));
   }
   GemmDev p{};
   p.scale_a = g.scale_a; p.scale_b = g.scale_b;
@@ -780,7 +793,16 @@ pd_status launch_tc_pair(const GemmArgs& g, cudaStream_t stream) {
   if (EPI == EPI_ROPE_KV) p.rope = *g.rope;
   const int units = ((p.tiles_m + 1) / 2) * p.tiles_n;
   p.n_units = units; p.main_tiles = units;
-  const int pairs = units < cap ? units : cap;
+  {
+    // the last wave holds `tail` tiles: if they occupy at most half of the pairs, run each as two 128-column halves
+    const int tail = units % cap;
+    if (tail > 0 && 2 * tail <= cap) {
+      p.main_tiles = units - tail;
+      p.n_units = units + tail;
+      p.tail_halves = 1;
+    }
+  }
+  const int pairs = p.n_units < cap ? p.n_units : cap;
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3(2 * pairs);
   cfg.blockDim = dim3(GEMM_THREADS);
@@ -791,7 +813,7 @@ pd_status launch_tc_pair(const GemmArgs& g, cudaStream_t stream) {
   attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  PD_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, ta, tb, p));
+  PD_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, ta, tb, tbh, p));
   count_launch();
   return PD_OK;
 }
