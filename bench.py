@@ -39,8 +39,8 @@ TTFT_SLO, TPOT_SLO, TP_TOTAL = 2.0, 0.050, 2e5
 # one layer (profiles/gemm_tc_prefill_8b_ncu_full.md, profiles/prefill_attn_tc_and_decode_kernels_ncu_full.md).
 # Set an entry to None whenever the kernel changes after the capture.
 NCU_TRAFFIC = {
-    "gemm_tc_kernel": {"bytes_per_launch": 328.4e6, "algorithmic_bytes_per_launch": 238.8e6,
-                       "note": "mean over the four prefill projections of a layer (1313.5 MB / 4)"},
+    "gemm_tc_kernel": {"bytes_per_launch": 362.1e6, "algorithmic_bytes_per_launch": 238.8e6,
+                       "note": "gemm_tc_pair_kernel, mean over the four prefill projections of a layer (1448.4 MB / 4)"},
     "decode_attn_kernel": {"bytes_per_launch": 2.1563e9, "algorithmic_bytes_per_launch": 2.1485e9,
                            "note": "B = 256 at KV length 2049; grows in proportion to the KV length"},
 }
@@ -553,7 +553,7 @@ def main():
                            "n_decode": alloc["n_decode"], "ratio_pd": alloc["ratio_pd"], "rho": alloc["rho"],
                            "mm1_sojourn_s": None if alloc["status"] else 1.0 / (alloc["mu"] - alloc["lam"]),
                            "replayed_sojourn_s_deterministic_service": sojourn},
-            "roofline": {"kernel": "gemm_tc_kernel (QKV, O, gate/up, down projections of the prefill pass)",
+            "roofline": {"kernel": "gemm_tc_pair_kernel (QKV, O, gate/up, down projections of the prefill pass)",
                          "bound": "tensor", "achieved": gemm_tf, "peak": peak_tf, "unit": "TFLOP/s",
                          "frac": gemm_tf / peak_tf, "frac_of_burst_peak": gemm_tf / peaks["bf16_tflops"],
                          "peak_source": peaks["source"] + " (sustained bf16)", "launches": gemm_n,
