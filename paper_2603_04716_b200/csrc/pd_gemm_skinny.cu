@@ -16,6 +16,8 @@
 // weight stream therefore keeps running across kernel boundaries.  (Pulling further weight tiles into L2
 // before the wait was measured too: no gain, the ring already covers the gap.)  The fp32 buffer of a K-split
 // projection is cleared by a row-wise kernel earlier in the chain instead of a memset.
+#include <cstdlib>
+
 #include "pd_common.cuh"
 #include "pd_ptx.cuh"
 
@@ -45,6 +47,53 @@ struct SkinnyDev {
   const float* scale_x;  // FP8 operands: per-row scales of X [B] and of W [N]
   const float* scale_w;
 };
+
+// One chunk of CH accumulator columns (batch rows b0 ..) of the thread that owns output feature n -> the fp32
+// buffer: vector store when K is not split, vector reduction otherwise; FP8 sums are scaled on the way.
+template <int CH, bool F8>
+__device__ __forceinline__ void skinny_store_chunk(const SkinnyDev& p, uint32_t (&v)[32], int n, int lane, int b0) {
+    // 4 x 4 transposes across groups of four lanes: afterwards lane 4q + r holds, for batch column
+    // c0 + 4m + r, the four consecutive features 4q .. 4q + 3 in v[4m .. 4m + 3], i.e. 16 contiguous bytes
+    // of the output row, so one vector store / vector reduction replaces four scalar ones (scalar fp32
+    // reductions into L2 were measured four times slower per byte).
+    const int r4 = lane & 3;
+#pragma unroll
+    for (int m = 0; m < CH; m += 4) {
+#pragma unroll
+      for (int s2 = 0; s2 < 4; s2 += 2) {
+        const uint32_t send = (r4 & 1) ? v[m + s2] : v[m + s2 + 1];
+        const uint32_t recv = __shfl_xor_sync(0xffffffffu, send, 1);
+        if (r4 & 1) v[m + s2] = recv; else v[m + s2 + 1] = recv;
+      }
+#pragma unroll
+      for (int s2 = 0; s2 < 2; ++s2) {
+        const uint32_t send = (r4 & 2) ? v[m + s2] : v[m + s2 + 2];
+        const uint32_t recv = __shfl_xor_sync(0xffffffffu, send, 2);
+        if (r4 & 2) v[m + s2] = recv; else v[m + s2 + 2] = recv;
+      }
+    }
+    const int n4 = n - r4;  // first of this lane's four features (n is a multiple of 4 per group of lanes)
+    if (n4 < p.n) {
+      float4 sw4 = make_float4(1.f, 1.f, 1.f, 1.f);
+      if constexpr (F8) sw4 = __ldg(reinterpret_cast<const float4*>(p.scale_w + n4));
+#pragma unroll
+      for (int m = 0; m < CH; m += 4) {
+        const int b = b0 + m + r4;
+        if (b < p.batch) {
+          if constexpr (F8) {
+            const float sx = __ldg(p.scale_x + b);
+            v[m] = __float_as_uint(__uint_as_float(v[m]) * (sx * sw4.x));
+            v[m + 1] = __float_as_uint(__uint_as_float(v[m + 1]) * (sx * sw4.y));
+            v[m + 2] = __float_as_uint(__uint_as_float(v[m + 2]) * (sx * sw4.z));
+            v[m + 3] = __float_as_uint(__uint_as_float(v[m + 3]) * (sx * sw4.w));
+          }
+          float* dst = p.acc + static_cast<size_t>(b) * p.n + n4;
+          if (p.splits > 1) ptx::red_add_v4_f32(dst, v[m], v[m + 1], v[m + 2], v[m + 3]);
+          else *reinterpret_cast<uint4*>(dst) = make_uint4(v[m], v[m + 1], v[m + 2], v[m + 3]);
+        }
+      }
+    }
+}
 
 // F8: both operands are E4M3 codes (a 128-byte shared-memory row then holds 128 K elements, one MMA covers 32)
 // and every partial sum is multiplied by scale_x[b] * scale_w[n] on its way out.
@@ -176,47 +225,7 @@ gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
         if constexpr (CH == 32) ptx::tmem_ld_32x32(t_row + c0, v);
         else ptx::tmem_ld_32x16(t_row + c0, v);
         ptx::tmem_ld_wait();
-        // 4 x 4 transposes across groups of four lanes: afterwards lane 4q + r holds, for batch column
-        // c0 + 4m + r, the four consecutive features 4q .. 4q + 3 in v[4m .. 4m + 3], i.e. 16 contiguous bytes
-        // of the output row, so one vector store / vector reduction replaces four scalar ones (scalar fp32
-        // reductions into L2 were measured four times slower per byte).
-        const int r4 = lane & 3;
-#pragma unroll
-        for (int m = 0; m < CH; m += 4) {
-#pragma unroll
-          for (int s2 = 0; s2 < 4; s2 += 2) {
-            const uint32_t send = (r4 & 1) ? v[m + s2] : v[m + s2 + 1];
-            const uint32_t recv = __shfl_xor_sync(0xffffffffu, send, 1);
-            if (r4 & 1) v[m + s2] = recv; else v[m + s2 + 1] = recv;
-          }
-#pragma unroll
-          for (int s2 = 0; s2 < 2; ++s2) {
-            const uint32_t send = (r4 & 2) ? v[m + s2] : v[m + s2 + 2];
-            const uint32_t recv = __shfl_xor_sync(0xffffffffu, send, 2);
-            if (r4 & 2) v[m + s2] = recv; else v[m + s2 + 2] = recv;
-          }
-        }
-        const int n4 = n - r4;  // first of this lane's four features (n is a multiple of 4 per group of lanes)
-        if (n4 < p.n) {
-          float4 sw4 = make_float4(1.f, 1.f, 1.f, 1.f);
-          if constexpr (F8) sw4 = __ldg(reinterpret_cast<const float4*>(p.scale_w + n4));
-#pragma unroll
-          for (int m = 0; m < CH; m += 4) {
-            const int b = tb * BNB + c0 + m + r4;
-            if (b < p.batch) {
-              if constexpr (F8) {
-                const float sx = __ldg(p.scale_x + b);
-                v[m] = __float_as_uint(__uint_as_float(v[m]) * (sx * sw4.x));
-                v[m + 1] = __float_as_uint(__uint_as_float(v[m + 1]) * (sx * sw4.y));
-                v[m + 2] = __float_as_uint(__uint_as_float(v[m + 2]) * (sx * sw4.z));
-                v[m + 3] = __float_as_uint(__uint_as_float(v[m + 3]) * (sx * sw4.w));
-              }
-              float* dst = p.acc + static_cast<size_t>(b) * p.n + n4;
-              if (p.splits > 1) ptx::red_add_v4_f32(dst, v[m], v[m + 1], v[m + 2], v[m + 3]);
-              else *reinterpret_cast<uint4*>(dst) = make_uint4(v[m], v[m + 1], v[m + 2], v[m + 3]);
-            }
-          }
-        }
+        skinny_store_chunk<CH, F8>(p, v, n, lane, tb * BNB + c0);
       }
       }
     }
@@ -228,6 +237,160 @@ gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
     __syncwarp();
     ptx::tc_fence_after();
     ptx::tmem_dealloc(tmem_base, Cfg::TMEM_COLS);
+  }
+}
+
+// ------------------------------------------------------------- CTA-pair variant (batch tiles of 128 and 256)
+// A cluster of two CTAs on one TPC owns 256 weight rows x the batch tile for one K slice.  Each CTA loads its own 128
+// weight rows and HALF of the activation tile (a stage is 32 KB instead of 48 KB at a 256-wide batch tile, so three
+// stages fit where two did and the activations cross from L2 once per pair), the even CTA issues
+// tcgen05.mma.cta_group::2 (M = 256) for both, and each CTA adds its 128 output features into the fp32 buffer.
+// Barrier protocol as in the prefill pair GEMM: `full` in the even CTA counts both CTAs' bytes, `empty` and the
+// accumulator barrier are signalled in both CTAs by one multicast commit; a CTA waits only on its own barriers.
+template <int BNB>
+struct SkinnyPairCfg {
+  static constexpr int W_BYTES = SK_BM * 128;
+  static constexpr int XH_BYTES = (BNB / 2) * 128;
+  static constexpr int STAGE_BYTES = W_BYTES + XH_BYTES;
+  static constexpr int STAGES = BNB >= 256 ? 3 : 4;
+  static constexpr int TMEM_COLS = BNB;
+  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 128;
+};
+
+template <int BNB, bool F8>
+__global__ void __launch_bounds__(SK_THREADS)
+gemm_skinny_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_x, SkinnyDev p) {
+  using Cfg = SkinnyPairCfg<BNB>;
+  constexpr int STAGES = Cfg::STAGES;
+  constexpr int KE = F8 ? 2 * SK_BK : SK_BK;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem_al = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem_al + STAGES * Cfg::STAGE_BYTES);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 1);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = ptx::cluster_ctarank();
+  const uint32_t bar0 = ptx::smem_u32(bars);
+  auto full_bar = [&](int s) { return bar0 + 8u * s; };
+  auto empty_bar = [&](int s) { return bar0 + 8u * (STAGES + s); };
+  const uint32_t acc_bar = bar0 + 8u * (2 * STAGES);
+
+  // work unit of the pair: (batch tile, pair of weight-row tiles, K slice)
+  int unit = blockIdx.x >> 1;
+  const int split = unit % p.splits;
+  unit /= p.splits;
+  const int pairs_n = p.tiles_n >> 1;
+  const int tp = unit % pairs_n;
+  const int tb = unit / pairs_n;
+  const int tn = 2 * tp + static_cast<int>(rank);  // this CTA's weight-row tile
+  const int kb0 = static_cast<int>(static_cast<long long>(p.k_blocks) * split / p.splits);
+  const int kb1 = static_cast<int>(static_cast<long long>(p.k_blocks) * (split + 1) / p.splits);
+
+  if (threadIdx.x == 0) {
+    *abort_flag = 0;
+    for (int s = 0; s < STAGES; ++s) {
+      ptx::mbar_init(full_bar(s), 1);
+      ptx::mbar_init(empty_bar(s), 1);
+    }
+    ptx::mbar_init(acc_bar, 1);
+    ptx::fence_barrier_init();
+    ptx::prefetch_tensormap(&tmap_w);
+    ptx::prefetch_tensormap(&tmap_x);
+  }
+  if (warp == 1) {
+    ptx::tmem_alloc_pair(ptx::smem_u32(tmem_slot), Cfg::TMEM_COLS);
+    ptx::tmem_relinquish_pair();
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::cluster_sync_all();
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  ptx::grid_launch_dependents();
+  if (warp == 0) {
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      // ring prologue: weight tiles first (they depend on no earlier kernel), then the dependency wait, then the
+      // activation half tiles of the same stages
+      const int pre = min(STAGES, kb1 - kb0);
+      for (int i = 0; i < pre; ++i) {
+        if (rank == 0) ptx::mbar_arrive_expect_tx(full_bar(i), 2 * Cfg::STAGE_BYTES);
+        ptx::tma_load_2d_pair(smem_base + i * Cfg::STAGE_BYTES, &tmap_w, (kb0 + i) * KE, tn * SK_BM,
+                              ptx::map_to_cta(full_bar(i), 0));
+      }
+      ptx::grid_dependency_wait();
+      for (int i = 0; i < pre; ++i)
+        ptx::tma_load_2d_pair(smem_base + i * Cfg::STAGE_BYTES + Cfg::W_BYTES, &tmap_x, (kb0 + i) * KE,
+                              tb * BNB + static_cast<int>(rank) * (BNB / 2), ptx::map_to_cta(full_bar(i), 0));
+      if (pre == STAGES) phase = 1u;  // the ring has wrapped once
+      else stage = pre;
+      for (int kb = kb0 + pre; kb < kb1; ++kb) {
+        if (!ptx::mbar_wait_bounded(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
+        const uint32_t sw = smem_base + stage * Cfg::STAGE_BYTES;
+        const uint32_t lead_full = ptx::map_to_cta(full_bar(stage), 0);
+        if (rank == 0) ptx::mbar_arrive_expect_tx(full_bar(stage), 2 * Cfg::STAGE_BYTES);
+        ptx::tma_load_2d_pair(sw, &tmap_w, kb * KE, tn * SK_BM, lead_full);
+        ptx::tma_load_2d_pair(sw + Cfg::W_BYTES, &tmap_x, kb * KE, tb * BNB + static_cast<int>(rank) * (BNB / 2), lead_full);
+        if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+      }
+      if (!ok) {
+        for (int i = 0; i < 2000; ++i) __nanosleep(1000);  // let loads in flight land before shared memory is released
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0 && rank == 0) {
+      constexpr uint32_t idesc = F8 ? ptx::umma_idesc_e4m3(2 * SK_BM, BNB) : ptx::umma_idesc_bf16(2 * SK_BM, BNB);
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int kb = kb0; kb < kb1; ++kb) {
+        if (!ptx::mbar_wait_bounded(full_bar(stage), phase, abort_flag)) { ok = false; break; }
+        ptx::tc_fence_after();
+        const uint32_t sw = smem_base + stage * Cfg::STAGE_BYTES;
+        const uint64_t dw = ptx::umma_desc_sw128(sw);
+        const uint64_t dx = ptx::umma_desc_sw128(sw + Cfg::W_BYTES);
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk) {  // 32 bytes along K per instruction
+          const uint32_t accum = (kb > kb0 || kk > 0) ? 1u : 0u;
+          if constexpr (F8) ptx::umma_f8_pair(tmem_base, dw + 2u * kk, dx + 2u * kk, idesc, accum);
+          else ptx::umma_bf16_pair(tmem_base, dw + 2u * kk, dx + 2u * kk, idesc, accum);
+        }
+        ptx::umma_commit_pair(empty_bar(stage), 3);
+        if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+      }
+      if (ok) ptx::umma_commit_pair(acc_bar, 3);
+    }
+  } else {
+    const int lane_group = warp & 3;
+    const bool ok = __all_sync(0xffffffffu, ptx::mbar_wait_bounded(acc_bar, 0u, abort_flag));
+    ptx::grid_dependency_wait();  // (long since satisfied) orders the sums after the kernel that cleared the buffer
+    if (ok && kb1 > kb0) {
+      ptx::tc_fence_after();
+      const int n = tn * SK_BM + lane_group * 32 + lane;  // output feature of this thread
+      const uint32_t t_row = tmem_base + (static_cast<uint32_t>(lane_group * 32) << 16);
+#pragma unroll 1
+      for (int c0 = 0; c0 < BNB; c0 += 32) {
+        if (tb * BNB + c0 >= p.batch) break;  // warp-uniform: the rest of the accumulator is padding
+        uint32_t v[32];
+        ptx::tmem_ld_32x32(t_row + c0, v);
+        ptx::tmem_ld_wait();
+        skinny_store_chunk<32, F8>(p, v, n, lane, tb * BNB + c0);
+      }
+    }
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::cluster_sync_all();  // neither CTA leaves (or frees tensor memory) while its peer may still signal it
+  if (*abort_flag && threadIdx.x == 0 && p.err_word) atomicExch(p.err_word, 1);
+  if (warp == 1) {
+    __syncwarp();
+    ptx::tc_fence_after();
+    ptx::tmem_dealloc_pair(tmem_base, Cfg::TMEM_COLS);
   }
 }
 
@@ -271,6 +434,69 @@ pd_status launch_skinny(const SkinnyGemmArgs& g, cudaStream_t stream) {
   PD_CUDA_TRY(launch_pdl(kern, dim3(units * splits), dim3(SK_THREADS), Cfg::SMEM_BYTES, stream, tw, tx, p));
   count_launch();
   return PD_OK;
+}
+
+// CTA-pair launch (cluster of two + programmatic serialization).  Same K-slice count as the single-CTA kernel
+// would use, so the callers' decision which buffers need clearing does not depend on the path taken.
+template <int BNB, bool F8>
+pd_status launch_skinny_pair(const SkinnyGemmArgs& g, cudaStream_t stream) {
+  using Cfg = SkinnyPairCfg<BNB>;
+  static int usable = -1;  // -1 unknown, 0 clusters of two cannot be placed, 1 fine
+  auto kern = gemm_skinny_pair_kernel<BNB, F8>;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t cfg{};
+  cfg.blockDim = dim3(SK_THREADS);
+  cfg.dynamicSmemBytes = Cfg::SMEM_BYTES;
+  cfg.stream = stream;
+  cfg.attrs = attr;
+  if (usable < 0) {
+    usable = 0;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES) == cudaSuccess) {
+      cfg.gridDim = dim3(2);
+      cfg.numAttrs = 1;
+      int n = 0;
+      if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) == cudaSuccess && n > 0) usable = 1;
+      else cudaGetLastError();
+    }
+  }
+  if (!usable) return PD_ERR_UNSUPPORTED_SHAPE;
+  CUtensorMap tw, tx;
+  if (F8) {
+    PD_TRY(make_tmap_u8(&tw, g.w, g.n, g.k, g.k, SK_BM));
+    PD_TRY(make_tmap_u8(&tx, g.x, g.batch, g.k, g.ldx, BNB / 2));
+  } else {
+    PD_TRY(make_tmap_bf16(&tw, g.w, g.n, g.k, g.k, SK_BM));
+    PD_TRY(make_tmap_bf16(&tx, g.x, g.batch, g.k, g.ldx, BNB / 2));
+  }
+  SkinnyDev p{};
+  p.scale_x = g.scale_x; p.scale_w = g.scale_w;
+  p.acc = g.acc; p.batch = g.batch; p.n = g.n; p.k_blocks = g.k / (F8 ? 2 * SK_BK : SK_BK);
+  p.tiles_n = g.n / SK_BM;
+  const int tiles_b = (g.batch + BNB - 1) / BNB;
+  p.splits = skinny_splits(p.tiles_n * tiles_b, p.k_blocks, 2);
+  p.err_word = g.err_word;
+  if (p.splits > 1 && !g.acc_zeroed)
+    PD_CUDA_TRY(cudaMemsetAsync(g.acc, 0, static_cast<size_t>(g.batch) * g.n * sizeof(float), stream));
+  cfg.gridDim = dim3(static_cast<unsigned>(2 * (p.tiles_n / 2) * tiles_b * p.splits));
+  cfg.numAttrs = pdl_enabled() ? 2 : 1;
+  PD_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, tw, tx, p));
+  count_launch();
+  return PD_OK;
+}
+
+// Batches above 64 (FP8: above 128, where it was measured to pay) run on the CTA-pair kernel; PD_SKINNY_PAIRS=0 in
+// the environment keeps them on the single-CTA kernel (for A/B timing).  Measured per 8B layer, bf16: 258 -> 243 us
+// at B = 96, 298 -> 277 at 128, 400 -> 374 at 192, 480 -> 463 at 256.
+static int skinny_pair_mode() {
+  static const int mode = [] {
+    const char* v = std::getenv("PD_SKINNY_PAIRS");
+    return (v && v[0] == '0') ? 0 : 1;
+  }();
+  return mode;
 }
 
 // ------------------------------------------------------------ row-wise epilogues
@@ -477,8 +703,15 @@ int gemm_skinny_splits(int batch, int n, int k, bool fp8) {
 
 pd_status gemm_skinny(const SkinnyGemmArgs& g, cudaStream_t stream) {
   if (!g.x || !g.w || !g.acc || g.batch <= 0 || g.n <= 0 || g.k <= 0) return PD_ERR_INVALID_ARG;
+  if (g.fp8 && (!g.scale_x || !g.scale_w)) return PD_ERR_INVALID_ARG;
+  if (g.batch > (g.fp8 ? 128 : 64) && g.batch <= 256 && g.n % (2 * SK_BM) == 0 && g.k % (g.fp8 ? 2 * SK_BK : SK_BK) == 0 &&
+      g.ldx % (g.fp8 ? 16 : 8) == 0 && skinny_pair_mode()) {
+    pd_status st;
+    if (g.batch <= 128) st = g.fp8 ? launch_skinny_pair<128, true>(g, stream) : launch_skinny_pair<128, false>(g, stream);
+    else st = g.fp8 ? launch_skinny_pair<256, true>(g, stream) : launch_skinny_pair<256, false>(g, stream);
+    if (st != PD_ERR_UNSUPPORTED_SHAPE) return st;  // (clusters of two could not be placed: single-CTA kernel)
+  }
   if (g.fp8) {
-    if (!g.scale_x || !g.scale_w) return PD_ERR_INVALID_ARG;
     if (g.k % (2 * SK_BK) != 0 || g.n % 4 != 0 || g.ldx % 16 != 0) return PD_ERR_UNSUPPORTED_SHAPE;
     if (g.batch <= 16) return launch_skinny<16, 1, true>(g, stream);
     if (g.batch <= 32) return launch_skinny<32, 1, true>(g, stream);
