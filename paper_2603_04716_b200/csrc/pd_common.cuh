@@ -135,10 +135,15 @@ struct SkinnyGemmArgs {
   int fp8;                 // 1: x and w hold E4M3 codes (one byte per element); sums are scaled by scale_x[b] * scale_w[n]
   const float* scale_x;    // [B]
   const float* scale_w;    // [N]
+  // Not NULL: w is a gate/up matrix (64 gate rows, 64 up rows, alternating) and the kernel writes
+  // silu(gate) * up as bf16 [B, N/2] here instead of the fp32 sums.  Only where gemm_skinny_fuses_swiglu() holds.
+  bf16* swiglu_out;
 };
 pd_status gemm_skinny(const SkinnyGemmArgs& g, cudaStream_t stream);
 // Number of K slices gemm_skinny will use (1: plain stores, acc need not be zero).
 int gemm_skinny_splits(int batch, int n, int k, bool fp8 = false);
+// True when the projection is not split along K for this batch, so that SwiGLU can be applied in its epilogue.
+bool gemm_skinny_fuses_swiglu(int batch, int n, int k, bool fp8 = false);
 // Row-wise kernels that turn the fp32 sums into the layer's stored tensors.
 // Every row-wise kernel can also clear the fp32 sums of a LATER projection (zero_ptr[batch, zero_cols], NULL to
 // skip): the buffer is idle while the kernel runs, and the projection then needs no memset of its own.

@@ -46,6 +46,8 @@ struct SkinnyDev {
   int* err_word;
   const float* scale_x;  // FP8 operands: per-row scales of X [B] and of W [N]
   const float* scale_w;
+  bf16* swiglu_out;      // not NULL (only with splits == 1): W is the gate/up matrix, write silu(gate) * up here
+  int swiglu_ld;         // its row pitch (= number of SwiGLU features)
 };
 
 // One chunk of CH accumulator columns (batch rows b0 ..) of the thread that owns output feature n -> the fp32
@@ -93,6 +95,67 @@ __device__ __forceinline__ void skinny_store_chunk(const SkinnyDev& p, uint32_t 
         }
       }
     }
+}
+
+// Named barrier 1 over the 128 epilogue threads (warps 2-5) and its AND-reduction form.
+__device__ __forceinline__ void epi_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+__device__ __forceinline__ bool epi_all(bool pred) {
+  uint32_t r;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "setp.ne.b32 p, %1, 0;\n\t"
+      "bar.red.and.pred q, 1, 128, p;\n\t"
+      "selp.u32 %0, 1, 0, q;\n\t}"
+      : "=r"(r) : "r"(static_cast<uint32_t>(pred)) : "memory");
+  return r != 0;
+}
+
+// SwiGLU straight from the accumulator of an unsplit gate/up tile: its 128 weight rows are 64 gate rows followed by
+// the 64 up rows of the same features, i.e. tensor-memory lanes r and r + 64, which belong to different warps.  The
+// up warps pass their chunk through shared memory (the operand stages are idle by now; two buffers so one barrier
+// per chunk suffices), the gate warps compute silu(gate) * up and store bf16: a warp writes 32 consecutive features
+// of one batch row.  Executed by all four epilogue warps; `ok` is made uniform over them first.
+template <int BNB, bool F8>
+__device__ __forceinline__ void skinny_swiglu_tile(const SkinnyDev& p, uint32_t t_row, int tn, int tb, int lane_group,
+                                                   int lane, float* xbuf, bool ok) {
+  if (!epi_all(ok)) return;
+  constexpr int CH = BNB < 32 ? BNB : 32;
+  const int r = lane_group * 32 + lane;   // weight row inside the tile
+  const int n = tn * SK_BM + r;
+  const int f = tn * 64 + (r & 63);       // SwiGLU feature of this row
+  float sw = 1.f;
+  if constexpr (F8) sw = n < p.n ? __ldg(p.scale_w + n) : 0.f;
+  int it = 0;
+#pragma unroll 1
+  for (int c0 = 0; c0 < BNB; c0 += CH, ++it) {
+    const int b0 = tb * BNB + c0;
+    if (b0 >= p.batch) break;  // uniform: the rest of the accumulator is padding
+    uint32_t v[32];
+    if constexpr (CH == 32) ptx::tmem_ld_32x32(t_row + c0, v);
+    else ptx::tmem_ld_32x16(t_row + c0, v);
+    ptx::tmem_ld_wait();
+    if constexpr (F8) {
+#pragma unroll
+      for (int j = 0; j < CH; ++j)
+        v[j] = __float_as_uint(__uint_as_float(v[j]) * (sw * (b0 + j < p.batch ? __ldg(p.scale_x + b0 + j) : 0.f)));
+    }
+    float* buf = xbuf + (it & 1) * (64 * 33);
+    if (lane_group >= 2) {
+#pragma unroll
+      for (int j = 0; j < CH; ++j) buf[(r - 64) * 33 + j] = __uint_as_float(v[j]);
+    }
+    epi_sync();
+    if (lane_group < 2 && n < p.n) {
+#pragma unroll
+      for (int j = 0; j < CH; ++j) {
+        if (b0 + j < p.batch) {
+          const float g = __uint_as_float(v[j]);
+          const float u = buf[r * 33 + j];
+          p.swiglu_out[static_cast<size_t>(b0 + j) * p.swiglu_ld + f] = __float2bfloat16(g / (1.f + __expf(-g)) * u);
+        }
+      }
+    }
+  }
 }
 
 // F8: both operands are E4M3 codes (a 128-byte shared-memory row then holds 128 K elements, one MMA covers 32)
@@ -212,7 +275,11 @@ gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
     const int lane_group = warp & 3;
     const bool ok = __all_sync(0xffffffffu, ptx::mbar_wait_bounded(acc_bar, 0u, abort_flag));
     ptx::grid_dependency_wait();  // (long since satisfied) orders the sums after the kernel that cleared the buffer
-    if (ok && kb1 > kb0) {
+    if (MT == 1 && p.swiglu_out) {  // block-uniform
+      ptx::tc_fence_after();
+      skinny_swiglu_tile<BNB, F8>(p, tmem_base + (static_cast<uint32_t>(lane_group * 32) << 16), tn, tb, lane_group, lane,
+                                  reinterpret_cast<float*>(smem_al), ok && kb1 > kb0);
+    } else if (ok && kb1 > kb0) {
       ptx::tc_fence_after();
       constexpr int CH = BNB < 32 ? BNB : 32;
 #pragma unroll 1
@@ -369,7 +436,11 @@ gemm_skinny_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid
     const int lane_group = warp & 3;
     const bool ok = __all_sync(0xffffffffu, ptx::mbar_wait_bounded(acc_bar, 0u, abort_flag));
     ptx::grid_dependency_wait();  // (long since satisfied) orders the sums after the kernel that cleared the buffer
-    if (ok && kb1 > kb0) {
+    if (p.swiglu_out) {  // block-uniform
+      ptx::tc_fence_after();
+      skinny_swiglu_tile<BNB, F8>(p, tmem_base + (static_cast<uint32_t>(lane_group * 32) << 16), tn, tb, lane_group, lane,
+                                  reinterpret_cast<float*>(smem_al), ok && kb1 > kb0);
+    } else if (ok && kb1 > kb0) {
       ptx::tc_fence_after();
       const int n = tn * SK_BM + lane_group * 32 + lane;  // output feature of this thread
       const uint32_t t_row = tmem_base + (static_cast<uint32_t>(lane_group * 32) << 16);
@@ -429,6 +500,10 @@ pd_status launch_skinny(const SkinnyGemmArgs& g, cudaStream_t stream) {
   const int splits = skinny_splits(units, p.k_blocks, Cfg::BLOCKS_PER_SM);  // (k_blocks already counts FP8 stages)
   p.splits = splits;
   p.err_word = g.err_word;
+  if (g.swiglu_out) {
+    if (splits != 1 || tiles_b != 1 || MT != 1 || g.n % SK_BM != 0) return PD_ERR_UNSUPPORTED_SHAPE;
+    p.swiglu_out = g.swiglu_out; p.swiglu_ld = g.n / 2;
+  }
   if (splits > 1 && !g.acc_zeroed)
     PD_CUDA_TRY(cudaMemsetAsync(g.acc, 0, static_cast<size_t>(g.batch) * g.n * sizeof(float), stream));
   PD_CUDA_TRY(launch_pdl(kern, dim3(units * splits), dim3(SK_THREADS), Cfg::SMEM_BYTES, stream, tw, tx, p));
@@ -479,6 +554,10 @@ pd_status launch_skinny_pair(const SkinnyGemmArgs& g, cudaStream_t stream) {
   const int tiles_b = (g.batch + BNB - 1) / BNB;
   p.splits = skinny_splits(p.tiles_n * tiles_b, p.k_blocks, 2);
   p.err_word = g.err_word;
+  if (g.swiglu_out) {
+    if (p.splits != 1 || tiles_b != 1) return PD_ERR_UNSUPPORTED_SHAPE;
+    p.swiglu_out = g.swiglu_out; p.swiglu_ld = g.n / 2;
+  }
   if (p.splits > 1 && !g.acc_zeroed)
     PD_CUDA_TRY(cudaMemsetAsync(g.acc, 0, static_cast<size_t>(g.batch) * g.n * sizeof(float), stream));
   cfg.gridDim = dim3(static_cast<unsigned>(2 * (p.tiles_n / 2) * tiles_b * p.splits));
@@ -694,6 +773,11 @@ __global__ void __launch_bounds__(256) skinny_swiglu_kernel(const float* __restr
 }
 
 }  // namespace
+
+bool gemm_skinny_fuses_swiglu(int batch, int n, int k, bool fp8) {
+  static const bool off = [] { const char* v = std::getenv("PD_FUSE_SWIGLU"); return v && v[0] == '0'; }();
+  return !off && batch <= 256 && n % SK_BM == 0 && gemm_skinny_splits(batch, n, k, fp8) == 1;
+}
 
 int gemm_skinny_splits(int batch, int n, int k, bool fp8) {
   const int bnb = skinny_bnb(batch);

@@ -275,6 +275,9 @@ pd_status decode_impl(pd_layer* L, const bf16* x, bf16* out, const int32_t* kv_l
   float* z_o = pd::gemm_skinny_splits(B, c.d_model, hq, f8) > 1 ? acc_o : nullptr;
   float* z_gu = pd::gemm_skinny_splits(B, n_gu, c.d_model, f8) > 1 ? acc_gu : nullptr;
   float* z_down = pd::gemm_skinny_splits(B, c.d_model, c.d_ff, f8) > 1 ? acc_down : nullptr;
+  // Gate/up is not split along K at these shapes: SwiGLU then runs in its epilogue (no fp32 round trip, one launch
+  // fewer) and the buffer of the down projection is cleared one kernel earlier.
+  const bool fuse_swiglu = pd::gemm_skinny_fuses_swiglu(B, n_gu, c.d_model, f8);
   // FP8 mode: a row-wise quantiser in front of every projection (same programmatic-serialization chain)
   uint8_t* q_act = ws + w.q_act;
   float* s_act = reinterpret_cast<float*>(ws + w.s_act);
@@ -314,15 +317,18 @@ pd_status decode_impl(pd_layer* L, const bf16* x, bf16* out, const int32_t* kv_l
     g.x = attn_o; g.w = L->w_o; g.acc = acc_o; g.n = c.d_model; g.k = hq; g.ldx = hq;
     PD_TRY(fp8_in(g, L->q_o, L->s_o, false));
     PD_TRY(pd::gemm_skinny(g, st));
-    PD_TRY(pd::launch_skinny_residual(acc_o, x, resid, L->g_mlp, norm, B, c.d_model, c.rms_eps, z_gu, n_gu, st,
+    PD_TRY(pd::launch_skinny_residual(acc_o, x, resid, L->g_mlp, norm, B, c.d_model, c.rms_eps,
+                                      fuse_swiglu ? z_down : z_gu, fuse_swiglu ? c.d_model : n_gu, st,
                                       f8 ? q_act : nullptr, f8 ? s_act : nullptr));
   }
   {
     pd::TraceScope ts(PD_K_GEMM_GATE_UP, st);
     g.x = norm; g.w = L->w_gu; g.acc = acc_gu; g.n = n_gu; g.k = c.d_model; g.ldx = c.d_model;
     PD_TRY(fp8_in(g, L->q_gu, L->s_gu, true));
+    g.swiglu_out = fuse_swiglu ? act : nullptr;
     PD_TRY(pd::gemm_skinny(g, st));
-    PD_TRY(pd::launch_skinny_swiglu(acc_gu, act, B, c.d_ff, z_down, c.d_model, st));
+    g.swiglu_out = nullptr;
+    if (!fuse_swiglu) PD_TRY(pd::launch_skinny_swiglu(acc_gu, act, B, c.d_ff, z_down, c.d_model, st));
   }
   {
     pd::TraceScope ts(PD_K_GEMM_DOWN, st);
