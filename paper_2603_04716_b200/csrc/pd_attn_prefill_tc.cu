@@ -107,6 +107,10 @@ prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
   __syncthreads();
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  // Programmatic dependent launch: the set-up above may overlap the tail of the QKV projection; q and the cache
+  // are read, and the output written, only after it has completed.
+  ptx::grid_launch_dependents();
+  ptx::grid_dependency_wait();
 
   if (warp == 0) {
     // ---------------------------------------------------------------- producer
@@ -376,9 +380,8 @@ pd_status launch_hd(const PrefillAttnArgs& a, int* err_word, cudaStream_t s) {
   p.n_q_heads = a.n_q_heads; p.n_kv_heads = a.n_kv_heads; p.len_cap = a.len_cap; p.batch_cap = a.batch_cap;
   p.err_word = err_word;
   dim3 grid((a.max_len + 2 * TQ - 1) / (2 * TQ), a.n_q_heads, a.n_req);
-  kern<<<grid, ATT_THREADS, Cfg::SMEM_BYTES, s>>>(tq, tk, tv, p);
+  PD_CUDA_TRY(launch_pdl(kern, grid, dim3(ATT_THREADS), Cfg::SMEM_BYTES, s, tq, tk, tv, p));
   count_launch();
-  PD_CUDA_TRY(cudaGetLastError());
   return PD_OK;
 }
 

@@ -187,9 +187,9 @@ pd_status launch_rmsnorm(const bf16* x, const bf16* gain, bf16* y, int rows, int
                          uint8_t* q_out, float* s_out) {
   if (rows == 0) return PD_OK;
   if (d % 8 != 0 || d > RMS_THREADS * RMS_MAX_CHUNKS * 8 || (q_out && !s_out)) return PD_ERR_UNSUPPORTED_SHAPE;
-  rmsnorm_kernel<<<rows, RMS_THREADS, 0, s>>>(x, gain, y, d, eps, nullptr, 0, q_out, s_out);
+  float* no_zero = nullptr;
+  PD_CUDA_TRY(launch_pdl(rmsnorm_kernel, dim3(rows), dim3(RMS_THREADS), 0, s, x, gain, y, d, eps, no_zero, 0, q_out, s_out));
   count_launch();
-  PD_CUDA_TRY(cudaGetLastError());
   return PD_OK;
 }
 

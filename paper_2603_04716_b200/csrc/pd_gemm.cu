@@ -368,12 +368,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
   const int n_units = p.n_units;
   const int k_blocks = p.k / KE;
 
+  // Programmatic dependent launch: the next kernel of the stream may start its own set-up now; this one touches
+  // global memory (operand loads, epilogue reads and writes) only after the kernels before it have completed.
+  ptx::grid_launch_dependents();
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
     if (lane == 0) {
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
+      ptx::grid_dependency_wait();
       for (int unit = blockIdx.x; unit < n_units && ok; unit += gridDim.x) {
         const UnitInfo ui = unit_info(unit, p.main_tiles, k_blocks, p.tail_halves);
         int tm, tn;
@@ -439,6 +443,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     int acc = 0;
     uint32_t acc_phase = 0;
     bool ok = true;
+    ptx::grid_dependency_wait();
     for (int unit = blockIdx.x; unit < n_units && ok; unit += gridDim.x) {
       const UnitInfo ui = unit_info(unit, p.main_tiles, k_blocks, p.tail_halves);
       int tm, tn;
@@ -579,11 +584,13 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
                                   // independent 128-column halves each (tail_halves), see unit_info
   const int group2 = max(1, p.raster_group >> 1);
 
+  ptx::grid_launch_dependents();  // (see gemm_tc_kernel)
   if (warp == 0) {
     if (lane == 0) {
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
+      ptx::grid_dependency_wait();
       for (int unit = pair_id; unit < n_units && ok; unit += n_pairs) {
         const UnitInfo ui = unit_info(unit, p.main_tiles, k_blocks, 1);
         int tm2, tn;
@@ -643,6 +650,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
     const int lane_group = warp & 3;
     int acc = 0;
     uint32_t acc_phase = 0;
+    ptx::grid_dependency_wait();
     for (int unit = pair_id; unit < n_units; unit += n_pairs) {
       const UnitInfo ui = unit_info(unit, p.main_tiles, k_blocks, 1);
       int tm2, tn;
@@ -738,9 +746,8 @@ pd_status launch_tc(const GemmArgs& g, cudaStream_t stream) {
     }
   }
   const int grid = p.n_units < sms ? p.n_units : sms;
-  kern<<<grid, GEMM_THREADS, Cfg::SMEM_BYTES, stream>>>(ta, tb, p);
+  PD_CUDA_TRY(launch_pdl(kern, dim3(grid), dim3(GEMM_THREADS), Cfg::SMEM_BYTES, stream, ta, tb, p));
   count_launch();
-  PD_CUDA_TRY(cudaGetLastError());
   return PD_OK;
 }
 
@@ -808,11 +815,13 @@ pd_status launch_tc_pair(const GemmArgs& g, cudaStream_t stream) {
   cfg.blockDim = dim3(GEMM_THREADS);
   cfg.dynamicSmemBytes = P2_SMEM_BYTES;
   cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = pdl_enabled() ? 2 : 1;
   PD_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, ta, tb, tbh, p));
   count_launch();
   return PD_OK;
