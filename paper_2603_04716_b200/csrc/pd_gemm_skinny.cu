@@ -54,47 +54,47 @@ struct SkinnyDev {
 // buffer: vector store when K is not split, vector reduction otherwise; FP8 sums are scaled on the way.
 template <int CH, bool F8>
 __device__ __forceinline__ void skinny_store_chunk(const SkinnyDev& p, uint32_t (&v)[32], int n, int lane, int b0) {
-    // 4 x 4 transposes across groups of four lanes: afterwards lane 4q + r holds, for batch column
-    // c0 + 4m + r, the four consecutive features 4q .. 4q + 3 in v[4m .. 4m + 3], i.e. 16 contiguous bytes
-    // of the output row, so one vector store / vector reduction replaces four scalar ones (scalar fp32
-    // reductions into L2 were measured four times slower per byte).
-    const int r4 = lane & 3;
+  // 4 x 4 transposes across groups of four lanes: afterwards lane 4q + r holds, for batch column
+  // c0 + 4m + r, the four consecutive features 4q .. 4q + 3 in v[4m .. 4m + 3], i.e. 16 contiguous bytes
+  // of the output row, so one vector store / vector reduction replaces four scalar ones (scalar fp32
+  // reductions into L2 were measured four times slower per byte).
+  const int r4 = lane & 3;
+#pragma unroll
+  for (int m = 0; m < CH; m += 4) {
+#pragma unroll
+    for (int s2 = 0; s2 < 4; s2 += 2) {
+      const uint32_t send = (r4 & 1) ? v[m + s2] : v[m + s2 + 1];
+      const uint32_t recv = __shfl_xor_sync(0xffffffffu, send, 1);
+      if (r4 & 1) v[m + s2] = recv; else v[m + s2 + 1] = recv;
+    }
+#pragma unroll
+    for (int s2 = 0; s2 < 2; ++s2) {
+      const uint32_t send = (r4 & 2) ? v[m + s2] : v[m + s2 + 2];
+      const uint32_t recv = __shfl_xor_sync(0xffffffffu, send, 2);
+      if (r4 & 2) v[m + s2] = recv; else v[m + s2 + 2] = recv;
+    }
+  }
+  const int n4 = n - r4;  // first of this lane's four features (n is a multiple of 4 per group of lanes)
+  if (n4 < p.n) {
+    float4 sw4 = make_float4(1.f, 1.f, 1.f, 1.f);
+    if constexpr (F8) sw4 = __ldg(reinterpret_cast<const float4*>(p.scale_w + n4));
 #pragma unroll
     for (int m = 0; m < CH; m += 4) {
-#pragma unroll
-      for (int s2 = 0; s2 < 4; s2 += 2) {
-        const uint32_t send = (r4 & 1) ? v[m + s2] : v[m + s2 + 1];
-        const uint32_t recv = __shfl_xor_sync(0xffffffffu, send, 1);
-        if (r4 & 1) v[m + s2] = recv; else v[m + s2 + 1] = recv;
-      }
-#pragma unroll
-      for (int s2 = 0; s2 < 2; ++s2) {
-        const uint32_t send = (r4 & 2) ? v[m + s2] : v[m + s2 + 2];
-        const uint32_t recv = __shfl_xor_sync(0xffffffffu, send, 2);
-        if (r4 & 2) v[m + s2] = recv; else v[m + s2 + 2] = recv;
-      }
-    }
-    const int n4 = n - r4;  // first of this lane's four features (n is a multiple of 4 per group of lanes)
-    if (n4 < p.n) {
-      float4 sw4 = make_float4(1.f, 1.f, 1.f, 1.f);
-      if constexpr (F8) sw4 = __ldg(reinterpret_cast<const float4*>(p.scale_w + n4));
-#pragma unroll
-      for (int m = 0; m < CH; m += 4) {
-        const int b = b0 + m + r4;
-        if (b < p.batch) {
-          if constexpr (F8) {
-            const float sx = __ldg(p.scale_x + b);
-            v[m] = __float_as_uint(__uint_as_float(v[m]) * (sx * sw4.x));
-            v[m + 1] = __float_as_uint(__uint_as_float(v[m + 1]) * (sx * sw4.y));
-            v[m + 2] = __float_as_uint(__uint_as_float(v[m + 2]) * (sx * sw4.z));
-            v[m + 3] = __float_as_uint(__uint_as_float(v[m + 3]) * (sx * sw4.w));
-          }
-          float* dst = p.acc + static_cast<size_t>(b) * p.n + n4;
-          if (p.splits > 1) ptx::red_add_v4_f32(dst, v[m], v[m + 1], v[m + 2], v[m + 3]);
-          else *reinterpret_cast<uint4*>(dst) = make_uint4(v[m], v[m + 1], v[m + 2], v[m + 3]);
+      const int b = b0 + m + r4;
+      if (b < p.batch) {
+        if constexpr (F8) {
+          const float sx = __ldg(p.scale_x + b);
+          v[m] = __float_as_uint(__uint_as_float(v[m]) * (sx * sw4.x));
+          v[m + 1] = __float_as_uint(__uint_as_float(v[m + 1]) * (sx * sw4.y));
+          v[m + 2] = __float_as_uint(__uint_as_float(v[m + 2]) * (sx * sw4.z));
+          v[m + 3] = __float_as_uint(__uint_as_float(v[m + 3]) * (sx * sw4.w));
         }
+        float* dst = p.acc + static_cast<size_t>(b) * p.n + n4;
+        if (p.splits > 1) ptx::red_add_v4_f32(dst, v[m], v[m + 1], v[m + 2], v[m + 3]);
+        else *reinterpret_cast<uint4*>(dst) = make_uint4(v[m], v[m + 1], v[m + 2], v[m + 3]);
       }
     }
+  }
 }
 
 // Named barrier 1 over the 128 epilogue threads (warps 2-5) and its AND-reduction form.
