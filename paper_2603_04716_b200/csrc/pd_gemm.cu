@@ -200,22 +200,39 @@ __device__ __forceinline__ void epilogue_tile(const GemmDev& p, int role, int n_
   if (role == 1 || !ok) {
     // nothing more to do for this unit
   } else if constexpr (EPI == EPI_STORE || EPI == EPI_RESIDUAL) {
+    // The residual of the NEXT chunk is requested before the current one is processed: a thread reads its own row
+    // (16 bytes per load, a different line for every lane), and without the lookahead that latency would be
+    // exposed once per chunk, which is what bounded the short-K projections.
+    uint4 r_next[4];
+    auto load_res = [&](int c0, uint4 (&dst)[4]) {
+      const bf16* rrow = p.r + static_cast<size_t>(row) * p.ldr + col_base + c0;
+#pragma unroll
+      for (int q = 0; q < 4; ++q)
+        dst[q] = (row < p.m && col_base + c0 + q * 8 < p.n) ? __ldcg(reinterpret_cast<const uint4*>(rrow + q * 8))
+                                                            : make_uint4(0u, 0u, 0u, 0u);
+    };
+    if constexpr (EPI == EPI_RESIDUAL) load_res(0, r_next);
 #pragma unroll 1
     for (int c0 = 0; c0 < acc_cols; c0 += 32) {
+      uint4 r_cur[4];
+      if constexpr (EPI == EPI_RESIDUAL) {
+#pragma unroll
+        for (int q = 0; q < 4; ++q) r_cur[q] = r_next[q];
+        if (c0 + 32 < acc_cols) load_res(c0 + 32, r_next);
+      }
       uint32_t v[32];
       load_acc(c0, v);
       const int col = col_base + c0;
       if (row < p.m) {
         bf16* crow = p.c + static_cast<size_t>(row) * p.ldc + col;
-        const bf16* rrow = (EPI == EPI_RESIDUAL) ? p.r + static_cast<size_t>(row) * p.ldr + col : nullptr;
 #pragma unroll
         for (int j = 0; j < 32; j += 8) {
           if (col + j < p.n) {
             float f[8];
 #pragma unroll
             for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(v[j + e]);
-            if (EPI == EPI_RESIDUAL) {
-              const uint4 rr = *reinterpret_cast<const uint4*>(rrow + j);
+            if constexpr (EPI == EPI_RESIDUAL) {
+              const uint4 rr = r_cur[j >> 3];
               f[0] += ptx::bf16_lo(rr.x); f[1] += ptx::bf16_hi(rr.x);
               f[2] += ptx::bf16_lo(rr.y); f[3] += ptx::bf16_hi(rr.y);
               f[4] += ptx::bf16_lo(rr.z); f[5] += ptx::bf16_hi(rr.z);
