@@ -292,12 +292,26 @@ __device__ __forceinline__ void epilogue_tile(const GemmDev& p, int role, int n_
     }
     const int n_heads = rp.n_q_heads + 2 * rp.n_kv_heads;
     const int heads_per_tile = acc_cols / hd;
+    // (cos, sin) of this row's position for 32 rotation pairs at a time: loaded once for all heads of the tile, and
+    // the next 32 pairs are requested before the current ones are used (the loads are private to the thread's row).
+    const bool any_rotate = col_base / hd < rp.n_q_heads + rp.n_kv_heads;  // warp-uniform
+    float4 t_next[16];
+    auto load_tab = [&](int i0, float4 (&dst)[16]) {
+      const float4* tab = reinterpret_cast<const float4*>(rp.rope_tab + static_cast<size_t>(pos) * half + i0);
+#pragma unroll
+      for (int q = 0; q < 16; ++q) dst[q] = row_ok ? __ldg(tab + q) : make_float4(1.f, 0.f, 1.f, 0.f);
+    };
+    if (any_rotate) load_tab(0, t_next);
 #pragma unroll 1
-    for (int hh = 0; hh < heads_per_tile; ++hh) {
-      const int head = col_base / hd + hh;
-      if (head >= n_heads) break;  // warp-uniform
+    for (int i0 = 0; i0 < half; i0 += 32) {
+      float4 t_cur[16];
+#pragma unroll
+      for (int q = 0; q < 16; ++q) t_cur[q] = t_next[q];
+      if (any_rotate && i0 + 32 < half) load_tab(i0 + 32, t_next);
 #pragma unroll 1
-      for (int i0 = 0; i0 < half; i0 += 32) {
+      for (int hh = 0; hh < heads_per_tile; ++hh) {
+        const int head = col_base / hd + hh;
+        if (head >= n_heads) break;  // warp-uniform
         uint32_t lo[32], hi[32];
         load_acc(hh * hd + i0, lo);
         load_acc(hh * hd + half + i0, hi);
@@ -313,7 +327,6 @@ __device__ __forceinline__ void epilogue_tile(const GemmDev& p, int role, int n_
                                   rp.len_cap + pos) * hd;
         }
         const bool rotate = head < rp.n_q_heads + rp.n_kv_heads;
-        const float4* tab = reinterpret_cast<const float4*>(rp.rope_tab + static_cast<size_t>(pos) * half + i0);
 #pragma unroll
         for (int j = 0; j < 32; j += 8) {
           float a[8], b[8];
@@ -322,7 +335,7 @@ __device__ __forceinline__ void epilogue_tile(const GemmDev& p, int role, int n_
           if (rotate) {
 #pragma unroll
             for (int e = 0; e < 8; e += 2) {
-              const float4 cs = tab[(j + e) >> 1];  // (cos, sin) of two consecutive pairs
+              const float4 cs = t_cur[(j + e) >> 1];  // (cos, sin) of two consecutive pairs
               const float a0 = a[e], b0 = b[e], a1 = a[e + 1], b1 = b[e + 1];
               a[e] = a0 * cs.x - b0 * cs.y;      b[e] = b0 * cs.x + a0 * cs.y;
               a[e + 1] = a1 * cs.z - b1 * cs.w;  b[e + 1] = b1 * cs.z + a1 * cs.w;
