@@ -39,8 +39,8 @@ TTFT_SLO, TPOT_SLO, TP_TOTAL = 2.0, 0.050, 2e5
 # one layer (profiles/gemm_tc_prefill_8b_ncu_full.md, profiles/prefill_attn_tc_and_decode_kernels_ncu_full.md).
 # Set an entry to None whenever the kernel changes after the capture.
 NCU_TRAFFIC = {
-    "gemm_tc_kernel": {"bytes_per_launch": 362.1e6, "algorithmic_bytes_per_launch": 238.8e6,
-                       "note": "gemm_tc_pair_kernel, mean over the four prefill projections of a layer (1448.4 MB / 4)"},
+    "gemm_tc_kernel": {"bytes_per_launch": 365.6e6, "algorithmic_bytes_per_launch": 238.8e6,
+                       "note": "gemm_tc_pair_kernel, mean over the four prefill projections of a layer (1462.4 MB / 4)"},
     "decode_attn_kernel": {"bytes_per_launch": 2.1563e9, "algorithmic_bytes_per_launch": 2.1485e9,
                            "note": "B = 256 at KV length 2049; grows in proportion to the KV length"},
 }
