@@ -91,9 +91,9 @@ def run_tiny(quick=False):
             "allocation": _alloc(1e4, 128, 16, 1.0, 0.050, m["prefill_tok_s"], m["batch"], m["tpot_s"])}
 
 
-def run_8b(quick=False):
+def run_8b(quick=False, fp8=False):
     peaks = _peaks()
-    cfg = pd.LayerConfig(**SHAPE_8B, max_pos=4096)
+    cfg = pd.LayerConfig(**SHAPE_8B, max_pos=4096, fp8_projections=fp8)
     nl = 8 if quick else 32
     grid = {}
     for l_in in ([4096] if quick else [1024, 2048, 4096]):
@@ -110,7 +110,7 @@ def run_8b(quick=False):
     for l_in in ([4096] if quick else [1024, 2048, 4096]):
         # sequential requests (n_req = 1) are what the M/M/1 model assumes; batched ones are reported above
         alloc[str(l_in)] = _alloc(2e5, l_in, 256, 2.0, 0.050, grid[f"{l_in}x1"]["tok_s"], d["batch"], d["tpot_s"])
-    return {"config": "8b", "layers_run": nl, "prefill_grid": grid, "decode": d, "allocation": alloc}
+    return {"config": "8b", "fp8_projections": fp8, "layers_run": nl, "prefill_grid": grid, "decode": d, "allocation": alloc}
 
 
 def run_long_input(quick=False):
@@ -283,8 +283,11 @@ def main(argv=None):
     ap.add_argument("config", choices=sorted(RUNNERS))
     ap.add_argument("--quick", action="store_true")
     ap.add_argument("--out", default="")
+    ap.add_argument("--fp8", action="store_true", help="8b only: run the projections in FP8 (E4M3)")
     args = ap.parse_args(argv)
-    res = RUNNERS[args.config](args.quick)
+    if args.fp8 and args.config != "8b":
+        ap.error("--fp8 is implemented for the 8b configuration")
+    res = run_8b(args.quick, fp8=True) if args.fp8 else RUNNERS[args.config](args.quick)
     res["peaks"] = _peaks()[2]
     text = json.dumps(res, indent=1)
     if args.out:

@@ -32,6 +32,21 @@ def test_measure_tiny_config_and_allocate(pdlib):
     assert got["tp_decode_eff"] == ref.tp_decode_eff and got["tp_prefill_eff"] == ref.tp_prefill_eff
 
 
+def test_measure_tiny_fp8_projections(pdlib):
+    """The harness with FP8 projections: it builds quantised layers from its own seeded weights and reports
+    the same quantities; the FP8 layer must not be slower than a generous multiple of the bf16 one."""
+    out = {}
+    for fp8 in (False, True):
+        cfg = pdlib.LayerConfig(**TINY, max_pos=256, fp8_projections=fp8)
+        out[fp8] = pdlib.pd_measure(cfg, n_layers_run=2, n_layers_model=2, warmup=2, reps=5, seed=0, l_in=[128, 100],
+                                    batch_sizes=[1, 4], kv_len_start=128, n_steps=8, step_stride=4,
+                                    peak_bf16_flops=1.4e15, peak_hbm_bytes_s=6.4e12)
+    assert out[True]["prefill_tok_s"] > 0 and all(t > 0 for t in out[True]["tpot_s"])
+    assert out[True]["prefill_flops"] == out[False]["prefill_flops"]
+    assert out[True]["gpu_launches"] > out[False]["gpu_launches"]          # the quantiser launches
+    assert out[True]["prefill_time_s"] < 5 * out[False]["prefill_time_s"]
+
+
 def test_measure_8b_shape_two_layers_scaled(pdlib):
     """Two 8B-shaped layers scaled to 32: ragged prefill batch, decode sweep with ragged KV lengths;
     TPOT must not decrease with the batch size beyond timing noise."""
