@@ -68,92 +68,108 @@ __global__ void __launch_bounds__(QNT_THREADS) quantize_rows_fp8_kernel(const bf
 // ------------------------------------------------------------------- RMSNorm
 // y = x * rsqrt(mean(x^2) + eps) * g; one block per row, row kept in registers.
 constexpr int RMS_THREADS = 256;
-constexpr int RMS_MAX_CHUNKS = 8;  // 8 chunks * 8 elements * 256 threads = d up to 16384
+constexpr int RMS_MAX_CHUNKS = 8;  // 8 chunks * 8 elements * 256 threads = d up to 16384 (largest instantiation)
 
 // With q_out != NULL the row is also quantised to E4M3 exactly as quantize_rows_fp8_kernel would quantise the
 // stored bf16 row (the maximum and the quotients are taken on the bf16-rounded values).
+// Rows are taken grid-stride (gridDim.x blocks, `rows` rows): while a row is being reduced and written, the loads of
+// the block's next row are already in flight.
+template <int NCH>  // 16-byte chunks per thread: d <= NCH * 8 * RMS_THREADS
 __global__ void __launch_bounds__(RMS_THREADS) rmsnorm_kernel(const bf16* __restrict__ x,
                                                                const bf16* __restrict__ gain, bf16* __restrict__ y,
-                                                               int d, float eps, float* zero_ptr, int zero_cols,
-                                                               uint8_t* __restrict__ q_out, float* __restrict__ s_out) {
-  const int row = blockIdx.x;
+                                                               int rows, int d, float eps, float* zero_ptr,
+                                                               int zero_cols, uint8_t* __restrict__ q_out,
+                                                               float* __restrict__ s_out) {
   ptx::grid_launch_dependents();
   ptx::grid_dependency_wait();
-  if (zero_ptr) {  // fp32 sums of a later decode projection, idle while this kernel runs
-    float4* q = reinterpret_cast<float4*>(zero_ptr + static_cast<size_t>(row) * zero_cols);
-    for (int i = threadIdx.x; i < zero_cols / 4; i += RMS_THREADS) q[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-  }
-  const uint4* xr = reinterpret_cast<const uint4*>(x + static_cast<size_t>(row) * d);
   const uint4* gr = reinterpret_cast<const uint4*>(gain);
-  uint4* yr = reinterpret_cast<uint4*>(y + static_cast<size_t>(row) * d);
   const int chunks = d / 8;
-  uint4 v[RMS_MAX_CHUNKS];
-  float ss = 0.f;
+  __shared__ float red[2][RMS_THREADS / 32];
+  uint4 v[NCH], nxt[NCH];
+  auto load_row = [&](int r, uint4 (&dst)[NCH]) {
+    const uint4* xr = reinterpret_cast<const uint4*>(x + static_cast<size_t>(r) * d);
 #pragma unroll
-  for (int i = 0; i < RMS_MAX_CHUNKS; ++i) {
-    const int c = threadIdx.x + i * RMS_THREADS;
-    if (c < chunks) {
-      v[i] = xr[c];
-      float f[8];
-      unpack8(v[i], f);
-#pragma unroll
-      for (int e = 0; e < 8; ++e) ss = fmaf(f[e], f[e], ss);
+    for (int i = 0; i < NCH; ++i) {
+      const int c = threadIdx.x + i * RMS_THREADS;
+      if (c < chunks) dst[i] = xr[c];
     }
-  }
-  __shared__ float red[RMS_THREADS / 32];
+  };
+  int row = blockIdx.x;
+  if (row < rows) load_row(row, nxt);
+  for (; row < rows; row += gridDim.x) {
 #pragma unroll
-  for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
-  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
-  __syncthreads();
-  float tot = 0.f;
-#pragma unroll
-  for (int w = 0; w < RMS_THREADS / 32; ++w) tot += red[w];
-  const float scale = rsqrtf(tot / static_cast<float>(d) + eps);
-  float amax = 0.f;
-#pragma unroll
-  for (int i = 0; i < RMS_MAX_CHUNKS; ++i) {
-    const int c = threadIdx.x + i * RMS_THREADS;
-    if (c < chunks) {
-      float f[8], g[8];
-      unpack8(v[i], f);
-      unpack8(gr[c], g);
-#pragma unroll
-      for (int e = 0; e < 8; ++e) f[e] = f[e] * scale * g[e];
-      v[i] = pack8(f);
-      yr[c] = v[i];
-      if (q_out) {
-        unpack8(v[i], f);
-#pragma unroll
-        for (int e = 0; e < 8; ++e) amax = fmaxf(amax, fabsf(f[e]));
-      }
+    for (int i = 0; i < NCH; ++i) v[i] = nxt[i];
+    if (row + static_cast<int>(gridDim.x) < rows) load_row(row + gridDim.x, nxt);
+    if (zero_ptr) {  // fp32 sums of a later decode projection, idle while this kernel runs
+      float4* q = reinterpret_cast<float4*>(zero_ptr + static_cast<size_t>(row) * zero_cols);
+      for (int i = threadIdx.x; i < zero_cols / 4; i += RMS_THREADS) q[i] = make_float4(0.f, 0.f, 0.f, 0.f);
     }
-  }
-  if (q_out) {  // block-uniform
-    __syncthreads();  // everyone has read red[]
+    uint4* yr = reinterpret_cast<uint4*>(y + static_cast<size_t>(row) * d);
+    float ss = 0.f;
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
-    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = amax;
-    __syncthreads();
-    float mx = 0.f;
-#pragma unroll
-    for (int w = 0; w < RMS_THREADS / 32; ++w) mx = fmaxf(mx, red[w]);
-    const float qs = mx > 0.f ? __fdiv_rn(mx, 448.f) : 1.f;
-    if (threadIdx.x == 0) s_out[row] = qs;
-    uint2* qr = reinterpret_cast<uint2*>(q_out + static_cast<size_t>(row) * d);
-#pragma unroll
-    for (int i = 0; i < RMS_MAX_CHUNKS; ++i) {
+    for (int i = 0; i < NCH; ++i) {
       const int c = threadIdx.x + i * RMS_THREADS;
       if (c < chunks) {
         float f[8];
         unpack8(v[i], f);
 #pragma unroll
-        for (int e = 0; e < 8; ++e) f[e] = __fdiv_rn(f[e], qs);
-        uint2 o;
-        o.x = ptx::cvt_e4m3x2(f[0], f[1]) | (ptx::cvt_e4m3x2(f[2], f[3]) << 16);
-        o.y = ptx::cvt_e4m3x2(f[4], f[5]) | (ptx::cvt_e4m3x2(f[6], f[7]) << 16);
-        qr[c] = o;
+        for (int e = 0; e < 8; ++e) ss = fmaf(f[e], f[e], ss);
       }
     }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+    if ((threadIdx.x & 31) == 0) red[0][threadIdx.x >> 5] = ss;
+    __syncthreads();
+    float tot = 0.f;
+#pragma unroll
+    for (int w = 0; w < RMS_THREADS / 32; ++w) tot += red[0][w];
+    const float scale = rsqrtf(tot / static_cast<float>(d) + eps);
+    float amax = 0.f;
+#pragma unroll
+    for (int i = 0; i < NCH; ++i) {
+      const int c = threadIdx.x + i * RMS_THREADS;
+      if (c < chunks) {
+        float f[8], g[8];
+        unpack8(v[i], f);
+        unpack8(gr[c], g);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) f[e] = f[e] * scale * g[e];
+        v[i] = pack8(f);
+        yr[c] = v[i];
+        if (q_out) {
+          unpack8(v[i], f);
+#pragma unroll
+          for (int e = 0; e < 8; ++e) amax = fmaxf(amax, fabsf(f[e]));
+        }
+      }
+    }
+    if (q_out) {  // block-uniform
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+      if ((threadIdx.x & 31) == 0) red[1][threadIdx.x >> 5] = amax;
+      __syncthreads();
+      float mx = 0.f;
+#pragma unroll
+      for (int w = 0; w < RMS_THREADS / 32; ++w) mx = fmaxf(mx, red[1][w]);
+      const float qs = mx > 0.f ? __fdiv_rn(mx, 448.f) : 1.f;
+      if (threadIdx.x == 0) s_out[row] = qs;
+      uint2* qr = reinterpret_cast<uint2*>(q_out + static_cast<size_t>(row) * d);
+#pragma unroll
+      for (int i = 0; i < NCH; ++i) {
+        const int c = threadIdx.x + i * RMS_THREADS;
+        if (c < chunks) {
+          float f[8];
+          unpack8(v[i], f);
+#pragma unroll
+          for (int e = 0; e < 8; ++e) f[e] = __fdiv_rn(f[e], qs);
+          uint2 o;
+          o.x = ptx::cvt_e4m3x2(f[0], f[1]) | (ptx::cvt_e4m3x2(f[2], f[3]) << 16);
+          o.y = ptx::cvt_e4m3x2(f[4], f[5]) | (ptx::cvt_e4m3x2(f[6], f[7]) << 16);
+          qr[c] = o;
+        }
+      }
+    }
+    __syncthreads();  // red[] is reused by the block's next row
   }
 }
 
@@ -183,12 +199,24 @@ __global__ void __launch_bounds__(256) fill_normal_kernel(bf16* dst, size_t n, u
 
 }  // namespace
 
+// Picks the instantiation for the row length; all blocks are resident (148 SMs x 4) and take further rows grid-stride.
+static cudaError_t launch_rmsnorm_any(const bf16* x, const bf16* gain, bf16* y, int rows, int d, float eps, float* zero_ptr,
+                                      int zero_cols, uint8_t* q_out, float* s_out, cudaStream_t s) {
+  const int grid = rows < 148 * 4 ? rows : 148 * 4;
+  const int per_thread = (d / 8 + RMS_THREADS - 1) / RMS_THREADS;
+  const dim3 g(grid), b(RMS_THREADS);
+  if (per_thread <= 1) return launch_pdl(rmsnorm_kernel<1>, g, b, 0, s, x, gain, y, rows, d, eps, zero_ptr, zero_cols, q_out, s_out);
+  if (per_thread <= 2) return launch_pdl(rmsnorm_kernel<2>, g, b, 0, s, x, gain, y, rows, d, eps, zero_ptr, zero_cols, q_out, s_out);
+  if (per_thread <= 4) return launch_pdl(rmsnorm_kernel<4>, g, b, 0, s, x, gain, y, rows, d, eps, zero_ptr, zero_cols, q_out, s_out);
+  return launch_pdl(rmsnorm_kernel<8>, g, b, 0, s, x, gain, y, rows, d, eps, zero_ptr, zero_cols, q_out, s_out);
+}
+
 pd_status launch_rmsnorm(const bf16* x, const bf16* gain, bf16* y, int rows, int d, float eps, cudaStream_t s,
                          uint8_t* q_out, float* s_out) {
   if (rows == 0) return PD_OK;
   if (d % 8 != 0 || d > RMS_THREADS * RMS_MAX_CHUNKS * 8 || (q_out && !s_out)) return PD_ERR_UNSUPPORTED_SHAPE;
   float* no_zero = nullptr;
-  PD_CUDA_TRY(launch_pdl(rmsnorm_kernel, dim3(rows), dim3(RMS_THREADS), 0, s, x, gain, y, d, eps, no_zero, 0, q_out, s_out));
+  PD_CUDA_TRY(launch_rmsnorm_any(x, gain, y, rows, d, eps, no_zero, 0, q_out, s_out, s));
   count_launch();
   return PD_OK;
 }
@@ -198,8 +226,7 @@ pd_status launch_rmsnorm_decode(const bf16* x, const bf16* gain, bf16* y, int ro
   if (rows == 0) return PD_OK;
   if (d % 8 != 0 || d > RMS_THREADS * RMS_MAX_CHUNKS * 8 || (zero_ptr && zero_cols % 4 != 0) || (q_out && !s_out))
     return PD_ERR_UNSUPPORTED_SHAPE;
-  PD_CUDA_TRY(launch_pdl(rmsnorm_kernel, dim3(rows), dim3(RMS_THREADS), 0, s, x, gain, y, d, eps, zero_ptr, zero_cols,
-                         q_out, s_out));
+  PD_CUDA_TRY(launch_rmsnorm_any(x, gain, y, rows, d, eps, zero_ptr, zero_cols, q_out, s_out, s));
   count_launch();
   return PD_OK;
 }
