@@ -11,6 +11,7 @@ pytestmark = pytest.mark.gpu
 @pytest.mark.parametrize("m,n,k", [
     (128, 256, 64), (128, 64, 128), (1, 768, 512), (37, 1536, 512), (200, 768, 512), (129, 512, 1536),
     (300, 3072, 512), (1000, 6144, 4096), (333, 4096, 14336), (2048, 28672, 4096), (16, 4096, 4096),
+    (512, 6144, 64), (300, 6144, 128), (2000, 4096, 8192),   # CTA-pair kernel: one K block; odd row tiles; tail halves
 ])
 def test_gemm_matches_float64(pdlib, m, n, k):
     import torch
