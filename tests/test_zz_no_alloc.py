@@ -36,7 +36,7 @@ def test_noalloc_matches_workspace_version_twice(pdlib):
     k0, v0 = gen.kv_cache(21, 4, hkv, cap, hd)
     dk, dv = to_dev(k0), to_dev(v0)
     cache = pdlib.kv_cache_struct(dk, dv, 4, cap)
-    # first call: 4 sequences, the KV range is split 8 ways -> the scratch is written
+    # first call: 4 sequences, the KV range is split 4 ways -> the scratch is written
     q1 = gen.normal_bf16(21, gen.S_X, (4, hq * hd), 1.0, sub=1)
     got1, ref1 = _both(pdlib, cfg, q1, [2303, 1500, 700, 5], cache, cap)
     assert_close(got1, ref1, "first call")
@@ -48,8 +48,8 @@ def test_noalloc_matches_workspace_version_twice(pdlib):
 
 
 def test_noalloc_rejects_oversized_problem(pdlib):
-    # 591 sequences x 1 KV head still get 2 splits each: 591 x 16 heads x 2 x 130 floats = 9.8 MB > the 8 MiB array
-    hq, hkv, hd, b, cap = 16, 1, 128, 591, 512
+    # 13 sequences x 8 KV heads still get 2 splits each: 13 x 128 heads x 2 x 130 floats = 1.7 MB > the 1 MiB array
+    hq, hkv, hd, b, cap = 128, 8, 128, 13, 1024
     cfg = pdlib.LayerConfig(hq * hd, hq, hkv, hd, 64)
     need = pdlib.pd_decode_attention_workspace_bytes(cfg, b, cap)
     assert need > pdlib.NOALLOC_SCRATCH_BYTES
