@@ -3,6 +3,8 @@
 // synchronises except pd_layer_create / pd_layer_destroy / pd_layer_check and the
 // host-I/O variants of the stack calls.
 #include <cmath>
+#include <cstdlib>
+#include <cstring>
 #include <new>
 #include <vector>
 
@@ -246,8 +248,18 @@ pd_status decode_impl_wide(pd_layer* L, const bf16* x, bf16* out, const int32_t*
   return PD_OK;
 }
 
+// How a decode layer is chained to its neighbours inside a stack call: the last row-wise kernel of a
+// layer can also produce the next layer's first RMSNorm (its gain is next_gain), in which case that next
+// layer is told that the normalised rows (and, with FP8 projections, their codes and scales) and the
+// cleared QKV accumulator are already in the workspace.
+struct DecodeLink {
+  bool norm_ready = false;
+  const bf16* next_gain = nullptr;
+};
+
 pd_status decode_impl(pd_layer* L, const bf16* x, bf16* out, const int32_t* kv_len_dev, int B, int max_kv_len,
-                      const pd_kv_cache* cache, uint8_t* ws, const Workspace& w, cudaStream_t st) {
+                      const pd_kv_cache* cache, uint8_t* ws, const Workspace& w, cudaStream_t st,
+                      const DecodeLink& link = DecodeLink{}) {
   if (B >= kWideDecodeBatch) return decode_impl_wide(L, x, out, kv_len_dev, B, max_kv_len, cache, ws, w, st);
   const pd_layer_cfg& c = L->cfg;
   const int hq = c.n_q_heads * c.head_dim;
@@ -290,7 +302,7 @@ pd_status decode_impl(pd_layer* L, const bf16* x, bf16* out, const int32_t* kv_l
     return PD_OK;
   };
 
-  {
+  if (!link.norm_ready) {
     pd::TraceScope ts(PD_K_RMSNORM, st);
     PD_TRY(pd::launch_rmsnorm_decode(x, L->g_attn, norm, B, c.d_model, c.rms_eps, z_qkv, L->n_qkv, st,
                                      f8 ? q_act : nullptr, f8 ? s_act : nullptr));
@@ -335,7 +347,11 @@ pd_status decode_impl(pd_layer* L, const bf16* x, bf16* out, const int32_t* kv_l
     g.x = act; g.w = L->w_down; g.acc = acc_down; g.n = c.d_model; g.k = c.d_ff; g.ldx = c.d_ff;
     PD_TRY(fp8_in(g, L->q_down, L->s_down, false));
     PD_TRY(pd::gemm_skinny(g, st));
-    PD_TRY(pd::launch_skinny_residual(acc_down, resid, out, nullptr, nullptr, B, c.d_model, c.rms_eps, nullptr, 0, st));
+    if (link.next_gain)  // out = h + down, and the next layer's first RMSNorm of it in the same pass
+      PD_TRY(pd::launch_skinny_residual(acc_down, resid, out, link.next_gain, norm, B, c.d_model, c.rms_eps, z_qkv,
+                                        L->n_qkv, st, f8 ? q_act : nullptr, f8 ? s_act : nullptr));
+    else
+      PD_TRY(pd::launch_skinny_residual(acc_down, resid, out, nullptr, nullptr, B, c.d_model, c.rms_eps, nullptr, 0, st));
   }
   return PD_OK;
 }
@@ -619,9 +635,20 @@ extern "C" pd_status pd_decode_stack(pd_layer* const* layers, const pd_kv_cache*
     kv_dev = reinterpret_cast<const int32_t*>(ws + w.meta);
     cur = buf[0];
   }
+  // Between two layers of the same shape the first RMSNorm of the second runs inside the last row-wise kernel
+  // of the first (one launch fewer per layer); PD_FUSE_NEXT_NORM=0 in the environment keeps them apart.
+  static const bool fuse_next_norm = [] {
+    const char* v = std::getenv("PD_FUSE_NEXT_NORM");
+    return !(v && v[0] == '0');
+  }();
+  DecodeLink link{};
   for (int i = 0; i < n_layers; ++i) {
     bf16* dst = (i == n_layers - 1 && !io_on_host) ? static_cast<bf16*>(out) : buf[(i + 1) & 1];
-    PD_TRY(decode_impl(layers[i], cur, dst, kv_dev, B, max_kv_len, &caches[i % n_caches], ws, w, st));
+    const bool fuse = fuse_next_norm && i + 1 < n_layers && B < kWideDecodeBatch &&
+                      std::memcmp(&layers[i]->cfg, &layers[i + 1]->cfg, sizeof(pd_layer_cfg)) == 0;
+    link.next_gain = fuse ? layers[i + 1]->g_attn : nullptr;
+    PD_TRY(decode_impl(layers[i], cur, dst, kv_dev, B, max_kv_len, &caches[i % n_caches], ws, w, st, link));
+    link.norm_ready = fuse;
     cur = dst;
   }
   if (io_on_host) {

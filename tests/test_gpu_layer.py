@@ -209,6 +209,66 @@ def test_two_layer_stack_matches_chained_oracle(pdlib):
     np.testing.assert_array_equal(oh.numpy(), dout.cpu().numpy())
 
 
+@pytest.mark.parametrize("fp8_mode", [False, True])
+@pytest.mark.parametrize("b", [5, 70])
+def test_three_layer_decode_stack_matches_chained_oracle(pdlib, b, fp8_mode):
+    """pd_decode_stack over three layers (the first RMSNorm of layers 1 and 2 runs inside the previous layer's
+    last row-wise kernel) against the oracle's layers chained, and against three pd_decode_layer calls."""
+    import torch
+    from oracle import fp8 as ofp8
+    cap = 40
+    ws_, ocfgs, ows, dls, pjs = [], [], [], [], []
+    for i in range(3):
+        w = gen.layer_weights(**TINY, seed=4, layer=i)
+        cfg = pdlib.LayerConfig(**TINY, max_pos=64, fp8_projections=fp8_mode)
+        dls.append(DeviceLayer(pdlib, cfg, w, 0, b, cap))
+        ows.append(L.LayerWeights(**w))
+        pjs.append(ofp8.Fp8Projector(ows[-1]) if fp8_mode else None)
+    ocfg = L.LayerConfig(**TINY)
+    kv_len = [int(v_) for v_ in gen.uniform_lengths(31, b, 0, cap - 1, sub=b)]
+    x = gen.activations(31, b, 512, sub=b)
+    k0s, v0s, caches_a, caches_b, keep = [], [], [], [], []
+    for i in range(3):
+        k0, v0 = gen.kv_cache(31 + i, b, 2, cap, 64)
+        k0s.append(k0); v0s.append(v0)
+        for lst in (caches_a, caches_b):
+            k, v, c = dls[i].make_cache(b, cap, k0, v0)
+            keep += [k, v]; lst.append(c)
+    dout = empty_bf16(b, 512)
+    pdlib.pd_decode_stack([d.layer for d in dls], caches_a, to_dev(x), dout, False, i32_dev(kv_len), b,
+                          max(kv_len) + 1, dls[0].ws, dls[0].ws_bytes)
+    for d in dls:
+        pdlib.pd_layer_check(d.layer)
+    torch.cuda.synchronize()
+    got = from_dev(dout)
+    # layer by layer through pd_decode_layer, each layer checked against the oracle on the input the GPU gave it
+    # (with FP8 projections an end-to-end bar over several layers is not meaningful: one flipped code in layer 0
+    # is a different input for layer 1)
+    cur_np, cur = x, to_dev(x)
+    chained = x
+    for i in range(3):
+        nxt = empty_bf16(b, 512)
+        pdlib.pd_decode_layer(dls[i].layer, cur, nxt, i32_dev(kv_len), b, max(kv_len) + 1, caches_b[i], dls[i].ws,
+                              dls[i].ws_bytes)
+        torch.cuda.synchronize()
+        kw = dict(store=store_bf16, proj=pjs[i]) if fp8_mode else {}
+        ref_i = L.decode_layer(ocfg, ows[i], cur_np, kv_len, k0s[i].astype(np.float64), v0s[i].astype(np.float64), **kw)
+        assert_close(from_dev(nxt), ref_i, f"layer {i} of the chain")
+        if not fp8_mode:
+            chained = L.decode_layer(ocfg, ows[i], chained, kv_len, k0s[i].astype(np.float64),
+                                     v0s[i].astype(np.float64))
+        cur, cur_np = nxt, from_dev(nxt)
+    one_by_one = cur_np
+    # the stack call computes the same values up to the order of the sum of squares in the fused RMSNorm
+    assert_close(got, one_by_one, "three-layer decode stack against the layer-by-layer calls", atol=3e-2)
+    if not fp8_mode:
+        assert_close(got, chained, "three-layer decode stack against the chained oracle")
+    # the appended K/V rows of the last layer agree as well
+    for s_ in (0, b - 1):
+        np.testing.assert_allclose(from_dev(keep[4 * 2])[s_, :, kv_len[s_]], from_dev(keep[4 * 2 + 2])[s_, :, kv_len[s_]],
+                                   rtol=2e-2, atol=2e-2)
+
+
 def test_argument_errors(pdlib):
     ocfg, ow, dl = setup(pdlib, TINY, 64, 64, 2, 64)
     k, v, cache = dl.make_cache(2, 64)
