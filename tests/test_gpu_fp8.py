@@ -56,7 +56,7 @@ def test_quantize_every_code_and_midpoint(pdlib):
 @pytest.mark.parametrize("m,n,k", [
     (128, 256, 128), (1, 768, 512), (37, 1536, 512), (200, 768, 1536), (129, 512, 512),
     (300, 3072, 512), (1000, 6144, 4096), (333, 4096, 14336), (2048, 28672, 4096), (16, 4096, 4096),
-    (512, 6144, 128), (300, 6144, 256),
+    (512, 6144, 128), (300, 6144, 256), (512, 4096, 1024), (384, 4096, 512),
 ])
 def test_gemm_fp8_matches_oracle(pdlib, m, n, k):
     import torch

@@ -12,6 +12,7 @@ pytestmark = pytest.mark.gpu
     (128, 256, 64), (128, 64, 128), (1, 768, 512), (37, 1536, 512), (200, 768, 512), (129, 512, 1536),
     (300, 3072, 512), (1000, 6144, 4096), (333, 4096, 14336), (2048, 28672, 4096), (16, 4096, 4096),
     (512, 6144, 64), (300, 6144, 128), (2000, 4096, 8192),   # CTA-pair kernel: one K block; odd row tiles; tail halves
+    (512, 4096, 1024), (384, 4096, 512), (130, 2048, 256),   # short batches against N = d_model: one wave of narrow tiles
 ])
 def test_gemm_matches_float64(pdlib, m, n, k):
     import torch
