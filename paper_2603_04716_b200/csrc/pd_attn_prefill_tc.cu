@@ -57,10 +57,13 @@ __global__ void __launch_bounds__(ATT_THREADS, 1)
 prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                        const __grid_constant__ CUtensorMap tmap_v, AttDev p) {
   using Cfg = AttCfg<HD>;
-  const int h = blockIdx.y, req = blockIdx.z;
+  // Launch order = longest blocks first over the whole grid: the block index that varies slowest is the row
+  // block, descending, so every head and request runs its last (longest-range) rows before anybody's short ones
+  // and no long block is left to start when the rest of the grid is about to drain.
+  const int h = blockIdx.x, req = blockIdx.y;
   const int start = p.cu_seqlens[req];
   const int len = p.cu_seqlens[req + 1] - start;
-  const int q0 = (gridDim.x - 1 - blockIdx.x) * (2 * TQ);  // long blocks first
+  const int q0 = (gridDim.z - 1 - blockIdx.z) * (2 * TQ);
   if (q0 >= len) return;
   const int slot = p.slots ? p.slots[req] : req;
   if (slot < 0 || slot >= p.batch_cap) return;  // reported by the QKV epilogue
@@ -379,7 +382,8 @@ pd_status launch_hd(const PrefillAttnArgs& a, int* err_word, cudaStream_t s) {
   p.o = a.o; p.cu_seqlens = a.cu_seqlens; p.slots = a.slots; p.prefix = a.prefix;
   p.n_q_heads = a.n_q_heads; p.n_kv_heads = a.n_kv_heads; p.len_cap = a.len_cap; p.batch_cap = a.batch_cap;
   p.err_word = err_word;
-  dim3 grid((a.max_len + 2 * TQ - 1) / (2 * TQ), a.n_q_heads, a.n_req);
+  dim3 grid(a.n_q_heads, a.n_req, (a.max_len + 2 * TQ - 1) / (2 * TQ));
+  if (grid.y > 65535u || grid.z > 65535u) return PD_ERR_UNSUPPORTED_SHAPE;
   PD_CUDA_TRY(launch_pdl(kern, grid, dim3(ATT_THREADS), Cfg::SMEM_BYTES, s, tq, tk, tv, p));
   count_launch();
   return PD_OK;
