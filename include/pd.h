@@ -163,10 +163,12 @@ pd_status pd_decode_attention(const pd_layer_cfg* cfg, const void* q, int32_t ld
  *
  * Arguments and results are those of pd_decode_attention without the workspace pair.
  * Limits and rules:
- *   - B * n_q_heads * splits * (head_dim + 2) * 4 bytes must fit the array (splits is chosen
- *     from B, n_kv_heads and max_kv_len as in pd_decode_attention: only while B * n_kv_heads is
- *     below about 110, so every shape with up to 8 query heads per KV head fits, and so does
- *     every batch large enough to need no split).  Otherwise the call returns
+ *   - B * n_q_heads * splits * (head_dim + 2) * 4 bytes must fit the array.  splits is chosen
+ *     from B, n_kv_heads and max_kv_len as in pd_decode_attention: small batches are split until
+ *     about 110 blocks exist, and any batch is split so that a block covers at most about 2048
+ *     keys (4096 from B * n_kv_heads = 592 on); a problem that needs no split always fits.
+ *     With 32 query heads and head_dim 128 the array holds B * splits up to 504, e.g. B = 256 at
+ *     up to 6143 keys or B = 126 at up to 18431.  Otherwise the call returns
  *     PD_ERR_WORKSPACE_TOO_SMALL and launches nothing.
  *   - The first call on each device looks up the array's device address (that device must be
  *     current); make this first call before any stream capture begins.
@@ -174,7 +176,7 @@ pd_status pd_decode_attention(const pd_layer_cfg* cfg, const void* q, int32_t ld
  *     when a call starts; nothing has to be cleared because each call overwrites every entry
  *     it later reads.  Two calls whose kernels can overlap on the GPU (different streams,
  *     different host threads) race on it: serialise them on one stream. */
-#define PD_NOALLOC_SCRATCH_BYTES (1u << 20)
+#define PD_NOALLOC_SCRATCH_BYTES (8u << 20)
 pd_status pd_decode_attention_noalloc(const pd_layer_cfg* cfg, const void* q, int32_t ldq, void* out,
                                       const int32_t* kv_len_dev, int32_t B, int32_t max_kv_len,
                                       const pd_kv_cache* cache, void* stream);

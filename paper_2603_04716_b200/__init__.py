@@ -313,7 +313,7 @@ def pd_decode_attention(cfg: LayerConfig, q, ldq: int, out, kv_len_dev, batch: i
                                     _stream_ptr(stream)), "pd_decode_attention")
 
 
-NOALLOC_SCRATCH_BYTES = 1 << 20
+NOALLOC_SCRATCH_BYTES = 8 << 20
 
 
 def pd_decode_attention_noalloc(cfg: LayerConfig, q, ldq: int, out, kv_len_dev, batch: int, max_kv_len: int,

@@ -48,8 +48,8 @@ def test_noalloc_matches_workspace_version_twice(pdlib):
 
 
 def test_noalloc_rejects_oversized_problem(pdlib):
-    # 13 sequences x 8 KV heads still get 2 splits each: 13 x 128 heads x 2 x 130 floats = 1.7 MB > the 1 MiB array
-    hq, hkv, hd, b, cap = 128, 8, 128, 13, 1024
+    # 130 sequences of up to 8192 keys get 2 splits each: 130 x 64 heads x 2 x 130 floats = 8.65 MB > the 8 MiB array
+    hq, hkv, hd, b, cap = 64, 8, 128, 130, 8192
     cfg = pdlib.LayerConfig(hq * hd, hq, hkv, hd, 64)
     need = pdlib.pd_decode_attention_workspace_bytes(cfg, b, cap)
     assert need > pdlib.NOALLOC_SCRATCH_BYTES
