@@ -166,9 +166,9 @@ pd_status pd_decode_attention(const pd_layer_cfg* cfg, const void* q, int32_t ld
  *   - B * n_q_heads * splits * (head_dim + 2) * 4 bytes must fit the array.  splits is chosen
  *     from B, n_kv_heads and max_kv_len as in pd_decode_attention: small batches are split until
  *     about 110 blocks exist, and any batch is split so that a block covers at most about 2048
- *     keys (4096 from B * n_kv_heads = 592 on); a problem that needs no split always fits.
- *     With 32 query heads and head_dim 128 the array holds B * splits up to 504, e.g. B = 256 at
- *     up to 6143 keys or B = 126 at up to 18431.  Otherwise the call returns
+ *     keys; a problem that needs no split always fits.  With 32 query heads and head_dim 128
+ *     the array holds B * splits up to 504, e.g. B = 256 at up to 3071 keys or B = 126 at up to
+ *     9215.  Otherwise the call returns
  *     PD_ERR_WORKSPACE_TOO_SMALL and launches nothing.
  *   - The first call on each device looks up the array's device address (that device must be
  *     current); make this first call before any stream capture begins.

@@ -287,12 +287,12 @@ int decode_attention_splits(int batch, int n_kv_heads, int max_kv_len) {
   // (partials, the merge kernel: 5-13 % at uniform lengths), except that the grid is sized from the LONGEST
   // sequence: with ragged lengths an unsplit long sequence is a block that runs on alone after the others
   // have drained (measured 0.48 of the HBM rate at B = 16 with lengths spread 1 : 9).  So a block's key range
-  // is capped at about 2048 keys while the grid is under two waves, at about 4096 beyond; short sequences
-  // leave their later splits empty.  A split shorter than 512 keys never paid.
+  // is capped at about 2048 keys; short sequences leave their later splits empty.  A split shorter than 512
+  // keys never paid.
   const long long blocks = 1ll * batch * n_kv_heads;
   if (blocks <= 0) return 1;
   long long want = (112 + blocks - 1) / blocks;
-  const long long by_len = blocks < 592 ? (max_kv_len + 1024ll) / 2048 : (max_kv_len + 2048ll) / 4096;
+  const long long by_len = (max_kv_len + 1024ll) / 2048;
   if (by_len > want) want = by_len;
   long long cap = max_kv_len / 512;
   if (cap < 1) cap = 1;

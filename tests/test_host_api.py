@@ -153,7 +153,7 @@ def test_workspace_bytes_and_config_validation(pdlib):
 def test_decode_attention_split_rule_through_the_workspace_size(pdlib):
     """pd_decode_attention_workspace_bytes is host arithmetic: B * n_q_heads * splits * (head_dim + 2) floats.  It
     pins the split rule the header documents: few blocks -> split up to about 112 blocks, never under 512 keys per
-    split, and a block's key range capped near 2048 keys (4096 from B * n_kv_heads = 592 on)."""
+    split, and a block's key range capped near 2048 keys."""
     cfg = pdlib.LayerConfig(4096, 32, 8, 128, 64)
 
     def splits(b, kv):
@@ -163,9 +163,9 @@ def test_decode_attention_split_rule_through_the_workspace_size(pdlib):
         return round(n / per) if n % per == 0 else -(-n // per)   # the size is rounded up to 256 bytes
 
     assert splits(256, 2304) == 1          # the benchmark's decode shape: one block per (sequence, KV head)
-    assert splits(256, 6143) == 1 and splits(256, 6144) == 2
+    assert splits(256, 3071) == 1 and splits(256, 3072) == 2
     assert splits(16, 2304) == 1 and splits(16, 9216) == 5
-    assert splits(64, 8192) == 4 and splits(128, 8192) == 2
+    assert splits(64, 8192) == 4 and splits(128, 8192) == 4
     assert splits(1, 2304) == 4            # 8 blocks: split, but not below 512 keys
     assert splits(1, 511) == 1 and splits(4, 100000) == 49 and splits(1, 100000) == 49
     assert splits(1, 200000) == 64         # upper limit

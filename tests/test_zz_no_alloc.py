@@ -48,7 +48,7 @@ def test_noalloc_matches_workspace_version_twice(pdlib):
 
 
 def test_noalloc_rejects_oversized_problem(pdlib):
-    # 130 sequences of up to 8192 keys get 2 splits each: 130 x 64 heads x 2 x 130 floats = 8.65 MB > the 8 MiB array
+    # 130 sequences of up to 8192 keys get 4 splits each: 130 x 64 heads x 4 x 130 floats = 17.3 MB > the 8 MiB array
     hq, hkv, hd, b, cap = 64, 8, 128, 130, 8192
     cfg = pdlib.LayerConfig(hq * hd, hq, hkv, hd, 64)
     need = pdlib.pd_decode_attention_workspace_bytes(cfg, b, cap)
