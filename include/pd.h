@@ -187,7 +187,11 @@ pd_status pd_decode_attention_noalloc(const pd_layer_cfg* cfg, const void* q, in
  * host pointers (pinned memory advised): the call copies the inputs to the device on `stream`,
  * runs the stack, copies `out` back and synchronises `stream` before returning; for prefill
  * `cu_seqlens_dev` is then ignored (the host copy is uploaded).  The workspace must come from
- * pd_workspace_bytes (it includes room for the staged activations). */
+ * pd_workspace_bytes (it includes room for the staged activations).
+ * In decode mode, between two layers of the same shape, the first RMSNorm of the second layer is
+ * computed by the last kernel of the first; the result equals that of chained pd_decode_layer calls
+ * up to the summation order of that norm's sum of squares (at most one bf16 unit in the last place
+ * of a normalised value). */
 pd_status pd_prefill_stack(pd_layer* const* layers, const pd_kv_cache* caches, int32_t n_layers, int32_t n_caches,
                            const void* x, void* out, int32_t io_on_host, const int32_t* cu_seqlens_dev,
                            const int32_t* cu_seqlens_host, int32_t n_req, void* workspace,
