@@ -14,6 +14,11 @@ Readings where the paper is silent:
   * the TPOT-feasible batch is the largest sweep point such that every sweep point
     up to and including it meets the SLO (no interpolation);
   * T_overhead is an explicit input;
+  * a workload of mixed input lengths ("Preliminaries" takes L_in and L_out as averages): the
+    maximum prefill throughput of the mix is its total tokens over its total service time,
+    and L_in in Eq. 5-13 is the mean length;
+  * the integer between two sweep points of the TPOT curve is found by measuring at the
+    midpoint of the bracket [largest feasible, smallest infeasible] until they are neighbours;
   * prefix caching ("Acquire prefill throughput under TTFT constraints", closing remark): the
     input length is replaced, everywhere it occurs in Eq. 1-13, by the length that misses
     the cache, L_in (1 - hit fraction); throughputs then count computed tokens;
@@ -222,3 +227,83 @@ def pollaczek_khinchine_sojourn(lam: float, mean_s: float, mean_s2: float) -> fl
     """Textbook M/G/1 mean sojourn: E[S] + lambda E[S^2] / (2 (1 - rho))."""
     rho = lam * mean_s
     return mean_s + lam * mean_s2 / (2.0 * (1.0 - rho))
+
+
+def _seq_sum(values) -> float:
+    """Left-to-right IEEE double sum (the built-in sum() compensates, which another
+    implementation need not do; the order is part of the definition here)."""
+    acc = 0.0
+    for v in values:
+        acc += float(v)
+    return acc
+
+
+def mixture_throughput(l_in, service_times):
+    """Maximum prefill throughput of a request mix served one request at a time.
+
+    Request i has l_in[i] tokens and takes service_times[i] seconds alone on a saturated
+    instance; the mix then runs at (sum of tokens) / (sum of times) tokens per second
+    ("Acquire prefill throughput under TTFT constraints": the maximum throughput is what the
+    instance sustains when continuously busy).  Returns (tp_max, mean input length).
+    """
+    n = len(l_in)
+    if n == 0 or n != len(service_times):
+        raise ValueError("need one service time per request")
+    tokens = _seq_sum(l_in)
+    busy = _seq_sum(service_times)
+    return tokens / busy, tokens / n
+
+
+def service_moments(service_times):
+    """(E[S], E[S^2]) of the sampled service times, sums taken left to right."""
+    n = len(service_times)
+    return _seq_sum(service_times) / n, _seq_sum(float(s) * float(s) for s in service_times) / n
+
+
+def mg1_sojourn(service_times, lam: float) -> float:
+    """Mean sojourn of an M/G/1 queue whose service-time distribution is the sample's
+    (Pollaczek-Khinchine); Eq. 12 is its special case for exponential service."""
+    es, es2 = service_moments(service_times)
+    if not lam * es < 1.0:
+        raise ValueError("arrival rate must keep the server utilisation below one")
+    return pollaczek_khinchine_sojourn(lam, es, es2)
+
+
+def interp_service_times(grid_l, grid_t, lengths):
+    """Service time of each length by linear interpolation between measured grid points
+    (grid_l strictly increasing); lengths outside the grid take the end values."""
+    out = []
+    n = len(grid_l)
+    for l in lengths:
+        if l <= grid_l[0]:
+            out.append(float(grid_t[0]))
+            continue
+        if l >= grid_l[n - 1]:
+            out.append(float(grid_t[n - 1]))
+            continue
+        i = 0
+        while grid_l[i + 1] < l:
+            i += 1
+        w = (float(l) - float(grid_l[i])) / (float(grid_l[i + 1]) - float(grid_l[i]))
+        out.append(grid_t[i] + (grid_t[i + 1] - grid_t[i]) * w)
+    return out
+
+
+def refine_next_batch(batch, tpot, tpot_slo) -> int:
+    """Next batch size to measure when refining the TPOT-feasible batch to an integer
+    ("Acquire decode throughput under TPOT constraints": determine the batch size that
+    satisfies the target TPOT).  With the points measured so far sorted by batch size, lo is
+    the largest one whose whole prefix meets the SLO and hi the first one that does not;
+    the next measurement goes to floor((lo + hi) / 2).  Returns 0 when nothing is left to
+    measure: no feasible point, no infeasible point, or lo and hi are neighbours."""
+    order = sorted(range(len(batch)), key=lambda i: batch[i])
+    lo = hi = 0
+    for i in order:
+        if tpot[i] <= tpot_slo:
+            lo = int(batch[i])
+        else:
+            hi = int(batch[i])
+            break
+    if lo == 0 or hi == 0 or hi - lo <= 1:
+        return 0
+    return (lo + hi) // 2

@@ -201,3 +201,70 @@ def test_prefix_cache_hits_shorten_the_effective_input():
         A.allocate_ext(**base, prefix_hit_frac=1.0)
     with pytest.raises(ValueError):
         A.allocate_ext(**base, dp_groups=0)
+
+
+def test_mixture_throughput_special_cases():
+    # equal requests: the mix runs at L / t; mean length L
+    tp, mean_l = A.mixture_throughput([4096] * 7, [0.05] * 7)
+    assert tp == pytest.approx(4096 / 0.05, rel=1e-12) and mean_l == 4096
+    # hand case: 1000 tokens in 1 s and 3000 tokens in 1 s -> 2000 tok/s, mean 2000
+    assert A.mixture_throughput([1000, 3000], [1.0, 1.0]) == (2000.0, 2000.0)
+    # a server that replays the mix back to back is busy sum(t) and emits sum(L): Eq. 9's mu = tp / mean_l
+    rnd = random.Random(4)
+    ls = [rnd.randint(100, 9000) for _ in range(500)]
+    ts = [1e-5 * l + 1e-9 * l * l for l in ls]
+    tp, mean_l = A.mixture_throughput(ls, ts)
+    assert A.service_rate(tp, mean_l) == pytest.approx(len(ls) / sum(ts), rel=1e-12)   # requests per busy second
+    with pytest.raises(ValueError):
+        A.mixture_throughput([1, 2], [1.0])
+
+
+def test_mg1_sojourn_reduces_to_md1_and_mm1_and_matches_a_replay():
+    mu = 5.0
+    assert A.mg1_sojourn([1 / mu] * 100, 3.0) == pytest.approx(A.md1_sojourn(mu, 3.0), rel=1e-12)
+    rng = np.random.Generator(np.random.Philox(key=17))
+    svc = rng.exponential(1 / mu, size=400_000)
+    # exponential samples: E[S^2] ~ 2 / mu^2, so the M/G/1 mean approaches Eq. 12
+    assert A.mg1_sojourn(svc.tolist(), 3.0) == pytest.approx(A.mm1_sojourn(mu, 3.0), rel=0.02)
+    # a two-point service distribution replayed through the queue agrees with the formula
+    two = np.where(rng.random(400_000) < 0.8, 0.05, 0.6)
+    lam = 0.7 / two.mean()
+    soj, _ = A.queue_replay(rng.exponential(1 / lam, size=two.size).tolist(), two.tolist())
+    assert soj == pytest.approx(A.mg1_sojourn(two.tolist(), lam), rel=0.05)
+    with pytest.raises(ValueError):
+        A.mg1_sojourn([1.0, 1.0], 1.0)
+
+
+def test_interp_service_times_against_numpy():
+    rnd = random.Random(6)
+    grid_l = sorted(rnd.sample(range(100, 40000), 9))
+    grid_t = sorted(rnd.uniform(0.01, 2.0) for _ in grid_l)
+    ls = [rnd.randint(50, 41000) for _ in range(300)] + grid_l
+    got = A.interp_service_times(grid_l, grid_t, ls)
+    np.testing.assert_allclose(got, np.interp(ls, grid_l, grid_t), rtol=1e-12)
+    # exact at the grid points and on a straight line
+    assert A.interp_service_times([10, 20], [1.0, 2.0], [10, 15, 20, 5, 30]) == [1.0, 1.5, 2.0, 1.0, 2.0]
+
+
+def test_refine_next_batch_brackets_the_largest_feasible_integer():
+    rnd = random.Random(5)
+    for _ in range(300):
+        a, b0 = rnd.uniform(1e-5, 2e-4), rnd.uniform(1e-3, 5e-3)
+        curve = lambda b: b0 + a * b                     # TPOT grows with the batch
+        batch = [1, 2, 4, 8, 16, 32, 64, 128, 256, 512]
+        tpot = [curve(b) for b in batch]
+        slo = rnd.uniform(b0 + a, b0 + 600 * a)
+        probes = 0
+        while True:
+            nxt = A.refine_next_batch(batch, tpot, slo)
+            if nxt == 0:
+                break
+            assert nxt not in batch
+            batch.append(nxt); tpot.append(curve(nxt)); probes += 1
+        feas = [b for b in range(1, 513) if curve(b) <= slo]       # brute force over every integer
+        _, b_star, capped = A.feasible_batch(batch, tpot, slo)
+        assert b_star == (max(feas) if feas else 0)
+        assert probes <= 8 and capped == (b_star == 512)
+    assert A.refine_next_batch([4, 8], [0.1, 0.2], 0.05) == 0       # nothing feasible
+    assert A.refine_next_batch([4, 8], [0.01, 0.02], 0.05) == 0     # nothing infeasible: capped by the sweep
+    assert A.refine_next_batch([8, 4, 5], [0.2, 0.01, 0.3], 0.05) == 0   # neighbours
