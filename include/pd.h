@@ -150,6 +150,24 @@ pd_status pd_decode_attention(const pd_layer_cfg* cfg, const void* q, int32_t ld
                               const int32_t* kv_len_dev, int32_t B, int32_t max_kv_len, const pd_kv_cache* cache,
                               void* workspace, size_t workspace_bytes, void* stream);
 
+/* The prefill-attention kernel on its own (causal grouped-query attention of the compute-bound prefill
+ * mode; paper, "Acquire prefill throughput under TTFT constraints" benchmarks the pass this kernel is the
+ * attention step of), for roofline measurement and unit tests.
+ *   q, out        device bf16 [T, ldq] / [T, Hq*hd]: row t of request r is query cu[r] + t at position
+ *                 prefix[r] + t; head h occupies columns h*hd .. of a row; ldq a multiple of 8, q 16-byte aligned
+ *   cu_seqlens    as for pd_prefill_layer (device copy and host copy)
+ *   prefix        tokens of each request already cached before its rows (device and host copy, both or
+ *                 neither; NULL = 0)
+ *   cache         must already hold K (after RoPE) and V of positions 0 .. prefix[r] + len_r - 1 of
+ *                 request r in sequence slots[r] (NULL: r)
+ *   err_word      optional device int32, set to 1 if a bounded wait inside the kernel gave up
+ * Query t attends to positions 0 .. prefix[r] + t of its own request.  Only n_q_heads, n_kv_heads and
+ * head_dim of cfg are used.  Enqueues one kernel; no workspace. */
+pd_status pd_prefill_attention(const pd_layer_cfg* cfg, const void* q, int32_t ldq, void* out,
+                               const int32_t* cu_seqlens_dev, const int32_t* cu_seqlens_host, int32_t n_req,
+                               const int32_t* prefix_dev, const int32_t* prefix_host, const int32_t* slots_dev,
+                               const pd_kv_cache* cache, int32_t* err_word, void* stream);
+
 /* pd_decode_attention for callers that may not allocate device memory.  (The paper has no
  * counterpart of this call; it exists for the library's users.)
  *
@@ -188,6 +206,10 @@ pd_status pd_decode_attention_noalloc(const pd_layer_cfg* cfg, const void* q, in
  * runs the stack, copies `out` back and synchronises `stream` before returning; for prefill
  * `cu_seqlens_dev` is then ignored (the host copy is uploaded).  The workspace must come from
  * pd_workspace_bytes (it includes room for the staged activations).
+ * Every layer of a stack must have the shape of layers[0] (d_model, head counts, head_dim, d_ff and the
+ * fp8_projections switch: the workspace and the inter-layer buffers are laid out once, for that shape);
+ * rms_eps, rope_theta and max_pos may differ.  A stack with a layer of another shape is refused with
+ * PD_ERR_INVALID_ARG before anything is enqueued.
  * In decode mode, between two layers of the same shape, the first RMSNorm of the second layer is
  * computed by the last kernel of the first; the result equals that of chained pd_decode_layer calls
  * up to the summation order of that norm's sum of squares (at most one bf16 unit in the last place
@@ -418,6 +440,43 @@ pd_status pd_allocate_ext(const pd_alloc_in* in, double prefix_hit_frac, int32_t
  * 1/(mu - lambda)) and the mean waiting time. */
 pd_status pd_queue_replay(const double* gaps, const double* service, int64_t n, double* mean_sojourn_s,
                           double* mean_wait_s);
+
+/* ------------------------------------------------- workload statistics (host) */
+
+/* Maximum prefill throughput of a mix of request lengths (paper, Preliminaries: L_in and L_out are
+ * averages; "Acquire prefill throughput under TTFT constraints": the maximum throughput is that of a
+ * continuously busy instance).  Request i has l_in[i] > 0 tokens and takes service_s[i] > 0 seconds when
+ * served alone; the mix sustains tp_max = sum(l_in) / sum(service_s) tokens/s, and mean_l_in = sum(l_in) / n
+ * is the L_in of Eq. 5-13 (so Eq. 9's mu = tp_max / mean_l_in is requests per busy second).  Sums run
+ * left to right in double. */
+pd_status pd_mixture_throughput(const int32_t* l_in, const double* service_s, int64_t n, double* tp_max_tok_s,
+                                double* mean_l_in);
+
+/* Service time of each request length by linear interpolation between measured prefill times
+ * (grid_l strictly increasing; lengths outside the grid take the end values):
+ * t = t_lo + (t_hi - t_lo) * ((l - l_lo) / (l_hi - l_lo)).  Feeds pd_mixture_throughput, pd_mg1_sojourn and
+ * pd_queue_replay when a length distribution is served from a grid of measured lengths. */
+pd_status pd_interp_service_times(const int32_t* grid_l, const double* grid_time_s, int32_t n_grid,
+                                  const int32_t* l_in, int64_t n, double* service_s);
+
+/* Eq. 12: mean sojourn time 1 / (mu - lambda) of the M/M/1 prefill queue.  PD_ERR_INFEASIBLE_TTFT when
+ * lambda >= mu (no steady state). */
+pd_status pd_mm1_sojourn(double mu, double lambda, double* sojourn_s);
+
+/* Mean sojourn time of the same queue when the service times follow the given sample instead of the
+ * exponential law Eq. 12 assumes (Pollaczek-Khinchine: E[S] + lambda E[S^2] / (2 (1 - lambda E[S]))); what
+ * the replayed queue is compared with for fixed or log-normal request lengths.  PD_ERR_INFEASIBLE_TTFT when
+ * lambda E[S] >= 1. */
+pd_status pd_mg1_sojourn(const double* service_s, int64_t n, double lambda, double* sojourn_s);
+
+/* One step of the integer refinement of the TPOT-feasible batch (paper, "Acquire decode throughput under
+ * TPOT constraints": determine the batch size that satisfies the target TPOT).  Given every (batch, TPOT)
+ * point measured so far, lo = the largest point whose whole prefix (in order of batch size) meets the SLO,
+ * hi = the first point that does not; *next_batch = lo + (hi - lo) / 2 is where to measure next, or 0 when
+ * nothing is left to measure (no feasible point, no infeasible point, or hi = lo + 1).  The caller measures,
+ * appends the point and calls again; pd_allocate on the final point set then returns B* = lo. */
+pd_status pd_refine_next_batch(const int32_t* batch, const double* tpot_s, int32_t n_points, double tpot_slo_s,
+                               int32_t* next_batch);
 
 #ifdef __cplusplus
 }

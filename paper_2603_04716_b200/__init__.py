@@ -38,6 +38,8 @@ EXPORTS = [
     "pd_decode_attention_noalloc", "pd_prefill_chunk_layer",
     "pd_model_create", "pd_model_destroy", "pd_model_workspace_bytes", "pd_model_prefill", "pd_model_decode_step",
     "pd_model_check", "pd_allocate_ext", "pd_quantize_fp8_rows", "pd_gemm_fp8", "pd_workspace_offsets",
+    "pd_prefill_attention", "pd_mixture_throughput", "pd_interp_service_times", "pd_mm1_sojourn", "pd_mg1_sojourn",
+    "pd_refine_next_batch",
 ]
 
 TRACE_CLASSES = ["gemm_qkv", "gemm_o", "gemm_gate_up", "gemm_down", "attn_prefill", "attn_decode", "rmsnorm",
@@ -145,10 +147,18 @@ _lib.pd_allocate.argtypes = [C.POINTER(pd_alloc_in), C.POINTER(pd_alloc_out)]
 _lib.pd_allocate_ext.argtypes = [C.POINTER(pd_alloc_in), C.c_double, C.c_int32, C.POINTER(pd_alloc_out)]
 _lib.pd_queue_replay.argtypes = [C.POINTER(C.c_double), C.POINTER(C.c_double), C.c_int64, C.POINTER(C.c_double),
                                  C.POINTER(C.c_double)]
+_DP, _IP = C.POINTER(C.c_double), C.POINTER(C.c_int32)
+_lib.pd_mixture_throughput.argtypes = [_IP, _DP, C.c_int64, _DP, _DP]
+_lib.pd_interp_service_times.argtypes = [_IP, _DP, C.c_int32, _IP, C.c_int64, _DP]
+_lib.pd_mm1_sojourn.argtypes = [C.c_double, C.c_double, _DP]
+_lib.pd_mg1_sojourn.argtypes = [_DP, C.c_int64, C.c_double, _DP]
+_lib.pd_refine_next_batch.argtypes = [_IP, _DP, C.c_int32, C.c_double, _IP]
 _lib.pd_decode_attention_workspace_bytes.argtypes = [C.POINTER(pd_layer_cfg), C.c_int32, C.c_int32,
                                                      C.POINTER(C.c_size_t)]
 _lib.pd_decode_attention.argtypes = [C.POINTER(pd_layer_cfg), _P, C.c_int32, _P, _P, C.c_int32, C.c_int32,
                                      C.POINTER(pd_kv_cache), _P, C.c_size_t, _P]
+_lib.pd_prefill_attention.argtypes = [C.POINTER(pd_layer_cfg), _P, C.c_int32, _P, _P, C.POINTER(C.c_int32), C.c_int32,
+                                      _P, C.POINTER(C.c_int32), _P, C.POINTER(pd_kv_cache), _P, _P]
 _lib.pd_decode_attention_noalloc.argtypes = [C.POINTER(pd_layer_cfg), _P, C.c_int32, _P, _P, C.c_int32, C.c_int32,
                                              C.POINTER(pd_kv_cache), _P]
 _lib.pd_model_create.argtypes = [C.POINTER(_P), C.c_int32, C.POINTER(pd_model_weights), _P, C.POINTER(_P)]
@@ -311,6 +321,15 @@ def pd_decode_attention(cfg: LayerConfig, q, ldq: int, out, kv_len_dev, batch: i
     _check(_lib.pd_decode_attention(C.byref(cfg.c_struct()), _ptr(q), ldq, _ptr(out), _ptr(kv_len_dev), batch,
                                     max_kv_len, C.byref(cache), _ptr(workspace), workspace_bytes,
                                     _stream_ptr(stream)), "pd_decode_attention")
+
+
+def pd_prefill_attention(cfg: LayerConfig, q, ldq: int, out, cu_seqlens_dev, cu_seqlens_host, cache: pd_kv_cache,
+                         prefix_dev=None, prefix_host=None, slots_dev=None, err_word=None, stream=None):
+    cu = _i32_array(cu_seqlens_host)
+    pre = _i32_array(prefix_host) if prefix_host is not None else None
+    _check(_lib.pd_prefill_attention(C.byref(cfg.c_struct()), _ptr(q), ldq, _ptr(out), _ptr(cu_seqlens_dev), cu,
+                                     len(cu_seqlens_host) - 1, _ptr(prefix_dev), pre, _ptr(slots_dev),
+                                     C.byref(cache), _ptr(err_word), _stream_ptr(stream)), "pd_prefill_attention")
 
 
 NOALLOC_SCRATCH_BYTES = 8 << 20
@@ -498,3 +517,61 @@ def pd_queue_replay(gaps, service):
     _check(_lib.pd_queue_replay(g.ctypes.data_as(dp), s.ctypes.data_as(dp), g.size, C.byref(soj), C.byref(wait)),
            "pd_queue_replay")
     return soj.value, wait.value
+
+
+def _np_i32(a):
+    import numpy as np
+    return np.ascontiguousarray(a, dtype=np.int32)
+
+
+def _np_f64(a):
+    import numpy as np
+    return np.ascontiguousarray(a, dtype=np.float64)
+
+
+def pd_mixture_throughput(l_in, service_s):
+    """(maximum prefill throughput of the request mix, mean input length)."""
+    l, s = _np_i32(l_in), _np_f64(service_s)
+    if l.shape != s.shape:
+        raise ValueError("one service time per request")
+    tp, mean_l = C.c_double(), C.c_double()
+    _check(_lib.pd_mixture_throughput(l.ctypes.data_as(_IP), s.ctypes.data_as(_DP), l.size, C.byref(tp),
+                                      C.byref(mean_l)), "pd_mixture_throughput")
+    return tp.value, mean_l.value
+
+
+def pd_interp_service_times(grid_l, grid_time_s, l_in):
+    """numpy float64 array: service time of each length, interpolated on the measured grid."""
+    import numpy as np
+    gl, gt, l = _np_i32(grid_l), _np_f64(grid_time_s), _np_i32(l_in)
+    if gl.shape != gt.shape:
+        raise ValueError("one time per grid length")
+    out = np.empty(l.size, dtype=np.float64)
+    _check(_lib.pd_interp_service_times(gl.ctypes.data_as(_IP), gt.ctypes.data_as(_DP), gl.size,
+                                        l.ctypes.data_as(_IP), l.size, out.ctypes.data_as(_DP)),
+           "pd_interp_service_times")
+    return out
+
+
+def pd_mm1_sojourn(mu: float, lam: float) -> float:
+    out = C.c_double()
+    _check(_lib.pd_mm1_sojourn(mu, lam, C.byref(out)), "pd_mm1_sojourn")
+    return out.value
+
+
+def pd_mg1_sojourn(service_s, lam: float) -> float:
+    s = _np_f64(service_s)
+    out = C.c_double()
+    _check(_lib.pd_mg1_sojourn(s.ctypes.data_as(_DP), s.size, lam, C.byref(out)), "pd_mg1_sojourn")
+    return out.value
+
+
+def pd_refine_next_batch(batch, tpot_s, tpot_slo_s: float) -> int:
+    """Next batch size to measure while refining the TPOT-feasible batch, 0 when done."""
+    b, t = _np_i32(batch), _np_f64(tpot_s)
+    if b.shape != t.shape:
+        raise ValueError("one TPOT per batch size")
+    out = C.c_int32()
+    _check(_lib.pd_refine_next_batch(b.ctypes.data_as(_IP), t.ctypes.data_as(_DP), b.size, tpot_slo_s,
+                                     C.byref(out)), "pd_refine_next_batch")
+    return out.value

@@ -263,11 +263,8 @@ __global__ void __launch_bounds__(HD) decode_combine_kernel(DecodeAttnArgs a) {
 template <int HD>
 pd_status launch_decode_hd(const DecodeAttnArgs& a, cudaStream_t s) {
   using SM = DecodeSmem<HD>;
-  static bool attr_set = false;
-  if (!attr_set) {
-    PD_CUDA_TRY(cudaFuncSetAttribute(decode_attn_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, SM::BYTES));
-    attr_set = true;
-  }
+  static PerDeviceInt smem_opt_in;
+  PD_TRY(opt_in_smem(smem_opt_in, decode_attn_kernel<HD>, SM::BYTES));
   dim3 grid(a.n_splits, a.n_kv_heads, a.batch);
   PD_CUDA_TRY(launch_pdl(decode_attn_kernel<HD>, grid, dim3(DC_THREADS), SM::BYTES, s, a));
   count_launch();

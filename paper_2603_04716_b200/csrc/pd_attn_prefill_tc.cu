@@ -367,12 +367,9 @@ prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
 template <int HD>
 pd_status launch_hd(const PrefillAttnArgs& a, int* err_word, cudaStream_t s) {
   using Cfg = AttCfg<HD>;
-  static bool attr_set = false;
+  static PerDeviceInt smem_opt_in;
   auto kern = prefill_attn_tc_kernel<HD>;
-  if (!attr_set) {
-    PD_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES));
-    attr_set = true;
-  }
+  PD_TRY(opt_in_smem(smem_opt_in, kern, Cfg::SMEM_BYTES));
   CUtensorMap tq, tk, tv;
   const uint64_t cache_rows = static_cast<uint64_t>(a.batch_cap) * a.n_kv_heads * a.len_cap;
   PD_TRY(make_tmap_bf16(&tq, a.q, a.n_tokens, static_cast<uint64_t>(a.n_q_heads) * HD, a.ldq, TQ));

@@ -6,6 +6,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "pd.h"
 
 namespace pd {
@@ -27,6 +29,32 @@ pd_status cuda_fail(cudaError_t e);  // records e for pd_last_cuda_error(), retu
   } while (0)
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// Per-device memo for launch set-up.  The opt-in to large dynamic shared memory (cudaFuncSetAttribute) and the
+// answers of the occupancy queries belong to one device, so a process that drives several GPUs needs them once
+// per device ordinal, not once per process.  Slot = ordinal of the current device (ordinals >= kMaxDevices share
+// the last slot's "unknown" state and simply redo the set-up on every call).
+constexpr int kMaxDevices = 64;
+inline int current_device_slot() {
+  int d = 0;
+  if (cudaGetDevice(&d) != cudaSuccess || d < 0 || d >= kMaxDevices) return -1;
+  return d;
+}
+struct PerDeviceInt {
+  std::atomic<int> v[kMaxDevices];
+  PerDeviceInt() { for (auto& e : v) e.store(-1, std::memory_order_relaxed); }
+  // -1 = not yet determined on the current device
+  int get() const { const int s = current_device_slot(); return s < 0 ? -1 : v[s].load(std::memory_order_acquire); }
+  void set(int value) { const int s = current_device_slot(); if (s >= 0) v[s].store(value, std::memory_order_release); }
+};
+// Opts `kern` in to `bytes` of dynamic shared memory on the current device, once per device.
+template <class K>
+pd_status opt_in_smem(PerDeviceInt& memo, K kern, int bytes) {
+  if (memo.get() == 1) return PD_OK;
+  PD_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+  memo.set(1);
+  return PD_OK;
+}
 
 // Counts kernel launches made by this thread (reported by pd_measure).
 extern thread_local long long g_launch_count;

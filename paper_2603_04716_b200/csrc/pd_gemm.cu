@@ -709,28 +709,26 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
   }
 }
 
-int g_sm_count = 0;
+// SM count of the current device (remembered per device ordinal).
 int sm_count() {
-  if (g_sm_count == 0) {
-    int dev = 0, n = 0;
-    if (cudaGetDevice(&dev) == cudaSuccess &&
-        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0)
-      g_sm_count = n;
-    else
-      g_sm_count = 148;
-  }
-  return g_sm_count;
+  static PerDeviceInt memo;
+  int n = memo.get();
+  if (n > 0) return n;
+  int dev = 0;
+  n = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
+    n = 148;
+  memo.set(n);
+  return n;
 }
 
 template <int BN, int EPI, bool F8>
 pd_status launch_tc(const GemmArgs& g, cudaStream_t stream) {
   using Cfg = GemmCfg<BN>;
-  static bool attr_set = false;
+  static PerDeviceInt smem_opt_in;
   auto kern = gemm_tc_kernel<BN, EPI, F8>;
-  if (!attr_set) {
-    PD_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES));
-    attr_set = true;
-  }
+  PD_TRY(opt_in_smem(smem_opt_in, kern, Cfg::SMEM_BYTES));
   CUtensorMap ta, tb;
   if (F8) {
     PD_TRY(make_tmap_u8(&ta, g.a, g.m, g.k, g.lda, BM));
@@ -784,10 +782,14 @@ pd_status launch_tc(const GemmArgs& g, cudaStream_t stream) {
 // CTA pairs resident at once for the pair kernel (0: clusters of two cannot be placed).
 template <int EPI, bool F8>
 int pair_capacity() {
-  static int cap = -1;
-  if (cap >= 0) return cap;
+  static PerDeviceInt memo;  // per device: the opt-in below and the occupancy answer are the device's
+  const int known = memo.get();
+  if (known >= 0) return known;
   auto kern = gemm_tc_pair_kernel<EPI, F8>;
-  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, P2_SMEM_BYTES) != cudaSuccess) return cap = 0;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, P2_SMEM_BYTES) != cudaSuccess) {
+    memo.set(0);
+    return 0;
+  }
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3(2 * sm_count());
   cfg.blockDim = dim3(GEMM_THREADS);
@@ -799,7 +801,8 @@ int pair_capacity() {
   cfg.numAttrs = 1;
   int n = 0;
   if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess) { cudaGetLastError(); n = 0; }
-  return cap = n;
+  memo.set(n);
+  return n;
 }
 
 template <int EPI, bool F8>

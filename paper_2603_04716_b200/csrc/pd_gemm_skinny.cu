@@ -477,12 +477,9 @@ int skinny_bnb(int batch) { return batch <= 16 ? 16 : batch <= 32 ? 32 : batch <
 template <int BNB, int MT, bool F8>
 pd_status launch_skinny(const SkinnyGemmArgs& g, cudaStream_t stream) {
   using Cfg = SkinnyCfg<BNB, MT>;
-  static bool attr_set = false;
+  static PerDeviceInt smem_opt_in;
   auto kern = gemm_skinny_kernel<BNB, MT, F8>;
-  if (!attr_set) {
-    PD_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES));
-    attr_set = true;
-  }
+  PD_TRY(opt_in_smem(smem_opt_in, kern, Cfg::SMEM_BYTES));
   CUtensorMap tw, tx;
   if (F8) {
     PD_TRY(make_tmap_u8(&tw, g.w, g.n, g.k, g.k, MT * SK_BM));
@@ -516,7 +513,8 @@ pd_status launch_skinny(const SkinnyGemmArgs& g, cudaStream_t stream) {
 template <int BNB, bool F8>
 pd_status launch_skinny_pair(const SkinnyGemmArgs& g, cudaStream_t stream) {
   using Cfg = SkinnyPairCfg<BNB>;
-  static int usable = -1;  // -1 unknown, 0 clusters of two cannot be placed, 1 fine
+  static PerDeviceInt usable_memo;  // per device: -1 unknown, 0 clusters of two cannot be placed, 1 fine
+  int usable = usable_memo.get();
   auto kern = gemm_skinny_pair_kernel<BNB, F8>;
   cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -537,6 +535,7 @@ pd_status launch_skinny_pair(const SkinnyGemmArgs& g, cudaStream_t stream) {
       if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) == cudaSuccess && n > 0) usable = 1;
       else cudaGetLastError();
     }
+    usable_memo.set(usable);
   }
   if (!usable) return PD_ERR_UNSUPPORTED_SHAPE;
   CUtensorMap tw, tx;

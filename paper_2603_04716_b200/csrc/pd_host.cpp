@@ -148,3 +148,82 @@ extern "C" pd_status pd_queue_replay(const double* gaps, const double* service, 
   *mean_wait_s = sum_wait / static_cast<double>(n);
   return PD_OK;
 }
+
+// ----------------------------------------------------------------- workload statistics
+// Everything below is sequential IEEE double arithmetic in a fixed order, so that an independent
+// implementation that follows the same order agrees bit for bit.
+
+extern "C" pd_status pd_mixture_throughput(const int32_t* l_in, const double* service_s, int64_t n,
+                                           double* tp_max_tok_s, double* mean_l_in) {
+  if (!l_in || !service_s || n <= 0 || !tp_max_tok_s || !mean_l_in) return PD_ERR_INVALID_ARG;
+  double tokens = 0.0, busy = 0.0;
+  for (int64_t i = 0; i < n; ++i) {
+    if (l_in[i] <= 0 || !(service_s[i] > 0.0)) return PD_ERR_INVALID_ARG;
+    tokens += static_cast<double>(l_in[i]);
+  }
+  for (int64_t i = 0; i < n; ++i) busy += service_s[i];
+  *tp_max_tok_s = tokens / busy;
+  *mean_l_in = tokens / static_cast<double>(n);
+  return PD_OK;
+}
+
+extern "C" pd_status pd_interp_service_times(const int32_t* grid_l, const double* grid_time_s, int32_t n_grid,
+                                             const int32_t* l_in, int64_t n, double* service_s) {
+  if (!grid_l || !grid_time_s || n_grid <= 0 || !l_in || n < 0 || !service_s) return PD_ERR_INVALID_ARG;
+  for (int i = 0; i + 1 < n_grid; ++i)
+    if (grid_l[i + 1] <= grid_l[i]) return PD_ERR_INVALID_ARG;
+  for (int64_t r = 0; r < n; ++r) {
+    const int32_t l = l_in[r];
+    if (l <= grid_l[0]) { service_s[r] = grid_time_s[0]; continue; }
+    if (l >= grid_l[n_grid - 1]) { service_s[r] = grid_time_s[n_grid - 1]; continue; }
+    int lo = 0, hi = n_grid - 1;  // grid_l[lo] < l <= grid_l[hi]
+    while (hi - lo > 1) {
+      const int mid = (lo + hi) / 2;
+      if (grid_l[mid] < l) lo = mid; else hi = mid;
+    }
+    const double w = (static_cast<double>(l) - static_cast<double>(grid_l[lo])) /
+                     (static_cast<double>(grid_l[hi]) - static_cast<double>(grid_l[lo]));
+    service_s[r] = grid_time_s[lo] + (grid_time_s[hi] - grid_time_s[lo]) * w;
+  }
+  return PD_OK;
+}
+
+extern "C" pd_status pd_mm1_sojourn(double mu, double lambda, double* sojourn_s) {
+  if (!sojourn_s || !(mu > 0.0) || !(lambda >= 0.0)) return PD_ERR_INVALID_ARG;
+  if (!(lambda < mu)) return PD_ERR_INFEASIBLE_TTFT;  // the queue has no steady state
+  *sojourn_s = 1.0 / (mu - lambda);                   // Eq. 12
+  return PD_OK;
+}
+
+extern "C" pd_status pd_mg1_sojourn(const double* service_s, int64_t n, double lambda, double* sojourn_s) {
+  if (!service_s || n <= 0 || !sojourn_s || !(lambda >= 0.0)) return PD_ERR_INVALID_ARG;
+  double s1 = 0.0, s2 = 0.0;
+  for (int64_t i = 0; i < n; ++i) {
+    if (!(service_s[i] >= 0.0)) return PD_ERR_INVALID_ARG;
+    s1 += service_s[i];
+  }
+  for (int64_t i = 0; i < n; ++i) s2 += service_s[i] * service_s[i];
+  const double es = s1 / static_cast<double>(n), es2 = s2 / static_cast<double>(n);
+  const double rho = lambda * es;
+  if (!(rho < 1.0)) return PD_ERR_INFEASIBLE_TTFT;
+  *sojourn_s = es + lambda * es2 / (2.0 * (1.0 - rho));  // Pollaczek-Khinchine
+  return PD_OK;
+}
+
+extern "C" pd_status pd_refine_next_batch(const int32_t* batch, const double* tpot_s, int32_t n_points,
+                                          double tpot_slo_s, int32_t* next_batch) {
+  if (!next_batch || n_points < 0 || (n_points > 0 && (!batch || !tpot_s)) || !(tpot_slo_s > 0.0))
+    return PD_ERR_INVALID_ARG;
+  for (int i = 0; i < n_points; ++i)
+    if (batch[i] <= 0 || !(tpot_s[i] > 0.0)) return PD_ERR_INVALID_ARG;
+  std::vector<int> order(n_points);
+  for (int i = 0; i < n_points; ++i) order[i] = i;
+  std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return batch[a] < batch[b]; });
+  int32_t lo = 0, hi = 0;
+  for (int idx : order) {
+    if (tpot_s[idx] <= tpot_slo_s) lo = batch[idx];
+    else { hi = batch[idx]; break; }
+  }
+  *next_batch = (lo == 0 || hi == 0 || hi - lo <= 1) ? 0 : lo + (hi - lo) / 2;
+  return PD_OK;
+}

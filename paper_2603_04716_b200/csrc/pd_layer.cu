@@ -93,6 +93,13 @@ pd_status use_fp8(pd_layer* L, pd::GemmArgs& g, const uint8_t* w_codes, const fl
   return PD_OK;
 }
 
+// The stack calls carve one workspace and one pair of inter-layer buffers from the first layer's shape, so
+// every layer of a stack must have that shape (the norm constants and the RoPE table length may differ).
+bool same_shape(const pd_layer_cfg& a, const pd_layer_cfg& b) {
+  return a.d_model == b.d_model && a.n_q_heads == b.n_q_heads && a.n_kv_heads == b.n_kv_heads &&
+         a.head_dim == b.head_dim && a.d_ff == b.d_ff && a.fp8_projections == b.fp8_projections;
+}
+
 pd_status check_cache(const pd_layer* L, const pd_kv_cache* c) {
   (void)L;
   if (!c || c->struct_size != sizeof(pd_kv_cache) || !c->k || !c->v || c->batch_cap <= 0 || c->len_cap <= 0)
@@ -568,6 +575,39 @@ extern "C" pd_status pd_decode_attention(const pd_layer_cfg* cfg, const void* q,
   return pd::launch_decode_attention(a, st);
 }
 
+extern "C" pd_status pd_prefill_attention(const pd_layer_cfg* cfg, const void* q, int32_t ldq, void* out,
+                                          const int32_t* cu_dev, const int32_t* cu_host, int32_t n_req,
+                                          const int32_t* prefix_dev, const int32_t* prefix_host,
+                                          const int32_t* slots_dev, const pd_kv_cache* cache, int32_t* err_word,
+                                          void* stream) {
+  PD_TRY(check_cfg(cfg));
+  if (!cu_host || n_req < 0 || n_req > 4095 || (prefix_dev == nullptr) != (prefix_host == nullptr))
+    return PD_ERR_INVALID_ARG;
+  PD_TRY(check_cache(nullptr, cache));
+  if (cu_host[0] != 0) return PD_ERR_INVALID_ARG;
+  int max_len = 0;
+  for (int r = 0; r < n_req; ++r) {
+    const int len = cu_host[r + 1] - cu_host[r];
+    const int pre = prefix_host ? prefix_host[r] : 0;
+    if (len < 0 || pre < 0 || pre > cache->len_cap - len) return PD_ERR_INVALID_ARG;
+    if (len > max_len) max_len = len;
+  }
+  if (!slots_dev && n_req > cache->batch_cap) return PD_ERR_INVALID_ARG;
+  const int tokens = cu_host[n_req];
+  if (tokens == 0) return PD_OK;
+  if (!q || !out || !cu_dev || ldq < cfg->n_q_heads * cfg->head_dim || ldq % 8 != 0) return PD_ERR_INVALID_ARG;
+  pd::PrefillAttnArgs a{};
+  a.q = static_cast<const bf16*>(q); a.ldq = ldq;
+  a.k_cache = static_cast<const bf16*>(cache->k); a.v_cache = static_cast<const bf16*>(cache->v);
+  a.o = static_cast<bf16*>(out); a.cu_seqlens = cu_dev; a.slots = slots_dev; a.prefix = prefix_dev;
+  a.n_req = n_req; a.n_tokens = tokens; a.max_len = max_len;
+  a.n_q_heads = cfg->n_q_heads; a.n_kv_heads = cfg->n_kv_heads; a.head_dim = cfg->head_dim;
+  a.len_cap = cache->len_cap; a.batch_cap = cache->batch_cap;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  pd::TraceScope ts(PD_K_ATTN_PREFILL, st);
+  return pd::launch_prefill_attention_tc(a, err_word, st);
+}
+
 extern "C" pd_status pd_prefill_stack(pd_layer* const* layers, const pd_kv_cache* caches, int32_t n_layers,
                                       int32_t n_caches, const void* x, void* out, int32_t io_on_host,
                                       const int32_t* cu_dev, const int32_t* cu_host, int32_t n_req, void* workspace,
@@ -575,7 +615,7 @@ extern "C" pd_status pd_prefill_stack(pd_layer* const* layers, const pd_kv_cache
   if (!layers || !caches || n_layers <= 0 || n_caches <= 0 || !layers[0]) return PD_ERR_INVALID_ARG;
   int tokens = 0, max_len = 0;
   for (int i = 0; i < n_layers; ++i) {
-    if (!layers[i]) return PD_ERR_INVALID_ARG;
+    if (!layers[i] || !same_shape(layers[i]->cfg, layers[0]->cfg)) return PD_ERR_INVALID_ARG;
     PD_TRY(validate_prefill(layers[i], cu_host, n_req, &caches[i % n_caches], true, &tokens, &max_len));
   }
   if (tokens == 0) return PD_OK;
@@ -613,7 +653,7 @@ extern "C" pd_status pd_decode_stack(pd_layer* const* layers, const pd_kv_cache*
   if (!layers || !caches || n_layers <= 0 || n_caches <= 0 || B < 0 || B > 4096) return PD_ERR_INVALID_ARG;
   if (B == 0) return PD_OK;
   for (int i = 0; i < n_layers; ++i) {
-    if (!layers[i]) return PD_ERR_INVALID_ARG;
+    if (!layers[i] || !layers[0] || !same_shape(layers[i]->cfg, layers[0]->cfg)) return PD_ERR_INVALID_ARG;
     const pd_kv_cache* c = &caches[i % n_caches];
     PD_TRY(check_cache(layers[i], c));
     if (B > c->batch_cap || max_kv_len <= 0 || max_kv_len > c->len_cap || max_kv_len > layers[i]->cfg.max_pos)

@@ -185,7 +185,7 @@ extern "C" pd_status pd_model_create(pd_layer* const* layers, int32_t n_layers, 
     if (!layers[i]) return PD_ERR_INVALID_ARG;
     const pd_layer_cfg &a = layers[i]->cfg, &b = layers[0]->cfg;
     if (a.d_model != b.d_model || a.n_q_heads != b.n_q_heads || a.n_kv_heads != b.n_kv_heads ||
-        a.head_dim != b.head_dim || a.d_ff != b.d_ff)
+        a.head_dim != b.head_dim || a.d_ff != b.d_ff || a.fp8_projections != b.fp8_projections)
       return PD_ERR_INVALID_ARG;
   }
   pd_model* m = new (std::nothrow) pd_model();

@@ -169,3 +169,48 @@ def test_decode_attention_split_rule_through_the_workspace_size(pdlib):
     assert splits(1, 2304) == 4            # 8 blocks: split, but not below 512 keys
     assert splits(1, 511) == 1 and splits(4, 100000) == 49 and splits(1, 100000) == 49
     assert splits(1, 200000) == 64         # upper limit
+
+
+def test_workload_statistics_match_oracle_bit_for_bit(pdlib):
+    rnd = random.Random(21)
+    rng = np.random.Generator(np.random.Philox(key=21))
+    for trial in range(200):
+        n = rnd.randint(1, 3000)
+        ls = rng.integers(16, 40000, size=n).astype(np.int32)
+        grid_l = sorted(rnd.sample(range(16, 40000), rnd.randint(1, 40)))
+        grid_t = sorted(rnd.uniform(1e-3, 3.0) for _ in grid_l)
+        svc = pdlib.pd_interp_service_times(grid_l, grid_t, ls)
+        o_svc = A.interp_service_times(grid_l, grid_t, ls.tolist())
+        assert svc.tolist() == o_svc
+        tp, mean_l = pdlib.pd_mixture_throughput(ls, svc)
+        assert (tp, mean_l) == A.mixture_throughput(ls.tolist(), o_svc)
+        mu = tp / mean_l
+        lam = rnd.uniform(0.05, 0.97) * mu
+        assert pdlib.pd_mm1_sojourn(mu, lam) == A.mm1_sojourn(mu, lam)
+        if lam * (sum(o_svc) / n) < 0.999:
+            assert pdlib.pd_mg1_sojourn(svc, lam) == A.mg1_sojourn(o_svc, lam)
+    with pytest.raises(pdlib.PdError) as e:
+        pdlib.pd_mm1_sojourn(1.0, 1.0)
+    assert e.value.status == pdlib.PD_ERR_INFEASIBLE_TTFT
+    with pytest.raises(pdlib.PdError) as e:
+        pdlib.pd_mg1_sojourn([1.0, 1.0], 1.0)
+    assert e.value.status == pdlib.PD_ERR_INFEASIBLE_TTFT
+    with pytest.raises(pdlib.PdError):
+        pdlib.pd_interp_service_times([10, 10], [1.0, 2.0], [5])
+    with pytest.raises(pdlib.PdError):
+        pdlib.pd_mixture_throughput([0], [1.0])
+
+
+def test_refine_next_batch_matches_oracle(pdlib):
+    rnd = random.Random(22)
+    for trial in range(2000):
+        n = rnd.randint(0, 14)
+        batch = rnd.sample(range(1, 600), n)
+        tpot = [rnd.uniform(0.002, 0.12) for _ in range(n)]
+        if trial % 2:
+            order = sorted(range(n), key=lambda i: batch[i])     # a monotone curve every other trial
+            srt = sorted(tpot)
+            for rank, i in enumerate(order):
+                tpot[i] = srt[rank]
+        slo = rnd.uniform(0.001, 0.13)
+        assert pdlib.pd_refine_next_batch(batch, tpot, slo) == A.refine_next_batch(batch, tpot, slo)
