@@ -221,6 +221,14 @@ pd_status pd_prefill_stack(pd_layer* const* layers, const pd_kv_cache* caches, i
 pd_status pd_decode_stack(pd_layer* const* layers, const pd_kv_cache* caches, int32_t n_layers, int32_t n_caches,
                           const void* x, void* out, int32_t io_on_host, const int32_t* kv_len, int32_t B,
                           int32_t max_kv_len, void* workspace, size_t workspace_bytes, void* stream);
+/* pd_prefill_chunk_layer over a stack: one chunk of every request through all layers (the unit a
+ * chunked-prefill engine schedules; paper, "Acquire prefill throughput under TTFT constraints": the maximum
+ * prefill throughput is a function of the chunked-prefill size).  Device pointers only; request r uses cache
+ * sequence r of caches[i % n_caches] in layer i; same shape rule as the other stack calls. */
+pd_status pd_prefill_chunk_stack(pd_layer* const* layers, const pd_kv_cache* caches, int32_t n_layers,
+                                 int32_t n_caches, const void* x, void* out, const int32_t* cu_seqlens_dev,
+                                 const int32_t* cu_seqlens_host, int32_t n_req, const int32_t* prefix_dev,
+                                 const int32_t* prefix_host, void* workspace, size_t workspace_bytes, void* stream);
 
 /* Reads and clears the device-side error word of the layer (set when a bounded wait inside
  * a kernel gave up).  Synchronises `stream`.  PD_OK or PD_ERR_DEVICE_TIMEOUT. */
@@ -351,6 +359,17 @@ pd_status pd_trace_end(pd_trace_report* out);
  * step_stride, ... < n_steps (and the last step) run the stack at kv_len = kv_len_start + t;
  * TPOT(B) is the mean step time scaled to n_layers_model layers.
  * Either part is skipped when its count (n_req / n_batch_sizes) is 0.
+ * chunk_tokens > 0 measures the prefill pass as chunked prefill: step s pushes rows s*chunk .. (s+1)*chunk-1
+ * of every request that still has rows through all layers (pd_prefill_chunk_stack), each chunk attending to
+ * its cached prefix; the reported time is that of the whole batch, all chunks.
+ * l_in_grid / n_grid (at most PD_MEASURE_GRID_MAX lengths): in addition every grid length is measured as one
+ * request on its own (same layers, same chunk size) and reported in grid_l / grid_time_s: the service-time
+ * curve t(L) that pd_interp_service_times, pd_mixture_throughput and pd_queue_replay take.
+ * Every layer of a timed stack has its own weights.  KV buffers: one per layer when memory allows, otherwise a
+ * ring of fewer buffers that the layers cycle through; the ring sizes are reported (prefill_kv_ring,
+ * decode_kv_ring).  Where the K/V bytes one attention-only timing pass touches are below twice the L2 size
+ * (small batches), attn_l2_resident is 1 and attn_frac_hbm_peak is left 0: the kernel time is then not an HBM
+ * figure.
  * With vocab > 0 the step is the whole-model step: the time of the token embedding, the final
  * RMSNorm, the LM head over a vocabulary of that size and the greedy sampling (once per step,
  * not per layer; timed on their own, median of `reps`) is added to prefill_time_s and TPOT(B)
@@ -367,7 +386,11 @@ typedef struct {
   int32_t kv_len_start, n_steps, step_stride;
   const int32_t* kv_len_mix; /* optional host int32[max batch]: per-sequence start lengths (ragged); NULL = kv_len_start */
   int32_t vocab;             /* 0: layer stack only; > 0 (a multiple of 4): whole-model step */
+  int32_t chunk_tokens;      /* 0: every request in one piece; > 0: chunked prefill with chunks of this many tokens */
+  const int32_t* l_in_grid;  /* optional host int32[n_grid]: lengths measured one request at a time */
+  int32_t n_grid;
 } pd_measure_cfg;
+#define PD_MEASURE_GRID_MAX 128
 
 typedef struct {
   uint32_t struct_size;
@@ -385,6 +408,13 @@ typedef struct {
   int32_t gpu_launches;             /* kernels launched inside the timed regions */
   double prefill_head_s;            /* embedding + final norm + LM head + sampling of the prefill pass (vocab > 0) */
   double decode_head_s[32];         /* the same for one decode step at batch[i] */
+  int32_t prefill_chunks;           /* stack passes per prefill measurement (1 unless chunk_tokens > 0) */
+  int32_t prefill_kv_ring;          /* distinct KV buffers the layers of the prefill stack cycle through */
+  int32_t decode_kv_ring[32];       /* the same for the decode stack at batch[i] */
+  int32_t attn_l2_resident[32];     /* 1: the attention-only pass fits L2, attn_frac_hbm_peak not reported */
+  int32_t n_grid;
+  int32_t grid_l[PD_MEASURE_GRID_MAX];
+  double grid_time_s[PD_MEASURE_GRID_MAX]; /* median time of one request of grid_l[i] tokens, n_layers_model layers */
 } pd_measurement;
 
 pd_status pd_measure(const pd_layer_cfg* cfg, const pd_measure_cfg* mcfg, double peak_bf16_flops,

@@ -156,21 +156,27 @@ class _ExactProjector:
 
 
 def _mlp_and_residuals(x_rows: np.ndarray, o_rows: np.ndarray, w: LayerWeights,
-                       cfg: LayerConfig, dt, st, pj) -> np.ndarray:
+                       cfg: LayerConfig, dt, st, pj, stages: dict | None = None) -> np.ndarray:
     h = st(x_rows + pj(o_rows, "w_o"))
     n2 = st(rmsnorm(h, w.g_mlp.astype(dt), cfg.rms_eps))
     a = st(silu(pj(n2, "w_gate")) * pj(n2, "w_up"))
+    if stages is not None:
+        stages.update(attn_o=o_rows, h=h, n2=n2, act=a)
     return st(h + pj(a, "w_down"))
 
 
 def prefill_layer(cfg: LayerConfig, w: LayerWeights, x: np.ndarray, cu_seqlens,
-                  rows=None, dtype=np.float64, probs_out: list | None = None, store=None, proj=None):
+                  rows=None, dtype=np.float64, probs_out: list | None = None, store=None, proj=None,
+                  stages: dict | None = None):
     """One layer over a packed ragged batch of requests.
 
     ``cu_seqlens`` has n_req + 1 entries; request r owns rows cu[r]..cu[r+1]-1 at
     positions 0..len_r-1 and attends only within itself (block-diagonal causal).
     ``rows`` (optional, sorted global row indices) restricts the expensive part
     to those query rows: K and V are still produced for every row.
+
+    ``stages`` (optional dict) receives the intermediates of the selected rows: q (after RoPE),
+    attn_o, h (residual stream after attention), n2, act (SwiGLU output).
 
     Returns (out, k, v): out[len(rows) or T, d]; k, v[T, Hkv, hd] (k after RoPE).
     """
@@ -199,13 +205,15 @@ def prefill_layer(cfg: LayerConfig, w: LayerWeights, x: np.ndarray, cu_seqlens,
             continue
         lo, hi = cu[r], cu[r + 1]
         o[mine] = _attend(q[mine], k[lo:hi], v[lo:hi], pos[sel][mine], pos[lo:hi], cfg, probs_out)
-    out = _mlp_and_residuals(x[sel], st(o), w, cfg, dt, st, pj)
+    if stages is not None:
+        stages["q"] = q
+    out = _mlp_and_residuals(x[sel], st(o), w, cfg, dt, st, pj, stages)
     return out, k, v
 
 
 def decode_layer(cfg: LayerConfig, w: LayerWeights, x: np.ndarray, kv_len,
                  k_cache: np.ndarray, v_cache: np.ndarray, dtype=np.float64,
-                 probs_out: list | None = None, store=None, proj=None) -> np.ndarray:
+                 probs_out: list | None = None, store=None, proj=None, stages: dict | None = None) -> np.ndarray:
     """One decode step for a batch of B sequences, one new token each.
 
     kv_len[b] tokens are already cached for sequence b; the new token has
@@ -236,7 +244,9 @@ def decode_layer(cfg: LayerConfig, w: LayerWeights, x: np.ndarray, kv_len,
         keys = np.ascontiguousarray(k_cache[b, :, :n + 1, :].transpose(1, 0, 2)).astype(dt)
         vals = np.ascontiguousarray(v_cache[b, :, :n + 1, :].transpose(1, 0, 2)).astype(dt)
         o[b:b + 1] = _attend(q[b:b + 1], keys, vals, kv_len[b:b + 1], np.arange(n + 1), cfg, probs_out)
-    return _mlp_and_residuals(x, st(o), w, cfg, dt, st, pj)
+    if stages is not None:
+        stages["q"] = q
+    return _mlp_and_residuals(x, st(o), w, cfg, dt, st, pj, stages)
 
 
 def extend_layer(cfg: LayerConfig, w: LayerWeights, x: np.ndarray, cu_seqlens, prefix_lens,

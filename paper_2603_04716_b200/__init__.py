@@ -39,7 +39,7 @@ EXPORTS = [
     "pd_model_create", "pd_model_destroy", "pd_model_workspace_bytes", "pd_model_prefill", "pd_model_decode_step",
     "pd_model_check", "pd_allocate_ext", "pd_quantize_fp8_rows", "pd_gemm_fp8", "pd_workspace_offsets",
     "pd_prefill_attention", "pd_mixture_throughput", "pd_interp_service_times", "pd_mm1_sojourn", "pd_mg1_sojourn",
-    "pd_refine_next_batch",
+    "pd_refine_next_batch", "pd_prefill_chunk_stack",
 ]
 
 TRACE_CLASSES = ["gemm_qkv", "gemm_o", "gemm_gate_up", "gemm_down", "attn_prefill", "attn_decode", "rmsnorm",
@@ -81,13 +81,17 @@ class pd_kv_cache(C.Structure):
                 ("batch_cap", C.c_int32), ("len_cap", C.c_int32)]
 
 
+MEASURE_GRID_MAX = 128
+
+
 class pd_measure_cfg(C.Structure):
     _fields_ = [("struct_size", C.c_uint32), ("n_layers_run", C.c_int32), ("n_layers_model", C.c_int32),
                 ("warmup", C.c_int32), ("reps", C.c_int32), ("seed", C.c_uint64),
                 ("l_in", C.POINTER(C.c_int32)), ("n_req", C.c_int32),
                 ("batch_sizes", C.POINTER(C.c_int32)), ("n_batch_sizes", C.c_int32),
                 ("kv_len_start", C.c_int32), ("n_steps", C.c_int32), ("step_stride", C.c_int32),
-                ("kv_len_mix", C.POINTER(C.c_int32)), ("vocab", C.c_int32)]
+                ("kv_len_mix", C.POINTER(C.c_int32)), ("vocab", C.c_int32), ("chunk_tokens", C.c_int32),
+                ("l_in_grid", C.POINTER(C.c_int32)), ("n_grid", C.c_int32)]
 
 
 class pd_measurement(C.Structure):
@@ -96,7 +100,10 @@ class pd_measurement(C.Structure):
                 ("n_points", C.c_int32), ("batch", C.c_int32 * 32), ("tpot_s", C.c_double * 32),
                 ("decode_bytes", C.c_double * 32), ("decode_frac_hbm_peak", C.c_double * 32),
                 ("attn_time_s", C.c_double * 32), ("attn_frac_hbm_peak", C.c_double * 32),
-                ("gpu_launches", C.c_int32), ("prefill_head_s", C.c_double), ("decode_head_s", C.c_double * 32)]
+                ("gpu_launches", C.c_int32), ("prefill_head_s", C.c_double), ("decode_head_s", C.c_double * 32),
+                ("prefill_chunks", C.c_int32), ("prefill_kv_ring", C.c_int32), ("decode_kv_ring", C.c_int32 * 32),
+                ("attn_l2_resident", C.c_int32 * 32), ("n_grid", C.c_int32), ("grid_l", C.c_int32 * MEASURE_GRID_MAX),
+                ("grid_time_s", C.c_double * MEASURE_GRID_MAX)]
 
 
 class pd_trace_report(C.Structure):
@@ -134,6 +141,8 @@ _lib.pd_prefill_chunk_layer.argtypes = [_P, _P, _P, _P, C.POINTER(C.c_int32), C.
 _lib.pd_decode_layer.argtypes = [_P, _P, _P, _P, C.c_int32, C.c_int32, C.POINTER(pd_kv_cache), _P, C.c_size_t, _P]
 _lib.pd_prefill_stack.argtypes = [C.POINTER(_P), C.POINTER(pd_kv_cache), C.c_int32, C.c_int32, _P, _P, C.c_int32, _P,
                                   C.POINTER(C.c_int32), C.c_int32, _P, C.c_size_t, _P]
+_lib.pd_prefill_chunk_stack.argtypes = [C.POINTER(_P), C.POINTER(pd_kv_cache), C.c_int32, C.c_int32, _P, _P, _P,
+                                        C.POINTER(C.c_int32), C.c_int32, _P, C.POINTER(C.c_int32), _P, C.c_size_t, _P]
 _lib.pd_decode_stack.argtypes = [C.POINTER(_P), C.POINTER(pd_kv_cache), C.c_int32, C.c_int32, _P, _P, C.c_int32, _P,
                                  C.c_int32, C.c_int32, _P, C.c_size_t, _P]
 _lib.pd_layer_check.argtypes = [_P, _P]
@@ -362,6 +371,16 @@ def pd_prefill_stack(layers, caches, x, out, io_on_host: bool, cu_seqlens_dev, c
                                  _ptr(workspace), workspace_bytes, _stream_ptr(stream)), "pd_prefill_stack")
 
 
+def pd_prefill_chunk_stack(layers, caches, x, out, cu_seqlens_dev, cu_seqlens_host, prefix_dev, prefix_host,
+                           workspace, workspace_bytes: int, stream=None):
+    cu = _i32_array(cu_seqlens_host)
+    pre = _i32_array(prefix_host)
+    _check(_lib.pd_prefill_chunk_stack(_layer_array(layers), _cache_array(caches), len(layers), len(caches), _ptr(x),
+                                       _ptr(out), _ptr(cu_seqlens_dev), cu, len(cu_seqlens_host) - 1, _ptr(prefix_dev),
+                                       pre, _ptr(workspace), workspace_bytes, _stream_ptr(stream)),
+           "pd_prefill_chunk_stack")
+
+
 def pd_decode_stack(layers, caches, x, out, io_on_host: bool, kv_len, batch: int, max_kv_len: int, workspace,
                     workspace_bytes: int, stream=None):
     _check(_lib.pd_decode_stack(_layer_array(layers), _cache_array(caches), len(layers), len(caches), _ptr(x),
@@ -449,14 +468,17 @@ def pd_gemm_fp8(a_codes, a_scales, b_codes, b_scales, c, m: int, n: int, k: int,
 def pd_measure(cfg: LayerConfig, *, n_layers_run: int, n_layers_model: int, warmup: int = 3, reps: int = 10,
                seed: int = 0, l_in=(), batch_sizes=(), kv_len_start: int = 0, n_steps: int = 1,
                step_stride: int = 1, kv_len_mix=None, peak_bf16_flops: float = 0.0,
-               peak_hbm_bytes_s: float = 0.0, vocab: int = 0) -> dict:
+               peak_hbm_bytes_s: float = 0.0, vocab: int = 0, chunk_tokens: int = 0, l_in_grid=()) -> dict:
     """vocab > 0 measures the whole-model step (embedding, final norm, LM head and greedy sampling added
-    to the prefill time and to every TPOT)."""
+    to the prefill time and to every TPOT); chunk_tokens > 0 measures chunked prefill; l_in_grid lists
+    lengths to be timed one request at a time (the service-time curve)."""
     l_arr = _i32_array(l_in) if len(l_in) else None
     b_arr = _i32_array(batch_sizes) if len(batch_sizes) else None
     mix = _i32_array(kv_len_mix) if kv_len_mix is not None else None
+    g_arr = _i32_array(l_in_grid) if len(l_in_grid) else None
     m = pd_measure_cfg(C.sizeof(pd_measure_cfg), n_layers_run, n_layers_model, warmup, reps, seed,
-                       l_arr, len(l_in), b_arr, len(batch_sizes), kv_len_start, n_steps, step_stride, mix, vocab)
+                       l_arr, len(l_in), b_arr, len(batch_sizes), kv_len_start, n_steps, step_stride, mix, vocab,
+                       chunk_tokens, g_arr, len(l_in_grid))
     out = pd_measurement()
     _check(_lib.pd_measure(C.byref(cfg.c_struct()), C.byref(m), peak_bf16_flops, peak_hbm_bytes_s, C.byref(out)),
            "pd_measure")
@@ -469,6 +491,9 @@ def pd_measure(cfg: LayerConfig, *, n_layers_run: int, n_layers_model: int, warm
         "attn_time_s": list(out.attn_time_s[:n]), "attn_frac_hbm_peak": list(out.attn_frac_hbm_peak[:n]),
         "gpu_launches": out.gpu_launches,
         "prefill_head_s": out.prefill_head_s, "decode_head_s": list(out.decode_head_s[:n]),
+        "prefill_chunks": out.prefill_chunks, "prefill_kv_ring": out.prefill_kv_ring,
+        "decode_kv_ring": list(out.decode_kv_ring[:n]), "attn_l2_resident": list(out.attn_l2_resident[:n]),
+        "grid_l": list(out.grid_l[:out.n_grid]), "grid_time_s": list(out.grid_time_s[:out.n_grid]),
     }
 
 

@@ -9,6 +9,12 @@ arrival stream through a FIFO server whose service times are the measured prefil
 compare the M/M/1 prediction of Eq. 12 with what a queue of real prefill passes does.
 Inputs are synthetic: shapes, length distributions and SLOs are those of the configurations.
 `--quick` shrinks grids and repetitions for smoke runs.
+
+This module holds loops and I/O only: every number comes from a call into the library (pd_measure,
+pd_allocate, pd_mixture_throughput, pd_interp_service_times, pd_mm1_sojourn, pd_mg1_sojourn,
+pd_refine_next_batch, pd_queue_replay).  Every allocation result is stored together with the exact
+inputs it was computed from ("inputs"), so that the result file can be re-checked later, on a machine
+without a GPU, against an independent implementation of the allocation equations.
 """
 from __future__ import annotations
 
@@ -36,50 +42,45 @@ def _peaks():
     return 1.4e15, 6.65e12, "fallback"
 
 
+ALLOC_KEYS = ("status", "tp_prefill_eff", "tp_decode_eff", "mu", "lam", "rho", "feasible_batch", "sweep_capped",
+              "n_prefill_frac", "n_decode_frac", "ratio_pd", "n_prefill", "n_decode", "n_prefill_ceil", "n_decode_ceil",
+              "achieved_total_tok_s")
+
+
 def _alloc(tp_total, l_in, l_out, ttft, tpot, tp_max, batch, tpot_s, t_overhead=0.0):
+    """pd_allocate, with the inputs recorded beside the result."""
     a = pd.pd_allocate(tp_total, l_in, l_out, ttft, tpot, tp_max, batch, tpot_s, t_overhead)
-    keys = ("status", "tp_prefill_eff", "tp_decode_eff", "rho", "feasible_batch", "sweep_capped", "n_prefill_frac",
-            "n_decode_frac", "ratio_pd", "n_prefill", "n_decode", "n_prefill_ceil", "n_decode_ceil",
-            "achieved_total_tok_s")
-    return {k: a[k] for k in keys}
+    out = {k: a[k] for k in ALLOC_KEYS}
+    out["inputs"] = {"tp_total_tok_s": float(tp_total), "l_in": float(l_in), "l_out": float(l_out),
+                     "ttft_slo_s": float(ttft), "tpot_slo_s": float(tpot), "prefill_max_tok_s": float(tp_max),
+                     "batch": [int(b) for b in batch], "tpot_s": [float(t) for t in tpot_s],
+                     "t_overhead_s": float(t_overhead)}
+    return out
 
 
 def _prefill_time_grid(cfg, lengths, n_layers_run, n_layers_model, reps, peaks):
-    """Measured prefill time of one request of each length (seconds, whole model)."""
-    out = {}
-    for ln in lengths:
-        m = pd.pd_measure(cfg, n_layers_run=n_layers_run, n_layers_model=n_layers_model, warmup=1, reps=reps, seed=0,
-                          l_in=[int(ln)], peak_bf16_flops=peaks[0], peak_hbm_bytes_s=peaks[1])
-        out[int(ln)] = {"time_s": m["prefill_time_s"], "frac_bf16_peak": m["prefill_frac_bf16_peak"]}
-    return out
+    """Measured prefill time of one request of each length (seconds, whole model): one pd_measure call, one
+    layer stack, every length timed on its own."""
+    m = pd.pd_measure(cfg, n_layers_run=n_layers_run, n_layers_model=n_layers_model, warmup=1, reps=reps, seed=0,
+                      l_in_grid=[int(l) for l in lengths], peak_bf16_flops=peaks[0], peak_hbm_bytes_s=peaks[1])
+    return {"l": m["grid_l"], "time_s": m["grid_time_s"]}
 
 
 def refine_feasible_batch(measure_tpot, batch, tpot_s, tpot_slo_s, max_probes=8):
     """Integer refinement of the TPOT-feasible batch (paper, "Acquire decode throughput ...": determine the batch
-    size that satisfies the target TPOT).  The sweep gives the largest feasible sweep point B_lo and the first
-    infeasible one B_hi; TPOT is measured at midpoints until the largest feasible integer is bracketed.
-    `measure_tpot(b)` returns the measured TPOT of batch b in seconds.  Returns (batch, tpot_s, probes)."""
-    pts = sorted(zip(batch, tpot_s))
-    lo = None
-    hi = None
-    for b, t in pts:
-        if t <= tpot_slo_s:
-            lo = (b, t)
-        else:
-            hi = (b, t)
+    size that satisfies the target TPOT): pd_refine_next_batch names the next batch size to measure until the
+    largest feasible integer is bracketed.  `measure_tpot(b)` returns the measured TPOT of batch b in seconds.
+    Returns the extended point lists (batch, tpot_s) and the probes made."""
+    batch, tpot_s, probes = list(batch), list(tpot_s), []
+    while len(probes) < max_probes:
+        nxt = pd.pd_refine_next_batch(batch, tpot_s, tpot_slo_s)
+        if nxt == 0:
             break
-    if lo is None or hi is None:
-        return (lo[0], lo[1], []) if lo else (0, float("nan"), [])
-    probes = []
-    while hi[0] - lo[0] > 1 and len(probes) < max_probes:
-        mid = (lo[0] + hi[0]) // 2
-        t = measure_tpot(mid)
-        probes.append((mid, t))
-        if t <= tpot_slo_s:
-            lo = (mid, t)
-        else:
-            hi = (mid, t)
-    return lo[0], lo[1], probes
+        t = measure_tpot(nxt)
+        batch.append(nxt)
+        tpot_s.append(t)
+        probes.append((nxt, t))
+    return batch, tpot_s, probes
 
 
 def run_tiny(quick=False):
@@ -118,36 +119,35 @@ def run_long_input(quick=False):
     cfg = pd.LayerConfig(**SHAPE_8B, max_pos=32768 + 256)
     nl = 4 if quick else 8
     lengths = gen.lognormal_lengths(1, 4096, 8192.0, 0.5, 2048, 32768)
-    grid_l = [2048, 8192, 32768] if quick else list(range(2048, 32768 + 1, 1024))
+    grid_l = [2048, 8192, 20480, 32768] if quick else list(range(2048, 32768 + 1, 512))
     grid = _prefill_time_grid(cfg, grid_l, nl, 32, 2 if quick else 3, peaks)
-    gl = np.array(sorted(grid))
-    gt = np.array([grid[int(l)]["time_s"] for l in gl])
     # interpolation check on seeded off-grid lengths
-    off = [int(v) for v in gen.uniform_lengths(2, 2 if quick else 8, 2100, 32000, sub=7)]
+    off = sorted(int(v) for v in gen.uniform_lengths(2, 2 if quick else 8, 2100, 32000, sub=7))
     off_meas = _prefill_time_grid(cfg, off, nl, 32, 2 if quick else 3, peaks)
-    interp_err = {str(l): float(np.interp(l, gl, gt) / off_meas[l]["time_s"] - 1.0) for l in off}
-    service = np.interp(lengths, gl, gt)
-    mean_l = float(lengths.mean())
-    tp_max = float(lengths.sum() / service.sum())          # mixture: total tokens over total time
-    mu = tp_max / mean_l                                    # Eq. 9 with the mean input length
+    off_interp = pd.pd_interp_service_times(grid["l"], grid["time_s"], off)
+    interp_check = [{"l": l, "measured_s": tm, "interpolated_s": float(ti)}
+                    for l, tm, ti in zip(off_meas["l"], off_meas["time_s"], off_interp)]
+    service = pd.pd_interp_service_times(grid["l"], grid["time_s"], lengths)
+    tp_max, mean_l = pd.pd_mixture_throughput(lengths, service)     # total tokens over total time; mean length
+    sweep = [1, 64] if quick else [1, 2, 4, 8, 16, 32, 64, 128, 256]
+    d = pd.pd_measure(cfg, n_layers_run=nl, n_layers_model=32, warmup=1, reps=3, seed=0, batch_sizes=sweep,
+                      kv_len_start=int(round(mean_l)), n_steps=256, step_stride=128,
+                      peak_bf16_flops=peaks[0], peak_hbm_bytes_s=peaks[1])
+    alloc = _alloc(2e5, mean_l, 256, 4.0, 0.050, tp_max, d["batch"], d["tpot_s"])
+    mu = alloc["mu"]                                                 # Eq. 9 with the mean input length
     n_arr = 20_000 if quick else 200_000
-    idx = np.arange(n_arr) % len(lengths)
-    svc = service[idx]
+    svc = service[np.arange(n_arr) % len(lengths)]
     replay = []
     for rho in ([0.5, 0.9] if quick else [0.1, 0.2, 0.3, 0.4, 0.5, 0.6, 0.7, 0.8, 0.9, 0.95]):
         lam = rho * mu
         gaps = gen.exponential_gaps(2, n_arr, lam)
         soj, wait = pd.pd_queue_replay(gaps, svc)
-        es, es2 = float(service.mean()), float((service ** 2).mean())
-        replay.append({"rho": rho, "lambda": lam, "mm1_sojourn_s": 1.0 / (mu - lam), "replayed_sojourn_s": soj,
-                       "pollaczek_khinchine_s": es + lam * es2 / (2.0 * (1.0 - lam * es))})
-    sweep = [1, 64] if quick else [1, 2, 4, 8, 16, 32, 64, 128, 256]
-    d = pd.pd_measure(cfg, n_layers_run=nl, n_layers_model=32, warmup=1, reps=3, seed=0, batch_sizes=sweep,
-                      kv_len_start=int(round(mean_l)), n_steps=256, step_stride=128,
-                      peak_bf16_flops=peaks[0], peak_hbm_bytes_s=peaks[1])
+        replay.append({"rho": rho, "lambda": lam, "mm1_sojourn_s": pd.pd_mm1_sojourn(mu, lam), "replayed_sojourn_s": soj,
+                       "pollaczek_khinchine_s": pd.pd_mg1_sojourn(service, lam)})
     return {"config": "long_input", "layers_run": nl, "sigma": 0.5, "mean_l_in": mean_l, "prefill_max_tok_s": tp_max,
-            "prefill_time_grid": grid, "interpolation_rel_err": interp_err, "queue": replay, "decode": d,
-            "allocation": _alloc(2e5, mean_l, 256, 4.0, 0.050, tp_max, d["batch"], d["tpot_s"])}
+            "prefill_time_grid": grid, "interpolation_check": interp_check, "queue": replay, "decode": d,
+            "lengths": {"generator": "pd_inputs.lognormal_lengths(1, 4096, 8192.0, 0.5, 2048, 32768)"},
+            "allocation": alloc}
 
 
 def run_decode_heavy(quick=False):
@@ -171,10 +171,9 @@ def run_decode_heavy(quick=False):
         a = _alloc(5e5, 512, 2048, 2.0, slo_ms * 1e-3, p["prefill_tok_s"], d["batch"], d["tpot_s"])
         if a["status"] == 0 and not a["sweep_capped"]:
             # the SLO binds between two sweep points: bracket the largest feasible integer batch by measurement
-            b_ref, t_ref, probes = refine_feasible_batch(tpot_at, d["batch"], d["tpot_s"], slo_ms * 1e-3,
+            b_all, t_all, probes = refine_feasible_batch(tpot_at, d["batch"], d["tpot_s"], slo_ms * 1e-3,
                                                          max_probes=3 if quick else 8)
-            a["refined"] = _alloc(5e5, 512, 2048, 2.0, slo_ms * 1e-3, p["prefill_tok_s"],
-                                  d["batch"] + [b_ref], d["tpot_s"] + [t_ref])
+            a["refined"] = _alloc(5e5, 512, 2048, 2.0, slo_ms * 1e-3, p["prefill_tok_s"], b_all, t_all)
             a["refined"]["probes"] = probes
         per_slo[str(slo_ms)] = a
     return {"config": "decode_heavy", "layers_run": nl, "ttft_slo_s": 2.0, "prefill": p, "decode": d,
@@ -194,11 +193,9 @@ def run_70b(quick=False):
     # mixed workload: L_in ~ U[1024, 8192], L_out ~ U[128, 1024]
     l_in = gen.uniform_lengths(3, 512, 1024, 8192, sub=0)
     l_out = gen.uniform_lengths(3, 512, 128, 1024, sub=1)
-    grid_l = [1024, 4096, 8192] if quick else list(range(1024, 8192 + 1, 1024))
+    grid_l = [1024, 4096, 8192] if quick else list(range(1024, 8192 + 1, 512))
     grid = _prefill_time_grid(cfg, grid_l, nl, 80, 2, peaks)
-    gl = np.array(sorted(grid))
-    gt = np.array([grid[int(l)]["time_s"] for l in gl])
-    tp_max_mix = float(l_in.sum() / np.interp(l_in, gl, gt).sum())
+    tp_max_mix, mean_l_in = pd.pd_mixture_throughput(l_in, pd.pd_interp_service_times(grid["l"], grid["time_s"], l_in))
     # stationary decode batch: sequence i sits at a uniformly random point of its output
     prog = gen.uniform_lengths(3, 512, 0, 10**6, sub=2) / 1e6
     mix = (l_in + np.floor(prog * l_out)).astype(np.int32)
@@ -207,70 +204,27 @@ def run_70b(quick=False):
                        peak_bf16_flops=peaks[0], peak_hbm_bytes_s=peaks[1])
     return {"config": "70b", "layers_run": nl, "layers_model": 80, "prefill": p, "decode": d,
             "allocation": _alloc(2e5, 4096, 256, 3.0, 0.060, p["prefill_tok_s"], d["batch"], d["tpot_s"]),
-            "mixed": {"mean_l_in": float(l_in.mean()), "mean_l_out": float(l_out.mean()),
+            "mixed": {"mean_l_in": mean_l_in, "mean_l_out": float(l_out.mean()),
                       "prefill_max_tok_s": tp_max_mix, "prefill_time_grid": grid, "decode": dm,
-                      "allocation": _alloc(2e5, float(l_in.mean()), float(l_out.mean()), 3.0, 0.060, tp_max_mix,
+                      "allocation": _alloc(2e5, mean_l_in, float(l_out.mean()), 3.0, 0.060, tp_max_mix,
                                            dm["batch"], dm["tpot_s"])}}
 
 
 def run_chunked(quick=False):
     """Maximum prefill throughput versus chunked-prefill size (paper, "Acquire prefill throughput ...": a larger
-    chunk raises the peak prefill throughput until saturation).  One request of L_in tokens is pushed through
-    the layer stack chunk by chunk with pd_prefill_chunk_layer; each chunk attends to the cached prefix."""
-    import statistics
-    import torch
+    chunk raises the peak prefill throughput until saturation).  One request of L_in tokens goes through the
+    layer stack chunk by chunk inside pd_measure (graph-captured like every other measured pass); each chunk
+    attends to the cached prefix."""
     peaks = _peaks()
     l_in = 4096 if quick else 8192
     nl = 2 if quick else 8
     cfg = pd.LayerConfig(**SHAPE_8B, max_pos=l_in)
-    dev = torch.device("cuda")
-    d = SHAPE_8B["d_model"]
-
-    def rnd(*shape, std=1.0, mean=0.0):
-        return (torch.randn(*shape, device=dev) * std + mean).to(torch.bfloat16)
-
-    layers, caches, keep = [], [], []
-    for _ in range(nl):
-        w = {"w_qkv": rnd(cfg.n_qkv, d, std=0.02), "w_o": rnd(d, d, std=0.02), "w_gate": rnd(SHAPE_8B["d_ff"], d, std=0.02),
-             "w_up": rnd(SHAPE_8B["d_ff"], d, std=0.02), "w_down": rnd(d, SHAPE_8B["d_ff"], std=0.02),
-             "g_attn": rnd(d, std=0.02, mean=1.0), "g_mlp": rnd(d, std=0.02, mean=1.0)}
-        layers.append(pd.Layer(cfg, w))
-        torch.cuda.synchronize()
-        k = torch.zeros((1, 8, l_in, 128), dtype=torch.bfloat16, device=dev)
-        v = torch.zeros_like(k)
-        keep += [k, v]
-        caches.append(pd.kv_cache_struct(k, v, 1, l_in))
-    ws_bytes = pd.pd_workspace_bytes(cfg, l_in, 0, 0)
-    ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
-    x = rnd(l_in, d)
-    bufs = [torch.empty_like(x), torch.empty_like(x)]
     out = {}
     for chunk in ([1024, 4096] if quick else [256, 512, 1024, 2048, 4096, 8192]):
-        metas = []
-        for c0 in range(0, l_in, chunk):
-            n = min(chunk, l_in - c0)
-            metas.append((c0, n, torch.tensor([0, n], dtype=torch.int32, device=dev),
-                          torch.tensor([c0], dtype=torch.int32, device=dev)))
-
-        def one_pass():
-            for c0, n, cu_dev, pre_dev in metas:          # chunk after chunk, each through the whole stack
-                src = x[c0:c0 + n]
-                for i, layer in enumerate(layers):
-                    dst = bufs[i & 1][:n]
-                    pd.pd_prefill_chunk_layer(layer, src, dst, cu_dev, [0, n], pre_dev, [c0], caches[i], ws, ws_bytes)
-                    src = dst
-        one_pass()
-        times = []
-        for _ in range(3 if quick else 5):
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record()
-            one_pass()
-            e1.record()
-            e1.synchronize()
-            times.append(e0.elapsed_time(e1) * 1e-3)
-        pd.pd_layer_check(layers[0])
-        t = statistics.median(times) * 32 / nl
-        out[str(chunk)] = {"time_s": t, "prefill_max_tok_s": l_in / t}
+        m = pd.pd_measure(cfg, n_layers_run=nl, n_layers_model=32, warmup=1, reps=3 if quick else 5, seed=0,
+                          l_in=[l_in], chunk_tokens=chunk, peak_bf16_flops=peaks[0], peak_hbm_bytes_s=peaks[1])
+        out[str(chunk)] = {"time_s": m["prefill_time_s"], "prefill_max_tok_s": m["prefill_tok_s"],
+                           "chunks": m["prefill_chunks"], "frac_bf16_peak": m["prefill_frac_bf16_peak"]}
     return {"config": "chunked", "l_in": l_in, "layers_run": nl, "chunk_sweep": out}
 
 

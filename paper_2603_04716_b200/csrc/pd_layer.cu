@@ -646,6 +646,36 @@ extern "C" pd_status pd_prefill_stack(pd_layer* const* layers, const pd_kv_cache
   return PD_OK;
 }
 
+extern "C" pd_status pd_prefill_chunk_stack(pd_layer* const* layers, const pd_kv_cache* caches, int32_t n_layers,
+                                            int32_t n_caches, const void* x, void* out, const int32_t* cu_dev,
+                                            const int32_t* cu_host, int32_t n_req, const int32_t* prefix_dev,
+                                            const int32_t* prefix_host, void* workspace, size_t workspace_bytes,
+                                            void* stream) {
+  if (!layers || !caches || n_layers <= 0 || n_caches <= 0 || !layers[0] || !prefix_dev || !prefix_host)
+    return PD_ERR_INVALID_ARG;
+  int tokens = 0, max_len = 0;
+  for (int i = 0; i < n_layers; ++i) {
+    if (!layers[i] || !same_shape(layers[i]->cfg, layers[0]->cfg)) return PD_ERR_INVALID_ARG;
+    PD_TRY(validate_prefill(layers[i], cu_host, n_req, &caches[i % n_caches], true, &tokens, &max_len, prefix_host));
+  }
+  if (tokens == 0) return PD_OK;
+  if (!x || !out || !workspace || !cu_dev) return PD_ERR_INVALID_ARG;
+  const Workspace w = carve(layers[0]->cfg, tokens, 0, 0);
+  if (workspace_bytes < w.total) return PD_ERR_WORKSPACE_TOO_SMALL;
+  if (reinterpret_cast<uintptr_t>(workspace) & 255u) return PD_ERR_INVALID_ARG;
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  bf16* buf[2] = {reinterpret_cast<bf16*>(ws + w.stage_a), reinterpret_cast<bf16*>(ws + w.stage_b)};
+  const bf16* cur = static_cast<const bf16*>(x);
+  for (int i = 0; i < n_layers; ++i) {
+    bf16* dst = (i == n_layers - 1) ? static_cast<bf16*>(out) : buf[(i + 1) & 1];
+    PD_TRY(prefill_impl(layers[i], cur, dst, cu_dev, n_req, tokens, max_len, nullptr, &caches[i % n_caches], ws, w, st,
+                        prefix_dev));
+    cur = dst;
+  }
+  return PD_OK;
+}
+
 extern "C" pd_status pd_decode_stack(pd_layer* const* layers, const pd_kv_cache* caches, int32_t n_layers,
                                      int32_t n_caches, const void* x, void* out, int32_t io_on_host,
                                      const int32_t* kv_len, int32_t B, int32_t max_kv_len, void* workspace,

@@ -189,53 +189,118 @@ extern "C" pd_status pd_measure(const pd_layer_cfg* cfg_in, const pd_measure_cfg
   long long timed_launches = 0;
 
   // ------------------------------------------------------------------ prefill
-  if (m->n_req > 0) {
-    std::vector<int32_t> cu(m->n_req + 1, 0);
+  // Median time of one prefill pass of the batch `lens` through the nl layers of the stack (not yet scaled to the
+  // model's layer count): in one piece, or, with chunk_tokens > 0, chunk after chunk, every chunk through all layers.
+  DevBuf x_keep, y_keep, cu_keep;  // buffers of the main batch, reused by the whole-model head below
+  auto measure_prefill = [&](const int32_t* lens, int n_req, bool keep, double* time_s, int* ring_out,
+                             int* chunks_out) -> pd_status {
+    std::vector<int32_t> cu(n_req + 1, 0);
     int max_len = 0;
+    for (int r = 0; r < n_req; ++r) {
+      if (lens[r] < 0 || lens[r] > cfg.max_pos) return PD_ERR_INVALID_ARG;
+      cu[r + 1] = cu[r] + lens[r];
+      max_len = std::max(max_len, lens[r]);
+    }
+    const int tokens = cu[n_req];
+    *time_s = 0.0; *ring_out = 0; *chunks_out = 0;
+    if (tokens == 0) return PD_OK;
+    const size_t cache_bytes = static_cast<size_t>(n_req) * max_len * kv_row;
+    const int ring = cache_ring(2 * cache_bytes, nl);
+    std::vector<DevBuf> kbuf(ring), vbuf(ring);
+    std::vector<pd_kv_cache> caches(ring);
+    for (int i = 0; i < ring; ++i) {
+      PD_CUDA_TRY(kbuf[i].alloc(cache_bytes));
+      PD_CUDA_TRY(vbuf[i].alloc(cache_bytes));
+      caches[i].struct_size = sizeof(pd_kv_cache);
+      caches[i].k = kbuf[i].p; caches[i].v = vbuf[i].p;
+      caches[i].batch_cap = n_req; caches[i].len_cap = max_len;
+    }
+    // chunk schedule: step s holds rows [s c, (s + 1) c) of every request that still has rows
+    const int chunk = m->chunk_tokens > 0 ? m->chunk_tokens : max_len;
+    const int n_steps = (max_len + chunk - 1) / chunk;
+    std::vector<int32_t> meta(static_cast<size_t>(n_steps) * (2 * n_req + 1));  // per step: cu[n_req + 1], prefix[n_req]
+    int max_chunk_tokens = 0;
+    for (int sidx = 0; sidx < n_steps; ++sidx) {
+      int32_t* cu_s = meta.data() + static_cast<size_t>(sidx) * (2 * n_req + 1);
+      int32_t* pre_s = cu_s + n_req + 1;
+      cu_s[0] = 0;
+      for (int r = 0; r < n_req; ++r) {
+        const int lo = std::min(lens[r], sidx * chunk), hi = std::min(lens[r], (sidx + 1) * chunk);
+        cu_s[r + 1] = cu_s[r] + (hi - lo);
+        pre_s[r] = lo;
+      }
+      max_chunk_tokens = std::max(max_chunk_tokens, cu_s[n_req]);
+    }
+    size_t ws_bytes = 0;
+    PD_TRY(pd_workspace_bytes(&cfg, max_chunk_tokens, 0, 0, &ws_bytes));
+    DevBuf ws, x_loc, y_loc, meta_dev;
+    DevBuf& x = keep ? x_keep : x_loc;
+    DevBuf& y = keep ? y_keep : y_loc;
+    PD_CUDA_TRY(ws.alloc(ws_bytes));
+    PD_CUDA_TRY(x.alloc(tokens * d * 2));
+    PD_CUDA_TRY(y.alloc(tokens * d * 2));
+    PD_CUDA_TRY(meta_dev.alloc(meta.size() * 4));
+    PD_CUDA_TRY(cudaMemcpyAsync(meta_dev.p, meta.data(), meta.size() * 4, cudaMemcpyHostToDevice, st));
+    if (keep) {
+      PD_CUDA_TRY(cu_keep.alloc(cu.size() * 4));
+      PD_CUDA_TRY(cudaMemcpyAsync(cu_keep.p, cu.data(), cu.size() * 4, cudaMemcpyHostToDevice, st));
+    }
+    PD_TRY(pd::launch_fill_normal(static_cast<bf16*>(x.p), tokens * d, m->seed, 1000, 0.f, 1.f, st));
+    std::vector<double> times;
+    long long per_run = 0;
+    PD_TRY(time_enqueued(
+        [&]() -> pd_status {
+          for (int sidx = 0; sidx < n_steps; ++sidx) {
+            const size_t off = static_cast<size_t>(sidx) * (2 * n_req + 1);
+            const int32_t* cu_h = meta.data() + off;
+            const int32_t* cu_d = static_cast<const int32_t*>(meta_dev.p) + off;
+            if (m->chunk_tokens > 0)
+              PD_TRY(pd_prefill_chunk_stack(stack.layers.data(), caches.data(), nl, ring, x.p, y.p, cu_d, cu_h, n_req,
+                                            cu_d + n_req + 1, cu_h + n_req + 1, ws.p, ws_bytes, st));
+            else
+              PD_TRY(pd_prefill_stack(stack.layers.data(), caches.data(), nl, ring, x.p, y.p, 0, cu_d, cu_h, n_req,
+                                      ws.p, ws_bytes, st));
+          }
+          return PD_OK;
+        },
+        st, ev, m->warmup, m->reps, &times, &per_run));
+    timed_launches += per_run * m->reps;
+    PD_TRY(pd_layer_check(stack.layers[0], st));
+    *time_s = median(times);
+    *ring_out = ring;
+    *chunks_out = n_steps;
+    return PD_OK;
+  };
+
+  if (m->n_grid < 0 || m->n_grid > PD_MEASURE_GRID_MAX || (m->n_grid > 0 && !m->l_in_grid) || m->chunk_tokens < 0)
+    return PD_ERR_INVALID_ARG;
+  for (int gi = 0; gi < m->n_grid; ++gi) {
+    if (m->l_in_grid[gi] <= 0) return PD_ERR_INVALID_ARG;
+    double t = 0.0;
+    int ring = 0, chunks = 0;
+    PD_TRY(measure_prefill(&m->l_in_grid[gi], 1, false, &t, &ring, &chunks));
+    out->grid_l[gi] = m->l_in_grid[gi];
+    out->grid_time_s[gi] = t * scale_layers;
+    out->n_grid = gi + 1;
+  }
+
+  if (m->n_req > 0) {
     double attn_flops = 0.0;
+    int tokens = 0;
     for (int r = 0; r < m->n_req; ++r) {
-      if (m->l_in[r] < 0 || m->l_in[r] > cfg.max_pos) return PD_ERR_INVALID_ARG;
-      cu[r + 1] = cu[r] + m->l_in[r];
-      max_len = std::max(max_len, m->l_in[r]);
       const double l = m->l_in[r];
       attn_flops += 4.0 * cfg.n_q_heads * cfg.head_dim * (l * (l + 1.0) / 2.0);
+      tokens += m->l_in[r] > 0 ? m->l_in[r] : 0;
     }
-    const int tokens = cu[m->n_req];
+    double t_run = 0.0;
+    PD_TRY(measure_prefill(m->l_in, m->n_req, true, &t_run, &out->prefill_kv_ring, &out->prefill_chunks));
     if (tokens > 0) {
       const double gemm_flops = 2.0 * tokens * static_cast<double>(layer_param_count(cfg));
       out->prefill_flops = (gemm_flops + attn_flops) * m->n_layers_model;
-
-      const size_t cache_bytes = static_cast<size_t>(m->n_req) * max_len * kv_row;
-      const int ring = cache_ring(2 * cache_bytes, nl);
-      std::vector<DevBuf> kbuf(ring), vbuf(ring);
-      std::vector<pd_kv_cache> caches(ring);
-      for (int i = 0; i < ring; ++i) {
-        PD_CUDA_TRY(kbuf[i].alloc(cache_bytes));
-        PD_CUDA_TRY(vbuf[i].alloc(cache_bytes));
-        caches[i].struct_size = sizeof(pd_kv_cache);
-        caches[i].k = kbuf[i].p; caches[i].v = vbuf[i].p;
-        caches[i].batch_cap = m->n_req; caches[i].len_cap = max_len;
-      }
-      size_t ws_bytes = 0;
-      PD_TRY(pd_workspace_bytes(&cfg, tokens, 0, 0, &ws_bytes));
-      DevBuf ws, x, y, cu_dev;
-      PD_CUDA_TRY(ws.alloc(ws_bytes));
-      PD_CUDA_TRY(x.alloc(tokens * d * 2));
-      PD_CUDA_TRY(y.alloc(tokens * d * 2));
-      PD_CUDA_TRY(cu_dev.alloc(cu.size() * 4));
-      PD_CUDA_TRY(cudaMemcpyAsync(cu_dev.p, cu.data(), cu.size() * 4, cudaMemcpyHostToDevice, st));
-      PD_TRY(pd::launch_fill_normal(static_cast<bf16*>(x.p), tokens * d, m->seed, 1000, 0.f, 1.f, st));
-      std::vector<double> times;
-      long long per_run = 0;
-      PD_TRY(time_enqueued(
-          [&] {
-            return pd_prefill_stack(stack.layers.data(), caches.data(), nl, ring, x.p, y.p, 0,
-                                    static_cast<const int32_t*>(cu_dev.p), cu.data(), m->n_req, ws.p, ws_bytes, st);
-          },
-          st, ev, m->warmup, m->reps, &times, &per_run));
-      timed_launches += per_run * m->reps;
-      PD_TRY(pd_layer_check(stack.layers[0], st));
-      out->prefill_time_s = median(times) * scale_layers;
+      out->prefill_time_s = t_run * scale_layers;
+      DevBuf& x = x_keep;
+      DevBuf& y = y_keep;
+      DevBuf& cu_dev = cu_keep;
       if (model.m) {  // embedding in front, final norm + LM head + sampling behind: once per pass
         const std::vector<int32_t> tok = synthetic_tokens(tokens, m->vocab, m->seed);
         DevBuf tok_dev, sel, norm, logits, next;
@@ -404,9 +469,18 @@ extern "C" pd_status pd_measure(const pd_layer_cfg* cfg_in, const pd_measure_cfg
       if (model.m)  // LM head once, embedding rows, logits written and read back by the sampler
         out->decode_bytes[pi] += static_cast<double>(m->vocab) * d * 2 + 2.0 * B * d * 2 + 2.0 * B * m->vocab * 4.0;
       out->attn_time_s[pi] = attn_time;
+      out->decode_kv_ring[pi] = ring;
+      // The attention-only pass walks `ring` distinct K/V buffers back to back.  When all of them together stay
+      // below twice the L2 size, part of the "HBM" stream is served from L2 and the rate is not an HBM figure.
+      {
+        int dev = 0, l2 = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&l2, cudaDevAttrL2CacheSize, dev) != cudaSuccess)
+          l2 = 128 << 20;
+        out->attn_l2_resident[pi] = (kv_bytes_layer * ring < 2.0 * l2) ? 1 : 0;
+      }
       if (peak_hbm_bytes_s > 0) {
         out->decode_frac_hbm_peak[pi] = out->decode_bytes[pi] / out->tpot_s[pi] / peak_hbm_bytes_s;
-        out->attn_frac_hbm_peak[pi] = kv_bytes_layer / attn_time / peak_hbm_bytes_s;
+        if (!out->attn_l2_resident[pi]) out->attn_frac_hbm_peak[pi] = kv_bytes_layer / attn_time / peak_hbm_bytes_s;
       }
     }
   }

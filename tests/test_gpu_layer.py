@@ -285,6 +285,16 @@ def test_argument_errors(pdlib):
     with pytest.raises(pdlib.PdError) as e:        # batch beyond the cache
         pdlib.pd_decode_layer(dl.layer, x, x, i32_dev([0, 0, 0]), 3, 1, cache, dl.ws, dl.ws_bytes)
     assert e.value.status == pdlib.PD_ERR_INVALID_ARG
+    # a stack whose layers differ in shape is refused before anything is launched
+    wide = dict(TINY, d_ff=3072)
+    _, _, dl_wide = setup(pdlib, wide, 64, 64, 2, 64)
+    for call in (lambda: pdlib.pd_prefill_stack([dl.layer, dl_wide.layer], [cache], x, x, False, i32_dev([0, 64]), [0, 64],
+                                                dl.ws, dl.ws_bytes),
+                 lambda: pdlib.pd_decode_stack([dl.layer, dl_wide.layer], [cache], x, x, False, i32_dev([3, 3]), 2, 4,
+                                               dl.ws, dl.ws_bytes)):
+        with pytest.raises(pdlib.PdError) as e:
+            call()
+        assert e.value.status == pdlib.PD_ERR_INVALID_ARG
     # empty inputs are accepted
     pdlib.pd_prefill_layer(dl.layer, x, x, i32_dev([0, 0]), [0, 0], cache, dl.ws, dl.ws_bytes)
     pdlib.pd_decode_layer(dl.layer, x, x, i32_dev([0]), 0, 1, cache, dl.ws, dl.ws_bytes)

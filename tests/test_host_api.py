@@ -33,7 +33,10 @@ def test_struct_sizes_match_c_layout(pdlib):
     assert ctypes.sizeof(pdlib.pd_kv_cache) == 32
     assert ctypes.sizeof(pdlib.pd_alloc_in) == 8 + 7 * 8 + 8 + 16
     assert ctypes.sizeof(pdlib.pd_alloc_out) == 8 + 5 * 8 + 8 + 3 * 8 + 16 + 8
-    assert ctypes.sizeof(pdlib.pd_measurement) == 8 + 4 * 8 + 8 + 32 * 4 + 5 * 32 * 8 + 8 + 8 + 32 * 8
+    assert ctypes.sizeof(pdlib.pd_measurement) == (8 + 4 * 8 + 8 + 32 * 4 + 5 * 32 * 8 + 8 + 8 + 32 * 8
+                                                   + 8 + 2 * 32 * 4 + 8 + 128 * 4 + 128 * 8)
+    # 5 x 4 (+4 pad) | seed 8 | l_in 8 | n_req 4 (+4) | batch_sizes 8 | 4 x 4 | kv_len_mix 8 | 2 x 4 | l_in_grid 8 | n_grid 4 (+4)
+    assert ctypes.sizeof(pdlib.pd_measure_cfg) == 24 + 8 + 8 + 8 + 8 + 16 + 8 + 8 + 8 + 8
 
 
 def _same(a, b):

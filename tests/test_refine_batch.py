@@ -21,12 +21,14 @@ def test_refinement_finds_largest_feasible_integer(pdlib):
         tp = [curve(b) for b in sweep]
         slo = rnd.uniform(b0 + a, b0 + 600 * a)
         calls = []
-        got, t, probes = cfgs.refine_feasible_batch(lambda b: (calls.append(b), curve(b))[1], sweep, tp, slo, max_probes=12)
+        b_all, t_all, probes = cfgs.refine_feasible_batch(lambda b: (calls.append(b), curve(b))[1], sweep, tp, slo,
+                                                          max_probes=12)
+        got = pdlib.pd_allocate(1e5, 512, 512, 2.0, slo, 5e4, b_all, t_all)["feasible_batch"]
         feas = [b for b in range(1, 513) if curve(b) <= slo]
         if not feas:
-            assert got == 0
+            assert got == 0 and not calls
         elif max(feas) == 512:
             assert got == 512 and not calls            # capped by the sweep: nothing to refine
         else:
-            assert got == max(feas) and t == curve(got)
-            assert len(calls) <= 9
+            assert got == max(feas) and t_all[b_all.index(got)] == curve(got)
+            assert len(calls) <= 9 and [p[0] for p in probes] == calls

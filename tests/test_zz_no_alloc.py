@@ -1,4 +1,4 @@
-"""GPU: the allocation-free decode attention against the ordinary entry point.
+"""GPU: the allocation-free decode attention against the ordinary entry point and against the oracle.
 
 pd_decode_attention_noalloc serves callers that cannot cudaMalloc a workspace (a process
 whose memory pool owns the device, code under stream capture, a loop that must avoid the
@@ -11,6 +11,7 @@ import numpy as np
 import pytest
 
 import pd_inputs as gen
+from oracle import decoder_layer as L
 from gpu_util import assert_close, from_dev, i32_dev, to_dev, empty_bf16
 
 pytestmark = pytest.mark.gpu
@@ -30,6 +31,18 @@ def _both(pd, cfg, q, kv_len, cache, cap):
     return from_dev(got), from_dev(ref)
 
 
+def _oracle(hq, hkv, hd, q, k0, v0, kv_len):
+    """The oracle's attention core on each sequence: entries 0 .. kv_len[b] of cache slot b."""
+    ocfg = L.LayerConfig(d_model=hq * hd, n_q_heads=hq, n_kv_heads=hkv, head_dim=hd, d_ff=64)
+    out = np.empty((len(kv_len), hq * hd))
+    for b, n in enumerate(kv_len):
+        keys = k0[b, :, :n + 1].transpose(1, 0, 2).astype(np.float64)
+        vals = v0[b, :, :n + 1].transpose(1, 0, 2).astype(np.float64)
+        qb = q[b].reshape(1, hq, hd).astype(np.float64)
+        out[b] = L._attend(qb, keys, vals, np.array([n]), np.arange(n + 1), ocfg, None)[0]
+    return out
+
+
 def test_noalloc_matches_workspace_version_twice(pdlib):
     hq, hkv, hd, cap = 32, 8, 128, 2304
     cfg = pdlib.LayerConfig(hq * hd, hq, hkv, hd, 64)
@@ -40,10 +53,12 @@ def test_noalloc_matches_workspace_version_twice(pdlib):
     q1 = gen.normal_bf16(21, gen.S_X, (4, hq * hd), 1.0, sub=1)
     got1, ref1 = _both(pdlib, cfg, q1, [2303, 1500, 700, 5], cache, cap)
     assert_close(got1, ref1, "first call")
+    assert_close(got1, _oracle(hq, hkv, hd, q1, k0, v0, [2303, 1500, 700, 5]), "first call against the oracle")
     # second call straight after: other inputs, fewer sequences, a different split count
     q2 = gen.normal_bf16(21, gen.S_X, (2, hq * hd), 1.0, sub=2)
     got2, ref2 = _both(pdlib, cfg, q2, [900, 1023], cache, 1024)
     assert_close(got2, ref2, "second call")
+    assert_close(got2, _oracle(hq, hkv, hd, q2, k0, v0, [900, 1023]), "second call against the oracle")
     assert np.abs(ref2).max() > 0.01
 
 
