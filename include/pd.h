@@ -328,6 +328,18 @@ pd_status pd_quantize_fp8_rows(const void* x, int32_t ldx, int32_t rows, int32_t
 pd_status pd_gemm_fp8(const void* a_codes, const float* a_scales, const void* b_codes, const float* b_scales,
                       void* c, int32_t m, int32_t n, int32_t k, int32_t* err_word, void* stream);
 
+/* Failure-detection test hook.  Every wait inside the tensor-core kernels (on a tile load, an accumulator, a
+ * partner block) is bounded by wall clock (4 s); when a wait gives up, the block raises its abort flag, leaves
+ * through the normal teardown (tensor memory freed, cluster barrier of a CTA pair passed) and sets the error
+ * word that pd_layer_check / the err_word arguments report as PD_ERR_DEVICE_TIMEOUT.  This call arms ONE such
+ * event for the calling thread: the next launch of the named kernel kind runs with the bound wait_limit_ns
+ * (between 0.1 ms and 4 s) and its producer leaves out one operand tile load, so that a wait runs into the
+ * bound.  Nothing faults or spins without a limit; the output of that launch is undefined, later launches are
+ * unaffected.  PD_INJECT_NONE disarms.  (The paper has no counterpart; it exists so that the timeout path can
+ * be exercised without a real fault.) */
+enum { PD_INJECT_NONE = 0, PD_INJECT_ATTN_PREFILL = 1, PD_INJECT_GEMM = 2, PD_INJECT_GEMM_PAIR = 3 };
+pd_status pd_test_inject_wait_timeout(int32_t kernel_kind, uint64_t wait_limit_ns);
+
 /* Kernels launched so far by the calling thread through this library. */
 int64_t pd_launch_count(void);
 

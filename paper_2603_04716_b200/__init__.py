@@ -39,7 +39,7 @@ EXPORTS = [
     "pd_model_create", "pd_model_destroy", "pd_model_workspace_bytes", "pd_model_prefill", "pd_model_decode_step",
     "pd_model_check", "pd_allocate_ext", "pd_quantize_fp8_rows", "pd_gemm_fp8", "pd_workspace_offsets",
     "pd_prefill_attention", "pd_mixture_throughput", "pd_interp_service_times", "pd_mm1_sojourn", "pd_mg1_sojourn",
-    "pd_refine_next_batch", "pd_prefill_chunk_stack",
+    "pd_refine_next_batch", "pd_prefill_chunk_stack", "pd_test_inject_wait_timeout",
 ]
 
 TRACE_CLASSES = ["gemm_qkv", "gemm_o", "gemm_gate_up", "gemm_down", "attn_prefill", "attn_decode", "rmsnorm",
@@ -237,6 +237,15 @@ class LayerConfig:
     @property
     def n_qkv(self) -> int:
         return (self.n_q_heads + 2 * self.n_kv_heads) * self.head_dim
+
+
+INJECT_NONE, INJECT_ATTN_PREFILL, INJECT_GEMM, INJECT_GEMM_PAIR = 0, 1, 2, 3
+_lib.pd_test_inject_wait_timeout.argtypes = [C.c_int32, C.c_uint64]
+
+
+def pd_test_inject_wait_timeout(kernel_kind: int, wait_limit_ns: int):
+    """Arms one injected wait timeout for the calling thread's next launch of that kernel kind."""
+    _check(_lib.pd_test_inject_wait_timeout(kernel_kind, wait_limit_ns), "pd_test_inject_wait_timeout")
 
 
 def pd_version() -> int:

@@ -77,6 +77,11 @@ cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t sme
   return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
 }
 
+// Test hook behind pd_test_inject_wait_timeout: true (once) if the calling thread armed an injection for this
+// kind of kernel; the launcher then gives the kernel the short wait bound and tells its producer to leave out
+// one tile load.
+bool take_wait_injection(int kind, unsigned long long* limit_ns);
+
 // Brackets the kernels launched in its scope with CUDA events while a trace is active
 // (pd_trace_begin .. pd_trace_end); free otherwise.
 class TraceScope {
@@ -214,6 +219,13 @@ struct PrefillAttnArgs {
   const int32_t* prefix;      // device [n_req] cached tokens before each request's rows, or NULL
   int n_req, n_tokens, max_len;
   int n_q_heads, n_kv_heads, head_dim, len_cap, batch_cap;
+  // Two device ints (work-item counter, finished-block counter) that are zero between launches; NULL takes a
+  // pair from a pool inside the library.  Launches sharing a pair must be ordered on one stream.
+  int* sched = nullptr;
+  // Test hooks: a shorter bound (ns) for the kernel's waits (0 = the default of 4 s), and a producer that leaves
+  // out one K tile load so that a wait runs into that bound.
+  unsigned long long wait_limit_ns = 0;
+  int test_skip_load = 0;
 };
 // Causal GQA attention of a packed ragged batch on tcgen05 / tensor memory.
 pd_status launch_prefill_attention_tc(const PrefillAttnArgs& a, int* err_word, cudaStream_t s);
@@ -255,4 +267,5 @@ struct pd_layer {
   float2* rope_tab;                        // [max_pos, hd/2]
   int* err_word;                           // device int32
   int* split_flags;                        // device int32[kSplitMaxTiles * 4], see GemmArgs
+  int* attn_sched;                         // device int32[2], work counters of the prefill-attention kernel
 };

@@ -107,6 +107,8 @@ struct GemmDev {
   int* split_flags;      // [tail tile][4], 1 while a partial waits to be consumed
   int split_enable;
   int* err_word;
+  unsigned long long wait_limit_ns;  // bound of every wait inside the kernel
+  int test_skip_load;                // test hook: the producer leaves out the A tile of its second K block
   const float* scale_a;  // FP8 operands: per-row scale of A [M] and of B [N]
   const float* scale_b;
   RopeEpilogue rope;  // EPI_ROPE_KV only
@@ -413,11 +415,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         int tm, tn;
         tile_coords(ui.tile, p.tiles_m, p.tiles_n, p.raster_group, tm, tn);
         for (int kb = ui.kb_lo; kb < ui.kb_hi; ++kb) {
-          if (!ptx::mbar_wait_bounded(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
+          if (!ptx::mbar_wait_bounded(empty_bar(stage), phase ^ 1u, abort_flag, p.wait_limit_ns)) { ok = false; break; }
           const uint32_t sa = smem_base + stage * Cfg::STAGE_BYTES;
           const uint32_t sb = sa + Cfg::A_BYTES;
           ptx::mbar_arrive_expect_tx(full_bar(stage), Cfg::STAGE_BYTES);
-          ptx::tma_load_2d(sa, &tmap_a, kb * KE, tm * BM, full_bar(stage));
+          if (!(p.test_skip_load && unit == static_cast<int>(blockIdx.x) && kb == ui.kb_lo + 1))
+            ptx::tma_load_2d(sa, &tmap_a, kb * KE, tm * BM, full_bar(stage));
           ptx::tma_load_2d(sb, &tmap_b, kb * KE, tn * BN, full_bar(stage));
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
@@ -439,11 +442,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       bool ok = true;
       for (int unit = blockIdx.x; unit < n_units && ok; unit += gridDim.x) {
         const UnitInfo ui = unit_info(unit, p.main_tiles, k_blocks, p.tail_halves);
-        if (!ptx::mbar_wait_bounded(acce_bar(acc), acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+        if (!ptx::mbar_wait_bounded(acce_bar(acc), acc_phase ^ 1u, abort_flag, p.wait_limit_ns)) { ok = false; break; }
         ptx::tc_fence_after();
         const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * Cfg::ACC_COLS);
         for (int kb = ui.kb_lo; kb < ui.kb_hi; ++kb) {
-          if (!ptx::mbar_wait_bounded(full_bar(stage), phase, abort_flag)) { ok = false; break; }
+          if (!ptx::mbar_wait_bounded(full_bar(stage), phase, abort_flag, p.wait_limit_ns)) { ok = false; break; }
           ptx::tc_fence_after();
           const uint32_t sa = smem_base + stage * Cfg::STAGE_BYTES;
           const uint32_t sb = sa + Cfg::A_BYTES;
@@ -479,7 +482,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       int tm, tn;
       tile_coords(ui.tile, p.tiles_m, p.tiles_n, p.raster_group, tm, tn);
       // warp-uniform outcome: tcgen05.ld below needs the whole warp
-      ok = __all_sync(0xffffffffu, ptx::mbar_wait_bounded(accf_bar(acc), acc_phase, abort_flag));
+      ok = __all_sync(0xffffffffu, ptx::mbar_wait_bounded(accf_bar(acc), acc_phase, abort_flag, p.wait_limit_ns));
       if (!ok) break;
       ptx::tc_fence_after();
       const int row = tm * BM + lane_group * 32 + lane;
@@ -512,7 +515,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             const uint64_t t0 = ptx::globaltimer_ns();
             uint32_t spins = 0;
             while (*reinterpret_cast<volatile int*>(flag) != 1) {
-              if ((++spins & 1023u) == 0u && (*abort_flag || ptx::globaltimer_ns() - t0 > 4000000000ull)) {
+              if ((++spins & 1023u) == 0u && (*abort_flag || ptx::globaltimer_ns() - t0 > p.wait_limit_ns)) {
                 *abort_flag = 1;
                 seen = false;
                 break;
@@ -627,12 +630,13 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
         tile_coords(ui.tile, tiles_m2, p.tiles_n, group2, tm2, tn);
         const bool half = ui.role == 3;  // this CTA then supplies 64 of the half tile's 128 rows of B
         for (int kb = 0; kb < k_blocks; ++kb) {
-          if (!ptx::mbar_wait_bounded(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
+          if (!ptx::mbar_wait_bounded(empty_bar(stage), phase ^ 1u, abort_flag, p.wait_limit_ns)) { ok = false; break; }
           const uint32_t sa = smem_base + stage * P2_STAGE_BYTES;
           const uint32_t sb = sa + BM * 128;
           const uint32_t lead_full = ptx::map_to_cta(full_bar(stage), 0);
           if (rank == 0) ptx::mbar_arrive_expect_tx(full_bar(stage), half ? 2 * (BM + 64) * 128 : 2 * P2_STAGE_BYTES);
-          ptx::tma_load_2d_pair(sa, &tmap_a, kb * KE, (2 * tm2 + static_cast<int>(rank)) * BM, lead_full);
+          if (!(p.test_skip_load && rank == 0 && unit == pair_id && kb == 1))
+            ptx::tma_load_2d_pair(sa, &tmap_a, kb * KE, (2 * tm2 + static_cast<int>(rank)) * BM, lead_full);
           if (half)
             ptx::tma_load_2d_pair(sb, &tmap_b_half, kb * KE, tn * BN + ui.n_half * 128 + static_cast<int>(rank) * 64, lead_full);
           else
@@ -653,11 +657,11 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
       bool ok = true;
       for (int unit = pair_id; unit < n_units && ok; unit += n_pairs) {
         const uint32_t idesc = unit < p.main_tiles ? idesc_full : idesc_half;
-        if (!ptx::mbar_wait_bounded(acce_bar(acc), acc_phase ^ 1u, abort_flag)) break;
+        if (!ptx::mbar_wait_bounded(acce_bar(acc), acc_phase ^ 1u, abort_flag, p.wait_limit_ns)) break;
         ptx::tc_fence_after();
         const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * BN);
         for (int kb = 0; kb < k_blocks; ++kb) {
-          if (!ptx::mbar_wait_bounded(full_bar(stage), phase, abort_flag)) { ok = false; break; }
+          if (!ptx::mbar_wait_bounded(full_bar(stage), phase, abort_flag, p.wait_limit_ns)) { ok = false; break; }
           ptx::tc_fence_after();
           const uint32_t sa = smem_base + stage * P2_STAGE_BYTES;
           const uint64_t da = ptx::umma_desc_sw128(sa);
@@ -686,7 +690,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
       int tm2, tn;
       tile_coords(ui.tile, tiles_m2, p.tiles_n, group2, tm2, tn);
       const int tm = 2 * tm2 + static_cast<int>(rank);
-      if (!__all_sync(0xffffffffu, ptx::mbar_wait_bounded(accf_bar(acc), acc_phase, abort_flag))) break;
+      if (!__all_sync(0xffffffffu, ptx::mbar_wait_bounded(accf_bar(acc), acc_phase, abort_flag, p.wait_limit_ns))) break;
       ptx::tc_fence_after();
       const int row = tm * BM + lane_group * 32 + lane;
       const uint32_t t_row = tmem_base + (static_cast<uint32_t>(lane_group * 32) << 16) + static_cast<uint32_t>(acc * BN);
@@ -743,6 +747,8 @@ pd_status launch_tc(const GemmArgs& g, cudaStream_t stream) {
   p.tiles_m = (g.m + BM - 1) / BM;
   p.tiles_n = (g.n + BN - 1) / BN;
   p.err_word = g.err_word;
+  p.wait_limit_ns = 4000000000ull;
+  if (take_wait_injection(PD_INJECT_GEMM, &p.wait_limit_ns)) p.test_skip_load = 1;
   {
     // keep a group's A slab (group x 128 rows x K) within about 40 MB of L2
     long long grp = (40ll << 20) / (static_cast<long long>(BM) * g.k * 2);
@@ -826,6 +832,8 @@ pd_status launch_tc_pair(const GemmArgs& g, cudaStream_t stream) {
   p.tiles_m = (g.m + BM - 1) / BM;
   p.tiles_n = g.n / 256;
   p.err_word = g.err_word;
+  p.wait_limit_ns = 4000000000ull;
+  if (take_wait_injection(PD_INJECT_GEMM_PAIR, &p.wait_limit_ns)) p.test_skip_load = 1;
   {
     long long grp = (40ll << 20) / (static_cast<long long>(BM) * g.k * (F8 ? 1 : 2));
     p.raster_group = static_cast<int>(grp < 4 ? 4 : (grp > 32 ? 32 : grp));

@@ -223,6 +223,7 @@ pd_status prefill_impl(pd_layer* L, const bf16* x, bf16* out, const int32_t* cu_
   a.n_req = n_req; a.n_tokens = tokens; a.max_len = max_len;
   a.n_q_heads = c.n_q_heads; a.n_kv_heads = c.n_kv_heads; a.head_dim = c.head_dim; a.len_cap = cache->len_cap;
   a.batch_cap = cache->batch_cap;
+  a.sched = L->attn_sched;
   {
     pd::TraceScope ts(PD_K_ATTN_PREFILL, st);
     PD_TRY(pd::launch_prefill_attention_tc(a, L->err_word, st));
@@ -416,6 +417,8 @@ extern "C" pd_status pd_layer_create(const pd_layer_cfg* cfg, const pd_layer_wei
   if ((e = cudaMalloc(&L->err_word, sizeof(int))) != cudaSuccess) return fail(e);
   if ((e = cudaMalloc(&L->split_flags, pd::kSplitMaxTiles * 4 * sizeof(int))) != cudaSuccess) return fail(e);
   if ((e = cudaMemsetAsync(L->split_flags, 0, pd::kSplitMaxTiles * 4 * sizeof(int), st)) != cudaSuccess) return fail(e);
+  if ((e = cudaMalloc(&L->attn_sched, 2 * sizeof(int))) != cudaSuccess) return fail(e);
+  if ((e = cudaMemsetAsync(L->attn_sched, 0, 2 * sizeof(int), st)) != cudaSuccess) return fail(e);
   const cudaMemcpyKind d2d = cudaMemcpyDeviceToDevice;
   if ((e = cudaMemcpyAsync(L->w_qkv, w->w_qkv, L->n_qkv * d * 2, d2d, st)) != cudaSuccess) return fail(e);
   if ((e = cudaMemcpyAsync(L->w_o, w->w_o, d * hq * 2, d2d, st)) != cudaSuccess) return fail(e);
@@ -469,6 +472,7 @@ extern "C" pd_status pd_layer_destroy(pd_layer* L) {
   cudaFree(L->q_qkv); cudaFree(L->q_o); cudaFree(L->q_gu); cudaFree(L->q_down);
   cudaFree(L->s_qkv); cudaFree(L->s_o); cudaFree(L->s_gu); cudaFree(L->s_down);
   cudaFree(L->g_attn); cudaFree(L->g_mlp); cudaFree(L->rope_tab); cudaFree(L->err_word); cudaFree(L->split_flags);
+  cudaFree(L->attn_sched);
   delete L;
   return PD_OK;
 }
@@ -483,6 +487,7 @@ extern "C" pd_status pd_layer_check(pd_layer* L, void* stream) {
     PD_CUDA_TRY(cudaMemsetAsync(L->err_word, 0, sizeof(int), st));
     // an aborted K-split GEMM may have left a hand-over flag raised
     PD_CUDA_TRY(cudaMemsetAsync(L->split_flags, 0, pd::kSplitMaxTiles * 4 * sizeof(int), st));
+    PD_CUDA_TRY(cudaMemsetAsync(L->attn_sched, 0, 2 * sizeof(int), st));
     return word == 2 ? PD_ERR_INVALID_ARG : PD_ERR_DEVICE_TIMEOUT;
   }
   return PD_OK;

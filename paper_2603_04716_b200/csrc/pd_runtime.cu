@@ -18,6 +18,18 @@ bool pdl_enabled() {
   return on;
 }
 
+namespace {
+thread_local int t_inject_kind = 0;
+thread_local unsigned long long t_inject_limit_ns = 0;
+}  // namespace
+
+bool take_wait_injection(int kind, unsigned long long* limit_ns) {
+  if (t_inject_kind != kind) return false;
+  t_inject_kind = 0;
+  *limit_ns = t_inject_limit_ns;
+  return true;
+}
+
 pd_status cuda_fail(cudaError_t e) {
   g_last_cuda_error = static_cast<int>(e);
   return PD_ERR_CUDA;
@@ -58,6 +70,14 @@ TraceScope::~TraceScope() {
 }
 
 }  // namespace pd
+
+extern "C" pd_status pd_test_inject_wait_timeout(int32_t kernel_kind, uint64_t wait_limit_ns) {
+  if (kernel_kind < PD_INJECT_NONE || kernel_kind > PD_INJECT_GEMM_PAIR) return PD_ERR_INVALID_ARG;
+  if (kernel_kind != PD_INJECT_NONE && (wait_limit_ns < 100000ull || wait_limit_ns > 4000000000ull)) return PD_ERR_INVALID_ARG;
+  pd::t_inject_kind = kernel_kind;
+  pd::t_inject_limit_ns = wait_limit_ns;
+  return PD_OK;
+}
 
 extern "C" int pd_last_cuda_error(void) { return pd::g_last_cuda_error; }
 extern "C" int64_t pd_launch_count(void) { return pd::g_launch_count; }
