@@ -4,8 +4,9 @@
 // softmax and MMAs ping-pong.  One block per SM stays resident and takes items, longest first, from a
 // counter in global memory until none is left, so that barrier and tensor-memory set-up happen once per
 // SM and the loads of the next item run while the current one drains.
-//   warp 0      : producer  - fetches and decodes items, publishes them in a shared-memory ring, loads Q
-//                             (one buffer per row tile) and the K / V tiles of 128 keys (3 K slots, 2 V slots)
+//   warp 0      : producer  - fetches and decodes items, publishes them in a shared-memory ring, loads the
+//                             K / V tiles of 128 keys (3 K slots, 2 V slots)
+//   warp 10     : Q loader  - loads each item's Q tiles (one buffer per row tile) as the buffers fall free
 //   warp 1      : MMA issuer - S = Q K^T (both operands in shared memory, fp32 S in tensor memory) and
 //                             O += P V (P read from tensor memory, V as an MN-major operand); event driven:
 //                             it issues whichever row tile's next product has its inputs ready, so a tile
@@ -33,7 +34,7 @@ namespace {
 
 constexpr int TQ = 128;                    // rows per tile
 constexpr int TK = 128;                    // keys per KV tile
-constexpr int ATT_THREADS = 320;
+constexpr int ATT_THREADS = 352;
 constexpr float LOG2E_F = 1.4426950408889634f;
 constexpr float RESCALE_THRESHOLD = 8.0f;  // in log2 units
 constexpr int K_SLOTS = 3, V_SLOTS = 2, ITEM_SLOTS = 4;
@@ -120,7 +121,7 @@ prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
       int count = 1;
       if (i >= B_PREADY && i < B_PREADY + 2) count = 4;             // the four softmax warps of the tile
       if (i >= B_OREAD && i < B_OREAD + 2) count = 4;
-      if (i >= B_IEMPTY && i < B_IEMPTY + ITEM_SLOTS) count = 10;   // eight softmax warps + the MMA thread once per tile
+      if (i >= B_IEMPTY && i < B_IEMPTY + ITEM_SLOTS) count = 11;   // eight softmax warps, the MMA thread once per tile, the Q loader
       ptx::mbar_init(bar(i), count);
     }
     ptx::fence_barrier_init();
@@ -145,7 +146,6 @@ prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
     // ---------------------------------------------------------------- producer
     if (lane == 0) {
       int it_pub = 0;               // items published so far (ring position)
-      int q_cnt[2] = {0, 0};        // Q loads so far per row tile
       int g_k = 0, g_v = 0;         // K / V tiles loaded so far (ring positions)
       bool ok = true;
       // the next item is fetched and decoded while the current one's tiles are being loaded
@@ -174,16 +174,6 @@ prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
         }
         if (last) break;
         const int n_max = max(it.n_kv0, it.n_kv1);
-        for (int t = 0; t < 2 && ok; ++t) {
-          if (t == 1 && it.n_kv1 == 0) break;
-          // the tile's Q buffer is free once the last Q K^T of its previous item has been executed
-          if (!ptx::mbar_wait_bounded(bar(B_QEMPTY + t), (q_cnt[t] & 1) ^ 1u, abort_flag, limit)) { ok = false; break; }
-          ptx::mbar_arrive_expect_tx(bar(B_QFULL + t), Cfg::TILE_BYTES);
-          for (int c = 0; c < Cfg::SUB; ++c)
-            ptx::tma_load_2d(smem_base + Cfg::Q_OFF + t * Cfg::TILE_BYTES + c * Cfg::SUB_BYTES, &tmap_q, it.h * HD + c * 64,
-                             it.start + it.q0 + t * TQ, bar(B_QFULL + t));
-          ++q_cnt[t];
-        }
         for (int j = 0; j < n_max && ok; ++j) {
           // K and V slots are released separately: K as soon as the Q K^T products that use it have run, V only
           // after the P V products, so later K tiles are on their way while the softmax runs
@@ -317,6 +307,35 @@ prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
         }
       }
     }
+  } else if (warp == 10) {
+    // ---------------------------------------------------------------- Q loader
+    // Its own thread, so that a wait for one tile's Q buffer never holds up the K / V stream of the other tile.
+    if (lane == 0) {
+      int seq = 0;
+      int q_cnt[2] = {0, 0};  // Q loads so far per row tile
+      bool ok = true;
+      while (ok) {
+        const int s = seq & (ITEM_SLOTS - 1);
+        if (!ptx::mbar_wait_bounded(bar(B_IFULL + s), (seq / ITEM_SLOTS) & 1, abort_flag, limit)) break;
+        const Item it = item_ring[s];
+        ptx::mbar_arrive(bar(B_IEMPTY + s));
+        ++seq;
+        if (it.n_kv0 < 0) break;
+        for (int t = 0; t < 2; ++t) {
+          if (t == 1 && it.n_kv1 == 0) break;
+          // the tile's Q buffer is free once the last Q K^T of its previous item has been executed
+          if (!ptx::mbar_wait_bounded(bar(B_QEMPTY + t), (q_cnt[t] & 1) ^ 1u, abort_flag, limit)) { ok = false; break; }
+          ptx::mbar_arrive_expect_tx(bar(B_QFULL + t), Cfg::TILE_BYTES);
+          for (int c = 0; c < Cfg::SUB; ++c)
+            ptx::tma_load_2d(smem_base + Cfg::Q_OFF + t * Cfg::TILE_BYTES + c * Cfg::SUB_BYTES, &tmap_q, it.h * HD + c * 64,
+                             it.start + it.q0 + t * TQ, bar(B_QFULL + t));
+          ++q_cnt[t];
+        }
+      }
+      if (!ok) {
+        for (int i = 0; i < 2000; ++i) __nanosleep(1000);
+      }
+    }
   } else {
     // ---------------------------------------------------------------- softmax
     const int t = (warp - 2) >> 2;       // row tile of this warpgroup
@@ -355,28 +374,28 @@ prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
         ptx::tc_fence_after();
         const int k0 = j * TK;
         uint32_t sv[4][32];
-  #pragma unroll
+#pragma unroll
         for (int c = 0; c < 4; ++c) ptx::tmem_ld_32x32(t_lane + Cfg::S_COL + c * 32, sv[c]);
         ptx::tmem_ld_wait();
         // raw scores stay in registers; the scale is folded into the exponent (scale > 0, so the
         // maximum can be taken on the raw values)
         const bool need_mask = (k0 + TK - 1 > it.pre + it.q0 + t * TQ) || (k0 + TK > kv_end);  // warp-uniform
         if (need_mask) {
-  #pragma unroll
+          // keys with index above `lim` (inside this tile) are invisible to this row: one compare per key
+          const int lim = min(row_pos, kv_end - 1) - k0;
+#pragma unroll
           for (int c = 0; c < 4; ++c) {
-  #pragma unroll
-            for (int e = 0; e < 32; ++e) {
-              const int key = k0 + c * 32 + e;
-              if (key > row_pos || key >= kv_end) sv[c][e] = 0xff800000u;  // -inf
-            }
+#pragma unroll
+            for (int e = 0; e < 32; ++e)
+              if (c * 32 + e > lim) sv[c][e] = 0xff800000u;  // -inf
           }
         }
         // row maximum: four independent chains of three-input maxima (the softmax warps set the pace of the
         // kernel, so their instruction count and dependency depth are what is being minimised here)
         float mx4[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F};
-  #pragma unroll
+#pragma unroll
         for (int c = 0; c < 4; ++c) {
-  #pragma unroll
+#pragma unroll
           for (int e = 0; e < 32; e += 2)
             mx4[(e >> 1) & 3] = ptx::fmax3(mx4[(e >> 1) & 3], __uint_as_float(sv[c][e]), __uint_as_float(sv[c][e + 1]));
         }
@@ -397,12 +416,12 @@ prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
           ok = __all_sync(0xffffffffu, ptx::mbar_wait_bounded(bar(B_ODONE + t), (step - 1) & 1, abort_flag, limit));
           if (!ok) break;
           ptx::tc_fence_after();
-  #pragma unroll 1
+#pragma unroll 1
           for (int c = 0; c < HD / 32; ++c) {
             uint32_t ov[32];
             ptx::tmem_ld_32x32(t_lane + Cfg::O_COL + c * 32, ov);
             ptx::tmem_ld_wait();
-  #pragma unroll
+#pragma unroll
             for (int e = 0; e < 32; ++e) ov[e] = __float_as_uint(__uint_as_float(ov[e]) * factor);
             ptx::tmem_st_32x32(t_lane + Cfg::O_COL + c * 32, ov);
           }
@@ -416,10 +435,10 @@ prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
         const uint64_t sl2_2 = ptx::pack_f32x2(sl2, sl2);
         const uint64_t negm_2 = ptx::pack_f32x2(-m_used, -m_used);
         uint64_t ps[4] = {0ull, 0ull, 0ull, 0ull};
-  #pragma unroll
+#pragma unroll
         for (int c = 0; c < 2; ++c) {
           uint32_t pk[32];
-  #pragma unroll
+#pragma unroll
           for (int e = 0; e < 32; ++e) {
             // packed column 32 c + e holds keys 2 (32 c + e) and 2 (32 c + e) + 1
             const int k_lo = (c * 32 + e) * 2;
@@ -467,26 +486,25 @@ prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
       ptx::tc_fence_after();
       const float inv = 1.f / l_sum;
       bf16* dst = p.o + static_cast<size_t>(it.start + row) * (p.n_q_heads * HD) + it.h * HD;
-#pragma unroll 1
-      for (int c = 0; c < HD / 32; ++c) {
-        uint32_t ov[32];
-        ptx::tmem_ld_32x32(t_lane + Cfg::O_COL + c * 32, ov);
-        ptx::tmem_ld_wait();
-        if (c == HD / 32 - 1) {
-          // O is in registers: the next item's first product may overwrite it
-          ptx::tc_fence_before();
-          __syncwarp();
-          if (lane == 0) ptx::mbar_arrive(bar(B_OREAD + t));
-        }
-        if (row < it.len) {
+      // the whole row first, so that the next item's first product may overwrite O as early as possible
+      uint32_t ov[HD / 32][32];
 #pragma unroll
-          for (int e = 0; e < 32; e += 8) {
-            uint4 o;
-            o.x = ptx::pack_bf16(__uint_as_float(ov[e]) * inv, __uint_as_float(ov[e + 1]) * inv);
-            o.y = ptx::pack_bf16(__uint_as_float(ov[e + 2]) * inv, __uint_as_float(ov[e + 3]) * inv);
-            o.z = ptx::pack_bf16(__uint_as_float(ov[e + 4]) * inv, __uint_as_float(ov[e + 5]) * inv);
-            o.w = ptx::pack_bf16(__uint_as_float(ov[e + 6]) * inv, __uint_as_float(ov[e + 7]) * inv);
-            *reinterpret_cast<uint4*>(dst + c * 32 + e) = o;
+      for (int c = 0; c < HD / 32; ++c) ptx::tmem_ld_32x32(t_lane + Cfg::O_COL + c * 32, ov[c]);
+      ptx::tmem_ld_wait();
+      ptx::tc_fence_before();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(bar(B_OREAD + t));
+      if (row < it.len) {
+        // a thread owns a row, so every store of a warp touches 32 different lines: 32-byte stores halve their number
+#pragma unroll
+        for (int c = 0; c < HD / 32; ++c) {
+#pragma unroll
+          for (int e = 0; e < 32; e += 16) {
+            uint32_t w[8];
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+              w[q] = ptx::pack_bf16(__uint_as_float(ov[c][e + 2 * q]) * inv, __uint_as_float(ov[c][e + 2 * q + 1]) * inv);
+            ptx::st_global_v8(dst + c * 32 + e, w);
           }
         }
       }
