@@ -143,7 +143,10 @@ pd_status pd_decode_layer(pd_layer* layer, const void* x, void* out, const int32
  *                 (kv_len[b]+1 entries, all of which must already be in the cache)
  *   workspace     scratch for the partial results of the KV-range splits, at least
  *                 pd_decode_attention_workspace_bytes(cfg, B, max_kv_len) bytes, 256-byte aligned
- * Only n_q_heads, n_kv_heads and head_dim of cfg are used. */
+ * Only n_q_heads, n_kv_heads and head_dim of cfg are used.  kv_len is read on the device and not validated by
+ * this call: a range that reaches past the cache (kv_len[b] + 1 > len_cap) is clamped to len_cap entries, and a
+ * sequence with kv_len[b] < 0 (no entry at all) gets an all-zero output row; neither is reported.  (The layer
+ * calls do report an out-of-range position, through pd_layer_check.) */
 pd_status pd_decode_attention_workspace_bytes(const pd_layer_cfg* cfg, int32_t B, int32_t max_kv_len,
                                               size_t* out_bytes);
 pd_status pd_decode_attention(const pd_layer_cfg* cfg, const void* q, int32_t ldq, void* out,
@@ -162,7 +165,9 @@ pd_status pd_decode_attention(const pd_layer_cfg* cfg, const void* q, int32_t ld
  *                 request r in sequence slots[r] (NULL: r)
  *   err_word      optional device int32, set to 1 if a bounded wait inside the kernel gave up
  * Query t attends to positions 0 .. prefix[r] + t of its own request.  Only n_q_heads, n_kv_heads and
- * head_dim of cfg are used.  Enqueues one kernel; no workspace. */
+ * head_dim of cfg are used; out must be 32-byte aligned.  Enqueues one kernel; no workspace.  The kernel
+ * keeps its work counter in a small pool inside the library: calls that follow each other on one stream
+ * are always safe, and up to 64 calls may overlap on the GPU. */
 pd_status pd_prefill_attention(const pd_layer_cfg* cfg, const void* q, int32_t ldq, void* out,
                                const int32_t* cu_seqlens_dev, const int32_t* cu_seqlens_host, int32_t n_req,
                                const int32_t* prefix_dev, const int32_t* prefix_host, const int32_t* slots_dev,
@@ -298,6 +303,17 @@ pd_status pd_model_check(pd_model* model, void* stream);
  * `err_word` device int32 (may be NULL), set non-zero if a bounded wait gave up. */
 pd_status pd_gemm_bf16(const void* a, const void* b, void* c, int32_t m, int32_t n, int32_t k,
                        int32_t* err_word, void* stream);
+
+/* pd_gemm_bf16 with the scratch the layer calls give their projections: with it the kernel may cut tiles in two
+ * along K and run the halves on different SMs (every tile when the problem has too few tiles to fill the SMs,
+ * e.g. a few hundred tokens against N = d_model; otherwise only the tiles of the last, partly filled wave when K
+ * is long).  The first half parks its fp32 partial tile in the workspace, the second adds it before the
+ * epilogue; the wait between them is bounded like every other wait.  workspace: device, 256-byte aligned, at
+ * least pd_gemm_workspace_bytes() bytes; the call clears the flags at its start, so calls sharing a workspace
+ * must be ordered on one stream. */
+pd_status pd_gemm_workspace_bytes(size_t* out_bytes);
+pd_status pd_gemm_bf16_ws(const void* a, const void* b, void* c, int32_t m, int32_t n, int32_t k, void* workspace,
+                          size_t workspace_bytes, int32_t* err_word, void* stream);
 
 /* Where a layer pass leaves its intermediates.  Byte offsets, inside the workspace handed to
  * pd_prefill_layer / pd_prefill_chunk_layer over `tokens` rows (or pd_decode_layer with B = tokens), of the

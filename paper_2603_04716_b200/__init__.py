@@ -40,6 +40,7 @@ EXPORTS = [
     "pd_model_check", "pd_allocate_ext", "pd_quantize_fp8_rows", "pd_gemm_fp8", "pd_workspace_offsets",
     "pd_prefill_attention", "pd_mixture_throughput", "pd_interp_service_times", "pd_mm1_sojourn", "pd_mg1_sojourn",
     "pd_refine_next_batch", "pd_prefill_chunk_stack", "pd_test_inject_wait_timeout",
+    "pd_gemm_workspace_bytes", "pd_gemm_bf16_ws",
 ]
 
 TRACE_CLASSES = ["gemm_qkv", "gemm_o", "gemm_gate_up", "gemm_down", "attn_prefill", "attn_decode", "rmsnorm",
@@ -147,6 +148,8 @@ _lib.pd_decode_stack.argtypes = [C.POINTER(_P), C.POINTER(pd_kv_cache), C.c_int3
                                  C.c_int32, C.c_int32, _P, C.c_size_t, _P]
 _lib.pd_layer_check.argtypes = [_P, _P]
 _lib.pd_gemm_bf16.argtypes = [_P, _P, _P, C.c_int32, C.c_int32, C.c_int32, _P, _P]
+_lib.pd_gemm_workspace_bytes.argtypes = [C.POINTER(C.c_size_t)]
+_lib.pd_gemm_bf16_ws.argtypes = [_P, _P, _P, C.c_int32, C.c_int32, C.c_int32, _P, C.c_size_t, _P, _P]
 _lib.pd_workspace_offsets.argtypes = [C.POINTER(pd_layer_cfg), C.c_int32, C.POINTER(pd_workspace_layout)]
 _lib.pd_quantize_fp8_rows.argtypes = [_P, C.c_int32, C.c_int32, C.c_int32, _P, _P, _P]
 _lib.pd_gemm_fp8.argtypes = [_P, _P, _P, _P, _P, C.c_int32, C.c_int32, C.c_int32, _P, _P]
@@ -454,6 +457,18 @@ def pd_layer_check(layer: Layer, stream=None):
 
 def pd_gemm_bf16(a, b, c, m: int, n: int, k: int, err_word=None, stream=None):
     _check(_lib.pd_gemm_bf16(_ptr(a), _ptr(b), _ptr(c), m, n, k, _ptr(err_word), _stream_ptr(stream)), "pd_gemm_bf16")
+
+
+def pd_gemm_workspace_bytes() -> int:
+    out = C.c_size_t(0)
+    _check(_lib.pd_gemm_workspace_bytes(C.byref(out)), "pd_gemm_workspace_bytes")
+    return out.value
+
+
+def pd_gemm_bf16_ws(a, b, c, m: int, n: int, k: int, workspace, workspace_bytes: int, err_word=None, stream=None):
+    """pd_gemm_bf16 with the K-split scratch (tiles may be cut in two along K and run on two SMs / CTA pairs)."""
+    _check(_lib.pd_gemm_bf16_ws(_ptr(a), _ptr(b), _ptr(c), m, n, k, _ptr(workspace), workspace_bytes, _ptr(err_word),
+                                _stream_ptr(stream)), "pd_gemm_bf16_ws")
 
 
 def pd_workspace_offsets(cfg: LayerConfig, tokens: int) -> dict:

@@ -223,7 +223,8 @@ __global__ void __launch_bounds__(DC_THREADS) decode_attn_kernel(DecodeAttnArgs 
       }
     }
     if (a.n_splits == 1) {
-      a.o[static_cast<size_t>(b) * (a.n_q_heads * HD) + (kvh * group + r) * HD + d] = __float2bfloat16(o / l);
+      // (a sequence with no visible entry at all, kv_len < 0, gives zeros rather than 0 / 0)
+      a.o[static_cast<size_t>(b) * (a.n_q_heads * HD) + (kvh * group + r) * HD + d] = __float2bfloat16(l > 0.f ? o / l : 0.f);
     } else {
       float* dst = a.partial +
                    (((static_cast<size_t>(b) * a.n_kv_heads + kvh) * a.n_splits + split) * group + r) * RS;
@@ -257,7 +258,7 @@ __global__ void __launch_bounds__(HD) decode_combine_kernel(DecodeAttnArgs a) {
     l += src[HD + 1] * sc;
     o += src[d] * sc;
   }
-  a.o[static_cast<size_t>(b) * (a.n_q_heads * HD) + hq * HD + d] = __float2bfloat16(o / l);
+  a.o[static_cast<size_t>(b) * (a.n_q_heads * HD) + hq * HD + d] = __float2bfloat16(l > 0.f ? o / l : 0.f);
 }
 
 template <int HD>

@@ -106,6 +106,7 @@ struct GemmDev {
   float* split_scratch;  // [tail tile][128][BN] fp32
   int* split_flags;      // [tail tile][4], 1 while a partial waits to be consumed
   int split_enable;
+  int split_all;         // CTA-pair kernel: EVERY tile is cut in two along K (unit 2 i = first half, 2 i + 1 = second half)
   int* err_word;
   unsigned long long wait_limit_ns;  // bound of every wait inside the kernel
   int test_skip_load;                // test hook: the producer leaves out the A tile of its second K block
@@ -179,7 +180,7 @@ __device__ __forceinline__ void epilogue_tile(const GemmDev& p, int role, int n_
     if (role == 2) {
 #pragma unroll
       for (int j = 0; j < 32; j += 4) {
-        const float4 q = __ldcg(reinterpret_cast<const float4*>(part_row + col_off + j));
+        const float4 q = __ldcg(reinterpret_cast<const float4*>(part_row + ((col_off + j) >> 2) * (BM * 4)));
         v[j] = __float_as_uint(__uint_as_float(v[j]) + q.x);
         v[j + 1] = __float_as_uint(__uint_as_float(v[j + 1]) + q.y);
         v[j + 2] = __float_as_uint(__uint_as_float(v[j + 2]) + q.z);
@@ -351,6 +352,47 @@ __device__ __forceinline__ void epilogue_tile(const GemmDev& p, int role, int n_
   }
 }
 
+// Hand-over of a K-split tile between its two units (one warp = one 32-row group of the tile).  The fp32 scratch
+// tile is laid out [column group of 4][row][4] so that the 32 rows of a warp access 512 contiguous bytes per
+// instruction (a thread's own row, 1 KB apart from its neighbours', would cost 32 lines per instruction); part_row
+// points at the thread's row inside column group 0.  role 1: park the accumulator rows and raise the group's flag.  role 2: wait (bounded) for the partner's
+// flag; the caller's epilogue then adds the parked rows.  Returns false when the wait gave up.
+template <int BN>
+__device__ __forceinline__ bool split_hand_over(const GemmDev& p, int role, int slot, int lane_group, int lane,
+                                                uint32_t t_row, float* part_row, volatile int* abort_flag) {
+  int* flag = p.split_flags + slot * 4 + lane_group;
+  if (role == 1) {
+#pragma unroll 1
+    for (int c0 = 0; c0 < BN; c0 += 32) {
+      uint32_t v[32];
+      ptx::tmem_ld_32x32(t_row + c0, v);
+      ptx::tmem_ld_wait();
+#pragma unroll
+      for (int j = 0; j < 32; j += 4)
+        __stcg(reinterpret_cast<uint4*>(part_row + ((c0 + j) >> 2) * (BM * 4)), make_uint4(v[j], v[j + 1], v[j + 2], v[j + 3]));
+    }
+    __threadfence();
+    __syncwarp();
+    if (lane == 0) *reinterpret_cast<volatile int*>(flag) = 1;
+    return true;
+  }
+  bool seen = true;
+  if (lane == 0) {
+    const uint64_t t0 = ptx::globaltimer_ns();
+    uint32_t spins = 0;
+    while (*reinterpret_cast<volatile int*>(flag) != 1) {
+      if ((++spins & 1023u) == 0u && (*abort_flag || ptx::globaltimer_ns() - t0 > p.wait_limit_ns)) {
+        *abort_flag = 1;
+        seen = false;
+        break;
+      }
+    }
+  }
+  const bool ok = __all_sync(0xffffffffu, seen);
+  __threadfence();
+  return ok;
+}
+
 template <int BN, int EPI, bool F8>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b, GemmDev p) {
@@ -492,39 +534,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       float* part_row = nullptr;
       if (ui.role == 1 || ui.role == 2) {
         const int slot = ui.tile - p.main_tiles;
-        part_row = p.split_scratch + (static_cast<size_t>(slot) * BM + lane_group * 32 + lane) * BN;
-        int* flag = p.split_flags + slot * 4 + lane_group;
-        if (ui.role == 1) {
-          // first K half: park the accumulator in global memory, publish, and skip the epilogue
-#pragma unroll 1
-          for (int c0 = 0; c0 < BN; c0 += 32) {
-            uint32_t v[32];
-            ptx::tmem_ld_32x32(t_row + c0, v);
-            ptx::tmem_ld_wait();
-#pragma unroll
-            for (int j = 0; j < 32; j += 4)
-              __stcg(reinterpret_cast<uint4*>(part_row + c0 + j), make_uint4(v[j], v[j + 1], v[j + 2], v[j + 3]));
-          }
-          __threadfence();
-          __syncwarp();
-          if (lane == 0) *reinterpret_cast<volatile int*>(flag) = 1;
-        } else {
-          // second K half: wait (bounded) for the partner's rows of this warp
-          bool seen = true;
-          if (lane == 0) {
-            const uint64_t t0 = ptx::globaltimer_ns();
-            uint32_t spins = 0;
-            while (*reinterpret_cast<volatile int*>(flag) != 1) {
-              if ((++spins & 1023u) == 0u && (*abort_flag || ptx::globaltimer_ns() - t0 > p.wait_limit_ns)) {
-                *abort_flag = 1;
-                seen = false;
-                break;
-              }
-            }
-          }
-          ok = __all_sync(0xffffffffu, seen);
-          __threadfence();
-        }
+        part_row = p.split_scratch + static_cast<size_t>(slot) * BM * BN + (lane_group * 32 + lane) * 4;
+        ok = split_hand_over<BN>(p, ui.role, slot, lane_group, lane, t_row, part_row, abort_flag);
       }
       epilogue_tile<BN, EPI, F8>(p, ui.role, ui.n_half, tm, tn, row, t_row, part_row, ok);
       // all of this warp's reads of the accumulator are complete: hand the buffer back
@@ -561,6 +572,19 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
 constexpr int P2_STAGE_BYTES = 2 * BM * 128;  // A rows + B rows of this CTA, 16 KB each
 constexpr int P2_STAGES = 7;
 constexpr int P2_SMEM_BYTES = P2_STAGES * P2_STAGE_BYTES + 1024 + 256;
+
+// Work unit of the CTA-pair kernel: whole tiles and half-width tail tiles as in unit_info, or, when the problem
+// has so few tiles that half of the pairs would idle (split_all), every tile as two K halves on two pairs.
+__device__ __forceinline__ UnitInfo pair_unit_info(const GemmDev& p, int unit, int k_blocks) {
+  if (!p.split_all) return unit_info(unit, p.main_tiles, k_blocks, 1);
+  UnitInfo u;
+  u.n_half = 0;
+  u.tile = unit >> 1;
+  const int kh = k_blocks >> 1;
+  if (unit & 1) { u.kb_lo = kh; u.kb_hi = k_blocks; u.role = 2; }
+  else { u.kb_lo = 0; u.kb_hi = kh; u.role = 1; }
+  return u;
+}
 
 template <int EPI, bool F8>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
@@ -625,17 +649,17 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
       bool ok = true;
       ptx::grid_dependency_wait();
       for (int unit = pair_id; unit < n_units && ok; unit += n_pairs) {
-        const UnitInfo ui = unit_info(unit, p.main_tiles, k_blocks, 1);
+        const UnitInfo ui = pair_unit_info(p, unit, k_blocks);
         int tm2, tn;
         tile_coords(ui.tile, tiles_m2, p.tiles_n, group2, tm2, tn);
         const bool half = ui.role == 3;  // this CTA then supplies 64 of the half tile's 128 rows of B
-        for (int kb = 0; kb < k_blocks; ++kb) {
+        for (int kb = ui.kb_lo; kb < ui.kb_hi; ++kb) {
           if (!ptx::mbar_wait_bounded(empty_bar(stage), phase ^ 1u, abort_flag, p.wait_limit_ns)) { ok = false; break; }
           const uint32_t sa = smem_base + stage * P2_STAGE_BYTES;
           const uint32_t sb = sa + BM * 128;
           const uint32_t lead_full = ptx::map_to_cta(full_bar(stage), 0);
           if (rank == 0) ptx::mbar_arrive_expect_tx(full_bar(stage), half ? 2 * (BM + 64) * 128 : 2 * P2_STAGE_BYTES);
-          if (!(p.test_skip_load && rank == 0 && unit == pair_id && kb == 1))
+          if (!(p.test_skip_load && rank == 0 && unit == pair_id && kb == ui.kb_lo + 1))
             ptx::tma_load_2d_pair(sa, &tmap_a, kb * KE, (2 * tm2 + static_cast<int>(rank)) * BM, lead_full);
           if (half)
             ptx::tma_load_2d_pair(sb, &tmap_b_half, kb * KE, tn * BN + ui.n_half * 128 + static_cast<int>(rank) * 64, lead_full);
@@ -656,11 +680,12 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
       uint32_t phase = 0, acc_phase = 0;
       bool ok = true;
       for (int unit = pair_id; unit < n_units && ok; unit += n_pairs) {
-        const uint32_t idesc = unit < p.main_tiles ? idesc_full : idesc_half;
+        const UnitInfo ui = pair_unit_info(p, unit, k_blocks);
+        const uint32_t idesc = ui.role == 3 ? idesc_half : idesc_full;
         if (!ptx::mbar_wait_bounded(acce_bar(acc), acc_phase ^ 1u, abort_flag, p.wait_limit_ns)) break;
         ptx::tc_fence_after();
         const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * BN);
-        for (int kb = 0; kb < k_blocks; ++kb) {
+        for (int kb = ui.kb_lo; kb < ui.kb_hi; ++kb) {
           if (!ptx::mbar_wait_bounded(full_bar(stage), phase, abort_flag, p.wait_limit_ns)) { ok = false; break; }
           ptx::tc_fence_after();
           const uint32_t sa = smem_base + stage * P2_STAGE_BYTES;
@@ -668,7 +693,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
           const uint64_t db = ptx::umma_desc_sw128(sa + BM * 128);
 #pragma unroll
           for (int kk = 0; kk < 4; ++kk) {
-            const uint32_t accum = (kb > 0 || kk > 0) ? 1u : 0u;
+            const uint32_t accum = (kb > ui.kb_lo || kk > 0) ? 1u : 0u;
             if constexpr (F8) ptx::umma_f8_pair(d_tmem, da + 2u * kk, db + 2u * kk, idesc, accum);
             else ptx::umma_bf16_pair(d_tmem, da + 2u * kk, db + 2u * kk, idesc, accum);
           }
@@ -686,7 +711,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
     uint32_t acc_phase = 0;
     ptx::grid_dependency_wait();
     for (int unit = pair_id; unit < n_units; unit += n_pairs) {
-      const UnitInfo ui = unit_info(unit, p.main_tiles, k_blocks, 1);
+      const UnitInfo ui = pair_unit_info(p, unit, k_blocks);
       int tm2, tn;
       tile_coords(ui.tile, tiles_m2, p.tiles_n, group2, tm2, tn);
       const int tm = 2 * tm2 + static_cast<int>(rank);
@@ -694,9 +719,22 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
       ptx::tc_fence_after();
       const int row = tm * BM + lane_group * 32 + lane;
       const uint32_t t_row = tmem_base + (static_cast<uint32_t>(lane_group * 32) << 16) + static_cast<uint32_t>(acc * BN);
-      epilogue_tile<BN, EPI, F8>(p, ui.role, ui.n_half, tm, tn, row, t_row, nullptr, true);
+      // K-split tile: this CTA's 128 rows of the fp32 partial live in scratch slot 2 * tile + rank
+      float* part_row = nullptr;
+      bool ok = true;
+      if (ui.role == 1 || ui.role == 2) {
+        const int slot = 2 * ui.tile + static_cast<int>(rank);
+        part_row = p.split_scratch + static_cast<size_t>(slot) * BM * BN + (lane_group * 32 + lane) * 4;
+        ok = split_hand_over<BN>(p, ui.role, slot, lane_group, lane, t_row, part_row, abort_flag);
+      }
+      epilogue_tile<BN, EPI, F8>(p, ui.role, ui.n_half, tm, tn, row, t_row, part_row, ok);
       ptx::tc_fence_before();
       __syncwarp();
+      if (ui.role == 2 && lane == 0) {
+        // the partner's partial has been consumed: lower the flag for the next launch
+        __threadfence();
+        *reinterpret_cast<volatile int*>(p.split_flags + (2 * ui.tile + static_cast<int>(rank)) * 4 + lane_group) = 0;
+      }
       if (lane == 0) ptx::mbar_arrive_cluster(ptx::map_to_cta(acce_bar(acc), 0));
       if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
     }
@@ -711,6 +749,18 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
     ptx::tc_fence_after();
     ptx::tmem_dealloc_pair(tmem_base, TMEM_COLS);
   }
+}
+
+// Bytes of L2 a raster group's A slab may occupy while the B tiles stream past it.  The slab stays resident because
+// every one of its tiles is re-read for each column tile; PD_RASTER_MB in the environment overrides the size (for
+// sweeps).
+long long raster_slab_bytes() {
+  static const long long bytes = [] {
+    const char* v = std::getenv("PD_RASTER_MB");
+    const long long mb = v ? std::atoll(v) : 0;
+    return (mb > 0 ? mb : 64) << 20;  // half of the 126 MB L2: with K = 14336 the weight matrix is then streamed twice, not three to four times
+  }();
+  return bytes;
 }
 
 // SM count of the current device (remembered per device ordinal).
@@ -750,8 +800,8 @@ pd_status launch_tc(const GemmArgs& g, cudaStream_t stream) {
   p.wait_limit_ns = 4000000000ull;
   if (take_wait_injection(PD_INJECT_GEMM, &p.wait_limit_ns)) p.test_skip_load = 1;
   {
-    // keep a group's A slab (group x 128 rows x K) within about 40 MB of L2
-    long long grp = (40ll << 20) / (static_cast<long long>(BM) * g.k * 2);
+    // keep a group's A slab (group x 128 rows x K) within the L2 share given to it
+    long long grp = raster_slab_bytes() / (static_cast<long long>(BM) * g.k * 2);
     p.raster_group = static_cast<int>(grp < 4 ? 4 : (grp > 32 ? 32 : grp));
   }
   if (EPI == EPI_ROPE_KV) p.rope = *g.rope;
@@ -835,13 +885,23 @@ pd_status launch_tc_pair(const GemmArgs& g, cudaStream_t stream) {
   p.wait_limit_ns = 4000000000ull;
   if (take_wait_injection(PD_INJECT_GEMM_PAIR, &p.wait_limit_ns)) p.test_skip_load = 1;
   {
-    long long grp = (40ll << 20) / (static_cast<long long>(BM) * g.k * (F8 ? 1 : 2));
+    long long grp = raster_slab_bytes() / (static_cast<long long>(BM) * g.k * (F8 ? 1 : 2));
     p.raster_group = static_cast<int>(grp < 4 ? 4 : (grp > 32 ? 32 : grp));
   }
   if (EPI == EPI_ROPE_KV) p.rope = *g.rope;
   const int units = ((p.tiles_m + 1) / 2) * p.tiles_n;
   p.n_units = units; p.main_tiles = units;
-  {
+  // Few tiles (short batches against N = d_model): when the tiles would fill at most half of the pairs, every tile
+  // is cut in two along K and the halves run on two pairs at once; the first parks its fp32 partial in the scratch,
+  // the second adds it before its epilogue (the hand-over of the single-CTA kernel's tail split).
+  const size_t split_need = static_cast<size_t>(2 * units) * BM * 256 * sizeof(float);
+  // (pays only for long K, like the tail split: the hand-over costs about as much as 4096 elements of K)
+  if (2 * units <= cap && g.k / (F8 ? BK_F8 : BK) >= 128 && g.split_scratch && g.split_flags &&
+      split_need <= g.split_scratch_bytes && 2 * units <= kSplitMaxTiles) {
+    p.split_all = 1;
+    p.n_units = 2 * units;
+    p.split_scratch = g.split_scratch; p.split_flags = g.split_flags;
+  } else {
     // the last wave holds `tail` tiles: if they occupy at most half of the pairs, run each as two 128-column halves
     const int tail = units % cap;
     if (tail > 0 && 2 * tail <= cap) {
@@ -943,7 +1003,17 @@ pd_status gemm(const GemmArgs& g, cudaStream_t stream) {
   PD_TRY(check_gemm_args(g));
   if (g.m == 0) return PD_OK;
   const int bn = gemm_block_n(g.m, g.n, g.epilogue);
-  if (bn == 256 && g.n % 256 == 0 && g.m > BM && pair_mode() != 0) {
+  // Short batches against a narrow N with a long K (the down projection at a few hundred tokens): the pair kernel
+  // with every tile cut in two along K keeps all SMs busy with 256-wide tiles, which beats one wave of narrow
+  // single-CTA tiles (measured 73.7 -> 61.5 us at 512 x 4096 x 14336; at K = 4096 the hand-over costs more than the
+  // half main loop it saves, 28.7 -> 34.8 us, so short K stays on the narrow tiles).
+  bool pair_split = false;
+  if (g.n % 256 == 0 && g.m > BM && g.split_scratch && g.split_flags) {
+    const int units = ((g.m + 2 * BM - 1) / (2 * BM)) * (g.n / 256);
+    pair_split = 2 * units <= sm_count() / 2 && g.k / (g.fp8 ? BK_F8 : BK) >= 128 &&
+                 static_cast<size_t>(2 * units) * BM * 256 * sizeof(float) <= g.split_scratch_bytes;
+  }
+  if ((bn == 256 || pair_split) && g.n % 256 == 0 && g.m > BM && pair_mode() != 0) {
     const pd_status st = g.fp8 ? launch_tc_pair_epi<true>(g, stream) : launch_tc_pair_epi<false>(g, stream);
     if (st != PD_ERR_UNSUPPORTED_SHAPE) return st;  // (clusters of two could not be placed: single-CTA kernel)
   }
@@ -975,6 +1045,35 @@ extern "C" pd_status pd_gemm_bf16(const void* a, const void* b, void* c, int32_t
   g.epilogue = pd::EPI_STORE;
   g.err_word = err_word;
   return pd::gemm(g, static_cast<cudaStream_t>(stream));
+}
+
+// Workspace layout of pd_gemm_bf16_ws: the hand-over flags (cleared by the call), then the fp32 partial tiles.
+static constexpr size_t kGemmWsFlagBytes = (pd::kSplitMaxTiles * 4 * sizeof(int) + 255) / 256 * 256;
+
+extern "C" pd_status pd_gemm_workspace_bytes(size_t* out_bytes) {
+  if (!out_bytes) return PD_ERR_INVALID_ARG;
+  *out_bytes = kGemmWsFlagBytes + pd::kSplitScratchBytes;
+  return PD_OK;
+}
+
+extern "C" pd_status pd_gemm_bf16_ws(const void* a, const void* b, void* c, int32_t m, int32_t n, int32_t k,
+                                     void* workspace, size_t workspace_bytes, int32_t* err_word, void* stream) {
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return PD_ERR_INVALID_ARG;
+  if (workspace_bytes < kGemmWsFlagBytes + pd::kSplitScratchBytes) return PD_ERR_WORKSPACE_TOO_SMALL;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  PD_CUDA_TRY(cudaMemsetAsync(workspace, 0, kGemmWsFlagBytes, st));
+  pd::GemmArgs g{};
+  g.a = static_cast<const pd::bf16*>(a);
+  g.b = static_cast<const pd::bf16*>(b);
+  g.c = static_cast<pd::bf16*>(c);
+  g.m = m; g.n = n; g.k = k;
+  g.lda = k; g.ldb = k; g.ldc = n; g.ldr = 0;
+  g.epilogue = pd::EPI_STORE;
+  g.err_word = err_word;
+  g.split_flags = static_cast<int*>(workspace);
+  g.split_scratch = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + kGemmWsFlagBytes);
+  g.split_scratch_bytes = pd::kSplitScratchBytes;
+  return pd::gemm(g, st);
 }
 
 extern "C" pd_status pd_gemm_fp8(const void* a_codes, const float* a_scales, const void* b_codes, const float* b_scales,

@@ -55,7 +55,7 @@ Workspace carve(const pd_layer_cfg& c, size_t tokens, size_t max_batch, int max_
   w.stage_a = take(tokens * d * 2);  // activations between layers of a stack / staged host input
   w.stage_b = take(tokens * d * 2);
   w.meta = take(4096 * 4);           // staged cu_seqlens / kv_len of the host-I/O stack calls
-  w.splitk = take(tokens > 256 ? pd::kSplitScratchBytes : 0);  // partial tiles of K-split GEMM tails (prefill only)
+  w.splitk = take(tokens > 128 ? pd::kSplitScratchBytes : 0);  // fp32 partial tiles of K-split GEMM tiles
   const size_t widest = f > hq ? (f > d ? f : d) : (hq > d ? hq : d);
   w.q_act = take(c.fp8_projections ? tokens * widest : 0);
   w.s_act = take(c.fp8_projections ? tokens * 4 : 0);
@@ -110,7 +110,7 @@ pd_status check_cache(const pd_layer* L, const pd_kv_cache* c) {
 
 // Lets a prefill GEMM cut the tiles of its last partial wave in two along K.
 void enable_tail_split(pd_layer* L, pd::GemmArgs& g, uint8_t* ws, const Workspace& w, size_t tokens) {
-  if (tokens <= 256) return;
+  if (tokens <= 128) return;
   g.split_scratch = reinterpret_cast<float*>(ws + w.splitk);
   g.split_scratch_bytes = pd::kSplitScratchBytes;
   g.split_flags = L->split_flags;
@@ -601,6 +601,7 @@ extern "C" pd_status pd_prefill_attention(const pd_layer_cfg* cfg, const void* q
   const int tokens = cu_host[n_req];
   if (tokens == 0) return PD_OK;
   if (!q || !out || !cu_dev || ldq < cfg->n_q_heads * cfg->head_dim || ldq % 8 != 0) return PD_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(out) & 31u) return PD_ERR_INVALID_ARG;
   pd::PrefillAttnArgs a{};
   a.q = static_cast<const bf16*>(q); a.ldq = ldq;
   a.k_cache = static_cast<const bf16*>(cache->k); a.v_cache = static_cast<const bf16*>(cache->v);
