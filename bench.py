@@ -39,12 +39,16 @@ TTFT_SLO, TPOT_SLO, TP_TOTAL = 2.0, 0.050, 2e5
 # one layer (profiles/gemm_tc_prefill_8b_ncu_full.md, profiles/prefill_attn_tc_and_decode_kernels_ncu_full.md).
 # Set an entry to None whenever the kernel changes after the capture.
 NCU_TRAFFIC = {
-    "gemm_tc_kernel": {"bytes_per_launch": 365.6e6, "algorithmic_bytes_per_launch": 238.8e6,
-                       "note": "gemm_tc_pair_kernel, mean over the four prefill projections of a layer (1462.4 MB / 4)"},
-    "decode_attn_kernel": {"bytes_per_launch": 2.1563e9, "algorithmic_bytes_per_launch": 2.1485e9,
-                           "note": "B = 256 at KV length 2049; grows in proportion to the KV length"},
+    "gemm_tc_kernel": {"bytes_per_launch": None, "algorithmic_bytes_per_launch": 238.8e6,
+                       "note": "gemm_tc_pair_kernel, mean over the four prefill projections of a layer; the kernel's raster "
+                               "changed after the last capture (365.6 MB per launch then)"},
+    "decode_attn_kernel": {"bytes_per_launch": None, "algorithmic_bytes_per_launch": 2.1485e9,
+                           "note": "B = 256 at KV length 2049; grows in proportion to the KV length (2.1563 GB before the "
+                                   "kernel's last change)"},
 }
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+# Datasheet figures of the part (dense bf16 without 2:4 sparsity; HBM3e of the HGX board), quoted beside the measured peaks.
+NOMINAL = {"bf16_tflops": 2250.0, "hbm_gbs": 7700.0}
 
 
 def load_peaks():
@@ -544,24 +548,33 @@ def main():
             "prefill": {"tok_s": prefill_tok_s, "ms_per_pass": pre_model_s * 1e3,
                         "tflops": flops_all * scale / pre_model_s / 1e12 * 1.0,
                         "frac_bf16_sustained": flops_all * scale / pre_model_s / 1e12 / peak_tf,
-                        "frac_bf16_burst": flops_all * scale / pre_model_s / 1e12 / peaks["bf16_tflops"]},
+                        "frac_bf16_burst": flops_all * scale / pre_model_s / 1e12 / peaks["bf16_tflops"],
+                        "frac_bf16_nominal": flops_all * scale / pre_model_s / 1e12 / NOMINAL["bf16_tflops"]},
             "decode": {"tok_s": decode_tok_s, "tpot_ms": tpot_s * 1e3, "feasible_batch": b_star,
                        "sweep_capped": bool(alloc["sweep_capped"]), "tpot_curve_ms": {str(k): v * 1e3 for k, v in curve.items()},
-                       "frac_hbm": dec_bytes_step * scale / tpot_s / 1e9 / peaks["hbm_gbs"]},
+                       "frac_hbm": dec_bytes_step * scale / tpot_s / 1e9 / peaks["hbm_gbs"],
+                       "frac_hbm_nominal": dec_bytes_step * scale / tpot_s / 1e9 / NOMINAL["hbm_gbs"]},
             "allocation": {"status": alloc["status"], "tp_prefill_eff": alloc["tp_prefill_eff"],
                            "tp_decode_eff": alloc["tp_decode_eff"], "n_prefill": alloc["n_prefill"],
                            "n_decode": alloc["n_decode"], "ratio_pd": alloc["ratio_pd"], "rho": alloc["rho"],
                            "mm1_sojourn_s": None if alloc["status"] else 1.0 / (alloc["mu"] - alloc["lam"]),
                            "replayed_sojourn_s_deterministic_service": sojourn},
+            # The launches are timed one by one with CUDA events (a traced pass), i.e. in isolation: the burst peak is
+            # the denominator; the sustained and the datasheet figure ride along.
             "roofline": {"kernel": "gemm_tc_pair_kernel (QKV, O, gate/up, down projections of the prefill pass)",
-                         "bound": "tensor", "achieved": gemm_tf, "peak": peak_tf, "unit": "TFLOP/s",
-                         "frac": gemm_tf / peak_tf, "frac_of_burst_peak": gemm_tf / peaks["bf16_tflops"],
-                         "peak_source": peaks["source"] + " (sustained bf16)", "launches": gemm_n,
-                         "avg_launch_ms": gemm_s / max(1, gemm_n) * 1e3, "traffic": NCU_TRAFFIC["gemm_tc_kernel"]["bytes_per_launch"], "traffic_unit": "DRAM bytes per launch (ncu)",
+                         "bound": "tensor", "achieved": gemm_tf, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                         "frac": gemm_tf / peaks["bf16_tflops"], "frac_of_sustained_peak": gemm_tf / peak_tf,
+                         "frac_of_nominal_peak": gemm_tf / NOMINAL["bf16_tflops"], "nominal_peak": NOMINAL["bf16_tflops"],
+                         "peak_source": peaks["source"] + " (burst bf16, torch.matmul 8192^3)", "launches": gemm_n,
+                         "avg_launch_ms": gemm_s / max(1, gemm_n) * 1e3,
+                         "traffic": NCU_TRAFFIC["gemm_tc_kernel"]["bytes_per_launch"], "traffic_unit": "DRAM bytes per launch (ncu)",
                          "traffic_detail": NCU_TRAFFIC["gemm_tc_kernel"],
                          "timing": "CUDA events around each launch in a separate traced pass of the same step"},
             "roofline_decode_attention": {"kernel": "decode_attn_kernel", "bound": "hbm", "achieved": attn_gbs,
                                           "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": attn_gbs / peaks["hbm_gbs"],
+                                          "frac_of_nominal_peak": attn_gbs / NOMINAL["hbm_gbs"], "nominal_peak": NOMINAL["hbm_gbs"],
+                                          "peak_source": peaks["source"] + " (device copy: read + write bytes; a pure read stream "
+                                                         "can exceed it slightly)",
                                           "launches": attn_dec_n, "avg_launch_ms": attn_dec_s / max(1, attn_dec_n) * 1e3,
                                           "traffic": NCU_TRAFFIC["decode_attn_kernel"]["bytes_per_launch"],
                                           "traffic_unit": "DRAM bytes per launch (ncu)",
