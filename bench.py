@@ -39,12 +39,10 @@ TTFT_SLO, TPOT_SLO, TP_TOTAL = 2.0, 0.050, 2e5
 # one layer (profiles/gemm_tc_prefill_8b_ncu_full.md, profiles/prefill_attn_tc_and_decode_kernels_ncu_full.md).
 # Set an entry to None whenever the kernel changes after the capture.
 NCU_TRAFFIC = {
-    "gemm_tc_kernel": {"bytes_per_launch": None, "algorithmic_bytes_per_launch": 238.8e6,
-                       "note": "gemm_tc_pair_kernel, mean over the four prefill projections of a layer; the kernel's raster "
-                               "changed after the last capture (365.6 MB per launch then)"},
-    "decode_attn_kernel": {"bytes_per_launch": None, "algorithmic_bytes_per_launch": 2.1485e9,
-                           "note": "B = 256 at KV length 2049; grows in proportion to the KV length (2.1563 GB before the "
-                                   "kernel's last change)"},
+    "gemm_tc_kernel": {"bytes_per_launch": 317.4e6, "algorithmic_bytes_per_launch": 238.8e6,
+                       "note": "gemm_tc_pair_kernel, mean over the four prefill projections of a layer (1269.8 MB / 4)"},
+    "decode_attn_kernel": {"bytes_per_launch": 2.1562e9, "algorithmic_bytes_per_launch": 2.1485e9,
+                           "note": "B = 256 at KV length 2049; grows in proportion to the KV length"},
 }
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # Datasheet figures of the part (dense bf16 without 2:4 sparsity; HBM3e of the HGX board), quoted beside the measured peaks.
