@@ -512,10 +512,13 @@ pd_status pd_mixture_throughput(const int32_t* l_in, const double* service_s, in
 
 /* Service time of each request length by linear interpolation between measured prefill times
  * (grid_l strictly increasing; lengths outside the grid take the end values):
- * t = t_lo + (t_hi - t_lo) * ((l - l_lo) / (l_hi - l_lo)).  Feeds pd_mixture_throughput, pd_mg1_sojourn and
- * pd_queue_replay when a length distribution is served from a grid of measured lengths. */
+ * t = t_lo + (t_hi - t_lo) * ((l - l_lo) / (l_hi - l_lo)), where l is the request length rounded up to a multiple
+ * of `quantum` >= 1: the prefill kernels work in tiles (256 rows per attention item and per GEMM tile pair), so the
+ * time is a step function of the length and a grid of tile multiples with quantum = the tile size has no
+ * interpolation error.  Feeds pd_mixture_throughput, pd_mg1_sojourn and pd_queue_replay when a length distribution
+ * is served from a grid of measured lengths. */
 pd_status pd_interp_service_times(const int32_t* grid_l, const double* grid_time_s, int32_t n_grid,
-                                  const int32_t* l_in, int64_t n, double* service_s);
+                                  const int32_t* l_in, int64_t n, int32_t quantum, double* service_s);
 
 /* Eq. 12: mean sojourn time 1 / (mu - lambda) of the M/M/1 prefill queue.  PD_ERR_INFEASIBLE_TTFT when
  * lambda >= mu (no steady state). */

@@ -269,12 +269,15 @@ def mg1_sojourn(service_times, lam: float) -> float:
     return pollaczek_khinchine_sojourn(lam, es, es2)
 
 
-def interp_service_times(grid_l, grid_t, lengths):
+def interp_service_times(grid_l, grid_t, lengths, quantum=1):
     """Service time of each length by linear interpolation between measured grid points
-    (grid_l strictly increasing); lengths outside the grid take the end values."""
+    (grid_l strictly increasing); lengths outside the grid take the end values.  A length is
+    first rounded up to a multiple of `quantum` (a server that works in tiles of that many
+    tokens takes as long for L tokens as for the next full tile)."""
     out = []
     n = len(grid_l)
     for l in lengths:
+        l = -(-int(l) // quantum) * quantum
         if l <= grid_l[0]:
             out.append(float(grid_t[0]))
             continue

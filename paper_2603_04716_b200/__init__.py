@@ -161,7 +161,7 @@ _lib.pd_queue_replay.argtypes = [C.POINTER(C.c_double), C.POINTER(C.c_double), C
                                  C.POINTER(C.c_double)]
 _DP, _IP = C.POINTER(C.c_double), C.POINTER(C.c_int32)
 _lib.pd_mixture_throughput.argtypes = [_IP, _DP, C.c_int64, _DP, _DP]
-_lib.pd_interp_service_times.argtypes = [_IP, _DP, C.c_int32, _IP, C.c_int64, _DP]
+_lib.pd_interp_service_times.argtypes = [_IP, _DP, C.c_int32, _IP, C.c_int64, C.c_int32, _DP]
 _lib.pd_mm1_sojourn.argtypes = [C.c_double, C.c_double, _DP]
 _lib.pd_mg1_sojourn.argtypes = [_DP, C.c_int64, C.c_double, _DP]
 _lib.pd_refine_next_batch.argtypes = [_IP, _DP, C.c_int32, C.c_double, _IP]
@@ -589,15 +589,16 @@ def pd_mixture_throughput(l_in, service_s):
     return tp.value, mean_l.value
 
 
-def pd_interp_service_times(grid_l, grid_time_s, l_in):
-    """numpy float64 array: service time of each length, interpolated on the measured grid."""
+def pd_interp_service_times(grid_l, grid_time_s, l_in, quantum: int = 1):
+    """numpy float64 array: service time of each length (rounded up to a multiple of `quantum`), interpolated on
+    the measured grid."""
     import numpy as np
     gl, gt, l = _np_i32(grid_l), _np_f64(grid_time_s), _np_i32(l_in)
     if gl.shape != gt.shape:
         raise ValueError("one time per grid length")
     out = np.empty(l.size, dtype=np.float64)
     _check(_lib.pd_interp_service_times(gl.ctypes.data_as(_IP), gt.ctypes.data_as(_DP), gl.size,
-                                        l.ctypes.data_as(_IP), l.size, out.ctypes.data_as(_DP)),
+                                        l.ctypes.data_as(_IP), l.size, quantum, out.ctypes.data_as(_DP)),
            "pd_interp_service_times")
     return out
 

@@ -119,15 +119,18 @@ def run_long_input(quick=False):
     cfg = pd.LayerConfig(**SHAPE_8B, max_pos=32768 + 256)
     nl = 4 if quick else 8
     lengths = gen.lognormal_lengths(1, 4096, 8192.0, 0.5, 2048, 32768)
-    grid_l = [2048, 8192, 20480, 32768] if quick else list(range(2048, 32768 + 1, 512))
+    # the kernels work in tiles of 256 rows: on a grid of 256-multiples, with lengths rounded up to the next one,
+    # the measured times are exact for every request length (no interpolation between tile counts)
+    quantum = 1 if quick else 256
+    grid_l = [2048, 8192, 20480, 32768] if quick else list(range(2048, 32768 + 1, 256))
     grid = _prefill_time_grid(cfg, grid_l, nl, 32, 2 if quick else 3, peaks)
     # interpolation check on seeded off-grid lengths
     off = sorted(int(v) for v in gen.uniform_lengths(2, 2 if quick else 8, 2100, 32000, sub=7))
     off_meas = _prefill_time_grid(cfg, off, nl, 32, 2 if quick else 3, peaks)
-    off_interp = pd.pd_interp_service_times(grid["l"], grid["time_s"], off)
+    off_interp = pd.pd_interp_service_times(grid["l"], grid["time_s"], off, quantum)
     interp_check = [{"l": l, "measured_s": tm, "interpolated_s": float(ti)}
                     for l, tm, ti in zip(off_meas["l"], off_meas["time_s"], off_interp)]
-    service = pd.pd_interp_service_times(grid["l"], grid["time_s"], lengths)
+    service = pd.pd_interp_service_times(grid["l"], grid["time_s"], lengths, quantum)
     tp_max, mean_l = pd.pd_mixture_throughput(lengths, service)     # total tokens over total time; mean length
     sweep = [1, 64] if quick else [1, 2, 4, 8, 16, 32, 64, 128, 256]
     d = pd.pd_measure(cfg, n_layers_run=nl, n_layers_model=32, warmup=1, reps=3, seed=0, batch_sizes=sweep,
@@ -144,7 +147,7 @@ def run_long_input(quick=False):
         soj, wait = pd.pd_queue_replay(gaps, svc)
         replay.append({"rho": rho, "lambda": lam, "mm1_sojourn_s": pd.pd_mm1_sojourn(mu, lam), "replayed_sojourn_s": soj,
                        "pollaczek_khinchine_s": pd.pd_mg1_sojourn(service, lam)})
-    return {"config": "long_input", "layers_run": nl, "sigma": 0.5, "mean_l_in": mean_l, "prefill_max_tok_s": tp_max,
+    return {"config": "long_input", "layers_run": nl, "sigma": 0.5, "tile_quantum": quantum, "mean_l_in": mean_l, "prefill_max_tok_s": tp_max,
             "prefill_time_grid": grid, "interpolation_check": interp_check, "queue": replay, "decode": d,
             "lengths": {"generator": "pd_inputs.lognormal_lengths(1, 4096, 8192.0, 0.5, 2048, 32768)"},
             "allocation": alloc}
@@ -193,9 +196,10 @@ def run_70b(quick=False):
     # mixed workload: L_in ~ U[1024, 8192], L_out ~ U[128, 1024]
     l_in = gen.uniform_lengths(3, 512, 1024, 8192, sub=0)
     l_out = gen.uniform_lengths(3, 512, 128, 1024, sub=1)
-    grid_l = [1024, 4096, 8192] if quick else list(range(1024, 8192 + 1, 512))
+    quantum = 1 if quick else 256
+    grid_l = [1024, 4096, 8192] if quick else list(range(1024, 8192 + 1, 256))
     grid = _prefill_time_grid(cfg, grid_l, nl, 80, 2, peaks)
-    tp_max_mix, mean_l_in = pd.pd_mixture_throughput(l_in, pd.pd_interp_service_times(grid["l"], grid["time_s"], l_in))
+    tp_max_mix, mean_l_in = pd.pd_mixture_throughput(l_in, pd.pd_interp_service_times(grid["l"], grid["time_s"], l_in, quantum))
     # stationary decode batch: sequence i sits at a uniformly random point of its output
     prog = gen.uniform_lengths(3, 512, 0, 10**6, sub=2) / 1e6
     mix = (l_in + np.floor(prog * l_out)).astype(np.int32)
@@ -204,7 +208,7 @@ def run_70b(quick=False):
                        peak_bf16_flops=peaks[0], peak_hbm_bytes_s=peaks[1])
     return {"config": "70b", "layers_run": nl, "layers_model": 80, "prefill": p, "decode": d,
             "allocation": _alloc(2e5, 4096, 256, 3.0, 0.060, p["prefill_tok_s"], d["batch"], d["tpot_s"]),
-            "mixed": {"mean_l_in": mean_l_in, "mean_l_out": float(l_out.mean()),
+            "mixed": {"mean_l_in": mean_l_in, "mean_l_out": float(l_out.mean()), "tile_quantum": quantum,
                       "prefill_max_tok_s": tp_max_mix, "prefill_time_grid": grid, "decode": dm,
                       "allocation": _alloc(2e5, mean_l_in, float(l_out.mean()), 3.0, 0.060, tp_max_mix,
                                            dm["batch"], dm["tpot_s"])}}

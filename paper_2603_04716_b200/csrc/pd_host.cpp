@@ -168,12 +168,13 @@ extern "C" pd_status pd_mixture_throughput(const int32_t* l_in, const double* se
 }
 
 extern "C" pd_status pd_interp_service_times(const int32_t* grid_l, const double* grid_time_s, int32_t n_grid,
-                                             const int32_t* l_in, int64_t n, double* service_s) {
-  if (!grid_l || !grid_time_s || n_grid <= 0 || !l_in || n < 0 || !service_s) return PD_ERR_INVALID_ARG;
+                                             const int32_t* l_in, int64_t n, int32_t quantum, double* service_s) {
+  if (!grid_l || !grid_time_s || n_grid <= 0 || !l_in || n < 0 || !service_s || quantum < 1) return PD_ERR_INVALID_ARG;
   for (int i = 0; i + 1 < n_grid; ++i)
     if (grid_l[i + 1] <= grid_l[i]) return PD_ERR_INVALID_ARG;
   for (int64_t r = 0; r < n; ++r) {
-    const int32_t l = l_in[r];
+    if (l_in[r] < 0 || l_in[r] > 2147483647 - quantum) return PD_ERR_INVALID_ARG;
+    const int32_t l = (l_in[r] + quantum - 1) / quantum * quantum;  // the next full tile
     if (l <= grid_l[0]) { service_s[r] = grid_time_s[0]; continue; }
     if (l >= grid_l[n_grid - 1]) { service_s[r] = grid_time_s[n_grid - 1]; continue; }
     int lo = 0, hi = n_grid - 1;  // grid_l[lo] < l <= grid_l[hi]

@@ -17,7 +17,29 @@ namespace {
 // Batches beyond one 256-wide batch tile run the projections on the prefill GEMM (fused epilogues, tail
 // tiles split): the weight-streaming kernel would read every weight once per batch tile (measured per
 // 8B-shaped layer: 327 -> 242 us at B = 384, 352 -> 275 us at B = 512; at B = 256 the two paths tie).
-constexpr int kWideDecodeBatch = 257;
+constexpr int kWideDecodeBatchDefault = 257;
+// (PD_WIDE_DECODE_BATCH in the environment overrides it, for A/B timing.)
+int wide_decode_batch() {
+  static const int v = [] {
+    const char* e = std::getenv("PD_WIDE_DECODE_BATCH");
+    const int n = e ? std::atoi(e) : kWideDecodeBatchDefault;
+    return n > 0 ? n : kWideDecodeBatchDefault;
+  }();
+  return v;
+}
+
+// From this batch on the gate/up projection of a decode step runs on the prefill GEMM (CTA pairs, SwiGLU in the
+// epilogue) instead of the weight-streaming kernel: with N = 2 d_ff it has enough 256-wide tiles to fill the pairs
+// even at one or two row tiles, and the tensor pipe, not the weight stream, is what bounds it there.
+// PD_GU_GEMM_BATCH in the environment overrides the threshold (for A/B timing; 0 = never).
+int gate_up_gemm_batch() {
+  static const int v = [] {
+    const char* e = std::getenv("PD_GU_GEMM_BATCH");
+    const int n = e ? std::atoi(e) : 129;
+    return n > 0 ? n : 1 << 30;
+  }();
+  return v;
+}
 
 struct Workspace {
   // byte offsets into the caller's workspace
@@ -43,7 +65,7 @@ Workspace carve(const pd_layer_cfg& c, size_t tokens, size_t max_batch, int max_
   w.act = take(tokens * f * 2);
   {  // fp32 sums of the four decode-mode projections, one buffer each (a buffer is cleared by a row-wise kernel
      // earlier in the chain while another one is in use); batches beyond the weight-streaming path need none
-    const size_t rows = max_batch < static_cast<size_t>(kWideDecodeBatch) ? max_batch : 0;
+    const size_t rows = max_batch < static_cast<size_t>(wide_decode_batch()) ? max_batch : 0;
     w.acc_qkv = take(rows * nqkv * 4);
     w.acc_o = take(rows * d * 4);
     w.acc_gu = take(rows * 2 * f * 4);
@@ -268,7 +290,7 @@ struct DecodeLink {
 pd_status decode_impl(pd_layer* L, const bf16* x, bf16* out, const int32_t* kv_len_dev, int B, int max_kv_len,
                       const pd_kv_cache* cache, uint8_t* ws, const Workspace& w, cudaStream_t st,
                       const DecodeLink& link = DecodeLink{}) {
-  if (B >= kWideDecodeBatch) return decode_impl_wide(L, x, out, kv_len_dev, B, max_kv_len, cache, ws, w, st);
+  if (B >= wide_decode_batch()) return decode_impl_wide(L, x, out, kv_len_dev, B, max_kv_len, cache, ws, w, st);
   const pd_layer_cfg& c = L->cfg;
   const int hq = c.n_q_heads * c.head_dim;
   bf16* norm = reinterpret_cast<bf16*>(ws + w.norm);
@@ -297,7 +319,8 @@ pd_status decode_impl(pd_layer* L, const bf16* x, bf16* out, const int32_t* kv_l
   float* z_down = pd::gemm_skinny_splits(B, c.d_model, c.d_ff, f8) > 1 ? acc_down : nullptr;
   // Gate/up is not split along K at these shapes: SwiGLU then runs in its epilogue (no fp32 round trip, one launch
   // fewer) and the buffer of the down projection is cleared one kernel earlier.
-  const bool fuse_swiglu = pd::gemm_skinny_fuses_swiglu(B, n_gu, c.d_model, f8);
+  const bool gu_gemm = B >= gate_up_gemm_batch() && B > 128;
+  const bool fuse_swiglu = gu_gemm || pd::gemm_skinny_fuses_swiglu(B, n_gu, c.d_model, f8);
   // FP8 mode: a row-wise quantiser in front of every projection (same programmatic-serialization chain)
   uint8_t* q_act = ws + w.q_act;
   float* s_act = reinterpret_cast<float*>(ws + w.s_act);
@@ -343,12 +366,20 @@ pd_status decode_impl(pd_layer* L, const bf16* x, bf16* out, const int32_t* kv_l
   }
   {
     pd::TraceScope ts(PD_K_GEMM_GATE_UP, st);
-    g.x = norm; g.w = L->w_gu; g.acc = acc_gu; g.n = n_gu; g.k = c.d_model; g.ldx = c.d_model;
-    PD_TRY(fp8_in(g, L->q_gu, L->s_gu, true));
-    g.swiglu_out = fuse_swiglu ? act : nullptr;
-    PD_TRY(pd::gemm_skinny(g, st));
-    g.swiglu_out = nullptr;
-    if (!fuse_swiglu) PD_TRY(pd::launch_skinny_swiglu(acc_gu, act, B, c.d_ff, z_down, c.d_model, st));
+    if (gu_gemm) {
+      pd::GemmArgs gg{};
+      gg.a = norm; gg.b = L->w_gu; gg.c = act; gg.m = B; gg.n = n_gu; gg.k = c.d_model;
+      gg.lda = c.d_model; gg.ldb = c.d_model; gg.ldc = c.d_ff; gg.epilogue = pd::EPI_SWIGLU; gg.err_word = L->err_word;
+      if (f8) PD_TRY(use_fp8(L, gg, L->q_gu, L->s_gu, ws, w, st, true));  // (the codes of norm are already in place)
+      PD_TRY(pd::gemm(gg, st));
+    } else {
+      g.x = norm; g.w = L->w_gu; g.acc = acc_gu; g.n = n_gu; g.k = c.d_model; g.ldx = c.d_model;
+      PD_TRY(fp8_in(g, L->q_gu, L->s_gu, true));
+      g.swiglu_out = fuse_swiglu ? act : nullptr;
+      PD_TRY(pd::gemm_skinny(g, st));
+      g.swiglu_out = nullptr;
+      if (!fuse_swiglu) PD_TRY(pd::launch_skinny_swiglu(acc_gu, act, B, c.d_ff, z_down, c.d_model, st));
+    }
   }
   {
     pd::TraceScope ts(PD_K_GEMM_DOWN, st);
@@ -720,7 +751,7 @@ extern "C" pd_status pd_decode_stack(pd_layer* const* layers, const pd_kv_cache*
   DecodeLink link{};
   for (int i = 0; i < n_layers; ++i) {
     bf16* dst = (i == n_layers - 1 && !io_on_host) ? static_cast<bf16*>(out) : buf[(i + 1) & 1];
-    const bool fuse = fuse_next_norm && i + 1 < n_layers && B < kWideDecodeBatch &&
+    const bool fuse = fuse_next_norm && i + 1 < n_layers && B < wide_decode_batch() &&
                       std::memcmp(&layers[i]->cfg, &layers[i + 1]->cfg, sizeof(pd_layer_cfg)) == 0;
     link.next_gain = fuse ? layers[i + 1]->g_attn : nullptr;
     PD_TRY(decode_impl(layers[i], cur, dst, kv_dev, B, max_kv_len, &caches[i % n_caches], ws, w, st, link));

@@ -69,7 +69,8 @@ def check_result(res, pd=None):
     if res.get("config") == "long_input":
         lengths = gen.lognormal_lengths(1, 4096, 8192.0, 0.5, 2048, 32768)
         g = res["prefill_time_grid"]
-        svc = A.interp_service_times(g["l"], g["time_s"], lengths.tolist())
+        quantum = res.get("tile_quantum", 1)
+        svc = A.interp_service_times(g["l"], g["time_s"], lengths.tolist(), quantum)
         tp, mean_l = A.mixture_throughput(lengths.tolist(), svc)
         assert tp == res["prefill_max_tok_s"] and mean_l == res["mean_l_in"]
         mu = A.service_rate(tp, mean_l)
@@ -85,11 +86,12 @@ def check_result(res, pd=None):
             if es2 <= 2.0 * es * es:
                 assert q["pollaczek_khinchine_s"] <= q["mm1_sojourn_s"] * (1 + 1e-12)
         for c in res["interpolation_check"]:
-            assert c["interpolated_s"] == A.interp_service_times(g["l"], g["time_s"], [c["l"]])[0]
+            assert c["interpolated_s"] == A.interp_service_times(g["l"], g["time_s"], [c["l"]], quantum)[0]
     if res.get("config") == "70b":
         m = res["mixed"]
         l_in = gen.uniform_lengths(3, 512, 1024, 8192, sub=0)
         g = m["prefill_time_grid"]
-        tp, mean_l = A.mixture_throughput(l_in.tolist(), A.interp_service_times(g["l"], g["time_s"], l_in.tolist()))
+        tp, mean_l = A.mixture_throughput(l_in.tolist(), A.interp_service_times(g["l"], g["time_s"], l_in.tolist(),
+                                                                                m.get("tile_quantum", 1)))
         assert tp == m["prefill_max_tok_s"] and mean_l == m["mean_l_in"]
     return n

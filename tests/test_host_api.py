@@ -182,8 +182,9 @@ def test_workload_statistics_match_oracle_bit_for_bit(pdlib):
         ls = rng.integers(16, 40000, size=n).astype(np.int32)
         grid_l = sorted(rnd.sample(range(16, 40000), rnd.randint(1, 40)))
         grid_t = sorted(rnd.uniform(1e-3, 3.0) for _ in grid_l)
-        svc = pdlib.pd_interp_service_times(grid_l, grid_t, ls)
-        o_svc = A.interp_service_times(grid_l, grid_t, ls.tolist())
+        quantum = rnd.choice([1, 1, 64, 256])
+        svc = pdlib.pd_interp_service_times(grid_l, grid_t, ls, quantum)
+        o_svc = A.interp_service_times(grid_l, grid_t, ls.tolist(), quantum)
         assert svc.tolist() == o_svc
         tp, mean_l = pdlib.pd_mixture_throughput(ls, svc)
         assert (tp, mean_l) == A.mixture_throughput(ls.tolist(), o_svc)

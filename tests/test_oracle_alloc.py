@@ -244,6 +244,9 @@ def test_interp_service_times_against_numpy():
     np.testing.assert_allclose(got, np.interp(ls, grid_l, grid_t), rtol=1e-12)
     # exact at the grid points and on a straight line
     assert A.interp_service_times([10, 20], [1.0, 2.0], [10, 15, 20, 5, 30]) == [1.0, 1.5, 2.0, 1.0, 2.0]
+    # tile quantum: a length counts as the next multiple of the quantum (a step function on a grid of multiples)
+    assert A.interp_service_times([8, 16, 24], [1.0, 2.0, 4.0], [1, 8, 9, 16, 17, 24], quantum=8) == [1.0, 1.0, 2.0, 2.0, 4.0, 4.0]
+    assert A.interp_service_times([8, 24], [1.0, 3.0], [9, 13], quantum=4) == [1.5, 2.0]
 
 
 def test_refine_next_batch_brackets_the_largest_feasible_integer():
