@@ -30,12 +30,15 @@ int wide_decode_batch() {
 
 // From this batch on the gate/up projection of a decode step runs on the prefill GEMM (CTA pairs, SwiGLU in the
 // epilogue) instead of the weight-streaming kernel: with N = 2 d_ff it has enough 256-wide tiles to fill the pairs
-// even at one or two row tiles, and the tensor pipe, not the weight stream, is what bounds it there.
+// even at one or two row tiles, and the tensor pipe, not the weight stream, is what bounds it there (measured per
+// 8B-shaped layer: gate/up 74.7 -> 66.0 us at B = 256, 68.6 -> 64.4 at 192, no gain at 129; the other three
+// projections are faster on the weight-streaming kernel up to B = 256: the whole layer on the prefill GEMM takes 483
+// against 455 us at B = 256).
 // PD_GU_GEMM_BATCH in the environment overrides the threshold (for A/B timing; 0 = never).
 int gate_up_gemm_batch() {
   static const int v = [] {
     const char* e = std::getenv("PD_GU_GEMM_BATCH");
-    const int n = e ? std::atoi(e) : 129;
+    const int n = e ? std::atoi(e) : 192;
     return n > 0 ? n : 1 << 30;
   }();
   return v;
