@@ -123,13 +123,16 @@ def run_long_input(quick=False):
     # the measured times are exact for every request length (no interpolation between tile counts)
     quantum = 1 if quick else 256
     grid_l = [2048, 8192, 20480, 32768] if quick else list(range(2048, 32768 + 1, 256))
-    grid = _prefill_time_grid(cfg, grid_l, nl, 32, 2 if quick else 3, peaks)
-    # interpolation check on seeded off-grid lengths
-    off = sorted(int(v) for v in gen.uniform_lengths(2, 2 if quick else 8, 2100, 32000, sub=7))
-    off_meas = _prefill_time_grid(cfg, off, nl, 32, 2 if quick else 3, peaks)
+    # interpolation check on seeded off-grid lengths, timed in the same pd_measure call as the grid (same clocks: under
+    # the power cap two calls differ by more than the interpolation does)
+    off = sorted(int(v) for v in gen.uniform_lengths(2, 2 if quick else 7, 2100, 32000, sub=7))
+    both = _prefill_time_grid(cfg, grid_l + off, nl, 32, 2 if quick else 3, peaks)
+    grid = {"l": both["l"][:len(grid_l)], "time_s": both["time_s"][:len(grid_l)]}
+    off_meas = {"l": both["l"][len(grid_l):], "time_s": both["time_s"][len(grid_l):]}
     off_interp = pd.pd_interp_service_times(grid["l"], grid["time_s"], off, quantum)
-    interp_check = [{"l": l, "measured_s": tm, "interpolated_s": float(ti)}
-                    for l, tm, ti in zip(off_meas["l"], off_meas["time_s"], off_interp)]
+    off_linear = pd.pd_interp_service_times(grid["l"], grid["time_s"], off, 1)
+    interp_check = [{"l": l, "measured_s": tm, "interpolated_s": float(ti), "linear_s": float(tl)}
+                    for l, tm, ti, tl in zip(off_meas["l"], off_meas["time_s"], off_interp, off_linear)]
     service = pd.pd_interp_service_times(grid["l"], grid["time_s"], lengths, quantum)
     tp_max, mean_l = pd.pd_mixture_throughput(lengths, service)     # total tokens over total time; mean length
     sweep = [1, 64] if quick else [1, 2, 4, 8, 16, 32, 64, 128, 256]
