@@ -22,6 +22,13 @@
 // use, because 0 * (uninitialised cache memory) must not produce NaN.
 // All barriers run on counters that continue across items (parity = counter bit).  Every wait is
 // wall-clock bounded and leaves through the common teardown.
+// The three single-thread roles are functions that are never inlined: each gets registers of its own, apart
+// from the softmax code, which needs every register the launch bounds allow.  The MMA issuer sets the pace
+// of the kernel: the tensor pipe takes a 128 x 128 x 16 product instruction about every 62 cycles, its
+// execution time, and queues hardly any, so the pipe is busy exactly while the thread issues and idles while
+// the thread polls, commits and keeps its books.  Hence the plain code of that loop: state of it in local
+// memory, polls placed between the instructions of a product, or a second issuing thread (the two
+// instruction streams interleave in the pipe and every product finishes later) were all measured slower.
 #include <math_constants.h>
 
 #include <atomic>
@@ -98,10 +105,220 @@ __device__ __forceinline__ bool decode_item(const AttDev& p, int idx, Item& it) 
   return true;
 }
 
+// The MMA issuer's loop, one thread.  A function of its own (never inlined), so that its registers are allocated
+// apart from the softmax code, whose pressure would otherwise push this loop's state into local memory.
+template <int HD>
+__device__ __noinline__ void mma_issuer(const uint32_t smem_base, const uint32_t tmem_base, const uint32_t bar0,
+                                        const Item* item_ring, volatile int* abort_flag, const uint64_t limit) {
+  using Cfg = AttCfg<HD>;
+  auto bar = [&](int i) { return bar0 + 8u * i; };
+  constexpr uint32_t idesc_qk = ptx::umma_idesc_bf16(TQ, TK);
+  constexpr uint32_t idesc_pv = ptx::umma_idesc_bf16_bmn(TQ, HD);
+  // Per row tile: the item it is working on and how far it has got.  The two tiles walk the same item
+  // sequence and share the K / V rings, but each advances as soon as its own inputs are ready.
+  Item cur[2];
+  bool have[2] = {false, false}, done[2] = {false, false};
+  int seq[2] = {0, 0};      // items taken from the ring so far
+  int base[2] = {0, 0};     // ring position of the current item's first K / V tile
+  int n[2] = {0, 0};        // K / V tiles of the current item for this row tile
+  int jq[2] = {0, 0};       // next Q K^T to issue
+  int jp[2] = {0, 0};       // next P V to issue
+  int act[2] = {0, 0};      // items with work for this row tile finished so far
+  int pv_cnt[2] = {0, 0};   // P V products issued so far (phase of p_ready)
+  uint32_t k_used = 0, v_used = 0;  // users that have consumed the tile in each ring slot, 4 bits per slot
+  uint64_t t_idle = 0;
+  uint32_t idle_polls = 0;
+  bool ok = true;
+  while (ok && !(done[0] && done[1])) {
+    bool progress = false;
+#pragma unroll
+    for (int t = 0; t < 2; ++t) {
+      if (done[t]) continue;
+      if (!have[t]) {
+        const int s = seq[t] & (ITEM_SLOTS - 1);
+        if (!ptx::mbar_test_wait(bar(B_IFULL + s), (seq[t] / ITEM_SLOTS) & 1)) continue;
+        cur[t] = item_ring[s];
+        ptx::mbar_arrive(bar(B_IEMPTY + s));
+        ++seq[t];
+        progress = true;
+        if (cur[t].n_kv0 < 0) { done[t] = true; continue; }
+        n[t] = t == 0 ? cur[t].n_kv0 : cur[t].n_kv1;
+        if (n[t] == 0) {  // this item has rows for the other tile only
+          base[t] += max(cur[t].n_kv0, cur[t].n_kv1);
+          continue;
+        }
+        have[t] = true; jq[t] = 0; jp[t] = 0;
+      }
+      const Item& it = cur[t];
+      if (jp[t] < jq[t]) {
+        // ---- O_t += P_t V_j
+        const int j = jp[t], g = base[t] + j, s = g % V_SLOTS;
+        if (!ptx::mbar_test_wait(bar(B_PREADY + t), pv_cnt[t] & 1)) continue;
+        if (!ptx::mbar_test_wait(bar(B_VFULL + s), (g / V_SLOTS) & 1)) continue;
+        // the first product of an item overwrites O: the previous item's output must have been read out
+        if (j == 0 && act[t] > 0 && !ptx::mbar_test_wait(bar(B_OREAD + t), (act[t] - 1) & 1)) continue;
+        ptx::tc_fence_after();
+        const uint32_t sv = smem_base + Cfg::V_OFF + s * Cfg::TILE_BYTES;
+        const uint32_t d = tmem_base + t * Cfg::TILE_COLS + Cfg::O_COL;
+        const uint32_t a = tmem_base + t * Cfg::TILE_COLS + Cfg::S_COL;
+#pragma unroll
+        for (int kk = 0; kk < TK / 16; ++kk) {
+          // 16 keys = 16 rows of 128 bytes further into the V tile; 8 packed columns further into P
+          ptx::umma_bf16_ts(d, a + kk * 8, ptx::umma_desc_mn_sw128(sv + kk * 2048, Cfg::SUB_BYTES), idesc_pv,
+                            (j > 0 || kk > 0) ? 1u : 0u);
+        }
+        ptx::umma_commit(bar(B_ODONE + t));
+        const uint32_t users = (j < it.n_kv0 ? 1u : 0u) + (j < it.n_kv1 ? 1u : 0u);
+        v_used += 1u << (4 * s);
+        if (((v_used >> (4 * s)) & 15u) == users) { ptx::umma_commit(bar(B_VEMPTY + s)); v_used &= ~(15u << (4 * s)); }
+        ++pv_cnt[t]; ++jp[t];
+        progress = true;
+        if (jp[t] == n[t]) {  // item finished for this tile
+          have[t] = false;
+          ++act[t];
+          base[t] += max(it.n_kv0, it.n_kv1);
+          continue;
+        }
+      }
+      if (jq[t] < n[t] && jq[t] == jp[t]) {
+        // ---- S_t = Q_t K_j^T (S is free: the P that aliased it has been consumed by the product above)
+        const int j = jq[t], g = base[t] + j, s = g % K_SLOTS;
+        if (j == 0 && !ptx::mbar_test_wait(bar(B_QFULL + t), act[t] & 1)) continue;
+        if (!ptx::mbar_test_wait(bar(B_KFULL + s), (g / K_SLOTS) & 1)) continue;
+        ptx::tc_fence_after();
+        const uint32_t sq = smem_base + Cfg::Q_OFF + t * Cfg::TILE_BYTES;
+        const uint32_t sk = smem_base + Cfg::K_OFF + s * Cfg::TILE_BYTES;
+        const uint32_t d = tmem_base + t * Cfg::TILE_COLS + Cfg::S_COL;
+#pragma unroll
+        for (int kk = 0; kk < HD / 16; ++kk) {
+          const uint32_t off = (kk >> 2) * Cfg::SUB_BYTES + (kk & 3) * 32;
+          ptx::umma_bf16(d, ptx::umma_desc_sw128(sq + off), ptx::umma_desc_sw128(sk + off), idesc_qk, kk > 0 ? 1u : 0u);
+        }
+        ptx::umma_commit(bar(B_SFULL + t));
+        const uint32_t users = (j < it.n_kv0 ? 1u : 0u) + (j < it.n_kv1 ? 1u : 0u);
+        k_used += 1u << (4 * s);
+        if (((k_used >> (4 * s)) & 15u) == users) { ptx::umma_commit(bar(B_KEMPTY + s)); k_used &= ~(15u << (4 * s)); }
+        ++jq[t];
+        if (jq[t] == n[t]) ptx::umma_commit(bar(B_QEMPTY + t));  // the tile's Q buffer may be refilled
+        progress = true;
+      }
+    }
+    if (progress) {
+      idle_polls = 0;
+      t_idle = 0;
+    } else if ((++idle_polls & 1023u) == 0u) {
+      // nothing could be issued for a while: look at the abort flag and the clock
+      if (*abort_flag) { ok = false; break; }
+      const uint64_t now = ptx::globaltimer_ns();
+      if (t_idle == 0) t_idle = now;
+      else if (now - t_idle > limit) { *abort_flag = 1; ok = false; }
+    }
+  }
+}
+
+// The producer's loop (one thread): work items, K and V tiles.  Like the MMA issuer a function of its own.
+template <int HD>
+__device__ __noinline__ void kv_producer(const CUtensorMap* tmap_k, const CUtensorMap* tmap_v, const AttDev& p,
+                                         const uint32_t smem_base, const uint32_t bar0, Item* item_ring,
+                                         volatile int* abort_flag, const uint64_t limit) {
+  using Cfg = AttCfg<HD>;
+  auto bar = [&](int i) { return bar0 + 8u * i; };
+  int it_pub = 0;               // items published so far (ring position)
+  int g_k = 0, g_v = 0;         // K / V tiles loaded so far (ring positions)
+  bool ok = true;
+  // the next item is fetched and decoded while the current one's tiles are being loaded
+  auto fetch = [&](Item& it) {
+    for (;;) {
+      const int idx = atomicAdd(p.sched, 1);
+      if (idx >= p.n_items) {
+        it.h = it.start = it.len = it.q0 = it.pre = it.kv_row0 = it.n_kv1 = 0;
+        it.n_kv0 = -1;
+        return;
+      }
+      if (decode_item(p, idx, it)) return;  // (rows beyond a request's length: nothing to do)
+    }
+  };
+  Item nxt;
+  fetch(nxt);
+  while (ok) {
+    const Item it = nxt;
+    const bool last = it.n_kv0 < 0;
+    {
+      const int s = it_pub & (ITEM_SLOTS - 1);
+      if (!ptx::mbar_wait_bounded(bar(B_IEMPTY + s), ((it_pub / ITEM_SLOTS) & 1) ^ 1u, abort_flag, limit)) { ok = false; break; }
+      item_ring[s] = it;
+      ptx::mbar_arrive(bar(B_IFULL + s));  // release: the item is visible to whoever sees the phase flip
+      ++it_pub;
+    }
+    if (last) break;
+    const int n_max = max(it.n_kv0, it.n_kv1);
+    for (int j = 0; j < n_max && ok; ++j) {
+      // K and V slots are released separately: K as soon as the Q K^T products that use it have run, V only
+      // after the P V products, so later K tiles are on their way while the softmax runs
+      const int sk_i = g_k % K_SLOTS;
+      if (!ptx::mbar_wait_bounded(bar(B_KEMPTY + sk_i), ((g_k / K_SLOTS) & 1) ^ 1u, abort_flag, limit)) { ok = false; break; }
+      if (!(p.test_skip_load && g_k == 1)) {
+        const uint32_t sk = smem_base + Cfg::K_OFF + sk_i * Cfg::TILE_BYTES;
+        ptx::mbar_arrive_expect_tx(bar(B_KFULL + sk_i), Cfg::TILE_BYTES);
+        for (int c = 0; c < Cfg::SUB; ++c)
+          ptx::tma_load_2d(sk + c * Cfg::SUB_BYTES, tmap_k, c * 64, it.kv_row0 + j * TK, bar(B_KFULL + sk_i));
+      }
+      ++g_k;
+      const int sv_i = g_v % V_SLOTS;
+      if (!ptx::mbar_wait_bounded(bar(B_VEMPTY + sv_i), ((g_v / V_SLOTS) & 1) ^ 1u, abort_flag, limit)) { ok = false; break; }
+      const uint32_t sv = smem_base + Cfg::V_OFF + sv_i * Cfg::TILE_BYTES;
+      ptx::mbar_arrive_expect_tx(bar(B_VFULL + sv_i), Cfg::TILE_BYTES);
+      for (int c = 0; c < Cfg::SUB; ++c)
+        ptx::tma_load_2d(sv + c * Cfg::SUB_BYTES, tmap_v, c * 64, it.kv_row0 + j * TK, bar(B_VFULL + sv_i));
+      ++g_v;
+      if (j == 0) fetch(nxt);  // (after this item's first loads are on their way)
+    }
+  }
+  if (!ok) {
+    // give loads already in flight time to land before the block's shared memory is released
+#pragma unroll 1
+    for (int i = 0; i < 2000; ++i) __nanosleep(1000);
+  }
+}
+
+// The Q loader's loop (one thread).  Its own thread, so that a wait for one tile's Q buffer never holds up the K / V
+// stream of the other tile.
+template <int HD>
+__device__ __noinline__ void q_loader(const CUtensorMap* tmap_q, const uint32_t smem_base, const uint32_t bar0,
+                                      const Item* item_ring, volatile int* abort_flag, const uint64_t limit) {
+  using Cfg = AttCfg<HD>;
+  auto bar = [&](int i) { return bar0 + 8u * i; };
+  int seq = 0;
+  int q_cnt[2] = {0, 0};  // Q loads so far per row tile
+  bool ok = true;
+  while (ok) {
+    const int s = seq & (ITEM_SLOTS - 1);
+    if (!ptx::mbar_wait_bounded(bar(B_IFULL + s), (seq / ITEM_SLOTS) & 1, abort_flag, limit)) break;
+    const Item it = item_ring[s];
+    ptx::mbar_arrive(bar(B_IEMPTY + s));
+    ++seq;
+    if (it.n_kv0 < 0) break;
+    for (int t = 0; t < 2; ++t) {
+      if (t == 1 && it.n_kv1 == 0) break;
+      // the tile's Q buffer is free once the last Q K^T of its previous item has been executed
+      if (!ptx::mbar_wait_bounded(bar(B_QEMPTY + t), (q_cnt[t] & 1) ^ 1u, abort_flag, limit)) { ok = false; break; }
+      ptx::mbar_arrive_expect_tx(bar(B_QFULL + t), Cfg::TILE_BYTES);
+      for (int c = 0; c < Cfg::SUB; ++c)
+        ptx::tma_load_2d(smem_base + Cfg::Q_OFF + t * Cfg::TILE_BYTES + c * Cfg::SUB_BYTES, tmap_q, it.h * HD + c * 64,
+                         it.start + it.q0 + t * TQ, bar(B_QFULL + t));
+      ++q_cnt[t];
+    }
+  }
+  if (!ok) {
+#pragma unroll 1
+    for (int i = 0; i < 2000; ++i) __nanosleep(1000);
+  }
+}
+
 template <int HD>
 __global__ void __launch_bounds__(ATT_THREADS, 1)
 prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
-                       const __grid_constant__ CUtensorMap tmap_v, AttDev p) {
+                       const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ AttDev p) {
   using Cfg = AttCfg<HD>;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -144,198 +361,13 @@ prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
 
   if (warp == 0) {
     // ---------------------------------------------------------------- producer
-    if (lane == 0) {
-      int it_pub = 0;               // items published so far (ring position)
-      int g_k = 0, g_v = 0;         // K / V tiles loaded so far (ring positions)
-      bool ok = true;
-      // the next item is fetched and decoded while the current one's tiles are being loaded
-      auto fetch = [&](Item& it) {
-        for (;;) {
-          const int idx = atomicAdd(p.sched, 1);
-          if (idx >= p.n_items) {
-            it.h = it.start = it.len = it.q0 = it.pre = it.kv_row0 = it.n_kv1 = 0;
-            it.n_kv0 = -1;
-            return;
-          }
-          if (decode_item(p, idx, it)) return;  // (rows beyond a request's length: nothing to do)
-        }
-      };
-      Item nxt;
-      fetch(nxt);
-      while (ok) {
-        const Item it = nxt;
-        const bool last = it.n_kv0 < 0;
-        {
-          const int s = it_pub & (ITEM_SLOTS - 1);
-          if (!ptx::mbar_wait_bounded(bar(B_IEMPTY + s), ((it_pub / ITEM_SLOTS) & 1) ^ 1u, abort_flag, limit)) { ok = false; break; }
-          item_ring[s] = it;
-          ptx::mbar_arrive(bar(B_IFULL + s));  // release: the item is visible to whoever sees the phase flip
-          ++it_pub;
-        }
-        if (last) break;
-        const int n_max = max(it.n_kv0, it.n_kv1);
-        for (int j = 0; j < n_max && ok; ++j) {
-          // K and V slots are released separately: K as soon as the Q K^T products that use it have run, V only
-          // after the P V products, so later K tiles are on their way while the softmax runs
-          const int sk_i = g_k % K_SLOTS;
-          if (!ptx::mbar_wait_bounded(bar(B_KEMPTY + sk_i), ((g_k / K_SLOTS) & 1) ^ 1u, abort_flag, limit)) { ok = false; break; }
-          if (!(p.test_skip_load && g_k == 1)) {
-            const uint32_t sk = smem_base + Cfg::K_OFF + sk_i * Cfg::TILE_BYTES;
-            ptx::mbar_arrive_expect_tx(bar(B_KFULL + sk_i), Cfg::TILE_BYTES);
-            for (int c = 0; c < Cfg::SUB; ++c)
-              ptx::tma_load_2d(sk + c * Cfg::SUB_BYTES, &tmap_k, c * 64, it.kv_row0 + j * TK, bar(B_KFULL + sk_i));
-          }
-          ++g_k;
-          const int sv_i = g_v % V_SLOTS;
-          if (!ptx::mbar_wait_bounded(bar(B_VEMPTY + sv_i), ((g_v / V_SLOTS) & 1) ^ 1u, abort_flag, limit)) { ok = false; break; }
-          const uint32_t sv = smem_base + Cfg::V_OFF + sv_i * Cfg::TILE_BYTES;
-          ptx::mbar_arrive_expect_tx(bar(B_VFULL + sv_i), Cfg::TILE_BYTES);
-          for (int c = 0; c < Cfg::SUB; ++c)
-            ptx::tma_load_2d(sv + c * Cfg::SUB_BYTES, &tmap_v, c * 64, it.kv_row0 + j * TK, bar(B_VFULL + sv_i));
-          ++g_v;
-          if (j == 0) fetch(nxt);  // (after this item's first loads are on their way)
-        }
-      }
-      if (!ok) {
-        // give loads already in flight time to land before the block's shared memory is released
-        for (int i = 0; i < 2000; ++i) __nanosleep(1000);
-      }
-    }
+    if (lane == 0) kv_producer<HD>(&tmap_k, &tmap_v, p, smem_base, bar0, item_ring, abort_flag, limit);
   } else if (warp == 1) {
     // -------------------------------------------------------------- MMA issuer
-    if (lane == 0) {
-      constexpr uint32_t idesc_qk = ptx::umma_idesc_bf16(TQ, TK);
-      constexpr uint32_t idesc_pv = ptx::umma_idesc_bf16_bmn(TQ, HD);
-      // Per row tile: the item it is working on and how far it has got.  The two tiles walk the same item
-      // sequence and share the K / V rings, but each advances as soon as its own inputs are ready.
-      Item cur[2];
-      bool have[2] = {false, false}, done[2] = {false, false};
-      int seq[2] = {0, 0};      // items taken from the ring so far
-      int base[2] = {0, 0};     // ring position of the current item's first K / V tile
-      int n[2] = {0, 0};        // K / V tiles of the current item for this row tile
-      int jq[2] = {0, 0};       // next Q K^T to issue
-      int jp[2] = {0, 0};       // next P V to issue
-      int act[2] = {0, 0};      // items with work for this row tile finished so far
-      int pv_cnt[2] = {0, 0};   // P V products issued so far (phase of p_ready)
-      uint32_t k_used = 0, v_used = 0;  // users that have consumed the tile in each ring slot, 4 bits per slot
-      uint64_t t_idle = 0;
-      uint32_t idle_polls = 0;
-      bool ok = true;
-      while (ok && !(done[0] && done[1])) {
-        bool progress = false;
-#pragma unroll
-        for (int t = 0; t < 2; ++t) {
-          if (done[t]) continue;
-          if (!have[t]) {
-            const int s = seq[t] & (ITEM_SLOTS - 1);
-            if (!ptx::mbar_test_wait(bar(B_IFULL + s), (seq[t] / ITEM_SLOTS) & 1)) continue;
-            cur[t] = item_ring[s];
-            ptx::mbar_arrive(bar(B_IEMPTY + s));
-            ++seq[t];
-            progress = true;
-            if (cur[t].n_kv0 < 0) { done[t] = true; continue; }
-            n[t] = t == 0 ? cur[t].n_kv0 : cur[t].n_kv1;
-            if (n[t] == 0) {  // this item has rows for the other tile only
-              base[t] += max(cur[t].n_kv0, cur[t].n_kv1);
-              continue;
-            }
-            have[t] = true; jq[t] = 0; jp[t] = 0;
-          }
-          const Item& it = cur[t];
-          if (jp[t] < jq[t]) {
-            // ---- O_t += P_t V_j
-            const int j = jp[t], g = base[t] + j, s = g % V_SLOTS;
-            if (!ptx::mbar_test_wait(bar(B_PREADY + t), pv_cnt[t] & 1)) continue;
-            if (!ptx::mbar_test_wait(bar(B_VFULL + s), (g / V_SLOTS) & 1)) continue;
-            // the first product of an item overwrites O: the previous item's output must have been read out
-            if (j == 0 && act[t] > 0 && !ptx::mbar_test_wait(bar(B_OREAD + t), (act[t] - 1) & 1)) continue;
-            ptx::tc_fence_after();
-            const uint32_t sv = smem_base + Cfg::V_OFF + s * Cfg::TILE_BYTES;
-            const uint32_t d = tmem_base + t * Cfg::TILE_COLS + Cfg::O_COL;
-            const uint32_t a = tmem_base + t * Cfg::TILE_COLS + Cfg::S_COL;
-#pragma unroll
-            for (int kk = 0; kk < TK / 16; ++kk) {
-              // 16 keys = 16 rows of 128 bytes further into the V tile; 8 packed columns further into P
-              ptx::umma_bf16_ts(d, a + kk * 8, ptx::umma_desc_mn_sw128(sv + kk * 2048, Cfg::SUB_BYTES), idesc_pv,
-                                (j > 0 || kk > 0) ? 1u : 0u);
-            }
-            ptx::umma_commit(bar(B_ODONE + t));
-            const uint32_t users = (j < it.n_kv0 ? 1u : 0u) + (j < it.n_kv1 ? 1u : 0u);
-            v_used += 1u << (4 * s);
-            if (((v_used >> (4 * s)) & 15u) == users) { ptx::umma_commit(bar(B_VEMPTY + s)); v_used &= ~(15u << (4 * s)); }
-            ++pv_cnt[t]; ++jp[t];
-            progress = true;
-            if (jp[t] == n[t]) {  // item finished for this tile
-              have[t] = false;
-              ++act[t];
-              base[t] += max(it.n_kv0, it.n_kv1);
-              continue;
-            }
-          }
-          if (jq[t] < n[t] && jq[t] == jp[t]) {
-            // ---- S_t = Q_t K_j^T (S is free: the P that aliased it has been consumed by the product above)
-            const int j = jq[t], g = base[t] + j, s = g % K_SLOTS;
-            if (j == 0 && !ptx::mbar_test_wait(bar(B_QFULL + t), act[t] & 1)) continue;
-            if (!ptx::mbar_test_wait(bar(B_KFULL + s), (g / K_SLOTS) & 1)) continue;
-            ptx::tc_fence_after();
-            const uint32_t sq = smem_base + Cfg::Q_OFF + t * Cfg::TILE_BYTES;
-            const uint32_t sk = smem_base + Cfg::K_OFF + s * Cfg::TILE_BYTES;
-            const uint32_t d = tmem_base + t * Cfg::TILE_COLS + Cfg::S_COL;
-#pragma unroll
-            for (int kk = 0; kk < HD / 16; ++kk) {
-              const uint32_t off = (kk >> 2) * Cfg::SUB_BYTES + (kk & 3) * 32;
-              ptx::umma_bf16(d, ptx::umma_desc_sw128(sq + off), ptx::umma_desc_sw128(sk + off), idesc_qk, kk > 0 ? 1u : 0u);
-            }
-            ptx::umma_commit(bar(B_SFULL + t));
-            const uint32_t users = (j < it.n_kv0 ? 1u : 0u) + (j < it.n_kv1 ? 1u : 0u);
-            k_used += 1u << (4 * s);
-            if (((k_used >> (4 * s)) & 15u) == users) { ptx::umma_commit(bar(B_KEMPTY + s)); k_used &= ~(15u << (4 * s)); }
-            ++jq[t];
-            if (jq[t] == n[t]) ptx::umma_commit(bar(B_QEMPTY + t));  // the tile's Q buffer may be refilled
-            progress = true;
-          }
-        }
-        if (progress) {
-          idle_polls = 0;
-          t_idle = 0;
-        } else if ((++idle_polls & 1023u) == 0u) {
-          // nothing could be issued for a while: look at the abort flag and the clock
-          if (*abort_flag) { ok = false; break; }
-          const uint64_t now = ptx::globaltimer_ns();
-          if (t_idle == 0) t_idle = now;
-          else if (now - t_idle > limit) { *abort_flag = 1; ok = false; }
-        }
-      }
-    }
+    if (lane == 0) mma_issuer<HD>(smem_base, tmem_base, bar0, item_ring, abort_flag, limit);
   } else if (warp == 10) {
     // ---------------------------------------------------------------- Q loader
-    // Its own thread, so that a wait for one tile's Q buffer never holds up the K / V stream of the other tile.
-    if (lane == 0) {
-      int seq = 0;
-      int q_cnt[2] = {0, 0};  // Q loads so far per row tile
-      bool ok = true;
-      while (ok) {
-        const int s = seq & (ITEM_SLOTS - 1);
-        if (!ptx::mbar_wait_bounded(bar(B_IFULL + s), (seq / ITEM_SLOTS) & 1, abort_flag, limit)) break;
-        const Item it = item_ring[s];
-        ptx::mbar_arrive(bar(B_IEMPTY + s));
-        ++seq;
-        if (it.n_kv0 < 0) break;
-        for (int t = 0; t < 2; ++t) {
-          if (t == 1 && it.n_kv1 == 0) break;
-          // the tile's Q buffer is free once the last Q K^T of its previous item has been executed
-          if (!ptx::mbar_wait_bounded(bar(B_QEMPTY + t), (q_cnt[t] & 1) ^ 1u, abort_flag, limit)) { ok = false; break; }
-          ptx::mbar_arrive_expect_tx(bar(B_QFULL + t), Cfg::TILE_BYTES);
-          for (int c = 0; c < Cfg::SUB; ++c)
-            ptx::tma_load_2d(smem_base + Cfg::Q_OFF + t * Cfg::TILE_BYTES + c * Cfg::SUB_BYTES, &tmap_q, it.h * HD + c * 64,
-                             it.start + it.q0 + t * TQ, bar(B_QFULL + t));
-          ++q_cnt[t];
-        }
-      }
-      if (!ok) {
-        for (int i = 0; i < 2000; ++i) __nanosleep(1000);
-      }
-    }
+    if (lane == 0) q_loader<HD>(&tmap_q, smem_base, bar0, item_ring, abort_flag, limit);
   } else {
     // ---------------------------------------------------------------- softmax
     const int t = (warp - 2) >> 2;       // row tile of this warpgroup
@@ -368,6 +400,7 @@ prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_
       const int kv_total = it.pre + it.len;          // keys this request has after the chunk
       const int kv_end = it.pre + min(it.len, it.q0 + t * TQ + TQ);
       float m_used = -CUDART_INF_F, l_sum = 0.f;
+#pragma unroll 1
       for (int j = 0; j < n_kv; ++j, ++step) {
         ok = __all_sync(0xffffffffu, ptx::mbar_wait_bounded(bar(B_SFULL + t), step & 1, abort_flag, limit));
         if (!ok) break;

@@ -469,6 +469,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       }
       if (!ok) {
         // give loads already in flight time to land before the block's shared memory is released
+#pragma unroll 1
         for (int i = 0; i < 2000; ++i) __nanosleep(1000);
       }
     }
@@ -669,6 +670,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
         }
       }
       if (!ok) {
+#pragma unroll 1
         for (int i = 0; i < 2000; ++i) __nanosleep(1000);
       }
     }

@@ -239,6 +239,7 @@ gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
         if (++stage == STAGES) { stage = 0; phase ^= 1u; }
       }
       if (!ok) {
+#pragma unroll 1
         for (int i = 0; i < 2000; ++i) __nanosleep(1000);  // let loads in flight land before shared memory is released
       }
     }
@@ -406,6 +407,7 @@ gemm_skinny_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid
         if (++stage == STAGES) { stage = 0; phase ^= 1u; }
       }
       if (!ok) {
+#pragma unroll 1
         for (int i = 0; i < 2000; ++i) __nanosleep(1000);  // let loads in flight land before shared memory is released
       }
     }
