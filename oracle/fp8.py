@@ -20,9 +20,16 @@ Scale and quotient are evaluated in IEEE float32 (one division each, round to ne
 so that the integer codes are decided in the same precision as on the GPU; an all-zero
 row gets scale 1.  Rounding to E4M3 is round-to-nearest-even with saturation to +-448.
 
+A second scaling scheme, one scale per 128 x 128 weight block and per token and 128 channels
+(quantize_groups, quantize_blocks, gemm_fp8_blockwise), is described where it is defined.
+
 Pins: tests/test_oracle_fp8.py (format constants of the published table, exhaustive
 decode/encode round trip, ties and saturation, brute-force nearest-value search, an
-independent library conversion, error bounds, exactly representable GEMM).
+independent library conversion, error bounds, exactly representable GEMM; for the
+block-wise scheme: reduction to the per-row scheme when K is one block and every output
+row its own block, element-by-element loops on small cases, exactness for operands that
+are representable block by block, scale invariance under per-block powers of two, and
+the error bound of the scheme against the unquantised product).
 """
 from __future__ import annotations
 
@@ -96,6 +103,66 @@ def gemm_fp8(qx, sx, qw, sw) -> np.ndarray:
     """Y[T, N] = (dec(qx) @ dec(qw)^T) * sx[:, None] * sw[None, :] in float64."""
     acc = e4m3_decode(qx) @ e4m3_decode(qw).T
     return acc * np.asarray(sx, np.float64)[:, None] * np.asarray(sw, np.float64)[None, :]
+
+
+# ----------------------------------------------------------------------------- block-wise scales
+# Reading for checkpoints that carry one scale per block instead of per channel (the public FP8 releases of
+# the model families the paper deploys state `weight_block_size = [128, 128]`): a weight matrix W[N, K] has one
+# fp32 scale per 128 x 128 block, an activation matrix X[T, K] one per token and group of 128 consecutive
+# channels, and the products of the codes are summed per 128-wide K block and scaled block by block:
+#   Y[t, n] = sum_kb ( sum_{k in kb} dec(qx[t, k]) dec(qw[n, k]) ) * sx[t, kb] * sw[n // 128, kb].
+# Scales and quotients are evaluated in float32 like the per-row ones; an all-zero block gets scale 1; N and K
+# need not be multiples of 128 (edge blocks are smaller).
+BLOCK = 128
+
+
+def quantize_groups(x, group: int = BLOCK):
+    """Per-row, per-K-group dynamic quantisation of x[T, K] -> (codes uint8 [T, K], scale float32 [T, ceil(K / group)])."""
+    x32 = np.ascontiguousarray(x, dtype=np.float32)
+    t, k = x32.shape
+    kb = (k + group - 1) // group
+    codes = np.zeros((t, k), dtype=np.uint8)
+    scale = np.ones((t, kb), dtype=np.float32)
+    for b in range(kb):
+        blk = x32[:, b * group:(b + 1) * group]
+        amax = np.max(np.abs(blk), axis=1)
+        sc = (amax / np.float32(E4M3_MAX)).astype(np.float32)
+        sc = np.where(amax > 0, sc, np.float32(1.0)).astype(np.float32)
+        codes[:, b * group:(b + 1) * group] = e4m3_encode((blk / sc[:, None]).astype(np.float32))
+        scale[:, b] = sc
+    return codes, scale
+
+
+def quantize_blocks(w, block_n: int = BLOCK, block_k: int = BLOCK):
+    """Per-block quantisation of w[N, K] -> (codes uint8 [N, K], scale float32 [ceil(N / block_n), ceil(K / block_k)])."""
+    w32 = np.ascontiguousarray(w, dtype=np.float32)
+    n, k = w32.shape
+    nb, kb = (n + block_n - 1) // block_n, (k + block_k - 1) // block_k
+    codes = np.zeros((n, k), dtype=np.uint8)
+    scale = np.ones((nb, kb), dtype=np.float32)
+    for i in range(nb):
+        for j in range(kb):
+            blk = w32[i * block_n:(i + 1) * block_n, j * block_k:(j + 1) * block_k]
+            amax = np.float32(np.max(np.abs(blk))) if blk.size else np.float32(0)
+            sc = np.float32(amax / np.float32(E4M3_MAX)) if amax > 0 else np.float32(1.0)
+            codes[i * block_n:(i + 1) * block_n, j * block_k:(j + 1) * block_k] = e4m3_encode((blk / sc).astype(np.float32))
+            scale[i, j] = sc
+    return codes, scale
+
+
+def gemm_fp8_blockwise(qx, sx, qw, sw, block_n: int = BLOCK, block_k: int = BLOCK) -> np.ndarray:
+    """Y[T, N] with one partial product per K block, each scaled by the token's group scale and the weight block's scale."""
+    dx, dw = e4m3_decode(qx), e4m3_decode(qw)
+    t, k = dx.shape
+    n = dw.shape[0]
+    sx = np.asarray(sx, np.float64)
+    sw = np.asarray(sw, np.float64)
+    y = np.zeros((t, n), dtype=np.float64)
+    row_block = np.arange(n) // block_n
+    for j in range((k + block_k - 1) // block_k):
+        part = dx[:, j * block_k:(j + 1) * block_k] @ dw[:, j * block_k:(j + 1) * block_k].T
+        y += part * sx[:, j][:, None] * sw[row_block, j][None, :]
+    return y
 
 
 class Fp8Projector:

@@ -124,6 +124,103 @@ def test_gemm_error_against_unquantised_product():
     assert np.allclose(fp8.gemm_fp8(*fp8.quantize_rows(b), *fp8.quantize_rows(a)), y.T, rtol=0, atol=1e-12)
 
 
+# ------------------------------------------------------------------- block-wise scales
+def test_blockwise_reduces_to_per_row_scheme():
+    """One K block and one output row per weight block: the block-wise scheme IS the per-row scheme."""
+    a = gen.normal_bf16(3, gen.S_X, (7, 96), 1.0).astype(np.float64)
+    b = gen.normal_bf16(3, gen.S_WQKV, (5, 96), 0.02).astype(np.float64)
+    qa, sa = fp8.quantize_groups(a, group=96)
+    qb, sb = fp8.quantize_blocks(b, block_n=1, block_k=96)
+    qa_r, sa_r = fp8.quantize_rows(a)
+    qb_r, sb_r = fp8.quantize_rows(b)
+    assert np.array_equal(qa, qa_r) and np.array_equal(sa[:, 0], sa_r)
+    assert np.array_equal(qb, qb_r) and np.array_equal(sb[:, 0], sb_r)
+    assert np.array_equal(fp8.gemm_fp8_blockwise(qa, sa, qb, sb, block_n=1, block_k=96), fp8.gemm_fp8(qa_r, sa_r, qb_r, sb_r))
+
+
+def test_blockwise_quantisers_by_element_loops():
+    """Scales and codes against loops over single elements (ragged edge blocks included)."""
+    rng = np.random.Generator(np.random.Philox(key=21))
+    x = (rng.standard_normal((5, 21)) * np.exp2(rng.integers(-4, 5, size=(5, 21)))).astype(np.float32)
+    x[2, 8:16] = 0.0                                               # an all-zero group
+    w = (rng.standard_normal((11, 21)) * 0.05).astype(np.float32)
+    qx, sx = fp8.quantize_groups(x, group=8)
+    qw, sw = fp8.quantize_blocks(w, block_n=4, block_k=8)
+    assert sx.shape == (5, 3) and sw.shape == (3, 3) and sx.dtype == np.float32 and sw.dtype == np.float32
+    for t in range(5):
+        for g in range(3):
+            seg = x[t, g * 8:(g + 1) * 8]
+            amax = np.float32(np.abs(seg).max())
+            want = np.float32(amax / np.float32(448.0)) if amax > 0 else np.float32(1.0)
+            assert sx[t, g] == want
+            for i, v in enumerate(seg):
+                assert qx[t, g * 8 + i] == fp8.e4m3_encode(np.float32(v / want))
+    for i in range(3):
+        for j in range(3):
+            blk = w[i * 4:(i + 1) * 4, j * 8:(j + 1) * 8]
+            amax = np.float32(np.abs(blk).max())
+            assert sw[i, j] == np.float32(amax / np.float32(448.0))
+            assert np.array_equal(qw[i * 4:(i + 1) * 4, j * 8:(j + 1) * 8], fp8.e4m3_encode((blk / sw[i, j]).astype(np.float32)))
+    assert sx[2, 1] == 1.0 and np.all(qx[2, 8:16] == 0)
+
+
+def test_blockwise_gemm_by_element_loops():
+    rng = np.random.Generator(np.random.Philox(key=22))
+    x = rng.standard_normal((4, 20)).astype(np.float32)
+    w = rng.standard_normal((7, 20)).astype(np.float32)
+    qx, sx = fp8.quantize_groups(x, group=8)
+    qw, sw = fp8.quantize_blocks(w, block_n=3, block_k=8)
+    dx, dw = fp8.e4m3_decode(qx), fp8.e4m3_decode(qw)
+    want = np.zeros((4, 7))
+    for t in range(4):
+        for n in range(7):
+            for k in range(20):
+                want[t, n] += dx[t, k] * dw[n, k] * float(sx[t, k // 8]) * float(sw[n // 3, k // 8])
+    got = fp8.gemm_fp8_blockwise(qx, sx, qw, sw, block_n=3, block_k=8)
+    assert np.allclose(got, want, rtol=1e-13, atol=1e-13)
+
+
+def test_blockwise_exact_for_blockwise_representable_operands():
+    """Small integers times one power of two per block: codes, scales and the product are exact."""
+    rng = np.random.Generator(np.random.Philox(key=23))
+    a = rng.integers(-7, 8, size=(6, 256)).astype(np.float64)
+    b = rng.integers(-7, 8, size=(256, 256)).astype(np.float64)
+    a[:, 0::128] = 7.0                                             # every 1 x 128 group has amax 7
+    b[0::128, 0::128] = -7.0                                       # every 128 x 128 block has amax 7
+    a = a.reshape(6, 2, 128) * np.exp2(rng.integers(-3, 4, size=(6, 2, 1)).astype(np.float64))
+    a = a.reshape(6, 256)
+    pw = np.exp2(rng.integers(-3, 4, size=(2, 2)).astype(np.float64))
+    b = b * np.kron(pw, np.ones((128, 128)))
+    qa, sa = fp8.quantize_groups(a)
+    qb, sb = fp8.quantize_blocks(b)
+    assert np.array_equal(fp8.e4m3_decode(qa) * np.repeat(sa.astype(np.float64), 128, axis=1), a)
+    assert np.array_equal(fp8.e4m3_decode(qb) * np.kron(sb.astype(np.float64), np.ones((128, 128))), b)
+    assert np.array_equal(fp8.gemm_fp8_blockwise(qa, sa, qb, sb), a @ b.T)
+
+
+def test_blockwise_scale_invariance_and_error_bound():
+    a = gen.normal_bf16(4, gen.S_X, (48, 512), 1.0).astype(np.float64)
+    b = gen.normal_bf16(4, gen.S_WQKV, (256, 512), 0.02).astype(np.float64)
+    qa, sa = fp8.quantize_groups(a)
+    qb, sb = fp8.quantize_blocks(b)
+    y = fp8.gemm_fp8_blockwise(qa, sa, qb, sb)
+    ref = a @ b.T
+    rel = np.linalg.norm(y - ref) / np.linalg.norm(ref)
+    assert 0.01 < rel < 0.06                                       # same error class as the per-row scheme
+    # multiplying one weight block and one activation group by powers of two changes only their scales
+    b2 = b.copy(); b2[128:256, 256:384] *= 8.0
+    a2 = a.copy(); a2[:, 128:256] *= 0.25
+    qb2, sb2 = fp8.quantize_blocks(b2)
+    qa2, sa2 = fp8.quantize_groups(a2)
+    assert np.array_equal(qb2, qb) and np.array_equal(qa2, qa)
+    assert sb2[1, 2] == sb[1, 2] * 8 and np.array_equal(sa2[:, 1], sa[:, 1] * np.float32(0.25))
+    # an outlier confined to one block leaves the codes of every other block untouched (what block scales are for)
+    b3 = b.copy(); b3[5, 7] = 3.0
+    qb3, sb3 = fp8.quantize_blocks(b3)
+    keep = np.ones_like(b, dtype=bool); keep[0:128, 0:128] = False
+    assert np.array_equal(qb3[keep], qb[keep]) and sb3[0, 0] > sb[0, 0] and np.array_equal(sb3.ravel()[1:], sb.ravel()[1:])
+
+
 CFG = L.LayerConfig(d_model=64, n_q_heads=4, n_kv_heads=2, head_dim=16, d_ff=96)
 
 
