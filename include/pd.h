@@ -344,6 +344,31 @@ pd_status pd_quantize_fp8_rows(const void* x, int32_t ldx, int32_t rows, int32_t
 pd_status pd_gemm_fp8(const void* a_codes, const float* a_scales, const void* b_codes, const float* b_scales,
                       void* c, int32_t m, int32_t n, int32_t k, int32_t* err_word, void* stream);
 
+/* FP8 (E4M3) with block-wise scales, the scaling scheme of checkpoints that state `weight_block_size = [128, 128]`
+ * (reading of the paper's FP8 deployment, Evaluation section: the TTFT experiment on an FP8 checkpoint; the paper does
+ * not say how that checkpoint is scaled):
+ *   a weight matrix W[n, k] carries one fp32 scale per 128 x 128 block, an activation matrix X[rows, k] one per row and
+ *   group of 128 consecutive k; scale = max|block| / 448 (1 for an all-zero block), code = E4M3(value / scale), both in
+ *   fp32, round to nearest even, saturating;
+ *   C[i, j] = sum over K blocks kb of ( sum_{k in kb} dec(A[i, k]) dec(B[j, k]) ) * a_scales[i, kb] * b_scales[j / 128, kb],
+ *   the inner sums exact in fp32 on the tensor cores (tcgen05 kind::f8f6f4), the scaled partial sums added in fp32.
+ *
+ * pd_quantize_fp8_groups: x device bf16 [rows, k], row pitch ldx elements (a multiple of 4) -> codes device uint8
+ * [rows, k] contiguous, scales device fp32 [rows, k / 128] contiguous.  k a multiple of 128.
+ * pd_quantize_fp8_blocks: w device bf16 [n, k], row pitch ldw elements (a multiple of 8) -> codes device uint8 [n, k]
+ * contiguous, scales device fp32 [ceil(n / 128), k / 128] contiguous (the last row of blocks may have fewer than 128
+ * rows).  k a multiple of 128.
+ * pd_gemm_fp8_blockwise: C[m, n] device bf16 contiguous from codes and scales laid out as above; code pointers 16-byte
+ * aligned, k a multiple of 128, n of 16.  `err_word` as in pd_gemm_bf16.  The caller owns every buffer; the three calls
+ * only enqueue work on `stream`; a shape outside these rules returns PD_ERR_UNSUPPORTED_SHAPE, a NULL pointer or a
+ * negative size PD_ERR_INVALID_ARG, and zero rows return PD_OK without a launch. */
+pd_status pd_quantize_fp8_groups(const void* x, int32_t ldx, int32_t rows, int32_t k, void* codes, float* scales,
+                                 void* stream);
+pd_status pd_quantize_fp8_blocks(const void* w, int32_t ldw, int32_t n, int32_t k, void* codes, float* scales,
+                                 void* stream);
+pd_status pd_gemm_fp8_blockwise(const void* a_codes, const float* a_scales, const void* b_codes, const float* b_scales,
+                                void* c, int32_t m, int32_t n, int32_t k, int32_t* err_word, void* stream);
+
 /* Failure-detection test hook.  Every wait inside the tensor-core kernels (on a tile load, an accumulator, a
  * partner block) is bounded by wall clock (4 s); when a wait gives up, the block raises its abort flag, leaves
  * through the normal teardown (tensor memory freed, cluster barrier of a CTA pair passed) and sets the error

@@ -41,6 +41,7 @@ EXPORTS = [
     "pd_prefill_attention", "pd_mixture_throughput", "pd_interp_service_times", "pd_mm1_sojourn", "pd_mg1_sojourn",
     "pd_refine_next_batch", "pd_prefill_chunk_stack", "pd_test_inject_wait_timeout",
     "pd_gemm_workspace_bytes", "pd_gemm_bf16_ws",
+    "pd_quantize_fp8_groups", "pd_quantize_fp8_blocks", "pd_gemm_fp8_blockwise",
 ]
 
 TRACE_CLASSES = ["gemm_qkv", "gemm_o", "gemm_gate_up", "gemm_down", "attn_prefill", "attn_decode", "rmsnorm",
@@ -153,6 +154,9 @@ _lib.pd_gemm_bf16_ws.argtypes = [_P, _P, _P, C.c_int32, C.c_int32, C.c_int32, _P
 _lib.pd_workspace_offsets.argtypes = [C.POINTER(pd_layer_cfg), C.c_int32, C.POINTER(pd_workspace_layout)]
 _lib.pd_quantize_fp8_rows.argtypes = [_P, C.c_int32, C.c_int32, C.c_int32, _P, _P, _P]
 _lib.pd_gemm_fp8.argtypes = [_P, _P, _P, _P, _P, C.c_int32, C.c_int32, C.c_int32, _P, _P]
+_lib.pd_quantize_fp8_groups.argtypes = [_P, C.c_int32, C.c_int32, C.c_int32, _P, _P, _P]
+_lib.pd_quantize_fp8_blocks.argtypes = [_P, C.c_int32, C.c_int32, C.c_int32, _P, _P, _P]
+_lib.pd_gemm_fp8_blockwise.argtypes = [_P, _P, _P, _P, _P, C.c_int32, C.c_int32, C.c_int32, _P, _P]
 _lib.pd_measure.argtypes = [C.POINTER(pd_layer_cfg), C.POINTER(pd_measure_cfg), C.c_double, C.c_double,
                             C.POINTER(pd_measurement)]
 _lib.pd_allocate.argtypes = [C.POINTER(pd_alloc_in), C.POINTER(pd_alloc_out)]
@@ -487,6 +491,23 @@ def pd_quantize_fp8_rows(x, rows: int, k: int, codes, scales, ldx: int = 0, stre
 def pd_gemm_fp8(a_codes, a_scales, b_codes, b_scales, c, m: int, n: int, k: int, err_word=None, stream=None):
     _check(_lib.pd_gemm_fp8(_ptr(a_codes), _ptr(a_scales), _ptr(b_codes), _ptr(b_scales), _ptr(c), m, n, k,
                             _ptr(err_word), _stream_ptr(stream)), "pd_gemm_fp8")
+
+
+def pd_quantize_fp8_groups(x, rows: int, k: int, codes, scales, ldx: int = 0, stream=None):
+    """x: device bf16 [rows, k] -> codes uint8 [rows, k], scales fp32 [rows, k / 128] (one per row and 128 channels)."""
+    _check(_lib.pd_quantize_fp8_groups(_ptr(x), ldx or k, rows, k, _ptr(codes), _ptr(scales), _stream_ptr(stream)),
+           "pd_quantize_fp8_groups")
+
+
+def pd_quantize_fp8_blocks(w, n: int, k: int, codes, scales, ldw: int = 0, stream=None):
+    """w: device bf16 [n, k] -> codes uint8 [n, k], scales fp32 [ceil(n / 128), k / 128] (one per 128 x 128 block)."""
+    _check(_lib.pd_quantize_fp8_blocks(_ptr(w), ldw or k, n, k, _ptr(codes), _ptr(scales), _stream_ptr(stream)),
+           "pd_quantize_fp8_blocks")
+
+
+def pd_gemm_fp8_blockwise(a_codes, a_scales, b_codes, b_scales, c, m: int, n: int, k: int, err_word=None, stream=None):
+    _check(_lib.pd_gemm_fp8_blockwise(_ptr(a_codes), _ptr(a_scales), _ptr(b_codes), _ptr(b_scales), _ptr(c), m, n, k,
+                                      _ptr(err_word), _stream_ptr(stream)), "pd_gemm_fp8_blockwise")
 
 
 def pd_measure(cfg: LayerConfig, *, n_layers_run: int, n_layers_model: int, warmup: int = 3, reps: int = 10,
