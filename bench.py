@@ -522,6 +522,38 @@ def main():
                    "kernel_time_ms_prefill": {k: v[0] * 1e3 for k, v in tr8.items() if v[1]},
                    "note": "E4M3 weights per output channel, activations per token; attention, norms, residual stream "
                            "and KV cache stay bf16; not part of `value`"}
+        # block-wise scales (one per 128 x 128 weight block and per token and 128 channels): the stand-alone GEMM on
+        # the down-projection shape of this workload, timed launch by launch (L2 flushed by the previous launches'
+        # operands: three weight matrices of 59 MB of codes take turns)
+        bw_m, bw_n, bw_k = L_IN, SHAPE["d_model"], SHAPE["d_ff"]
+        bw_a = torch.randn(bw_m, bw_k, device=dev).to(torch.bfloat16)
+        bw_qa = torch.empty((bw_m, bw_k), dtype=torch.uint8, device=dev)
+        bw_sa = torch.empty((bw_m, bw_k // 128), dtype=torch.float32, device=dev)
+        bw_c = torch.empty((bw_m, bw_n), dtype=torch.bfloat16, device=dev)
+        bw_w = []
+        for _ in range(3):
+            w_ = (torch.randn(bw_n, bw_k, device=dev) * 0.02).to(torch.bfloat16)
+            q_ = torch.empty((bw_n, bw_k), dtype=torch.uint8, device=dev)
+            s_ = torch.empty(((bw_n + 127) // 128, bw_k // 128), dtype=torch.float32, device=dev)
+            pd.pd_quantize_fp8_blocks(w_, bw_n, bw_k, q_, s_)
+            bw_w.append((q_, s_))
+            del w_
+        pd.pd_quantize_fp8_groups(bw_a, bw_m, bw_k, bw_qa, bw_sa)
+        bw_i = [0]
+
+        def bw_step():
+            q_, s_ = bw_w[bw_i[0] % 3]
+            bw_i[0] += 1
+            pd.pd_gemm_fp8_blockwise(bw_qa, bw_sa, q_, s_, bw_c, bw_m, bw_n, bw_k)
+        bw_s = timed(bw_step, reps=9)
+        bwq_s = timed(lambda: pd.pd_quantize_fp8_groups(bw_a, bw_m, bw_k, bw_qa, bw_sa), reps=5)
+        fp8_out["blockwise_gemm"] = {"shape_mnk": [bw_m, bw_n, bw_k], "ms": bw_s * 1e3,
+                                     "tflops": 2.0 * bw_m * bw_n * bw_k / bw_s / 1e12,
+                                     "frac_of_fp8_peak": 2.0 * bw_m * bw_n * bw_k / bw_s / 1e12 / peak8,
+                                     "activation_quantiser_ms": bwq_s * 1e3,
+                                     "note": "pd_gemm_fp8_blockwise: 128 x 128 tiles on single CTAs, scaled accumulation in "
+                                             "registers per K block; not used by the layer passes above"}
+        del bw_w, bw_a, bw_qa, bw_sa, bw_c
         del layers8, ws8
 
     cpu = None

@@ -6,10 +6,11 @@
 //   * C[m, n] = sum over K blocks kb of ( sum_{k in kb} dec(qx[m, k]) dec(qw[n, k]) ) * sx[m, kb] * sw[n / 128, kb].
 // The tensor cores sum the codes' products of ONE K block (128 elements = one shared-memory stage = four
 // tcgen05.mma kind::f8f6f4 instructions of K = 32) into a tensor-memory accumulator that starts from zero; four
-// warps then read that accumulator, multiply it by the two scales and add it to fp32 sums they keep in registers
-// (one output row per thread, 128 columns), while the products of the next K block run into the second accumulator.
-// Tile 128 x 128, one tile per block.
-//   warp 0: TMA producer (one lane), warp 1: MMA issuer (one lane), warps 2-5: scaled accumulation and the store.
+// eight warps then read that accumulator, multiply it by the two scales and add it to fp32 sums they keep in registers
+// (half an output row per thread: 64 columns, as packed f32x2 FMAs), while the products of the next K block run into
+// the second accumulator.  Tile 128 x 128, one tile per block.
+//   warp 0: TMA producer (one lane), warp 1: MMA issuer (one lane), warps 2-9: scaled accumulation and the store
+//   (warps 2-5 columns 0-63, warps 6-9 columns 64-127 of the tensor-memory lanes their number allows them to read).
 // Every wait is wall-clock bounded and leaves through the common teardown.
 #include "pd_common.cuh"
 #include "pd_ptx.cuh"
@@ -18,7 +19,7 @@ namespace pd {
 namespace {
 
 constexpr int FB_TILE = 128;       // rows and columns of an output tile, and K elements per block (128 bytes per row)
-constexpr int FB_THREADS = 192;
+constexpr int FB_THREADS = 320;
 constexpr int FB_STAGES = 6;
 constexpr int FB_OPERAND_BYTES = FB_TILE * 128;          // 128 rows of 128 one-byte codes
 constexpr int FB_STAGE_BYTES = 2 * FB_OPERAND_BYTES;     // A rows + B rows
@@ -59,7 +60,7 @@ gemm_f8_block_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
     }
     for (int a = 0; a < 2; ++a) {
       ptx::mbar_init(accf_bar(a), 1);
-      ptx::mbar_init(acce_bar(a), 4);  // the four accumulating warps
+      ptx::mbar_init(acce_bar(a), 8);  // the eight accumulating warps
     }
     ptx::fence_barrier_init();
     ptx::prefetch_tensormap(&tmap_a);
@@ -124,51 +125,58 @@ gemm_f8_block_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
       }
     }
   } else {
-    // ------------------------------------------------------------ scaled accumulation, one output row per thread
-    const int lane_group = warp & 3;  // the tensor-memory lanes this warp may touch
+    // ------------------------------------------------------------ scaled accumulation, half an output row per thread
+    const int lane_group = warp & 3;         // the tensor-memory lanes this warp may touch
+    const int half = (warp - 2) >> 2;        // columns 64 * half .. + 63 of the tile
     const int row = tm * FB_TILE + lane_group * 32 + lane;
-    const uint32_t t_row = tmem_base + (static_cast<uint32_t>(lane_group * 32) << 16);
+    const uint32_t t_row = tmem_base + (static_cast<uint32_t>(lane_group * 32) << 16) + static_cast<uint32_t>(half * 64);
     const bool row_ok = row < p.m;
     const float* sa_row = p.scale_a + static_cast<size_t>(row_ok ? row : 0) * k_blocks;
     const float* sb_row = p.scale_b + static_cast<size_t>(tn) * k_blocks;
-    float sum[FB_TILE];
+    uint64_t sum[32];  // 64 fp32 sums, two to a register pair
 #pragma unroll
-    for (int c = 0; c < FB_TILE; ++c) sum[c] = 0.f;
+    for (int c = 0; c < 32; ++c) sum[c] = 0ull;
     ptx::grid_dependency_wait();
     bool ok = true;
     float s_next = k_blocks > 0 ? sa_row[0] * sb_row[0] : 0.f;
     for (int kb = 0; kb < k_blocks; ++kb) {
       const int acc = kb & 1;
-      const float s = s_next;
+      const uint64_t s2 = ptx::pack_f32x2(s_next, s_next);
       if (kb + 1 < k_blocks) s_next = sa_row[kb + 1] * sb_row[kb + 1];
       ok = __all_sync(0xffffffffu, ptx::mbar_wait_bounded(accf_bar(acc), (kb >> 1) & 1, abort_flag, limit));
       if (!ok) break;
       ptx::tc_fence_after();
+      uint32_t v[2][32];
+      ptx::tmem_ld_32x32(t_row + static_cast<uint32_t>(acc * FB_TILE), v[0]);
+      ptx::tmem_ld_32x32(t_row + static_cast<uint32_t>(acc * FB_TILE + 32), v[1]);
+      ptx::tmem_ld_wait();
+      // the accumulator is in registers: the products of K block kb + 2 may overwrite it
+      ptx::tc_fence_before();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(acce_bar(acc));
 #pragma unroll
-      for (int ch = 0; ch < FB_TILE / 32; ++ch) {
-        uint32_t v[32];
-        ptx::tmem_ld_32x32(t_row + static_cast<uint32_t>(acc * FB_TILE + ch * 32), v);
-        ptx::tmem_ld_wait();
-        if (ch == FB_TILE / 32 - 1) {  // the accumulator is in registers: the products of K block kb + 2 may overwrite it
-          ptx::tc_fence_before();
-          __syncwarp();
-          if (lane == 0) ptx::mbar_arrive(acce_bar(acc));
+      for (int ch = 0; ch < 2; ++ch) {
+#pragma unroll
+        for (int e = 0; e < 32; e += 2) {
+          const uint64_t x2 = ptx::pack_f32x2(__uint_as_float(v[ch][e]), __uint_as_float(v[ch][e + 1]));
+          sum[ch * 16 + (e >> 1)] = ptx::fma_f32x2(x2, s2, sum[ch * 16 + (e >> 1)]);
         }
-#pragma unroll
-        for (int e = 0; e < 32; ++e) sum[ch * 32 + e] = fmaf(__uint_as_float(v[e]), s, sum[ch * 32 + e]);
       }
     }
     if (ok && row_ok) {
-      bf16* dst = p.c + static_cast<size_t>(row) * p.ldc + tn * FB_TILE;
-      const int cols = min(FB_TILE, p.n - tn * FB_TILE);  // a multiple of 16
+      bf16* dst = p.c + static_cast<size_t>(row) * p.ldc + tn * FB_TILE + half * 64;
+      const int cols = min(FB_TILE, p.n - tn * FB_TILE) - half * 64;  // a multiple of 16, may be <= 0
 #pragma unroll
-      for (int c = 0; c < FB_TILE; c += 8) {
+      for (int c = 0; c < 64; c += 8) {
         if (c < cols) {
+          float f[8];
+#pragma unroll
+          for (int q = 0; q < 4; ++q) ptx::unpack_f32x2(sum[(c >> 1) + q], f[2 * q], f[2 * q + 1]);
           uint4 o;
-          o.x = ptx::pack_bf16(sum[c + 0], sum[c + 1]);
-          o.y = ptx::pack_bf16(sum[c + 2], sum[c + 3]);
-          o.z = ptx::pack_bf16(sum[c + 4], sum[c + 5]);
-          o.w = ptx::pack_bf16(sum[c + 6], sum[c + 7]);
+          o.x = ptx::pack_bf16(f[0], f[1]);
+          o.y = ptx::pack_bf16(f[2], f[3]);
+          o.z = ptx::pack_bf16(f[4], f[5]);
+          o.w = ptx::pack_bf16(f[6], f[7]);
           *reinterpret_cast<uint4*>(dst + c) = o;
         }
       }
