@@ -5,7 +5,7 @@
 //   * X[M, K]: one fp32 scale per row and group of 128 consecutive K elements, computed the same way;
 //   * C[m, n] = sum over K blocks kb of ( sum_{k in kb} dec(qx[m, k]) dec(qw[n, k]) ) * sx[m, kb] * sw[n / 128, kb].
 // The tensor cores sum the codes' products of ONE K block (128 elements = one shared-memory stage = four
-// tcgen05.mma kind::f8f6f4 instructions of K = 32) into a tensor-memory accumulator that starts from zero; four
+// tcgen05.mma kind::f8f6f4 instructions of K = 32) into a tensor-memory accumulator that starts from zero;
 // eight warps then read that accumulator, multiply it by the two scales and add it to fp32 sums they keep in registers
 // (half an output row per thread: 64 columns, as packed f32x2 FMAs), while the products of the next K block run into
 // the second accumulator.  Tile 128 x 128, one tile per block.
