@@ -8,7 +8,9 @@
 // tcgen05.mma kind::f8f6f4 instructions of K = 32) into a tensor-memory accumulator that starts from zero;
 // eight warps then read that accumulator, multiply it by the two scales and add it to fp32 sums they keep in registers
 // (half an output row per thread: 64 columns, as packed f32x2 FMAs), while the products of the next K block run into
-// the second accumulator.  Tile 128 x 128, one tile per block.
+// the second accumulator.  Tile 128 x 128; the grid is persistent (one block per SM walks the tiles row by row of
+// tiles, so that the blocks of a wave share their rows of A and the whole of B in L2), and barrier phases and the
+// accumulator turn run on one K-block counter that continues across tiles.
 //   warp 0: TMA producer (one lane), warp 1: MMA issuer (one lane), warps 2-9: scaled accumulation and the store
 //   (warps 2-5 columns 0-63, warps 6-9 columns 64-127 of the tensor-memory lanes their number allows them to read).
 // Every wait is wall-clock bounded and leaves through the common teardown.
@@ -30,7 +32,7 @@ struct F8BlockDev {
   bf16* c;
   const float* scale_a;  // [m, k_blocks]
   const float* scale_b;  // [ceil(n / 128), k_blocks]
-  int m, n, k_blocks, ldc, tiles_n;
+  int m, n, k_blocks, ldc, tiles_n, n_tiles;
   int* err_word;
   unsigned long long wait_limit_ns;
 };
@@ -75,7 +77,6 @@ gemm_f8_block_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  const int tm = blockIdx.x / p.tiles_n, tn = blockIdx.x % p.tiles_n;
   const int k_blocks = p.k_blocks;
 
   ptx::grid_launch_dependents();
@@ -86,13 +87,16 @@ gemm_f8_block_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
       uint32_t phase = 0;
       bool ok = true;
       ptx::grid_dependency_wait();
-      for (int kb = 0; kb < k_blocks; ++kb) {
-        if (!ptx::mbar_wait_bounded(empty_bar(stage), phase ^ 1u, abort_flag, limit)) { ok = false; break; }
-        const uint32_t sa = smem_base + stage * FB_STAGE_BYTES;
-        ptx::mbar_arrive_expect_tx(full_bar(stage), FB_STAGE_BYTES);
-        ptx::tma_load_2d(sa, &tmap_a, kb * FB_TILE, tm * FB_TILE, full_bar(stage));
-        ptx::tma_load_2d(sa + FB_OPERAND_BYTES, &tmap_b, kb * FB_TILE, tn * FB_TILE, full_bar(stage));
-        if (++stage == FB_STAGES) { stage = 0; phase ^= 1u; }
+      for (int tile = blockIdx.x; tile < p.n_tiles && ok; tile += gridDim.x) {
+        const int tm = tile / p.tiles_n, tn = tile % p.tiles_n;
+        for (int kb = 0; kb < k_blocks; ++kb) {
+          if (!ptx::mbar_wait_bounded(empty_bar(stage), phase ^ 1u, abort_flag, limit)) { ok = false; break; }
+          const uint32_t sa = smem_base + stage * FB_STAGE_BYTES;
+          ptx::mbar_arrive_expect_tx(full_bar(stage), FB_STAGE_BYTES);
+          ptx::tma_load_2d(sa, &tmap_a, kb * FB_TILE, tm * FB_TILE, full_bar(stage));
+          ptx::tma_load_2d(sa + FB_OPERAND_BYTES, &tmap_b, kb * FB_TILE, tn * FB_TILE, full_bar(stage));
+          if (++stage == FB_STAGES) { stage = 0; phase ^= 1u; }
+        }
       }
       if (!ok) {
         // give loads already in flight time to land before the block's shared memory is released
@@ -106,10 +110,12 @@ gemm_f8_block_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
       constexpr uint32_t idesc = ptx::umma_idesc_e4m3(FB_TILE, FB_TILE);
       int stage = 0;
       uint32_t phase = 0;
-      for (int kb = 0; kb < k_blocks; ++kb) {
-        const int acc = kb & 1;
-        // the accumulator's previous content (K block kb - 2) has been read out
-        if (!ptx::mbar_wait_bounded(acce_bar(acc), ((kb >> 1) & 1) ^ 1u, abort_flag, limit)) break;
+      const long long total = static_cast<long long>((p.n_tiles - static_cast<int>(blockIdx.x) + static_cast<int>(gridDim.x) - 1) /
+                                                     static_cast<int>(gridDim.x)) * k_blocks;  // K blocks of this block's tiles
+      for (long long it = 0; it < total; ++it) {
+        const int acc = static_cast<int>(it & 1);
+        // the accumulator's previous content (two K blocks ago) has been read out
+        if (!ptx::mbar_wait_bounded(acce_bar(acc), (static_cast<uint32_t>(it >> 1) & 1u) ^ 1u, abort_flag, limit)) break;
         if (!ptx::mbar_wait_bounded(full_bar(stage), phase, abort_flag, limit)) break;
         ptx::tc_fence_after();
         const uint32_t sa = smem_base + stage * FB_STAGE_BYTES;
@@ -128,56 +134,60 @@ gemm_f8_block_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
     // ------------------------------------------------------------ scaled accumulation, half an output row per thread
     const int lane_group = warp & 3;         // the tensor-memory lanes this warp may touch
     const int half = (warp - 2) >> 2;        // columns 64 * half .. + 63 of the tile
-    const int row = tm * FB_TILE + lane_group * 32 + lane;
     const uint32_t t_row = tmem_base + (static_cast<uint32_t>(lane_group * 32) << 16) + static_cast<uint32_t>(half * 64);
-    const bool row_ok = row < p.m;
-    const float* sa_row = p.scale_a + static_cast<size_t>(row_ok ? row : 0) * k_blocks;
-    const float* sb_row = p.scale_b + static_cast<size_t>(tn) * k_blocks;
-    uint64_t sum[32];  // 64 fp32 sums, two to a register pair
-#pragma unroll
-    for (int c = 0; c < 32; ++c) sum[c] = 0ull;
     ptx::grid_dependency_wait();
     bool ok = true;
-    float s_next = k_blocks > 0 ? sa_row[0] * sb_row[0] : 0.f;
-    for (int kb = 0; kb < k_blocks; ++kb) {
-      const int acc = kb & 1;
-      const uint64_t s2 = ptx::pack_f32x2(s_next, s_next);
-      if (kb + 1 < k_blocks) s_next = sa_row[kb + 1] * sb_row[kb + 1];
-      ok = __all_sync(0xffffffffu, ptx::mbar_wait_bounded(accf_bar(acc), (kb >> 1) & 1, abort_flag, limit));
-      if (!ok) break;
-      ptx::tc_fence_after();
-      uint32_t v[2][32];
-      ptx::tmem_ld_32x32(t_row + static_cast<uint32_t>(acc * FB_TILE), v[0]);
-      ptx::tmem_ld_32x32(t_row + static_cast<uint32_t>(acc * FB_TILE + 32), v[1]);
-      ptx::tmem_ld_wait();
-      // the accumulator is in registers: the products of K block kb + 2 may overwrite it
-      ptx::tc_fence_before();
-      __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(acce_bar(acc));
+    long long it = 0;  // K blocks taken so far, over all tiles of this block (accumulator turn and barrier phase)
+    for (int tile = blockIdx.x; tile < p.n_tiles && ok; tile += gridDim.x) {
+      const int tm = tile / p.tiles_n, tn = tile % p.tiles_n;
+      const int row = tm * FB_TILE + lane_group * 32 + lane;
+      const bool row_ok = row < p.m;
+      const float* sa_row = p.scale_a + static_cast<size_t>(row_ok ? row : 0) * k_blocks;
+      const float* sb_row = p.scale_b + static_cast<size_t>(tn) * k_blocks;
+      uint64_t sum[32];  // 64 fp32 sums, two to a register pair
 #pragma unroll
-      for (int ch = 0; ch < 2; ++ch) {
+      for (int c = 0; c < 32; ++c) sum[c] = 0ull;
+      float s_next = sa_row[0] * sb_row[0];
+      for (int kb = 0; kb < k_blocks; ++kb, ++it) {
+        const int acc = static_cast<int>(it & 1);
+        const uint64_t s2 = ptx::pack_f32x2(s_next, s_next);
+        if (kb + 1 < k_blocks) s_next = sa_row[kb + 1] * sb_row[kb + 1];
+        ok = __all_sync(0xffffffffu, ptx::mbar_wait_bounded(accf_bar(acc), static_cast<uint32_t>(it >> 1) & 1u, abort_flag, limit));
+        if (!ok) break;
+        ptx::tc_fence_after();
+        uint32_t v[2][32];
+        ptx::tmem_ld_32x32(t_row + static_cast<uint32_t>(acc * FB_TILE), v[0]);
+        ptx::tmem_ld_32x32(t_row + static_cast<uint32_t>(acc * FB_TILE + 32), v[1]);
+        ptx::tmem_ld_wait();
+        // the accumulator is in registers: the products two K blocks on may overwrite it
+        ptx::tc_fence_before();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(acce_bar(acc));
 #pragma unroll
-        for (int e = 0; e < 32; e += 2) {
-          const uint64_t x2 = ptx::pack_f32x2(__uint_as_float(v[ch][e]), __uint_as_float(v[ch][e + 1]));
-          sum[ch * 16 + (e >> 1)] = ptx::fma_f32x2(x2, s2, sum[ch * 16 + (e >> 1)]);
+        for (int ch = 0; ch < 2; ++ch) {
+#pragma unroll
+          for (int e = 0; e < 32; e += 2) {
+            const uint64_t x2 = ptx::pack_f32x2(__uint_as_float(v[ch][e]), __uint_as_float(v[ch][e + 1]));
+            sum[ch * 16 + (e >> 1)] = ptx::fma_f32x2(x2, s2, sum[ch * 16 + (e >> 1)]);
+          }
         }
       }
-    }
-    if (ok && row_ok) {
-      bf16* dst = p.c + static_cast<size_t>(row) * p.ldc + tn * FB_TILE + half * 64;
-      const int cols = min(FB_TILE, p.n - tn * FB_TILE) - half * 64;  // a multiple of 16, may be <= 0
+      if (ok && row_ok) {
+        bf16* dst = p.c + static_cast<size_t>(row) * p.ldc + tn * FB_TILE + half * 64;
+        const int cols = min(FB_TILE, p.n - tn * FB_TILE) - half * 64;  // a multiple of 16, may be <= 0
 #pragma unroll
-      for (int c = 0; c < 64; c += 8) {
-        if (c < cols) {
-          float f[8];
+        for (int c = 0; c < 64; c += 8) {
+          if (c < cols) {
+            float f[8];
 #pragma unroll
-          for (int q = 0; q < 4; ++q) ptx::unpack_f32x2(sum[(c >> 1) + q], f[2 * q], f[2 * q + 1]);
-          uint4 o;
-          o.x = ptx::pack_bf16(f[0], f[1]);
-          o.y = ptx::pack_bf16(f[2], f[3]);
-          o.z = ptx::pack_bf16(f[4], f[5]);
-          o.w = ptx::pack_bf16(f[6], f[7]);
-          *reinterpret_cast<uint4*>(dst + c) = o;
+            for (int q = 0; q < 4; ++q) ptx::unpack_f32x2(sum[(c >> 1) + q], f[2 * q], f[2 * q + 1]);
+            uint4 o;
+            o.x = ptx::pack_bf16(f[0], f[1]);
+            o.y = ptx::pack_bf16(f[2], f[3]);
+            o.z = ptx::pack_bf16(f[4], f[5]);
+            o.w = ptx::pack_bf16(f[6], f[7]);
+            *reinterpret_cast<uint4*>(dst + c) = o;
+          }
         }
       }
     }
@@ -300,10 +310,14 @@ pd_status launch_gemm_f8_block(const uint8_t* a, const float* sa, const uint8_t*
   F8BlockDev p{};
   p.c = c; p.scale_a = sa; p.scale_b = sb;
   p.m = m; p.n = n; p.k_blocks = k / FB_TILE; p.ldc = n; p.tiles_n = static_cast<int>(tiles_n);
+  p.n_tiles = static_cast<int>(tiles_m * tiles_n);
   p.err_word = err_word;
   p.wait_limit_ns = 4000000000ull;
-  PD_CUDA_TRY(launch_pdl(gemm_f8_block_kernel, dim3(static_cast<unsigned>(tiles_m * tiles_n)), dim3(FB_THREADS), FB_SMEM_BYTES,
-                         st, ta, tb, p));
+  int dev = 0, sms = 0;
+  PD_CUDA_TRY(cudaGetDevice(&dev));
+  PD_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+  const int grid = p.n_tiles < sms ? p.n_tiles : sms;
+  PD_CUDA_TRY(launch_pdl(gemm_f8_block_kernel, dim3(static_cast<unsigned>(grid)), dim3(FB_THREADS), FB_SMEM_BYTES, st, ta, tb, p));
   count_launch();
   return PD_OK;
 }
