@@ -353,7 +353,7 @@ pd_status pd_gemm_fp8(const void* a_codes, const float* a_scales, const void* b_
  *   C[i, j] = sum over K blocks kb of ( sum_{k in kb} dec(A[i, k]) dec(B[j, k]) ) * a_scales[i, kb] * b_scales[j / 128, kb],
  *   the inner sums exact in fp32 on the tensor cores (tcgen05 kind::f8f6f4), the scaled partial sums added in fp32.
  *
- * pd_quantize_fp8_groups: x device bf16 [rows, k], row pitch ldx elements (a multiple of 4) -> codes device uint8
+ * pd_quantize_fp8_groups: x device bf16 [rows, k], row pitch ldx elements (a multiple of 8) -> codes device uint8
  * [rows, k] contiguous, scales device fp32 [rows, k / 128] contiguous.  k a multiple of 128.
  * pd_quantize_fp8_blocks: w device bf16 [n, k], row pitch ldw elements (a multiple of 8) -> codes device uint8 [n, k]
  * contiguous, scales device fp32 [ceil(n / 128), k / 128] contiguous (the last row of blocks may have fewer than 128

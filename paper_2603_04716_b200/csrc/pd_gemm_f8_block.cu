@@ -208,11 +208,6 @@ gemm_f8_block_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
 // nearest even with saturation, so that the codes are decided in one fixed precision.  An all-zero group or block gets
 // scale 1.
 
-__device__ __forceinline__ void unpack4(uint2 v, float (&f)[4]) {
-  f[0] = ptx::bf16_lo(v.x); f[1] = ptx::bf16_hi(v.x);
-  f[2] = ptx::bf16_lo(v.y); f[3] = ptx::bf16_hi(v.y);
-}
-
 __device__ __forceinline__ void unpack8(const uint4& v, float (&f)[8]) {
   f[0] = ptx::bf16_lo(v.x); f[1] = ptx::bf16_hi(v.x);
   f[2] = ptx::bf16_lo(v.y); f[3] = ptx::bf16_hi(v.y);
@@ -220,29 +215,40 @@ __device__ __forceinline__ void unpack8(const uint4& v, float (&f)[8]) {
   f[6] = ptx::bf16_lo(v.w); f[7] = ptx::bf16_hi(v.w);
 }
 
-// X[rows, k]: one warp per (row, group of 128 elements), four elements per lane.
+// X[rows, k]: half a warp per (row, group of 128 elements), eight elements (16 bytes) per lane.
 constexpr int QG_THREADS = 256;
 __global__ void __launch_bounds__(QG_THREADS) quantize_groups_fp8_kernel(const bf16* __restrict__ x, int ldx, int rows,
                                                                          int groups, uint8_t* __restrict__ codes, int ldq,
                                                                          float* __restrict__ scale_out) {
   ptx::grid_launch_dependents();
   ptx::grid_dependency_wait();
-  const int lane = threadIdx.x & 31;
-  const long long unit = static_cast<long long>(blockIdx.x) * (QG_THREADS / 32) + (threadIdx.x >> 5);
-  if (unit >= static_cast<long long>(rows) * groups) return;
-  const int row = static_cast<int>(unit / groups), g = static_cast<int>(unit % groups);
-  const uint2 v = *reinterpret_cast<const uint2*>(x + static_cast<size_t>(row) * ldx + g * 128 + lane * 4);
-  float f[4];
-  unpack4(v, f);
-  float amax = fmaxf(fmaxf(fabsf(f[0]), fabsf(f[1])), fmaxf(fabsf(f[2]), fabsf(f[3])));
+  const int sub = threadIdx.x & 15;  // lane inside the half warp
+  const long long n_units = static_cast<long long>(rows) * groups;
+  const long long stride = static_cast<long long>(gridDim.x) * (QG_THREADS / 16);
+  // whole warps stay in the loop together (the shuffles below name all 32 lanes): the bound is rounded up to a pair
+  for (long long unit = static_cast<long long>(blockIdx.x) * (QG_THREADS / 16) + (threadIdx.x >> 4); unit < ((n_units + 1) & ~1ll);
+       unit += stride) {
+    const bool live = unit < n_units;
+    const int row = live ? static_cast<int>(unit / groups) : 0, g = live ? static_cast<int>(unit % groups) : 0;
+    const uint4 v = *reinterpret_cast<const uint4*>(x + static_cast<size_t>(row) * ldx + g * 128 + sub * 8);
+    float f[8];
+    unpack8(v, f);
+    float amax = 0.f;
 #pragma unroll
-  for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
-  const float scale = amax > 0.f ? __fdiv_rn(amax, 448.f) : 1.f;
-  if (lane == 0) scale_out[static_cast<size_t>(row) * groups + g] = scale;
+    for (int e = 0; e < 8; ++e) amax = fmaxf(amax, fabsf(f[e]));
 #pragma unroll
-  for (int e = 0; e < 4; ++e) f[e] = __fdiv_rn(f[e], scale);
-  const uint32_t o = ptx::cvt_e4m3x2(f[0], f[1]) | (ptx::cvt_e4m3x2(f[2], f[3]) << 16);
-  *reinterpret_cast<uint32_t*>(codes + static_cast<size_t>(row) * ldq + g * 128 + lane * 4) = o;
+    for (int o = 8; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+    const float scale = amax > 0.f ? __fdiv_rn(amax, 448.f) : 1.f;
+    if (live) {
+      if (sub == 0) scale_out[static_cast<size_t>(row) * groups + g] = scale;
+#pragma unroll
+      for (int e = 0; e < 8; ++e) f[e] = __fdiv_rn(f[e], scale);
+      uint2 o;
+      o.x = ptx::cvt_e4m3x2(f[0], f[1]) | (ptx::cvt_e4m3x2(f[2], f[3]) << 16);
+      o.y = ptx::cvt_e4m3x2(f[4], f[5]) | (ptx::cvt_e4m3x2(f[6], f[7]) << 16);
+      *reinterpret_cast<uint2*>(codes + static_cast<size_t>(row) * ldq + g * 128 + sub * 8) = o;
+    }
+  }
 }
 
 // W[n, k]: one thread block per 128 x 128 block (fewer rows in the last row of blocks); a thread holds half a row.
@@ -328,11 +334,11 @@ extern "C" pd_status pd_quantize_fp8_groups(const void* x, int32_t ldx, int32_t 
                                             void* stream) {
   if (rows == 0) return PD_OK;
   if (!x || !codes || !scales || rows < 0 || k <= 0) return PD_ERR_INVALID_ARG;
-  if (k % 128 != 0 || ldx % 4 != 0 || ldx < k) return PD_ERR_UNSUPPORTED_SHAPE;
+  if (k % 128 != 0 || ldx % 8 != 0 || ldx < k) return PD_ERR_UNSUPPORTED_SHAPE;
   const int groups = k / 128;
   const long long units = static_cast<long long>(rows) * groups;
-  const long long blocks = (units + pd::QG_THREADS / 32 - 1) / (pd::QG_THREADS / 32);
-  if (blocks > 0x7fffffffll) return PD_ERR_UNSUPPORTED_SHAPE;
+  long long blocks = (units + pd::QG_THREADS / 16 - 1) / (pd::QG_THREADS / 16);
+  if (blocks > 148 * 16) blocks = 148 * 16;  // resident blocks take further units grid-stride
   PD_CUDA_TRY(pd::launch_pdl(pd::quantize_groups_fp8_kernel, dim3(static_cast<unsigned>(blocks)), dim3(pd::QG_THREADS), 0,
                              static_cast<cudaStream_t>(stream), static_cast<const pd::bf16*>(x), ldx, rows, groups,
                              static_cast<uint8_t*>(codes), k, scales));
