@@ -378,7 +378,8 @@ pd_status pd_gemm_fp8_blockwise(const void* a_codes, const float* a_scales, cons
  * bound.  Nothing faults or spins without a limit; the output of that launch is undefined, later launches are
  * unaffected.  PD_INJECT_NONE disarms.  (The paper has no counterpart; it exists so that the timeout path can
  * be exercised without a real fault.) */
-enum { PD_INJECT_NONE = 0, PD_INJECT_ATTN_PREFILL = 1, PD_INJECT_GEMM = 2, PD_INJECT_GEMM_PAIR = 3 };
+enum { PD_INJECT_NONE = 0, PD_INJECT_ATTN_PREFILL = 1, PD_INJECT_GEMM = 2, PD_INJECT_GEMM_PAIR = 3,
+       PD_INJECT_GEMM_FP8_BLOCKWISE = 4 };
 pd_status pd_test_inject_wait_timeout(int32_t kernel_kind, uint64_t wait_limit_ns);
 
 /* Kernels launched so far by the calling thread through this library. */

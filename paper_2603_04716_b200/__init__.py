@@ -246,7 +246,7 @@ class LayerConfig:
         return (self.n_q_heads + 2 * self.n_kv_heads) * self.head_dim
 
 
-INJECT_NONE, INJECT_ATTN_PREFILL, INJECT_GEMM, INJECT_GEMM_PAIR = 0, 1, 2, 3
+INJECT_NONE, INJECT_ATTN_PREFILL, INJECT_GEMM, INJECT_GEMM_PAIR, INJECT_GEMM_FP8_BLOCKWISE = 0, 1, 2, 3, 4
 _lib.pd_test_inject_wait_timeout.argtypes = [C.c_int32, C.c_uint64]
 
 

@@ -35,6 +35,7 @@ struct F8BlockDev {
   int m, n, k_blocks, ldc, tiles_n, n_tiles;
   int* err_word;
   unsigned long long wait_limit_ns;
+  int test_skip_load;  // test hook: the producer leaves out one A tile load
 };
 
 __global__ void __launch_bounds__(FB_THREADS, 1)
@@ -93,7 +94,8 @@ gemm_f8_block_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
           if (!ptx::mbar_wait_bounded(empty_bar(stage), phase ^ 1u, abort_flag, limit)) { ok = false; break; }
           const uint32_t sa = smem_base + stage * FB_STAGE_BYTES;
           ptx::mbar_arrive_expect_tx(full_bar(stage), FB_STAGE_BYTES);
-          ptx::tma_load_2d(sa, &tmap_a, kb * FB_TILE, tm * FB_TILE, full_bar(stage));
+          if (!(p.test_skip_load && tile == static_cast<int>(blockIdx.x) && kb == 0))
+            ptx::tma_load_2d(sa, &tmap_a, kb * FB_TILE, tm * FB_TILE, full_bar(stage));
           ptx::tma_load_2d(sa + FB_OPERAND_BYTES, &tmap_b, kb * FB_TILE, tn * FB_TILE, full_bar(stage));
           if (++stage == FB_STAGES) { stage = 0; phase ^= 1u; }
         }
@@ -319,6 +321,7 @@ pd_status launch_gemm_f8_block(const uint8_t* a, const float* sa, const uint8_t*
   p.n_tiles = static_cast<int>(tiles_m * tiles_n);
   p.err_word = err_word;
   p.wait_limit_ns = 4000000000ull;
+  if (take_wait_injection(PD_INJECT_GEMM_FP8_BLOCKWISE, &p.wait_limit_ns)) p.test_skip_load = 1;
   int dev = 0, sms = 0;
   PD_CUDA_TRY(cudaGetDevice(&dev));
   PD_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));

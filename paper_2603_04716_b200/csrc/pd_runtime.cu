@@ -72,7 +72,7 @@ TraceScope::~TraceScope() {
 }  // namespace pd
 
 extern "C" pd_status pd_test_inject_wait_timeout(int32_t kernel_kind, uint64_t wait_limit_ns) {
-  if (kernel_kind < PD_INJECT_NONE || kernel_kind > PD_INJECT_GEMM_PAIR) return PD_ERR_INVALID_ARG;
+  if (kernel_kind < PD_INJECT_NONE || kernel_kind > PD_INJECT_GEMM_FP8_BLOCKWISE) return PD_ERR_INVALID_ARG;
   if (kernel_kind != PD_INJECT_NONE && (wait_limit_ns < 100000ull || wait_limit_ns > 4000000000ull)) return PD_ERR_INVALID_ARG;
   pd::t_inject_kind = kernel_kind;
   pd::t_inject_limit_ns = wait_limit_ns;

@@ -41,6 +41,32 @@ def test_gemm_wait_runs_out_and_the_next_launch_is_correct(pdlib, kind, shape):
     pdlib.pd_test_inject_wait_timeout(pdlib.INJECT_NONE, 0)
 
 
+def test_blockwise_fp8_gemm_wait_runs_out_and_the_next_launch_is_correct(pdlib):
+    import torch
+    from oracle import fp8
+    m, n, k = 300, 512, 512
+    a = gen.normal_bf16(62, 40, (m, k), 1.0, sub=m)
+    b = gen.normal_bf16(62, 41, (n, k), 0.05, sub=n)
+    qa = torch.zeros((m, k), dtype=torch.uint8, device="cuda"); sa = torch.zeros((m, k // 128), dtype=torch.float32, device="cuda")
+    qb = torch.zeros((n, k), dtype=torch.uint8, device="cuda"); sb = torch.zeros((n // 128, k // 128), dtype=torch.float32, device="cuda")
+    pdlib.pd_quantize_fp8_groups(to_dev(a), m, k, qa, sa)
+    pdlib.pd_quantize_fp8_blocks(to_dev(b), n, k, qb, sb)
+    dc = empty_bf16(m, n)
+    err = torch.zeros(1, dtype=torch.int32, device="cuda")
+    pdlib.pd_test_inject_wait_timeout(pdlib.INJECT_GEMM_FP8_BLOCKWISE, LIMIT_NS)
+    pdlib.pd_gemm_fp8_blockwise(qa, sa, qb, sb, dc, m, n, k, err_word=err)
+    torch.cuda.synchronize()
+    assert int(err.item()) == 1, "the injected timeout was not reported"
+    err.zero_()
+    pdlib.pd_gemm_fp8_blockwise(qa, sa, qb, sb, dc, m, n, k, err_word=err)
+    torch.cuda.synchronize()
+    assert int(err.item()) == 0
+    ref = fp8.gemm_fp8_blockwise(qa.cpu().numpy(), sa.cpu().numpy(), qb.cpu().numpy(), sb.cpu().numpy())
+    got = from_dev(dc).astype(np.float64)
+    assert np.all(np.abs(got - ref) <= 2.0 ** -8 * np.abs(ref) + 1e-5 * np.sqrt(k) * 0.05)
+    pdlib.pd_test_inject_wait_timeout(pdlib.INJECT_NONE, 0)
+
+
 def test_prefill_attention_wait_runs_out_and_layer_check_reports_it(pdlib):
     import torch
     shape = dict(d_model=512, n_q_heads=8, n_kv_heads=2, head_dim=64, d_ff=1536)
