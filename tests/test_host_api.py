@@ -218,3 +218,20 @@ def test_refine_next_batch_matches_oracle(pdlib):
                 tpot[i] = srt[rank]
         slo = rnd.uniform(0.001, 0.13)
         assert pdlib.pd_refine_next_batch(batch, tpot, slo) == A.refine_next_batch(batch, tpot, slo)
+
+
+def test_binding_constants_match_the_header(pdlib):
+    """Status codes and wait-injection kinds of the Python binding are the header's enumerators."""
+    import os
+    import re
+    hdr = open(os.path.join(os.path.dirname(__file__), "..", "include", "pd.h")).read()
+    enums = dict((m.group(1), int(m.group(2))) for m in re.finditer(r"\b(PD_[A-Z0-9_]+)\s*=\s*(-?\d+)", hdr))
+    for name in ("PD_OK", "PD_ERR_INVALID_ARG", "PD_ERR_UNSUPPORTED_SHAPE", "PD_ERR_DEVICE_TIMEOUT"):
+        assert getattr(pdlib, name) == enums[name], name
+    for name in ("NONE", "ATTN_PREFILL", "GEMM", "GEMM_PAIR", "GEMM_FP8_BLOCKWISE"):
+        assert getattr(pdlib, "INJECT_" + name) == enums["PD_INJECT_" + name], name
+    # an injection kind outside the enumeration is refused (no GPU needed: the check precedes any device call)
+    with pytest.raises(pdlib.PdError) as e:
+        pdlib.pd_test_inject_wait_timeout(max(v for k, v in enums.items() if k.startswith("PD_INJECT_")) + 1, 1_000_000)
+    assert e.value.status == pdlib.PD_ERR_INVALID_ARG
+    pdlib.pd_test_inject_wait_timeout(pdlib.INJECT_NONE, 0)
